@@ -1,0 +1,329 @@
+"""Pins for the float64 oracle: each checks it against something the paper or the
+mathematics fixes (closed forms, the SVD polar factor, brute force on tiny inputs,
+printed values), never against the oracle's own formula retyped."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+
+RNG = np.random.default_rng(20260516)
+
+
+def f_scalar(x, k):
+    """Scalar Newton-Schulz map x -> x (3 - x^2) / 2 applied k times (what Alg. 4 does to a singular value)."""
+    for _ in range(k):
+        x = 0.5 * x * (3.0 - x * x)
+    return x
+
+
+# ----------------------------------------------------------------------------- momentum
+def test_momentum_constant_gradient_closed_form():
+    g = RNG.normal(size=(5, 7))
+    w = RNG.normal(size=(5, 7))
+    beta = 0.9
+    mom = np.zeros_like(g)
+    for t in range(1, 13):
+        mom = O.momentum_update(mom, g, w, beta, 0.0)
+        assert np.allclose(mom, (1.0 - beta ** t) * g, rtol=1e-13, atol=0)
+
+
+def test_momentum_beta_zero_and_weight_decay():
+    g = RNG.normal(size=(4, 3))
+    w = RNG.normal(size=(4, 3))
+    old = RNG.normal(size=(4, 3))
+    out = O.momentum_update(old, g, w, 0.0, 0.25)
+    assert np.allclose(out, g + 0.25 * w, rtol=1e-15)
+    # one hand-computed entry: beta=0.5, lambda=0.1, mom=2, g=4, w=10 -> 0.5*2 + 0.5*(4+1) = 3.5
+    assert O.momentum_update(np.array([[2.0]]), np.array([[4.0]]), np.array([[10.0]]), 0.5, 0.1)[0, 0] == 3.5
+
+
+# ----------------------------------------------------------------------------- Newton-Schulz
+@pytest.mark.parametrize("shape", [(3, 5), (8, 8), (16, 4), (1, 9), (7, 1)])
+@pytest.mark.parametrize("K", [0, 1, 3, 5])
+def test_polar_ns_matches_svd_closed_form(shape, K):
+    x = RNG.normal(size=shape)
+    u, s, vt = np.linalg.svd(x, full_matrices=False)
+    sigma = math.sqrt(np.sum(s ** 2))
+    expect = (u * f_scalar(s / sigma, K)) @ vt
+    got = O.polar_ns(x, K, 1e-12)
+    assert np.allclose(got, expect, rtol=1e-10, atol=1e-13)
+    got_short = O.polar_ns_short_side(x, K, 1e-12)
+    assert np.allclose(got_short, expect, rtol=1e-10, atol=1e-13)
+
+
+def test_polar_ns_literal_equals_short_side_larger():
+    x = RNG.normal(size=(24, 70))
+    a = O.polar_ns(x, 5)
+    b = O.polar_ns_short_side(x, 5)
+    assert np.max(np.abs(a - b)) <= 1e-13 * np.max(np.abs(a))
+
+
+@pytest.mark.parametrize("K", [1, 2, 3, 4, 5])
+def test_newton_schulz_polar_error_bound(K):
+    # tall 9 x 2 with singular values 0.8, 0.6: ||X||_F = 1, rho = ||I - X^T X||_op = 0.64
+    q1, _ = np.linalg.qr(RNG.normal(size=(9, 2)))
+    q2, _ = np.linalg.qr(RNG.normal(size=(2, 2)))
+    x = (q1 * np.array([0.8, 0.6])) @ q2.T
+    polar = q1 @ q2.T
+    rho = np.linalg.norm(np.eye(2) - x.T @ x, 2)
+    assert abs(rho - 0.64) < 1e-12
+    y = O.polar_ns(x, K)                      # Frobenius scaling is the identity here
+    assert np.linalg.norm(y, 2) <= 1.0 + 1e-12
+    assert np.linalg.norm(y - polar, 2) <= rho ** (2 ** K) + 1e-12
+    if K == 5:
+        # <X, polar(X)> = nuclear norm
+        assert abs(np.sum(x * y) - 1.4) < 1e-6
+
+
+def test_newton_schulz_bare_loop_band():
+    # Alg. 6 with a caller-chosen scaling: singular values in [0.6, 1.0] -> rho = 0.64
+    u, _ = np.linalg.qr(RNG.normal(size=(10, 6)))
+    v, _ = np.linalg.qr(RNG.normal(size=(6, 6)))
+    s = np.array([1.0, 0.95, 0.9, 0.8, 0.7, 0.6])
+    y0 = (u * s) @ v.T
+    y5 = O.newton_schulz(y0, 5)
+    assert np.linalg.norm(y5 - u @ v.T, 2) <= 0.64 ** 32 + 1e-12
+    sv = np.linalg.svd(y5, compute_uv=False)
+    assert np.all(sv <= 1 + 1e-12) and np.all(sv >= f_scalar(0.6, 5) - 1e-12)
+
+
+def test_polar_ns_special_cases():
+    # orthogonal s x s: all singular values 1 -> after fro scaling 1/sqrt(s)
+    q, _ = np.linalg.qr(RNG.normal(size=(6, 6)))
+    assert np.allclose(O.polar_ns(q, 4), f_scalar(1 / math.sqrt(6), 4) * q, rtol=1e-11, atol=1e-14)
+    # diagonal matrix: entrywise scalar recurrence, signs preserved
+    dvals = np.array([3.0, -2.0, 0.5, 1.0])
+    sigma = math.sqrt(np.sum(dvals ** 2))
+    got = O.polar_ns(np.diag(dvals), 3)
+    assert np.allclose(np.diag(got), np.sign(dvals) * f_scalar(np.abs(dvals) / sigma, 3), rtol=1e-12)
+    assert np.allclose(got - np.diag(np.diag(got)), 0, atol=1e-15)
+    # 1 x n: positive multiple of the input (so its sign pattern is that of the input)
+    row = RNG.normal(size=(1, 11))
+    out = O.polar_ns(row, 5)
+    ratio = out / row
+    assert np.all(ratio > 0) and np.allclose(ratio, ratio[0, 0], rtol=1e-12)
+    # K = 0: plain Frobenius normalisation
+    x = RNG.normal(size=(3, 4))
+    assert np.allclose(O.polar_ns(x, 0), x / np.linalg.norm(x), rtol=1e-15)
+    # all-zero input: sigma = 0 -> divide by eps -> zeros -> every bit is 1
+    z = O.polar_ns(np.zeros((3, 3)), 5)
+    assert np.all(z == 0) and np.all(O.encode_bits(z) == 1)
+
+
+def test_planted_mistakes_fail_the_svd_pin():
+    """The SVD pin has teeth: plausible slips in the iteration give different results."""
+    x = RNG.normal(size=(5, 5))
+    u, s, vt = np.linalg.svd(x)
+    expect = (u * f_scalar(s / np.linalg.norm(x), 2)) @ vt
+    y = x / np.linalg.norm(x)
+    wrong_sign = y.copy()
+    wrong_side = y.copy()
+    for _ in range(2):
+        wrong_sign = 0.5 * wrong_sign @ (3 * np.eye(5) + wrong_sign.T @ wrong_sign)
+        wrong_side = 0.5 * wrong_side @ (3 * np.eye(5) - wrong_side @ wrong_side.T)
+    assert not np.allclose(wrong_sign, expect, rtol=1e-6)
+    assert not np.allclose(wrong_side, expect, rtol=1e-6)
+    assert np.allclose(O.polar_ns(x, 2), expect, rtol=1e-11)
+
+
+# ----------------------------------------------------------------------------- sign / pack
+def test_sign_and_encoding_table():
+    u = np.array([3.0, -2.0, 0.0, -0.0, np.nan, 1e-300, -1e-300])
+    assert O.sign_pm1(u).tolist() == [1, -1, 1, 1, -1, 1, -1]
+    assert O.encode_bits(u).tolist() == [1, 0, 1, 1, 0, 1, 0]
+    assert O.decode_bits(np.array([0, 1])).tolist() == [-1, 1]
+    assert np.array_equal(O.decode_bits(O.encode_bits(u)), O.sign_pm1(u))
+
+
+def test_pack_bit_order_hand_example():
+    bits = [1, 0, 0, 0, 0, 0, 0, 0,   0, 1, 0, 0, 0, 0, 0, 1,   1]
+    assert O.pack_bits(bits).tolist() == [0x01, 0x82, 0x01]
+    assert O.bytes_to_words(O.pack_bits(bits)).tolist() == [0x00018201]
+
+
+@pytest.mark.parametrize("d", [1, 7, 8, 9, 31, 32, 33, 64, 1000, 4099])
+def test_pack_roundtrip_and_size(d):
+    bits = RNG.integers(0, 2, size=d).astype(np.uint8)
+    packed = O.pack_bits(bits)
+    assert packed.size == math.ceil(d / 8) == O.payload_bytes(d)
+    assert np.array_equal(O.unpack_bits(packed, d), bits)
+    # independent library check: numpy's own bit packer in little-endian bit order
+    assert np.array_equal(packed, np.packbits(bits, bitorder="little"))
+    # pad bits are zero
+    if d % 8:
+        assert packed[-1] >> (d % 8) == 0
+    assert np.array_equal(O.words_to_bytes(O.bytes_to_words(packed), d), packed)
+
+
+def test_payload_ratios_and_worked_example():
+    d = 2 ** 20
+    assert 4 * d / O.payload_bytes(d, 1) == 32       # bit-packed vs float32
+    assert 4 * d / O.payload_bytes(d, 8) == 4        # int8 vs float32
+    path = os.path.join(os.path.dirname(__file__), "golden", "payload_worked_example.txt")
+    vals = {}
+    for line in open(path):
+        if line.strip() and not line.startswith("#"):
+            k, v = line.split()
+            vals[k] = float(v)
+    dd = int(vals["d_entries"])
+    assert round(4 * dd / 1e6) == vals["fp32_megabytes"]
+    assert round(O.payload_bytes(dd, 1) / 2 ** 20, 1) == vals["onebit_mebibytes"]
+    assert O.payload_bytes(dd, 8) / 1e6 == vals["int8_megabytes"]
+    assert 4 * dd / O.payload_bytes(dd, 1) == vals["ratio_onebit"]
+    assert 4 * dd / O.payload_bytes(dd, 8) == vals["ratio_int8"]
+
+
+# ----------------------------------------------------------------------------- vote
+def brute_force_vote(bits_per_worker):
+    """Count +1 and -1 ballots entry by entry in plain Python."""
+    M = len(bits_per_worker)
+    d = len(bits_per_worker[0])
+    out = []
+    for i in range(d):
+        plus = sum(1 for m in range(M) if bits_per_worker[m][i] == 1)
+        minus = M - plus
+        out.append(1 if plus >= minus else 0)
+    return out
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 8, 16, 31, 32])
+def test_vote_matches_brute_force_and_int8_sum(M):
+    d = 77
+    bits = RNG.integers(0, 2, size=(M, d)).astype(np.uint8)
+    packed = [O.pack_bits(b) for b in bits]
+    vote = O.majority_vote_popcount(packed, d)
+    assert vote.tolist() == brute_force_vote(bits.tolist())
+    # Alg. 2 formulation: sign of the int8 sum of +-1 signs
+    s = O.majority_vote_sum(O.decode_bits(bits))
+    assert np.array_equal(O.decode_bits(vote), s)
+    if M == 1:
+        assert np.array_equal(vote, bits[0])
+    if M % 2 == 1:
+        comp = [O.pack_bits(1 - b) for b in bits]
+        assert np.array_equal(O.majority_vote_popcount(comp, d), 1 - vote)
+
+
+def test_vote_exhaustive_tiny():
+    for M in (1, 2, 3, 4):
+        for ballots in itertools.product([0, 1], repeat=M):
+            packed = [O.pack_bits([b]) for b in ballots]
+            got = int(O.majority_vote_popcount(packed, 1)[0])
+            assert got == (1 if 2 * sum(ballots) >= M else 0)
+
+
+def test_vote_even_tie_goes_to_plus():
+    bits = np.array([[1, 0, 1, 0], [0, 1, 1, 0]], dtype=np.uint8)
+    packed = [O.pack_bits(b) for b in bits]
+    assert O.majority_vote_popcount(packed, 4).tolist() == [1, 1, 1, 0]
+    assert O.majority_vote_sum(O.decode_bits(bits)).tolist() == [1, 1, 1, -1]
+
+
+# ----------------------------------------------------------------------------- local polar / update
+def test_local_polar_norm_and_bound():
+    s = O.decode_bits(RNG.integers(0, 2, size=(6, 10))).astype(np.float64)
+    assert O.frobenius_norm(s) == math.sqrt(60)
+    d = O.local_polar(s, 5)
+    assert np.allclose(d, O.newton_schulz(s / math.sqrt(60), 5), rtol=1e-13)
+    assert np.linalg.norm(d, 2) <= 1 + 1e-12
+    u, sv, vt = np.linalg.svd(s, full_matrices=False)
+    assert np.allclose(d, (u * f_scalar(sv / math.sqrt(60), 5)) @ vt, rtol=1e-10, atol=1e-13)
+
+
+def test_round_to_bf16_matches_torch_and_fixes_double_rounding():
+    x32 = RNG.normal(size=4096).astype(np.float32) * np.float32(0.02)
+    ours = O.round_to_bf16(x32.astype(np.float64))
+    ref = torch.from_numpy(x32).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(ours, ref)
+    # 1 + 2^-8 is a bf16 tie (between 1 and 1 + 2^-7); a float64 just below it must round down,
+    # although float32 rounding alone would land exactly on the tie and then round to even (up? no: 1.0 is even)
+    tie = 1.0 + 2.0 ** -8
+    assert O.round_to_bf16(np.array([tie]))[0] == 1.0                        # tie -> even
+    assert O.round_to_bf16(np.array([tie + 2.0 ** -40]))[0] == np.float32(1.0 + 2.0 ** -7)
+    tie_odd = 1.0 + 3 * 2.0 ** -8                                             # between 1+2^-7 (odd) and 1+2^-6 (even)
+    assert O.round_to_bf16(np.array([tie_odd]))[0] == np.float32(1.0 + 2.0 ** -6)
+    assert O.round_to_bf16(np.array([tie_odd - 2.0 ** -40]))[0] == np.float32(1.0 + 2.0 ** -7)
+
+
+def signum_reference_python(w, g, mom, beta, lr):
+    """Textbook signSGD with momentum, scalar loops: m = beta m + (1-beta) g ; w -= lr * sign(m), sign(0)=+1."""
+    new_w = [row[:] for row in w]
+    new_m = [row[:] for row in mom]
+    for i in range(len(w)):
+        for j in range(len(w[0])):
+            new_m[i][j] = beta * mom[i][j] + (1 - beta) * g[i][j]
+            new_w[i][j] = w[i][j] - lr * (1.0 if new_m[i][j] >= 0 else -1.0)
+    return new_w, new_m
+
+
+def test_step_reduces_to_signum_for_single_worker_no_ns():
+    spec = O.ParamSpec(4, 6, "matrix")
+    cfg = O.OracleConfig(num_workers=1, momentum=0.9, lr=0.01, ns_steps=0, local_polar=False)
+    st = O.init_state([spec], cfg)
+    w = RNG.normal(size=(4, 6))
+    mom_py = [[0.0] * 6 for _ in range(4)]
+    w_py = w.tolist()
+    for t in range(4):
+        g = RNG.normal(size=(1, 4, 6))
+        new_w, _ = O.step([spec], cfg, st, [w], [g])
+        w_py, mom_py = signum_reference_python(w_py, g[0].tolist(), mom_py, 0.9, 0.01)
+        w = new_w[0]
+        assert np.allclose(w, np.array(w_py), rtol=0, atol=1e-15)
+        assert np.allclose(st.mom[0][0], np.array(mom_py), rtol=1e-15)
+
+
+def test_step_update_is_plus_minus_eta_and_plain_kind():
+    for kind in ("matrix", "plain"):
+        spec = O.ParamSpec(5, 8, kind)
+        cfg = O.OracleConfig(num_workers=3, lr=0.125, ns_steps=3)
+        st = O.init_state([spec], cfg)
+        w = RNG.normal(size=(5, 8))
+        g = RNG.normal(size=(3, 5, 8))
+        new_w, tr = O.step([spec], cfg, st, [w], [g])
+        delta = new_w[0] - w
+        assert set(np.unique(np.round(delta / 0.125, 12)).tolist()) <= {-1.0, 1.0}
+        assert np.array_equal(delta < 0, tr[0].vote_bits.reshape(5, 8) == 1)
+        # the vote of the trace equals brute force over the per-worker bits
+        assert tr[0].vote_bits.tolist() == brute_force_vote(tr[0].bits.tolist())
+        if kind == "plain":
+            assert np.array_equal(tr[0].bits, (tr[0].mom.reshape(3, -1) >= 0).astype(np.uint8))
+
+
+def test_step_matrix_sign_is_scale_invariant_and_eq2_scale():
+    spec = O.ParamSpec(6, 4, "matrix")
+    w = RNG.normal(size=(6, 4))
+    g = RNG.normal(size=(2, 6, 4))
+    outs = []
+    for scale in (1.0, 1e-6):
+        cfg = O.OracleConfig(num_workers=2, lr=0.5, ns_steps=5)
+        st = O.init_state([spec], cfg)
+        _, tr = O.step([spec], cfg, st, [w], [g * scale])
+        outs.append(tr[0].bits)
+    assert np.array_equal(outs[0], outs[1])
+    cfg = O.OracleConfig(num_workers=2, lr=0.5, ns_steps=5, update_scale=1)
+    st = O.init_state([spec], cfg)
+    new_w, tr = O.step([spec], cfg, st, [w], [g])
+    assert np.allclose(np.abs(new_w[0] - w), 0.5 / math.sqrt(24), rtol=1e-12)
+    assert abs(O.frobenius_norm(tr[0].direction) - 1.0) < 1e-12      # ||D||_F = 1 (Eq. 2)
+
+
+def test_step_local_polar_direction():
+    spec = O.ParamSpec(8, 5, "matrix")
+    cfg = O.OracleConfig(num_workers=4, lr=0.1, ns_steps=5, local_polar=True)
+    st = O.init_state([spec], cfg)
+    w = RNG.normal(size=(8, 5))
+    g = RNG.normal(size=(4, 8, 5))
+    new_w, tr = O.step([spec], cfg, st, [w], [g])
+    s_bar = O.decode_bits(tr[0].vote_bits).reshape(8, 5).astype(np.float64)
+    u, sv, vt = np.linalg.svd(s_bar, full_matrices=False)
+    expect_d = (u * f_scalar(sv / math.sqrt(40), 5)) @ vt
+    assert np.allclose(tr[0].direction, expect_d, rtol=1e-10, atol=1e-13)
+    assert np.allclose(new_w[0], w - 0.1 * expect_d, rtol=1e-12, atol=1e-15)
+    # override path: feeding another vote changes the direction accordingly
+    flipped = 1 - tr[0].vote_bits
+    tr2 = O.step_param(spec, cfg, np.zeros((4, 8, 5)), w, g, vote_bits_override=flipped)
+    assert np.allclose(tr2.direction, -expect_d, rtol=1e-10, atol=1e-13)
