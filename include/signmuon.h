@@ -1,0 +1,189 @@
+/*
+ * signmuon.h - C ABI of the SignMuon optimizer step for NVIDIA B200 (sm_100a).
+ *
+ * One object computes, for M data-parallel workers held on one GPU as a batch
+ * axis, the step of Alg. 2 / Alg. 3 of the SignMuon paper:
+ *
+ *   per worker m:   G~ = G_m + lambda W                      (weight decay)
+ *                   Mom_m <- beta Mom_m + (1 - beta) G~       (momentum)
+ *                   U_m = PolarNS(Mom_m; K, eps, fro)         (Alg. 4)
+ *                   B_m = PackBits(sign(U_m))                 (>= 0 -> 1, < 0 -> 0)
+ *   shared:         S = sign(sum_m S_m) = sign(2 c - M)       (majority vote, ties -> +1;
+ *                                                              c = popcount over workers)
+ *                   D = S, or S / sqrt(rows cols) (Eq. 2), or PolarNS(S) (local polar step)
+ *                   W <- W - eta D
+ *
+ * The sum all-reduce / all-gather of the paper is replaced by an on-device
+ * reduction over the worker axis; there is no collective.
+ *
+ * Conventions
+ *   - Every pointer is tagged HOST or DEVICE below.  Device pointers must be
+ *     16-byte aligned.  All matrices are row-major and contiguous.
+ *   - The library allocates no device memory: the caller provides the state
+ *     buffer (momenta; persistent across steps) and the workspace (scratch;
+ *     contents meaningful only between a step and the next one).
+ *   - signmuon_step only enqueues work on the given stream and never
+ *     synchronises.  One context must not be used from two streams at once.
+ *   - Every function returns SIGNMUON_OK (0) or a negative error code; nothing
+ *     throws, aborts or prints.
+ *
+ * Packed payload format (App. B, "Packed 1-bit representation"; Alg. 3 note):
+ *   parameters are concatenated in creation order, each padded to a 32-bit
+ *   word; entry i of a parameter (flat row-major index) is bit (i & 31) of word
+ *   (i >> 5), i.e. bit (i & 7) of byte (i >> 3); 1 <-> +1, 0 <-> -1; pad bits
+ *   are 0.  One worker's payload is 4 * sum_p ceil(d_p / 32) bytes
+ *   (= ceil(d / 8) when every d_p is a multiple of 32): one bit per entry,
+ *   1/32 of a float32 gradient.
+ */
+#ifndef SIGNMUON_H_
+#define SIGNMUON_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct signmuon_ctx signmuon_ctx;   /* opaque host object */
+
+enum {
+  SIGNMUON_OK = 0,
+  SIGNMUON_ERR_INVALID_ARG = -1,      /* null pointer, out-of-range scalar */
+  SIGNMUON_ERR_BAD_SHAPE = -2,        /* rows/cols < 1 or too large */
+  SIGNMUON_ERR_NOT_BOUND = -3,        /* step/payload before signmuon_bind */
+  SIGNMUON_ERR_BUFFER_TOO_SMALL = -4, /* state/workspace smaller than signmuon_state_bytes says */
+  SIGNMUON_ERR_CUDA = -5,             /* a CUDA call or launch failed (sticky) */
+  SIGNMUON_ERR_TIMEOUT = -6,          /* a bounded device-side wait ran out (see signmuon_status) */
+  SIGNMUON_ERR_UNSUPPORTED_ARCH = -7, /* current device is not compute capability 10.x */
+  SIGNMUON_ERR_MISALIGNED = -8        /* a device pointer is not 16-byte aligned */
+};
+
+typedef enum { SIGNMUON_F32 = 0, SIGNMUON_BF16 = 1 } signmuon_dtype;
+
+typedef enum {
+  SIGNMUON_PARAM_MATRIX = 0, /* Newton-Schulz path (Alg. 2 with Alg. 4) */
+  SIGNMUON_PARAM_PLAIN = 1   /* vector-like parameter: sign of the momentum, no Newton-Schulz
+                                (App. B treats vectors as m x n with one dimension 1, for which
+                                PolarNS keeps every sign) */
+} signmuon_kind;
+
+typedef struct {
+  int64_t rows, cols;          /* conv weights arrive reshaped to out x (in*kh*kw) */
+  int32_t kind;                /* signmuon_kind */
+  int32_t weight_dtype;        /* signmuon_dtype of W */
+  int32_t grad_dtype;          /* signmuon_dtype of G */
+} signmuon_param;
+
+typedef struct {
+  int32_t num_params;
+  const signmuon_param* params; /* HOST, copied by signmuon_create */
+  int32_t num_workers;          /* M >= 1 (at most 255) */
+  float momentum;               /* beta in [0, 1)                       (Alg. 1 input) */
+  float lr;                     /* eta; signmuon_step may override it per call */
+  int32_t ns_steps;             /* K >= 0; K = 0 gives the sign of the momentum */
+  int32_t local_polar;          /* 0/1: D = PolarNS(S) after the vote (Sec. 3, "Sign-Muon update") */
+  float weight_decay;           /* lambda >= 0, coupled: G~ = G + lambda W */
+  float eps;                    /* Alg. 4 stability constant; <= 0 selects 1e-12 */
+  int32_t update_scale;         /* 0: W -= eta S (Alg. 2)   1: W -= eta S / sqrt(rows cols) (Eq. 2) */
+  int32_t flags;                /* SIGNMUON_FLAG_* */
+} signmuon_config;
+
+enum {
+  SIGNMUON_FLAG_KEEP_POLAR = 1,   /* also store U_m = Y_K (bf16) so that signmuon_debug_tap can return it */
+  SIGNMUON_FLAG_SIMT_GEMM = 2     /* diagnostic: run the Newton-Schulz products on a plain CUDA-core
+                                     kernel instead of the tensor-core kernel (slow; for fault isolation) */
+};
+
+/* Stages of one step, for signmuon_run_stages (bit mask). A full step is all of them in this order. */
+enum {
+  SIGNMUON_STAGE_MOMENTUM = 1,    /* weight decay, momentum, Frobenius norms, plain-parameter update */
+  SIGNMUON_STAGE_NS = 2,          /* K Newton-Schulz iterations per worker, sign + pack */
+  SIGNMUON_STAGE_VOTE = 4,        /* majority vote (+ weight update when local polar is off) */
+  SIGNMUON_STAGE_LOCAL_POLAR = 8, /* PolarNS of the vote matrix + weight update (local polar on) */
+  SIGNMUON_STAGE_ALL = 15
+};
+
+/* What signmuon_debug_tap can return. */
+enum {
+  SIGNMUON_TAP_MOMENTUM = 0,   /* float32 [rows*cols] of (param, worker) */
+  SIGNMUON_TAP_POLAR = 1,      /* bf16 [rows][ld] Y_K of (param, worker); needs SIGNMUON_FLAG_KEEP_POLAR */
+  SIGNMUON_TAP_VOTE_BITS = 2,  /* uint32 words of the vote of a param (worker ignored) */
+  SIGNMUON_TAP_WORKER_BITS = 3,/* uint32 words of (param, worker) inside the payload */
+  SIGNMUON_TAP_NORM = 4        /* float32 [2]: 1/max(sigma,eps)^2 and 1/max(sigma,eps) of (param, worker) */
+};
+
+/* Creates a context from a HOST config (Alg. 2 "Input"). Touches no GPU.
+ * Errors: INVALID_ARG (null, M outside [1,255], beta outside [0,1), K < 0, lambda < 0,
+ * unknown enum), BAD_SHAPE. On error *out is set to NULL. */
+int signmuon_create(const signmuon_config* config, signmuon_ctx** out);
+
+/* Bytes the caller must provide: `state` = momenta of all workers (float32 [M][d] per parameter,
+ * parameters in creation order) - the only persistent optimizer state; `workspace` = scratch
+ * (bf16 Newton-Schulz operands, Gram matrices, packed bits, norms, tile tables);
+ * `host_staging` = extra device bytes needed only by signmuon_step_host (may be queried as NULL). */
+int signmuon_state_bytes(const signmuon_ctx* ctx, size_t* state, size_t* workspace, size_t* host_staging);
+
+/* Attaches DEVICE buffers (owned by the caller, must outlive the context's use of them) and
+ * prepares the device-side tables on `cuda_stream` (a cudaStream_t, NULL = legacy default stream).
+ * `zero_state` != 0 clears the momenta (Mom_0 = 0); pass 0 when restoring a checkpointed state.
+ * `dev_staging` may be NULL when signmuon_step_host is not used.
+ * Errors: BUFFER_TOO_SMALL, MISALIGNED, UNSUPPORTED_ARCH, CUDA. */
+int signmuon_bind(signmuon_ctx* ctx, void* dev_state, size_t state_bytes, void* dev_workspace,
+                  size_t workspace_bytes, void* dev_staging, size_t staging_bytes, int zero_state,
+                  void* cuda_stream);
+
+/* One optimizer step (Alg. 2 / Alg. 3 loop body) enqueued on `cuda_stream`.
+ *   weights: HOST array of num_params DEVICE pointers, W_p [rows][cols] in weight_dtype, updated in place
+ *   grads:   HOST array of num_params DEVICE pointers, G_p [M][rows][cols] in grad_dtype (worker-major), read only
+ *   lr:      eta_t for this step; a negative value selects config.lr
+ * Errors: NOT_BOUND, INVALID_ARG, MISALIGNED, CUDA (sticky launch error). */
+int signmuon_step(signmuon_ctx* ctx, void* const* weights, const void* const* grads, float lr,
+                  void* cuda_stream);
+
+/* Same step, restricted to the stages in `stage_mask` (SIGNMUON_STAGE_*), run in step order.
+ * Lets a caller time or inspect the stages separately; running all stages in order over
+ * several calls equals one signmuon_step. */
+int signmuon_run_stages(signmuon_ctx* ctx, int32_t stage_mask, void* const* weights,
+                        const void* const* grads, float lr, void* cuda_stream);
+
+/* Same step with HOST-resident weights and gradients (same layouts as signmuon_step, but HOST
+ * pointers inside the HOST arrays; pinned memory recommended): copies them to the staging
+ * buffer bound by signmuon_bind, runs the step, copies the weights back, all on `cuda_stream`,
+ * without synchronising.  Errors as signmuon_step, plus NOT_BOUND when no staging was bound. */
+int signmuon_step_host(signmuon_ctx* ctx, void* const* host_weights, const void* const* host_grads,
+                       float lr, void* cuda_stream);
+
+/* The bytes worker `worker` would transmit for the last step (Alg. 3 "PackBits"; App. B s_1):
+ * DEVICE pointer into the workspace (valid until the next step), its size in bytes and the
+ * number of sign entries it carries.  May be called before bind with dev_ptr == NULL to get sizes. */
+int signmuon_packed_payload(const signmuon_ctx* ctx, int32_t worker, const uint32_t** dev_ptr,
+                            size_t* bytes, size_t* entries);
+
+/* Word offset of parameter `param` inside a worker's payload and its word count. */
+int signmuon_payload_segment(const signmuon_ctx* ctx, int32_t param, size_t* word_offset, size_t* words);
+
+/* DEVICE pointer + size of an intermediate result of the last step (SIGNMUON_TAP_*);
+ * `ld` (may be NULL) receives the row pitch in elements for matrix-shaped taps. */
+int signmuon_debug_tap(const signmuon_ctx* ctx, int32_t what, int32_t param, int32_t worker,
+                       const void** dev_ptr, size_t* bytes, int64_t* ld);
+
+/* Synchronises `cuda_stream`, then reads the device status word: OK, TIMEOUT (a bounded wait in a
+ * kernel gave up; results of that step are invalid) or CUDA. */
+int signmuon_status(signmuon_ctx* ctx, void* cuda_stream);
+
+/* Number of kernels signmuon_step launches per call with the current configuration. */
+int signmuon_launches_per_step(const signmuon_ctx* ctx, int32_t* launches);
+
+/* Newton-Schulz floating-point operations of one step: 4 s^2 l K per matrix and worker (plus one
+ * more "worker" for the local polar step), s = min(rows, cols), l = max(rows, cols). */
+int signmuon_ns_flops_per_step(const signmuon_ctx* ctx, double* flops);
+
+void signmuon_destroy(signmuon_ctx* ctx);
+
+const char* signmuon_error_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SIGNMUON_H_ */

@@ -1,0 +1,290 @@
+"""Thin ctypes binding over libsignmuon.so (argument marshalling only).
+
+The functions below carry the names of the C ABI in include/signmuon.h.  `SignMuon`
+bundles a context with the torch tensors that back its state and workspace; torch is
+used for device memory and streams only.  There is no fallback: if the native library
+is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libsignmuon.so")
+
+OK = 0
+F32, BF16 = 0, 1
+PARAM_MATRIX, PARAM_PLAIN = 0, 1
+FLAG_KEEP_POLAR, FLAG_SIMT_GEMM = 1, 2
+STAGE_MOMENTUM, STAGE_NS, STAGE_VOTE, STAGE_LOCAL_POLAR, STAGE_ALL = 1, 2, 4, 8, 15
+TAP_MOMENTUM, TAP_POLAR, TAP_VOTE_BITS, TAP_WORKER_BITS, TAP_NORM = 0, 1, 2, 3, 4
+
+EXPORTS = [
+    "signmuon_create", "signmuon_state_bytes", "signmuon_bind", "signmuon_step", "signmuon_run_stages",
+    "signmuon_step_host", "signmuon_packed_payload", "signmuon_payload_segment", "signmuon_debug_tap",
+    "signmuon_status", "signmuon_launches_per_step", "signmuon_ns_flops_per_step", "signmuon_destroy",
+    "signmuon_error_string",
+]
+
+
+class ParamStruct(C.Structure):
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("kind", C.c_int32),
+                ("weight_dtype", C.c_int32), ("grad_dtype", C.c_int32)]
+
+
+class ConfigStruct(C.Structure):
+    _fields_ = [("num_params", C.c_int32), ("params", C.POINTER(ParamStruct)),
+                ("num_workers", C.c_int32), ("momentum", C.c_float), ("lr", C.c_float),
+                ("ns_steps", C.c_int32), ("local_polar", C.c_int32), ("weight_decay", C.c_float),
+                ("eps", C.c_float), ("update_scale", C.c_int32), ("flags", C.c_int32)]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads the native library; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2605_16311_b200.build` "
+                           "(there is no fallback implementation)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, f32, sz = C.c_void_p, C.c_int32, C.c_float, C.c_size_t
+    lib.signmuon_create.argtypes = [C.POINTER(ConfigStruct), C.POINTER(vp)]
+    lib.signmuon_state_bytes.argtypes = [vp, C.POINTER(sz), C.POINTER(sz), C.POINTER(sz)]
+    lib.signmuon_bind.argtypes = [vp, vp, sz, vp, sz, vp, sz, C.c_int, vp]
+    lib.signmuon_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), f32, vp]
+    lib.signmuon_run_stages.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), f32, vp]
+    lib.signmuon_step_host.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), f32, vp]
+    lib.signmuon_packed_payload.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(sz), C.POINTER(sz)]
+    lib.signmuon_payload_segment.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
+    lib.signmuon_debug_tap.argtypes = [vp, i32, i32, i32, C.POINTER(vp), C.POINTER(sz), C.POINTER(C.c_int64)]
+    lib.signmuon_status.argtypes = [vp, vp]
+    lib.signmuon_launches_per_step.argtypes = [vp, C.POINTER(i32)]
+    lib.signmuon_ns_flops_per_step.argtypes = [vp, C.POINTER(C.c_double)]
+    lib.signmuon_destroy.argtypes = [vp]
+    lib.signmuon_destroy.restype = None
+    lib.signmuon_error_string.argtypes = [C.c_int]
+    lib.signmuon_error_string.restype = C.c_char_p
+    for name in EXPORTS[:-2]:
+        getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+class SignMuonError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = load_library().signmuon_error_string(code).decode()
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise SignMuonError(code, where)
+
+
+# ------------------------------------------------------------------------- C-ABI mirrors
+def signmuon_create(params: Sequence[tuple], num_workers: int, momentum: float, lr: float, ns_steps: int,
+                    local_polar: bool, weight_decay: float = 0.0, eps: float = 1e-12, update_scale: int = 0,
+                    flags: int = 0) -> int:
+    """params: (rows, cols, kind, weight_dtype, grad_dtype) tuples. Returns the context handle."""
+    lib = load_library()
+    arr = (ParamStruct * max(len(params), 1))()
+    for i, (r, c, k, wd, gd) in enumerate(params):
+        arr[i] = ParamStruct(r, c, k, wd, gd)
+    cfg = ConfigStruct(len(params), arr, num_workers, momentum, lr, ns_steps, int(local_polar), weight_decay,
+                       eps, update_scale, flags)
+    out = C.c_void_p()
+    _check(lib.signmuon_create(C.byref(cfg), C.byref(out)), "signmuon_create")
+    return out.value
+
+
+def signmuon_create_raw(cfg: Optional[ConfigStruct]):
+    """Direct call for error-path tests: returns (code, handle)."""
+    lib = load_library()
+    out = C.c_void_p()
+    code = lib.signmuon_create(C.byref(cfg) if cfg is not None else None, C.byref(out))
+    return code, out.value
+
+
+def signmuon_state_bytes(ctx: int):
+    lib = load_library()
+    a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    _check(lib.signmuon_state_bytes(ctx, C.byref(a), C.byref(b), C.byref(c)), "signmuon_state_bytes")
+    return a.value, b.value, c.value
+
+
+def signmuon_bind(ctx: int, state_ptr: int, state_bytes: int, ws_ptr: int, ws_bytes: int, staging_ptr: int,
+                  staging_bytes: int, zero_state: bool, stream: int):
+    _check(load_library().signmuon_bind(ctx, state_ptr, state_bytes, ws_ptr, ws_bytes, staging_ptr or None,
+                                        staging_bytes, int(zero_state), stream or None), "signmuon_bind")
+
+
+def _ptr_array(ptrs: Sequence[int]):
+    arr = (C.c_void_p * len(ptrs))()
+    for i, p in enumerate(ptrs):
+        arr[i] = p
+    return arr
+
+
+def signmuon_step(ctx: int, weight_ptrs, grad_ptrs, lr: float, stream: int):
+    _check(load_library().signmuon_step(ctx, weight_ptrs, grad_ptrs, lr, stream or None), "signmuon_step")
+
+
+def signmuon_run_stages(ctx: int, mask: int, weight_ptrs, grad_ptrs, lr: float, stream: int):
+    _check(load_library().signmuon_run_stages(ctx, mask, weight_ptrs, grad_ptrs, lr, stream or None),
+           "signmuon_run_stages")
+
+
+def signmuon_step_host(ctx: int, weight_ptrs, grad_ptrs, lr: float, stream: int):
+    _check(load_library().signmuon_step_host(ctx, weight_ptrs, grad_ptrs, lr, stream or None), "signmuon_step_host")
+
+
+def signmuon_packed_payload(ctx: int, worker: int, want_ptr: bool = True):
+    lib = load_library()
+    p, b, e = C.c_void_p(), C.c_size_t(), C.c_size_t()
+    _check(lib.signmuon_packed_payload(ctx, worker, C.byref(p) if want_ptr else None, C.byref(b), C.byref(e)),
+           "signmuon_packed_payload")
+    return p.value, b.value, e.value
+
+
+def signmuon_payload_segment(ctx: int, param: int):
+    lib = load_library()
+    o, w = C.c_size_t(), C.c_size_t()
+    _check(lib.signmuon_payload_segment(ctx, param, C.byref(o), C.byref(w)), "signmuon_payload_segment")
+    return o.value, w.value
+
+
+def signmuon_debug_tap(ctx: int, what: int, param: int, worker: int):
+    lib = load_library()
+    p, b, ld = C.c_void_p(), C.c_size_t(), C.c_int64()
+    _check(lib.signmuon_debug_tap(ctx, what, param, worker, C.byref(p), C.byref(b), C.byref(ld)),
+           "signmuon_debug_tap")
+    return p.value, b.value, ld.value
+
+
+def signmuon_status(ctx: int, stream: int) -> int:
+    return load_library().signmuon_status(ctx, stream or None)
+
+
+def signmuon_launches_per_step(ctx: int) -> int:
+    n = C.c_int32()
+    _check(load_library().signmuon_launches_per_step(ctx, C.byref(n)), "signmuon_launches_per_step")
+    return n.value
+
+
+def signmuon_ns_flops_per_step(ctx: int) -> float:
+    f = C.c_double()
+    _check(load_library().signmuon_ns_flops_per_step(ctx, C.byref(f)), "signmuon_ns_flops_per_step")
+    return f.value
+
+
+def signmuon_destroy(ctx: int):
+    load_library().signmuon_destroy(ctx)
+
+
+# ------------------------------------------------------------------------- convenience wrapper
+_DT = {"f32": F32, "bf16": BF16}
+_KIND = {"matrix": PARAM_MATRIX, "plain": PARAM_PLAIN}
+
+
+def _view_device(ptr: int, nbytes: int, dtype: torch.dtype, owner: torch.Tensor, base_ptr: int) -> torch.Tensor:
+    """A tensor view of `nbytes` at device address `ptr`, which lies inside `owner` (uint8)."""
+    off = ptr - base_ptr
+    return owner[off: off + nbytes].view(dtype)
+
+
+class SignMuon:
+    """Owns a context plus the torch buffers behind it. `params` are workloads.Param-like objects
+    (rows, cols, kind, dtype)."""
+
+    def __init__(self, params, num_workers: int, momentum: float = 0.9, lr: float = 1e-3, ns_steps: int = 5,
+                 local_polar: bool = False, weight_decay: float = 0.0, eps: float = 1e-12, update_scale: int = 0,
+                 flags: int = 0, device: str = "cuda:0", host_staging: bool = False):
+        self.params = list(params)
+        self.num_workers = num_workers
+        self.ns_steps = ns_steps
+        self.device = torch.device(device)
+        tuples = [(p.rows, p.cols, _KIND[p.kind], _DT[p.dtype], _DT[p.dtype]) for p in self.params]
+        self.ctx = signmuon_create(tuples, num_workers, momentum, lr, ns_steps, local_polar, weight_decay, eps,
+                                   update_scale, flags)
+        self.state_bytes, self.workspace_bytes, self.staging_bytes = signmuon_state_bytes(self.ctx)
+        with torch.cuda.device(self.device):
+            self.state = torch.empty(self.state_bytes, dtype=torch.uint8, device=self.device)
+            # over-allocate so the workspace can start on a 1024-byte boundary
+            self._ws_raw = torch.empty(self.workspace_bytes + 1024, dtype=torch.uint8, device=self.device)
+            off = (-self._ws_raw.data_ptr()) % 1024
+            self.workspace = self._ws_raw[off: off + self.workspace_bytes]
+            self.staging = (torch.empty(self.staging_bytes, dtype=torch.uint8, device=self.device)
+                            if host_staging else None)
+            stream = torch.cuda.current_stream(self.device).cuda_stream
+            signmuon_bind(self.ctx, self.state.data_ptr(), self.state_bytes, self.workspace.data_ptr(),
+                          self.workspace_bytes, self.staging.data_ptr() if host_staging else 0,
+                          self.staging_bytes if host_staging else 0, True, stream)
+        self._ptr_cache = None
+
+    def close(self):
+        if self.ctx:
+            signmuon_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _ptrs(self, weights: List[torch.Tensor], grads: List[torch.Tensor]):
+        key = (tuple(w.data_ptr() for w in weights), tuple(g.data_ptr() for g in grads))
+        if self._ptr_cache is None or self._ptr_cache[0] != key:
+            self._ptr_cache = (key, _ptr_array(key[0]), _ptr_array(key[1]))
+        return self._ptr_cache[1], self._ptr_cache[2]
+
+    def step(self, weights, grads, lr: float = -1.0, stages: int = STAGE_ALL):
+        wp, gp = self._ptrs(weights, grads)
+        stream = torch.cuda.current_stream(self.device).cuda_stream
+        if stages == STAGE_ALL:
+            signmuon_step(self.ctx, wp, gp, lr, stream)
+        else:
+            signmuon_run_stages(self.ctx, stages, wp, gp, lr, stream)
+
+    def step_host(self, host_weights, host_grads, lr: float = -1.0):
+        wp, gp = self._ptrs(host_weights, host_grads)
+        signmuon_step_host(self.ctx, wp, gp, lr, torch.cuda.current_stream(self.device).cuda_stream)
+
+    def status(self) -> int:
+        return signmuon_status(self.ctx, torch.cuda.current_stream(self.device).cuda_stream)
+
+    def payload(self, worker: int) -> torch.Tensor:
+        """uint8 view of the bytes worker `worker` would transmit (valid until the next step)."""
+        ptr, nbytes, _ = signmuon_packed_payload(self.ctx, worker)
+        return _view_device(ptr, nbytes, torch.uint8, self.workspace, self.workspace.data_ptr())
+
+    def tap(self, what: int, param: int, worker: int = 0) -> torch.Tensor:
+        ptr, nbytes, ld = signmuon_debug_tap(self.ctx, what, param, worker)
+        p = self.params[param]
+        if what == TAP_MOMENTUM:
+            return _view_device(ptr, nbytes, torch.float32, self.state, self.state.data_ptr()).view(p.rows, p.cols)
+        base = self.workspace.data_ptr()
+        if what == TAP_POLAR:
+            return _view_device(ptr, nbytes, torch.bfloat16, self.workspace, base).view(p.rows, ld)[:, : p.cols]
+        if what in (TAP_VOTE_BITS, TAP_WORKER_BITS):
+            return _view_device(ptr, nbytes, torch.uint8, self.workspace, base)
+        if what == TAP_NORM:
+            return _view_device(ptr, nbytes, torch.float32, self.workspace, base)
+        raise ValueError(what)
+
+    @property
+    def launches_per_step(self) -> int:
+        return signmuon_launches_per_step(self.ctx)
+
+    @property
+    def ns_flops_per_step(self) -> float:
+        return signmuon_ns_flops_per_step(self.ctx)

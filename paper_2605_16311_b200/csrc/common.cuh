@@ -1,0 +1,210 @@
+// Shared device-side structures of the SignMuon step (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace signmuon {
+
+typedef __nv_bfloat16 bf16;
+
+// Device status word values (first word of the status area in the workspace).
+enum : uint32_t { STATUS_OK = 0, STATUS_TIMEOUT = 1 };
+
+// One entry per parameter block, uploaded when the caller's pointers change.
+struct ParamDev {
+  void* W;              // [rows][cols] weight_dtype, in/out
+  const void* G;        // [M][rows][cols] grad_dtype
+  float* mom;           // [M][rows*cols] float32 momentum (state buffer)
+  bf16* y0;             // matrix params: Newton-Schulz operand buffer 0, [M][rows][ldy]
+  bf16* y1;             // matrix params: operand buffer 1 (ping-pong partner)
+  float* scales;        // matrix params: [M][2] = {1/max(sigma,eps)^2, 1/max(sigma,eps)}
+  float* partials;      // matrix params: [M][chunks_per_worker] per-block sums of squares
+  int64_t d;            // rows*cols
+  int32_t rows, cols;
+  int32_t ldy;          // row pitch of the bf16 operand buffers (cols rounded up to 8)
+  int32_t kind, wdtype, gdtype;
+  uint32_t word_off;    // first word of this parameter inside a worker's payload
+  uint32_t n_words;     // ceil(d / 32)
+  uint32_t chunks_per_worker;  // momentum-kernel blocks (= norm partials) per worker
+  float upd_scale;      // 1, or 1/sqrt(rows*cols) for the Eq. 2 normalisation
+  int32_t vec_ok;       // 16-byte vector path allowed (d % 8 == 0 and ldy == cols)
+};
+
+// Epilogues of the Newton-Schulz products.
+//
+// The iterate is kept as a bf16 pair: `hi` = bf16(y) is the tensor-core operand, `lo` = bf16(y - hi)
+// the remainder, so that the dominant term 1.5 * Y_k of  Y_{k+1} = 1.5 Y_k + (-A/2) Y_k  enters
+// with ~16 mantissa bits while the product uses `hi` only.  An entry of Y_K near zero is the
+// difference of its own term and the product term; carrying its own term in bf16 alone would
+// decide such signs with a 2^-9 relative error of a term that is not small.
+enum : int32_t {
+  EPI_GRAM = 0,          // out = bf16(-0.5 * scale * acc)                      (the "-A/2" of 3I/2 - A/2)
+  EPI_APPLY = 1,         // y = scale * (acc + 1.5 * C); out = hi(y), out_lo = lo(y)   (Y_{k+1})
+  EPI_APPLY_PACK = 2,    // sign bits of y -> payload words (hi(y) optionally stored)
+  EPI_APPLY_UPDATE = 3   // W -= lr * y                                          (local polar step)
+};
+
+enum : int32_t {
+  C_BF16 = 0,            // C = hi only (exact for the +-1 vote matrix)
+  C_HILO = 1,            // C = hi + lo
+  C_F32 = 2              // C = float32 momentum (first iteration)
+};
+
+// One product D[M x N] = A * B^T-like contraction over K with bf16 operands.
+//   a(i,k) = A[i*a_sm + k*a_sk],  b(j,k) = B[j*b_sn + k*b_sk]   (element strides)
+struct GemmProblem {
+  const bf16* A;
+  const bf16* B;
+  int64_t a_sm, a_sk, b_sn, b_sk;
+  int32_t M, N, K;
+  int32_t tmapA, tmapB;   // indices into the tensor-map array (tensor-core kernel)
+  int32_t batch;          // third TMA coordinate (worker slot)
+  int32_t a_mn, b_mn;     // 1: operand is contiguous along M/N (not along K)
+  int32_t epi;
+  void* out;              // bf16 output (GRAM: -A/2; APPLY*: hi part of Y_{k+1})
+  bf16* out_lo;           // APPLY: lo part of Y_{k+1} (same pitch as out)
+  int64_t ld_out;
+  const void* C;          // APPLY*: Y_k (bf16 hi, or float32 momentum when c_mode == C_F32)
+  const bf16* C_lo;       // APPLY*: lo part of Y_k when c_mode == C_HILO
+  int64_t ldc;
+  const float* scale_ptr; // optional per-problem scale read from memory (else scale_imm)
+  float scale_imm;
+  int32_t c_mode;
+  int32_t store_out;      // APPLY_PACK: also write hi(y)
+  int32_t param;          // APPLY_UPDATE: index into the ParamDev table
+  uint32_t* bits_out;     // APPLY_PACK: first payload word of this (param, worker)
+};
+
+struct TileEntry {
+  uint32_t problem;       // index relative to the launch's first problem
+  uint16_t tm, tn;        // tile coordinates (units of 128 rows / BN columns)
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// Stores 32 floats as bf16 (hi) and optionally the bf16 remainders (lo) at row pointer offsets.
+__device__ __forceinline__ void store_hi_lo(bf16* o, bf16* olo, const float (&v)[32], bool vec, int n_valid) {
+  if (vec) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t w[4], wl[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float a = v[q * 8 + 2 * e], b = v[q * 8 + 2 * e + 1];
+        w[e] = pack_bf16x2(a, b);
+        wl[e] = pack_bf16x2(a - __uint_as_float(w[e] << 16), b - __uint_as_float(w[e] & 0xffff0000u));
+      }
+      reinterpret_cast<uint4*>(o)[q] = make_uint4(w[0], w[1], w[2], w[3]);
+      if (olo) reinterpret_cast<uint4*>(olo)[q] = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+    }
+  } else {
+    for (int j = 0; j < n_valid; ++j) {
+      const bf16 h = __float2bfloat16_rn(v[j]);
+      o[j] = h;
+      if (olo) olo[j] = __float2bfloat16_rn(v[j] - __bfloat162float(h));
+    }
+  }
+}
+
+// Applies one epilogue to 32 consecutive columns [col0, col0+32) of output row `row`.
+// `v` holds the fp32 accumulators.  Rows/columns outside the problem are skipped.
+__device__ __forceinline__ void epilogue_row32(const GemmProblem& pr, const ParamDev* params, float lr,
+                                               int row, int col0, float (&v)[32]) {
+  if (row >= pr.M || col0 >= pr.N) return;
+  const float scale = pr.scale_ptr ? __ldg(pr.scale_ptr) : pr.scale_imm;
+  const bool full = (col0 + 32 <= pr.N);
+  const int n_valid = full ? 32 : pr.N - col0;
+  if (pr.epi == EPI_GRAM) {
+    const float f = -0.5f * scale;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] *= f;
+    bf16* o = reinterpret_cast<bf16*>(pr.out) + (int64_t)row * pr.ld_out + col0;
+    store_hi_lo(o, nullptr, v, full && ((pr.ld_out & 7) == 0), n_valid);
+    return;
+  }
+  // APPLY family: y = scale * (acc + 1.5 * C)
+  if (pr.c_mode == C_F32) {
+    const float* c = reinterpret_cast<const float*>(pr.C) + (int64_t)row * pr.ldc + col0;
+    if (full && ((pr.ldc & 3) == 0)) {
+      const float4* c4 = reinterpret_cast<const float4*>(c);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const float4 t = __ldg(c4 + q);
+        v[4 * q] = scale * fmaf(1.5f, t.x, v[4 * q]);
+        v[4 * q + 1] = scale * fmaf(1.5f, t.y, v[4 * q + 1]);
+        v[4 * q + 2] = scale * fmaf(1.5f, t.z, v[4 * q + 2]);
+        v[4 * q + 3] = scale * fmaf(1.5f, t.w, v[4 * q + 3]);
+      }
+    } else {
+      for (int j = 0; j < 32; ++j) v[j] = (j < n_valid) ? scale * fmaf(1.5f, __ldg(c + j), v[j]) : 0.f;
+    }
+  } else {
+    const bf16* c = reinterpret_cast<const bf16*>(pr.C) + (int64_t)row * pr.ldc + col0;
+    const bf16* cl = pr.c_mode == C_HILO ? pr.C_lo + (int64_t)row * pr.ldc + col0 : nullptr;
+    if (full && ((pr.ldc & 7) == 0)) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 t = __ldg(reinterpret_cast<const uint4*>(c) + q);
+        uint4 u = make_uint4(0, 0, 0, 0);
+        if (cl) u = *(reinterpret_cast<const uint4*>(cl) + q);
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+        const uint32_t wl[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float c0 = __uint_as_float(w[e] << 16) + __uint_as_float(wl[e] << 16);
+          const float c1 = __uint_as_float(w[e] & 0xffff0000u) + __uint_as_float(wl[e] & 0xffff0000u);
+          v[q * 8 + 2 * e] = scale * fmaf(1.5f, c0, v[q * 8 + 2 * e]);
+          v[q * 8 + 2 * e + 1] = scale * fmaf(1.5f, c1, v[q * 8 + 2 * e + 1]);
+        }
+      }
+    } else {
+      for (int j = 0; j < 32; ++j) {
+        float cv = 0.f;
+        if (j < n_valid) cv = __bfloat162float(c[j]) + (cl ? __bfloat162float(cl[j]) : 0.f);
+        v[j] = (j < n_valid) ? scale * fmaf(1.5f, cv, v[j]) : 0.f;
+      }
+    }
+  }
+  if (pr.epi == EPI_APPLY || (pr.epi == EPI_APPLY_PACK && pr.store_out)) {
+    bf16* o = reinterpret_cast<bf16*>(pr.out) + (int64_t)row * pr.ld_out + col0;
+    bf16* ol = (pr.epi == EPI_APPLY && pr.out_lo) ? pr.out_lo + (int64_t)row * pr.ld_out + col0 : nullptr;
+    store_hi_lo(o, ol, v, full && ((pr.ld_out & 7) == 0), n_valid);
+  }
+  if (pr.epi == EPI_APPLY_PACK) {
+    // Only issued for parameters with cols % 32 == 0: the 32 columns are one payload word.
+    uint32_t word = 0;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) word |= (v[j] >= 0.f ? 1u : 0u) << j;
+    pr.bits_out[((int64_t)row * pr.N + col0) >> 5] = word;
+  } else if (pr.epi == EPI_APPLY_UPDATE) {
+    const ParamDev& pd = params[pr.param];
+    const float step = lr;
+    if (pd.wdtype == 0) {
+      float* w = reinterpret_cast<float*>(pd.W) + (int64_t)row * pr.N + col0;
+      if (full && ((pr.N & 3) == 0)) {
+        float4* w4 = reinterpret_cast<float4*>(w);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          float4 t = w4[q];
+          t.x = fmaf(-step, v[4 * q], t.x);
+          t.y = fmaf(-step, v[4 * q + 1], t.y);
+          t.z = fmaf(-step, v[4 * q + 2], t.z);
+          t.w = fmaf(-step, v[4 * q + 3], t.w);
+          w4[q] = t;
+        }
+      } else {
+        for (int j = 0; j < n_valid; ++j) w[j] = fmaf(-step, v[j], w[j]);
+      }
+    } else {
+      bf16* w = reinterpret_cast<bf16*>(pd.W) + (int64_t)row * pr.N + col0;
+      for (int j = 0; j < n_valid; ++j) w[j] = __float2bfloat16_rn(fmaf(-step, v[j], __bfloat162float(w[j])));
+    }
+  }
+}
+
+}  // namespace signmuon

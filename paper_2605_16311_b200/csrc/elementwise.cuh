@@ -1,0 +1,379 @@
+// Memory-bound kernels of the SignMuon step: momentum (+ Frobenius norm + bf16 operand),
+// fused plain-parameter update, stand-alone sign pack, and majority vote + weight update.
+#pragma once
+
+#include "common.cuh"
+
+namespace signmuon {
+
+constexpr int EW_THREADS = 256;
+constexpr int MOM_CHUNK = 8192;        // entries per block of the momentum kernel (256 threads x 8 x 4)
+constexpr int PLAIN_CHUNK = 1024;      // entries per block of the plain-parameter kernel (8 warps x 128)
+constexpr int VOTE_WORDS = 256;        // payload words per block of the vote kernel (8 warps x 32)
+constexpr int PACK_CHUNK = 8192;       // entries per block of the stand-alone pack kernel
+
+// Finds the list slot whose block range contains `block` (`starts` is ascending, one entry per slot).
+__device__ __forceinline__ int find_slot(const uint32_t* __restrict__ starts, int n, uint32_t block) {
+  int lo = 0, hi = n - 1;
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if (__ldg(starts + mid) <= block) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+template <typename T> __device__ __forceinline__ float load_as_float(const T* p);
+template <> __device__ __forceinline__ float load_as_float<float>(const float* p) { return __ldg(p); }
+template <> __device__ __forceinline__ float load_as_float<bf16>(const bf16* p) {
+  return __bfloat162float(*p);
+}
+
+// Loads 8 consecutive elements (16-byte aligned for bf16, 32-byte span for float) as floats.
+__device__ __forceinline__ void load8(const float* p, float (&x)[8]) {
+  const float4 a = __ldcs(reinterpret_cast<const float4*>(p));
+  const float4 b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+  x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+__device__ __forceinline__ void load8(const bf16* p, float (&x)[8]) {
+  const uint4 a = __ldcs(reinterpret_cast<const uint4*>(p));
+  const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    x[2 * e] = __uint_as_float(w[e] << 16);
+    x[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Momentum of the matrix parameters (Alg. 2: weight decay + momentum; Alg. 4: ||Mom||_F):
+//   Mom <- beta Mom + (1-beta)(G + lambda W);  Y0 = bf16(Mom);  partial[block] = sum Mom^2.
+// Grid: one block per MOM_CHUNK entries of one (parameter, worker).
+// ---------------------------------------------------------------------------------------------
+template <typename GT, typename WT>
+__device__ __forceinline__ void momentum_block(const ParamDev& pd, int m, uint32_t chunk, float beta,
+                                               float lambda, float& sumsq) {
+  const int64_t d = pd.d;
+  const GT* g = reinterpret_cast<const GT*>(pd.G) + (int64_t)m * d;
+  const WT* w = reinterpret_cast<const WT*>(pd.W);
+  float* mom = pd.mom + (int64_t)m * d;
+  bf16* y = pd.y0 + (int64_t)m * pd.rows * pd.ldy;
+  const int64_t base = (int64_t)chunk * MOM_CHUNK;
+  const float omb = 1.f - beta;
+  if (pd.vec_ok) {
+#pragma unroll
+    for (int it = 0; it < MOM_CHUNK / (EW_THREADS * 8); ++it) {
+      const int64_t i = base + ((int64_t)it * EW_THREADS + threadIdx.x) * 8;
+      if (i < d) {   // d % 8 == 0 on this path
+        float gv[8], mv[8];
+        load8(g + i, gv);
+        load8(mom + i, mv);
+        if (lambda != 0.f) {
+          float wv[8];
+          load8(w + i, wv);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) gv[e] = fmaf(lambda, wv[e], gv[e]);
+        }
+        uint32_t packed[4];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          mv[e] = fmaf(beta, mv[e], omb * gv[e]);
+          sumsq = fmaf(mv[e], mv[e], sumsq);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __nv_bfloat162 h = __floats2bfloat162_rn(mv[2 * e], mv[2 * e + 1]);
+          packed[e] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        float4* mo = reinterpret_cast<float4*>(mom + i);
+        mo[0] = make_float4(mv[0], mv[1], mv[2], mv[3]);
+        mo[1] = make_float4(mv[4], mv[5], mv[6], mv[7]);
+        *reinterpret_cast<uint4*>(y + i) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+      }
+    }
+  } else {
+    const int64_t end = (base + MOM_CHUNK < d) ? base + MOM_CHUNK : d;
+    for (int64_t i = base + threadIdx.x; i < end; i += EW_THREADS) {
+      float gv = load_as_float<GT>(g + i);
+      if (lambda != 0.f) gv = fmaf(lambda, load_as_float<WT>(w + i), gv);
+      const float mv = fmaf(beta, mom[i], omb * gv);
+      mom[i] = mv;
+      sumsq = fmaf(mv, mv, sumsq);
+      const int64_t r = i / pd.cols;
+      const int64_t c = i - r * pd.cols;
+      y[r * pd.ldy + c] = __float2bfloat16_rn(mv);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(EW_THREADS) momentum_kernel(const ParamDev* __restrict__ params,
+                                                              const int32_t* __restrict__ list,
+                                                              const uint32_t* __restrict__ starts, int n_list,
+                                                              float beta, float lambda) {
+  const int slot = find_slot(starts, n_list, blockIdx.x);
+  const ParamDev pd = params[list[slot]];
+  const uint32_t local = blockIdx.x - starts[slot];
+  const int m = local / pd.chunks_per_worker;
+  const uint32_t chunk = local - m * pd.chunks_per_worker;
+  float sumsq = 0.f;
+  if (pd.gdtype == 0) {
+    if (pd.wdtype == 0) momentum_block<float, float>(pd, m, chunk, beta, lambda, sumsq);
+    else momentum_block<float, bf16>(pd, m, chunk, beta, lambda, sumsq);
+  } else {
+    if (pd.wdtype == 0) momentum_block<bf16, float>(pd, m, chunk, beta, lambda, sumsq);
+    else momentum_block<bf16, bf16>(pd, m, chunk, beta, lambda, sumsq);
+  }
+  __shared__ float red[EW_THREADS / 32];
+  sumsq = warp_sum(sumsq);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sumsq;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < EW_THREADS / 32; ++i) t += red[i];
+    pd.partials[(int64_t)m * pd.chunks_per_worker + chunk] = t;
+  }
+}
+
+// One warp per (matrix parameter, worker): fixed-order sum of the block partials in double,
+// then the two scale factors the Newton-Schulz epilogues use.
+__global__ void finalize_norms_kernel(const ParamDev* __restrict__ params, const int32_t* __restrict__ list,
+                                      int n_list, int num_workers, float eps) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (warp >= n_list * num_workers) return;
+  const ParamDev& pd = params[list[warp / num_workers]];
+  const int m = warp % num_workers;
+  const float* part = pd.partials + (int64_t)m * pd.chunks_per_worker;
+  double acc = 0.0;
+  for (uint32_t i = lane; i < pd.chunks_per_worker; i += 32) acc += (double)part[i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) {
+    const double sigma = fmax(sqrt(acc), (double)eps);
+    pd.scales[2 * m] = (float)(1.0 / (sigma * sigma));
+    pd.scales[2 * m + 1] = (float)(1.0 / sigma);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Plain parameters: the whole step in one pass (no Newton-Schulz): momentum of every worker,
+// bit = (Mom >= 0), ballot-packed payload words, majority vote in registers, weight update.
+// Each warp owns 128 consecutive entries; lane l holds entries base + 32 k + l, k = 0..3, so that
+// one __ballot_sync per (worker, k) yields one payload word.
+// ---------------------------------------------------------------------------------------------
+template <typename GT, typename WT>
+__device__ __forceinline__ void plain_block(const ParamDev& pd, uint32_t chunk, int M, float beta,
+                                            float lambda, float step, uint32_t* __restrict__ bits,
+                                            uint32_t* __restrict__ vote_words, int64_t words_per_worker) {
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int64_t d = pd.d;
+  const int64_t base = (int64_t)chunk * PLAIN_CHUNK + warp * 128;
+  if (base >= d) return;
+  const GT* g = reinterpret_cast<const GT*>(pd.G);
+  WT* w = reinterpret_cast<WT*>(pd.W);
+  const float omb = 1.f - beta;
+  int count[4] = {0, 0, 0, 0};
+  float wv[4];
+  bool valid[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int64_t i = base + 32 * k + lane;
+    valid[k] = i < d;
+    wv[k] = valid[k] ? load_as_float<WT>(w + i) : 0.f;
+  }
+  const int64_t word0 = base >> 5;
+  for (int m = 0; m < M; ++m) {
+    const GT* gm = g + (int64_t)m * d;
+    float* mm = pd.mom + (int64_t)m * d;
+    float mv[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int64_t i = base + 32 * k + lane;
+      float gv = valid[k] ? load_as_float<GT>(gm + i) : 0.f;
+      float old = valid[k] ? __ldcs(mm + i) : 0.f;
+      gv = fmaf(lambda, wv[k], gv);
+      mv[k] = fmaf(beta, old, omb * gv);
+    }
+    uint32_t mine = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int64_t i = base + 32 * k + lane;
+      if (valid[k]) __stcs(mm + i, mv[k]);
+      const bool b = valid[k] && (mv[k] >= 0.f);
+      count[k] += b ? 1 : 0;
+      const uint32_t word = __ballot_sync(0xffffffffu, b);
+      if (lane == k) mine = word;
+    }
+    if (lane < 4 && word0 + lane < pd.n_words)
+      bits[(int64_t)m * words_per_worker + pd.word_off + word0 + lane] = mine;
+  }
+  uint32_t vmine = 0;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int64_t i = base + 32 * k + lane;
+    const bool plus = valid[k] && (2 * count[k] >= M);
+    const uint32_t word = __ballot_sync(0xffffffffu, plus);
+    if (lane == k) vmine = word;
+    if (valid[k]) {
+      const float nw = wv[k] - (plus ? step : -step);
+      if (sizeof(WT) == 4) reinterpret_cast<float*>(w)[i] = nw;
+      else reinterpret_cast<bf16*>(w)[i] = __float2bfloat16_rn(nw);
+    }
+  }
+  if (lane < 4 && word0 + lane < pd.n_words) vote_words[pd.word_off + word0 + lane] = vmine;
+}
+
+__global__ void __launch_bounds__(EW_THREADS) plain_params_kernel(const ParamDev* __restrict__ params,
+                                                                  const int32_t* __restrict__ list,
+                                                                  const uint32_t* __restrict__ starts, int n_list,
+                                                                  int M, float beta, float lambda, float lr,
+                                                                  uint32_t* __restrict__ bits,
+                                                                  uint32_t* __restrict__ vote_words,
+                                                                  int64_t words_per_worker) {
+  const int slot = find_slot(starts, n_list, blockIdx.x);
+  const ParamDev pd = params[list[slot]];
+  const uint32_t chunk = blockIdx.x - starts[slot];
+  const float step = lr * pd.upd_scale;
+  if (pd.gdtype == 0) {
+    if (pd.wdtype == 0) plain_block<float, float>(pd, chunk, M, beta, lambda, step, bits, vote_words, words_per_worker);
+    else plain_block<float, bf16>(pd, chunk, M, beta, lambda, step, bits, vote_words, words_per_worker);
+  } else {
+    if (pd.wdtype == 0) plain_block<bf16, float>(pd, chunk, M, beta, lambda, step, bits, vote_words, words_per_worker);
+    else plain_block<bf16, bf16>(pd, chunk, M, beta, lambda, step, bits, vote_words, words_per_worker);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stand-alone sign + pack (Alg. 3 "PackBits") for matrix parameters whose rows do not hold whole
+// payload words (cols % 32 != 0), and for K = 0.  Source: bf16 Y_K [M][rows][ldy], or for K = 0
+// the float32 momentum itself.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) pack_kernel(const ParamDev* __restrict__ params,
+                                                          const int32_t* __restrict__ list,
+                                                          const uint32_t* __restrict__ starts, int n_list,
+                                                          int src_buf, int from_momentum,
+                                                          uint32_t* __restrict__ bits, int64_t words_per_worker) {
+  const int slot = find_slot(starts, n_list, blockIdx.x);
+  const ParamDev pd = params[list[slot]];
+  const uint32_t local = blockIdx.x - starts[slot];
+  const uint32_t cpw = (uint32_t)((pd.d + PACK_CHUNK - 1) / PACK_CHUNK);
+  const int m = local / cpw;
+  const uint32_t chunk = local - m * cpw;
+  const int lane = threadIdx.x & 31;
+  const bf16* y = (src_buf ? pd.y1 : pd.y0) + (int64_t)m * pd.rows * pd.ldy;
+  const float* mom = pd.mom + (int64_t)m * pd.d;
+  const int64_t base = (int64_t)chunk * PACK_CHUNK;
+#pragma unroll 4
+  for (int it = 0; it < PACK_CHUNK / EW_THREADS; ++it) {
+    const int64_t i = base + (int64_t)it * EW_THREADS + threadIdx.x;
+    bool b = false;
+    if (i < pd.d) {
+      if (from_momentum) {
+        b = mom[i] >= 0.f;
+      } else {
+        const int64_t r = i / pd.cols;
+        const int64_t c = i - r * pd.cols;
+        b = __bfloat162float(y[r * pd.ldy + c]) >= 0.f;
+      }
+    }
+    const uint32_t word = __ballot_sync(0xffffffffu, b);
+    const int64_t wi = i >> 5;
+    if (lane == 0 && wi < pd.n_words) bits[(int64_t)m * words_per_worker + pd.word_off + wi] = word;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Majority vote from the packed words (App. B: c = sum_m b^(m), S = sign(2c - M), ties -> +1) and
+// the weight update W <- W - eta S (Alg. 3), or, for the local polar step, S as a bf16 +-1 matrix.
+// Lane t of a warp loads word (base + t) of every worker (coalesced rows) and keeps the 32
+// per-position counts as bit-sliced counter planes; the comparison c >= ceil(M/2) is the carry
+// out of a bit-sliced addition of 2^PLANES - ceil(M/2).  The vote words are then exchanged by
+// shuffle so that lane l updates entry 32 k + l of word k: coalesced weight traffic.
+// ---------------------------------------------------------------------------------------------
+template <int PLANES>
+__device__ __forceinline__ uint32_t vote_word(const uint32_t* __restrict__ bits, int64_t words_per_worker,
+                                              int64_t word_index, int M) {
+  uint32_t c[PLANES];
+#pragma unroll
+  for (int b = 0; b < PLANES; ++b) c[b] = 0;
+  for (int m = 0; m < M; ++m) {
+    uint32_t carry = __ldcs(bits + (int64_t)m * words_per_worker + word_index);
+#pragma unroll
+    for (int b = 0; b < PLANES; ++b) {
+      const uint32_t t = c[b] & carry;
+      c[b] ^= carry;
+      carry = t;
+    }
+  }
+  const uint32_t add = (1u << PLANES) - (uint32_t)((M + 1) >> 1);
+  uint32_t carry = 0;
+#pragma unroll
+  for (int b = 0; b < PLANES; ++b) {
+    const uint32_t kb = ((add >> b) & 1u) ? 0xffffffffu : 0u;
+    carry = (c[b] & kb) | (carry & (c[b] ^ kb));
+  }
+  return carry;   // bit set <=> count >= ceil(M/2) <=> 2c - M >= 0
+}
+
+template <int PLANES, typename WT>
+__device__ __forceinline__ void vote_block(const ParamDev& pd, uint32_t chunk, int M, float step, int write_sbar,
+                                           const uint32_t* __restrict__ bits, uint32_t* __restrict__ vote_words,
+                                           int64_t words_per_worker) {
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int64_t wbase = (int64_t)chunk * VOTE_WORDS + warp * 32;
+  if (wbase >= pd.n_words) return;
+  const int64_t my_word = wbase + lane;
+  uint32_t v = 0;
+  if (my_word < pd.n_words) {
+    v = vote_word<PLANES>(bits, words_per_worker, pd.word_off + my_word, M);
+    vote_words[pd.word_off + my_word] = v;
+  }
+  WT* w = reinterpret_cast<WT*>(pd.W);
+  bf16* sbar = pd.y0 + (int64_t)M * pd.rows * pd.ldy;   // slot M of operand buffer 0: input of the local polar step
+#pragma unroll 4
+  for (int k = 0; k < 32; ++k) {
+    const uint32_t vk = __shfl_sync(0xffffffffu, v, k);
+    const int64_t i = (wbase + k) * 32 + lane;
+    if (i < pd.d) {
+      const bool plus = (vk >> lane) & 1u;
+      if (write_sbar) {
+        int64_t o = i;
+        if (pd.ldy != pd.cols) {
+          const int64_t r = i / pd.cols;
+          o = r * pd.ldy + (i - r * pd.cols);
+        }
+        sbar[o] = __float2bfloat16_rn(plus ? 1.f : -1.f);
+      } else {
+        const float nw = load_as_float<WT>(w + i) - (plus ? step : -step);
+        if (sizeof(WT) == 4) reinterpret_cast<float*>(w)[i] = nw;
+        else reinterpret_cast<bf16*>(w)[i] = __float2bfloat16_rn(nw);
+      }
+    }
+  }
+}
+
+template <int PLANES>
+__global__ void __launch_bounds__(EW_THREADS) vote_update_kernel(const ParamDev* __restrict__ params,
+                                                                 const int32_t* __restrict__ list,
+                                                                 const uint32_t* __restrict__ starts, int n_list,
+                                                                 int M, float lr, int write_sbar,
+                                                                 const uint32_t* __restrict__ bits,
+                                                                 uint32_t* __restrict__ vote_words,
+                                                                 int64_t words_per_worker) {
+  const int slot = find_slot(starts, n_list, blockIdx.x);
+  const ParamDev pd = params[list[slot]];
+  const uint32_t chunk = blockIdx.x - starts[slot];
+  const float step = lr * pd.upd_scale;
+  if (pd.wdtype == 0) vote_block<PLANES, float>(pd, chunk, M, step, write_sbar, bits, vote_words, words_per_worker);
+  else vote_block<PLANES, bf16>(pd, chunk, M, step, write_sbar, bits, vote_words, words_per_worker);
+}
+
+}  // namespace signmuon

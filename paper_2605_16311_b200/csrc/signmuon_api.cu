@@ -1,0 +1,830 @@
+// Host side of the SignMuon C ABI: validation, memory layout, tile scheduling and the
+// launch sequence of one optimizer step.  See include/signmuon.h for the contract.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <queue>
+#include <vector>
+
+#include "../../include/signmuon.h"
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "ns_gemm_simt.cuh"
+#include "ns_gemm_sm100.cuh"
+
+using namespace signmuon;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+constexpr int MAX_CTAS = 1024;
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct ParamPlan {
+  int64_t rows, cols, d;
+  int32_t kind, wdtype, gdtype;
+  int64_t s, l;
+  bool wide;             // rows <= cols: Gram matrix is Y Y^T (rows x rows)
+  int32_t ldy, ldq;
+  uint32_t n_words, word_off;
+  uint32_t chunks_per_worker;
+  bool fused_pack;       // sign+pack happens in the last apply epilogue
+  size_t mom_off;        // bytes into the state buffer
+  size_t y_off[2], lo_off, q_off, scales_off, partials_off;   // bytes into the workspace (matrix params)
+  int tmap_base;         // first of this parameter's 8 tensor maps
+  size_t stage_w_off, stage_g_off;                    // bytes into the host-staging buffer
+};
+
+// indices of a parameter's tensor maps relative to tmap_base
+enum { TM_Y0_K128 = 0, TM_Y0_KBN, TM_Y0_MN, TM_Y1_K128, TM_Y1_KBN, TM_Y1_MN, TM_Q_K128, TM_Q_KBN, TM_PER_PARAM };
+
+struct LaunchPlan {        // one grouped GEMM launch
+  size_t problem_base;     // index of its first problem in the problem array
+  int tile_table;          // which tile table (0 gram, 1 apply, 2 gram local-polar, 3 apply local-polar)
+};
+
+struct TileTable {
+  std::vector<TileEntry> tiles;         // ordered by CTA
+  std::vector<uint32_t> cta_start;      // [grid + 1]
+  int grid = 0;
+  int bn = 128;
+  size_t tiles_off = 0, cta_off = 0;    // bytes into the workspace
+};
+
+}  // namespace
+
+struct signmuon_ctx {
+  signmuon_config cfg;
+  std::vector<signmuon_param> params;
+  std::vector<ParamPlan> plan;
+  std::vector<int32_t> matrix_list, plain_list, packfb_list;
+  std::vector<uint32_t> mom_starts, plain_starts, vote_starts, packfb_starts;
+  uint32_t mom_blocks = 0, plain_blocks = 0, vote_blocks = 0, packfb_blocks = 0;
+  uint64_t words_per_worker = 0;
+  int64_t entries = 0;
+  size_t state_bytes = 0, workspace_bytes = 0, staging_bytes = 0;
+  // workspace offsets
+  size_t off_status = 0, off_paramdev = 0, off_lists = 0, off_bits = 0, off_vote = 0, off_tmaps = 0,
+         off_problems = 0, off_tables_end = 0;
+  size_t off_list_matrix = 0, off_list_plain = 0, off_list_packfb = 0, off_starts_mom = 0, off_starts_plain = 0,
+         off_starts_vote = 0, off_starts_packfb = 0;
+  // GEMM plans
+  std::vector<GemmProblem> problems;      // pointers filled at bind
+  std::vector<LaunchPlan> ns_launches, lp_launches;
+  TileTable tables[4];
+  int num_tmaps = 0;
+  // binding
+  bool bound = false;
+  uint8_t* d_state = nullptr;
+  uint8_t* d_ws = nullptr;
+  uint8_t* d_staging = nullptr;
+  int num_sms = 0;
+  std::vector<ParamDev> paramdev;         // host copy of the device table
+  bool paramdev_uploaded = false;
+  int sticky = SIGNMUON_OK;
+};
+
+namespace {
+
+bool valid_dtype(int32_t t) { return t == SIGNMUON_F32 || t == SIGNMUON_BF16; }
+size_t dtype_size(int32_t t) { return t == SIGNMUON_F32 ? 4 : 2; }
+
+// ------------------------------------------------------------------ tile scheduling (host)
+// Longest-processing-time-first assignment of tiles to `grid` persistent CTAs; cost = K blocks
+// of the main loop plus a constant for the epilogue.
+void build_tile_table(TileTable& tt, const std::vector<GemmProblem>& probs, size_t pbase, size_t pcount, int bn,
+                      int grid_limit) {
+  struct T { TileEntry e; int cost; };
+  std::vector<T> all;
+  for (size_t i = 0; i < pcount; ++i) {
+    const GemmProblem& pr = probs[pbase + i];
+    const int tm = (pr.M + GEMM_BM - 1) / GEMM_BM, tn = (pr.N + bn - 1) / bn;
+    const int cost = (pr.K + GEMM_BK - 1) / GEMM_BK + 2;
+    for (int a = 0; a < tm; ++a)
+      for (int b = 0; b < tn; ++b) all.push_back({{(uint32_t)i, (uint16_t)a, (uint16_t)b}, cost});
+  }
+  tt.bn = bn;
+  tt.grid = (int)std::min<size_t>((size_t)grid_limit, std::max<size_t>(all.size(), 1));
+  std::stable_sort(all.begin(), all.end(), [](const T& x, const T& y) { return x.cost > y.cost; });
+  std::vector<std::vector<TileEntry>> per(tt.grid);
+  typedef std::pair<long long, int> Load;   // (load, cta)
+  std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+  for (int c = 0; c < tt.grid; ++c) heap.push({0, c});
+  for (const T& t : all) {
+    Load top = heap.top();
+    heap.pop();
+    per[top.second].push_back(t.e);
+    heap.push({top.first + t.cost, top.second});
+  }
+  tt.tiles.clear();
+  tt.cta_start.assign(tt.grid + 1, 0);
+  for (int c = 0; c < tt.grid; ++c) {
+    tt.cta_start[c] = (uint32_t)tt.tiles.size();
+    tt.tiles.insert(tt.tiles.end(), per[c].begin(), per[c].end());
+  }
+  tt.cta_start[tt.grid] = (uint32_t)tt.tiles.size();
+}
+
+size_t count_tiles(const std::vector<GemmProblem>& probs, size_t pbase, size_t pcount, int bn) {
+  size_t n = 0;
+  for (size_t i = 0; i < pcount; ++i) {
+    const GemmProblem& pr = probs[pbase + i];
+    n += (size_t)((pr.M + GEMM_BM - 1) / GEMM_BM) * ((pr.N + bn - 1) / bn);
+  }
+  return n;
+}
+
+// ------------------------------------------------------------------ GEMM problem construction
+// Builds the problem list of the Gram (`gram` = true) or apply product of Newton-Schulz
+// iteration k for `workers` batch slots.  Device pointers are left as byte offsets into the
+// workspace (resolved at bind) in the pointer fields.
+void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, int k, int K, int workers,
+                     bool local_polar_phase) {
+  const bool keep = (c->cfg.flags & SIGNMUON_FLAG_KEEP_POLAR) != 0;
+  for (int32_t p : c->matrix_list) {
+    const ParamPlan& pl = c->plan[p];
+    const int src = k & 1, dst = (k + 1) & 1;
+    for (int w = 0; w < workers; ++w) {
+      // the local polar step works in its own slot (index M) so the workers' results stay readable
+      const int m = local_polar_phase ? c->cfg.num_workers : w;
+      GemmProblem pr;
+      std::memset(&pr, 0, sizeof(pr));
+      const size_t ybytes = (size_t)pl.rows * pl.ldy * 2, qbytes = (size_t)pl.s * pl.ldq * 2;
+      const size_t ysrc = pl.y_off[src] + m * ybytes, ydst = pl.y_off[dst] + m * ybytes;
+      const size_t q = pl.q_off + m * qbytes;
+      pr.batch = m;
+      pr.param = p;
+      const int ty = src ? TM_Y1_K128 : TM_Y0_K128;   // first map of the source buffer
+      if (gram) {
+        pr.M = pr.N = (int32_t)pl.s;
+        pr.K = (int32_t)pl.l;
+        pr.A = pr.B = reinterpret_cast<const bf16*>(ysrc);
+        if (pl.wide) {
+          pr.a_sm = pr.b_sn = pl.ldy; pr.a_sk = pr.b_sk = 1;
+          pr.tmapA = pl.tmap_base + ty; pr.tmapB = pl.tmap_base + ty + 1;
+        } else {
+          pr.a_sm = pr.b_sn = 1; pr.a_sk = pr.b_sk = pl.ldy; pr.a_mn = pr.b_mn = 1;
+          pr.tmapA = pr.tmapB = pl.tmap_base + ty + 2;
+        }
+        pr.epi = EPI_GRAM;
+        pr.out = reinterpret_cast<void*>(q);
+        pr.ld_out = pl.ldq;
+        if (k == 0) {
+          if (local_polar_phase) pr.scale_imm = (float)(1.0 / ((double)pl.rows * (double)pl.cols));
+          else pr.scale_ptr = reinterpret_cast<const float*>(pl.scales_off + (size_t)m * 8);
+        } else {
+          pr.scale_imm = 1.f;
+        }
+      } else {
+        pr.M = (int32_t)pl.rows; pr.N = (int32_t)pl.cols; pr.K = (int32_t)pl.s;
+        if (pl.wide) {                      // Y' = (3/2 I - A/2) Y : A operand Q, B operand Y (contiguous along N)
+          pr.A = reinterpret_cast<const bf16*>(q); pr.a_sm = pl.ldq; pr.a_sk = 1;
+          pr.B = reinterpret_cast<const bf16*>(ysrc); pr.b_sn = 1; pr.b_sk = pl.ldy; pr.b_mn = 1;
+          pr.tmapA = pl.tmap_base + TM_Q_K128; pr.tmapB = pl.tmap_base + ty + 2;
+        } else {                            // Y' = Y (3/2 I - A/2) : A operand Y, B operand Q (symmetric)
+          pr.A = reinterpret_cast<const bf16*>(ysrc); pr.a_sm = pl.ldy; pr.a_sk = 1;
+          pr.B = reinterpret_cast<const bf16*>(q); pr.b_sn = pl.ldq; pr.b_sk = 1;
+          pr.tmapA = pl.tmap_base + ty; pr.tmapB = pl.tmap_base + TM_Q_KBN;
+        }
+        const size_t lo = pl.lo_off + m * ybytes;
+        if (k == 0 && !local_polar_phase) {          // own term from the float32 momentum itself
+          pr.c_mode = C_F32;
+          pr.C = reinterpret_cast<const void*>(pl.mom_off + (size_t)m * pl.d * 4);   // offset into the state buffer
+          pr.ldc = pl.cols;
+        } else {
+          pr.c_mode = (k == 0) ? C_BF16 : C_HILO;    // the +-1 vote matrix is exact in bf16
+          pr.C = reinterpret_cast<const void*>(ysrc);
+          pr.C_lo = (k == 0) ? nullptr : reinterpret_cast<const bf16*>(lo);
+          pr.ldc = pl.ldy;
+        }
+        pr.out = reinterpret_cast<void*>(ydst);
+        pr.out_lo = reinterpret_cast<bf16*>(lo);
+        pr.ld_out = pl.ldy;
+        if (k == 0) {
+          if (local_polar_phase) pr.scale_imm = (float)(1.0 / std::sqrt((double)pl.rows * (double)pl.cols));
+          else pr.scale_ptr = reinterpret_cast<const float*>(pl.scales_off + (size_t)m * 8 + 4);
+        } else {
+          pr.scale_imm = 1.f;
+        }
+        const bool last = (k == K - 1);
+        if (!last) pr.epi = EPI_APPLY;
+        else if (local_polar_phase) pr.epi = EPI_APPLY_UPDATE;
+        else if (pl.fused_pack) {
+          pr.epi = EPI_APPLY_PACK;
+          pr.store_out = keep ? 1 : 0;
+          // payload word of this (param, worker): resolved at bind from off_bits
+          pr.bits_out = reinterpret_cast<uint32_t*>((size_t)m * c->words_per_worker * 4 + (size_t)pl.word_off * 4);
+        } else pr.epi = EPI_APPLY;
+      }
+      out.push_back(pr);
+    }
+  }
+}
+
+int plan_layout(signmuon_ctx* c) {
+  const int M = c->cfg.num_workers;
+  const int K = c->cfg.ns_steps;
+  size_t state = 0;
+  uint64_t words = 0;
+  for (size_t p = 0; p < c->params.size(); ++p) {
+    const signmuon_param& sp = c->params[p];
+    ParamPlan pl;
+    std::memset(&pl, 0, sizeof(pl));
+    pl.rows = sp.rows; pl.cols = sp.cols; pl.d = sp.rows * sp.cols;
+    pl.kind = sp.kind; pl.wdtype = sp.weight_dtype; pl.gdtype = sp.grad_dtype;
+    pl.s = std::min(sp.rows, sp.cols); pl.l = std::max(sp.rows, sp.cols);
+    pl.wide = sp.rows <= sp.cols;
+    pl.ldy = (int32_t)round_up((size_t)sp.cols, 8);
+    pl.ldq = (int32_t)round_up((size_t)pl.s, 8);
+    pl.n_words = (uint32_t)((pl.d + 31) / 32);
+    pl.word_off = (uint32_t)words;
+    words += pl.n_words;
+    pl.chunks_per_worker = (uint32_t)((pl.d + MOM_CHUNK - 1) / MOM_CHUNK);
+    pl.fused_pack = (sp.kind == SIGNMUON_PARAM_MATRIX) && K > 0 && (sp.cols % 32 == 0);
+    pl.mom_off = state;
+    state += round_up((size_t)M * pl.d * 4, ALIGN);
+    c->plan.push_back(pl);
+    if (sp.kind == SIGNMUON_PARAM_MATRIX) c->matrix_list.push_back((int32_t)p);
+    else c->plain_list.push_back((int32_t)p);
+    c->entries += pl.d;
+  }
+  if (words >= (1ull << 32)) return SIGNMUON_ERR_BAD_SHAPE;
+  c->words_per_worker = words;
+  c->state_bytes = state;
+
+  // block ranges of the element-wise kernels
+  uint64_t b = 0;
+  for (int32_t p : c->matrix_list) { c->mom_starts.push_back((uint32_t)b); b += (uint64_t)M * c->plan[p].chunks_per_worker; }
+  if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
+  c->mom_blocks = (uint32_t)b;
+  b = 0;
+  for (int32_t p : c->plain_list) { c->plain_starts.push_back((uint32_t)b); b += (uint64_t)((c->plan[p].d + PLAIN_CHUNK - 1) / PLAIN_CHUNK); }
+  if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
+  c->plain_blocks = (uint32_t)b;
+  b = 0;
+  for (int32_t p : c->matrix_list) { c->vote_starts.push_back((uint32_t)b); b += (c->plan[p].n_words + VOTE_WORDS - 1) / VOTE_WORDS; }
+  c->vote_blocks = (uint32_t)b;
+  b = 0;
+  for (int32_t p : c->matrix_list) {
+    if (c->plan[p].fused_pack) continue;
+    c->packfb_list.push_back(p);
+    c->packfb_starts.push_back((uint32_t)b);
+    b += (uint64_t)M * ((c->plan[p].d + PACK_CHUNK - 1) / PACK_CHUNK);
+  }
+  if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
+  c->packfb_blocks = (uint32_t)b;
+
+  // workspace layout: small tables first, then the large buffers
+  size_t off = 0;
+  c->off_status = off; off += ALIGN;
+  c->off_paramdev = off; off += round_up(c->params.size() * sizeof(ParamDev), ALIGN);
+  auto place = [&](size_t& slot, size_t bytes) { slot = off; off += round_up(std::max<size_t>(bytes, 4), ALIGN); };
+  place(c->off_list_matrix, c->matrix_list.size() * 4);
+  place(c->off_list_plain, c->plain_list.size() * 4);
+  place(c->off_list_packfb, c->packfb_list.size() * 4);
+  place(c->off_starts_mom, c->mom_starts.size() * 4);
+  place(c->off_starts_plain, c->plain_starts.size() * 4);
+  place(c->off_starts_vote, c->vote_starts.size() * 4);
+  place(c->off_starts_packfb, c->packfb_starts.size() * 4);
+  for (int32_t p : c->matrix_list) {
+    ParamPlan& pl = c->plan[p];
+    pl.scales_off = off; off += round_up((size_t)M * 8, ALIGN);
+    pl.partials_off = off; off += round_up((size_t)M * pl.chunks_per_worker * 4, ALIGN);
+  }
+  c->off_bits = off; off += round_up((size_t)M * words * 4, ALIGN);
+  c->off_vote = off; off += round_up((size_t)words * 4, ALIGN);
+  // tensor maps
+  c->off_tmaps = off;
+  int nt = 0;
+  for (int32_t p : c->matrix_list) { c->plan[p].tmap_base = nt; nt += TM_PER_PARAM; }
+  c->num_tmaps = nt;
+  off += round_up((size_t)std::max(nt, 1) * sizeof(CUtensorMap), ALIGN);
+  // Newton-Schulz operand buffers
+  for (int32_t p : c->matrix_list) {
+    ParamPlan& pl = c->plan[p];
+    const size_t slots = (size_t)M + (c->cfg.local_polar ? 1 : 0);
+    const size_t ybytes = round_up(slots * pl.rows * pl.ldy * 2, 1024);
+    pl.y_off[0] = off; off += ybytes;
+    pl.y_off[1] = off; off += ybytes;
+    pl.lo_off = off; off += ybytes;
+    pl.q_off = off; off += round_up(slots * pl.s * pl.ldq * 2, 1024);
+  }
+  // GEMM problems: K x (gram, apply) for the workers, and again for the local polar step
+  c->problems.clear();
+  c->ns_launches.clear();
+  c->lp_launches.clear();
+  if (!c->matrix_list.empty()) {
+    for (int k = 0; k < K; ++k) {
+      c->ns_launches.push_back({c->problems.size(), 0});
+      append_problems(c, c->problems, true, k, K, M, false);
+      c->ns_launches.push_back({c->problems.size(), 1});
+      append_problems(c, c->problems, false, k, K, M, false);
+    }
+    if (c->cfg.local_polar) {
+      for (int k = 0; k < K; ++k) {
+        c->lp_launches.push_back({c->problems.size(), 2});
+        append_problems(c, c->problems, true, k, K, 1, true);
+        c->lp_launches.push_back({c->problems.size(), 3});
+        append_problems(c, c->problems, false, k, K, 1, true);
+      }
+    }
+  }
+  c->off_problems = off; off += round_up(c->problems.size() * sizeof(GemmProblem), ALIGN);
+  // tile tables (sizes do not depend on the SM count; the CTA split is made at bind)
+  const size_t nm = c->matrix_list.size();
+  for (int t = 0; t < 4; ++t) {
+    TileTable& tt = c->tables[t];
+    tt.bn = 128;
+    size_t ntiles = 0;
+    const std::vector<LaunchPlan>& ls = (t < 2) ? c->ns_launches : c->lp_launches;
+    const size_t per = (t < 2) ? nm * M : nm;
+    if (!ls.empty()) ntiles = count_tiles(c->problems, ls[t & 1].problem_base, per, tt.bn);
+    tt.tiles_off = off; off += round_up(std::max<size_t>(ntiles, 1) * sizeof(TileEntry), ALIGN);
+    tt.cta_off = off; off += round_up((MAX_CTAS + 1) * 4, ALIGN);
+  }
+  c->off_tables_end = off;
+  c->workspace_bytes = off;
+
+  // host staging: W and G of every parameter
+  size_t st = 0;
+  for (ParamPlan& pl : c->plan) {
+    pl.stage_w_off = st; st += round_up((size_t)pl.d * dtype_size(pl.wdtype), ALIGN);
+    pl.stage_g_off = st; st += round_up((size_t)M * pl.d * dtype_size(pl.gdtype), ALIGN);
+  }
+  c->staging_bytes = st;
+  return SIGNMUON_OK;
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+  }
+  return fn;
+}
+
+// 3-D bf16 tensor {inner, rows, batch} with a {64, box_rows, 1} box and 128-byte swizzle.
+bool encode_map(CUtensorMap* map, void* base, uint64_t inner, uint64_t rows, uint64_t batch, uint64_t pitch_elems,
+                uint64_t batch_elems, uint32_t box_rows) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[3] = {inner, rows, batch};
+  cuuint64_t gstr[2] = {pitch_elems * 2, batch_elems * 2};
+  cuuint32_t box[3] = {64, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int check_launch(signmuon_ctx* c) {
+  if (cudaGetLastError() != cudaSuccess) c->sticky = SIGNMUON_ERR_CUDA;
+  return c->sticky;
+}
+
+template <int BN, int STAGES>
+void launch_tc(const GemmLaunchArgs& a, int grid, cudaStream_t s) {
+  static bool configured = false;
+  constexpr size_t smem = ns_gemm_tc_smem_bytes<BN, STAGES>();
+  if (!configured) {
+    cudaFuncSetAttribute(ns_gemm_tc_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    configured = true;
+  }
+  ns_gemm_tc_kernel<BN, STAGES><<<grid, GEMM_THREADS, smem, s>>>(a);
+}
+
+void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s) {
+  const TileTable& tt = c->tables[lp.tile_table];
+  if (tt.tiles.empty()) return;
+  const GemmProblem* probs = reinterpret_cast<const GemmProblem*>(c->d_ws + c->off_problems) + lp.problem_base;
+  const TileEntry* tiles = reinterpret_cast<const TileEntry*>(c->d_ws + tt.tiles_off);
+  const ParamDev* pd = reinterpret_cast<const ParamDev*>(c->d_ws + c->off_paramdev);
+  if (c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) {
+    ns_gemm_simt_kernel<<<(unsigned)tt.tiles.size(), 128, 0, s>>>(probs, tiles, tt.bn, pd, lr);
+    return;
+  }
+  GemmLaunchArgs a;
+  a.tmaps = reinterpret_cast<const CUtensorMap*>(c->d_ws + c->off_tmaps);
+  a.problems = probs;
+  a.tiles = tiles;
+  a.cta_tile_start = reinterpret_cast<const uint32_t*>(c->d_ws + tt.cta_off);
+  a.params = pd;
+  a.status = reinterpret_cast<uint32_t*>(c->d_ws + c->off_status);
+  a.lr = lr;
+  if (tt.bn == 256) launch_tc<256, 4>(a, tt.grid, s);
+  else launch_tc<128, 6>(a, tt.grid, s);
+}
+
+template <int PLANES>
+void launch_vote(signmuon_ctx* c, float lr, int write_sbar, cudaStream_t s) {
+  vote_update_kernel<PLANES><<<c->vote_blocks, EW_THREADS, 0, s>>>(
+      reinterpret_cast<const ParamDev*>(c->d_ws + c->off_paramdev),
+      reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_matrix),
+      reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_vote), (int)c->matrix_list.size(),
+      c->cfg.num_workers, lr, write_sbar, reinterpret_cast<const uint32_t*>(c->d_ws + c->off_bits),
+      reinterpret_cast<uint32_t*>(c->d_ws + c->off_vote), (int64_t)c->words_per_worker);
+}
+
+int upload_params(signmuon_ctx* c, void* const* weights, const void* const* grads, cudaStream_t s) {
+  bool changed = !c->paramdev_uploaded;
+  for (size_t p = 0; p < c->params.size(); ++p) {
+    if (!weights[p] || !grads[p]) return SIGNMUON_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(weights[p]) & 15) || (reinterpret_cast<uintptr_t>(grads[p]) & 15))
+      return SIGNMUON_ERR_MISALIGNED;
+    if (c->paramdev[p].W != weights[p] || c->paramdev[p].G != grads[p]) {
+      c->paramdev[p].W = weights[p];
+      c->paramdev[p].G = grads[p];
+      changed = true;
+    }
+  }
+  if (changed) {
+    // pageable source: the runtime stages it before returning, so the host copy may change afterwards
+    if (cudaMemcpyAsync(c->d_ws + c->off_paramdev, c->paramdev.data(), c->paramdev.size() * sizeof(ParamDev),
+                        cudaMemcpyHostToDevice, s) != cudaSuccess) {
+      c->sticky = SIGNMUON_ERR_CUDA;
+      return c->sticky;
+    }
+    c->paramdev_uploaded = true;
+  }
+  return SIGNMUON_OK;
+}
+
+int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const void* const* grads, float lr,
+                    cudaStream_t s) {
+  if (!c) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  if (c->sticky != SIGNMUON_OK) return c->sticky;
+  if (!weights || !grads) return SIGNMUON_ERR_INVALID_ARG;
+  if (lr < 0.f) lr = c->cfg.lr;
+  int rc = upload_params(c, weights, grads, s);
+  if (rc != SIGNMUON_OK) return rc;
+  const int M = c->cfg.num_workers, K = c->cfg.ns_steps;
+  const ParamDev* pd = reinterpret_cast<const ParamDev*>(c->d_ws + c->off_paramdev);
+  uint32_t* bits = reinterpret_cast<uint32_t*>(c->d_ws + c->off_bits);
+  uint32_t* vote = reinterpret_cast<uint32_t*>(c->d_ws + c->off_vote);
+  const int nm = (int)c->matrix_list.size(), np = (int)c->plain_list.size();
+  const float eps = c->cfg.eps;
+
+  if (mask & SIGNMUON_STAGE_MOMENTUM) {
+    if (nm) {
+      momentum_kernel<<<c->mom_blocks, EW_THREADS, 0, s>>>(
+          pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_matrix),
+          reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_mom), nm, c->cfg.momentum, c->cfg.weight_decay);
+      const int warps = nm * M;
+      finalize_norms_kernel<<<(warps * 32 + 255) / 256, 256, 0, s>>>(
+          pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_matrix), nm, M, eps);
+    }
+    if (np) {
+      plain_params_kernel<<<c->plain_blocks, EW_THREADS, 0, s>>>(
+          pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_plain),
+          reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_plain), np, M, c->cfg.momentum,
+          c->cfg.weight_decay, lr, bits, vote, (int64_t)c->words_per_worker);
+    }
+  }
+  if ((mask & SIGNMUON_STAGE_NS) && nm) {
+    for (const LaunchPlan& lp : c->ns_launches) launch_gemm(c, lp, lr, s);
+    if (c->packfb_blocks) {
+      pack_kernel<<<c->packfb_blocks, EW_THREADS, 0, s>>>(
+          pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_packfb),
+          reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_packfb), (int)c->packfb_list.size(), K & 1,
+          K == 0 ? 1 : 0, bits, (int64_t)c->words_per_worker);
+    }
+  }
+  const bool lp_ns = c->cfg.local_polar && K > 0;
+  if ((mask & SIGNMUON_STAGE_VOTE) && nm) {
+    // local polar with K = 0 degenerates to S / ||S||_F: plain update with the Eq. 2 scale
+    const int write_sbar = lp_ns ? 1 : 0;
+    if (M <= 7) launch_vote<3>(c, lr, write_sbar, s);
+    else if (M <= 63) launch_vote<6>(c, lr, write_sbar, s);
+    else launch_vote<8>(c, lr, write_sbar, s);
+  }
+  if ((mask & SIGNMUON_STAGE_LOCAL_POLAR) && nm && lp_ns) {
+    for (const LaunchPlan& lp : c->lp_launches) launch_gemm(c, lp, lr, s);
+  }
+  return check_launch(c);
+}
+
+}  // namespace
+
+// =============================================================================== C ABI
+extern "C" {
+
+int signmuon_create(const signmuon_config* config, signmuon_ctx** out) {
+  if (!out) return SIGNMUON_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config || config->num_params < 1 || !config->params) return SIGNMUON_ERR_INVALID_ARG;
+  if (config->num_workers < 1 || config->num_workers > 255) return SIGNMUON_ERR_INVALID_ARG;
+  if (!(config->momentum >= 0.f && config->momentum < 1.f)) return SIGNMUON_ERR_INVALID_ARG;
+  if (config->ns_steps < 0 || config->ns_steps > 64) return SIGNMUON_ERR_INVALID_ARG;
+  if (!(config->weight_decay >= 0.f)) return SIGNMUON_ERR_INVALID_ARG;
+  if (!(config->lr == config->lr)) return SIGNMUON_ERR_INVALID_ARG;
+  if (config->update_scale != 0 && config->update_scale != 1) return SIGNMUON_ERR_INVALID_ARG;
+  if (config->local_polar != 0 && config->local_polar != 1) return SIGNMUON_ERR_INVALID_ARG;
+  for (int i = 0; i < config->num_params; ++i) {
+    const signmuon_param& p = config->params[i];
+    if (p.rows < 1 || p.cols < 1 || p.rows > (1 << 24) || p.cols > (1 << 24)) return SIGNMUON_ERR_BAD_SHAPE;
+    if (p.kind != SIGNMUON_PARAM_MATRIX && p.kind != SIGNMUON_PARAM_PLAIN) return SIGNMUON_ERR_INVALID_ARG;
+    if (!valid_dtype(p.weight_dtype) || !valid_dtype(p.grad_dtype)) return SIGNMUON_ERR_INVALID_ARG;
+    if (p.kind == SIGNMUON_PARAM_MATRIX && std::min(p.rows, p.cols) > 65536 * 2) return SIGNMUON_ERR_BAD_SHAPE;
+    if (p.rows * p.cols > (1ll << 36)) return SIGNMUON_ERR_BAD_SHAPE;
+  }
+  signmuon_ctx* c = new (std::nothrow) signmuon_ctx();
+  if (!c) return SIGNMUON_ERR_INVALID_ARG;
+  c->cfg = *config;
+  if (!(c->cfg.eps > 0.f)) c->cfg.eps = 1e-12f;
+  c->params.assign(config->params, config->params + config->num_params);
+  c->cfg.params = nullptr;
+  int rc = plan_layout(c);
+  if (rc != SIGNMUON_OK) { delete c; return rc; }
+  *out = c;
+  return SIGNMUON_OK;
+}
+
+int signmuon_state_bytes(const signmuon_ctx* c, size_t* state, size_t* workspace, size_t* host_staging) {
+  if (!c) return SIGNMUON_ERR_INVALID_ARG;
+  if (state) *state = c->state_bytes;
+  if (workspace) *workspace = c->workspace_bytes;
+  if (host_staging) *host_staging = c->staging_bytes;
+  return SIGNMUON_OK;
+}
+
+int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* dev_workspace, size_t workspace_bytes,
+                  void* dev_staging, size_t staging_bytes, int zero_state, void* cuda_stream) {
+  if (!c || !dev_state || !dev_workspace) return SIGNMUON_ERR_INVALID_ARG;
+  if (state_bytes < c->state_bytes || workspace_bytes < c->workspace_bytes) return SIGNMUON_ERR_BUFFER_TOO_SMALL;
+  if (dev_staging && staging_bytes < c->staging_bytes) return SIGNMUON_ERR_BUFFER_TOO_SMALL;
+  if ((reinterpret_cast<uintptr_t>(dev_state) & 255) || (reinterpret_cast<uintptr_t>(dev_workspace) & 1023) ||
+      (reinterpret_cast<uintptr_t>(dev_staging) & 255))
+    return SIGNMUON_ERR_MISALIGNED;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  int dev = 0, major = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SIGNMUON_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SIGNMUON_ERR_CUDA;
+  if (major != 10) return SIGNMUON_ERR_UNSUPPORTED_ARCH;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  c->num_sms = std::max(1, std::min(sms, MAX_CTAS));
+  c->d_state = static_cast<uint8_t*>(dev_state);
+  c->d_ws = static_cast<uint8_t*>(dev_workspace);
+  c->d_staging = static_cast<uint8_t*>(dev_staging);
+  const int M = c->cfg.num_workers;
+
+  // host image of the table area [0, off_tables_end) minus the big buffers: assemble piecewise
+  auto up = [&](size_t off, const void* src, size_t bytes) -> bool {
+    if (bytes == 0) return true;
+    return cudaMemcpyAsync(c->d_ws + off, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  };
+  bool ok = cudaMemsetAsync(c->d_ws + c->off_status, 0, ALIGN, s) == cudaSuccess;
+  if (zero_state) ok = ok && cudaMemsetAsync(c->d_state, 0, c->state_bytes, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->d_ws + c->off_bits, 0, (size_t)M * c->words_per_worker * 4, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->d_ws + c->off_vote, 0, (size_t)c->words_per_worker * 4, s) == cudaSuccess;
+
+  // parameter table (W/G filled in at the first step)
+  c->paramdev.assign(c->params.size(), ParamDev());
+  for (size_t p = 0; p < c->params.size(); ++p) {
+    const ParamPlan& pl = c->plan[p];
+    ParamDev& d = c->paramdev[p];
+    std::memset(&d, 0, sizeof(d));
+    d.mom = reinterpret_cast<float*>(c->d_state + pl.mom_off);
+    if (pl.kind == SIGNMUON_PARAM_MATRIX) {
+      d.y0 = reinterpret_cast<bf16*>(c->d_ws + pl.y_off[0]);
+      d.y1 = reinterpret_cast<bf16*>(c->d_ws + pl.y_off[1]);
+      d.scales = reinterpret_cast<float*>(c->d_ws + pl.scales_off);
+      d.partials = reinterpret_cast<float*>(c->d_ws + pl.partials_off);
+    }
+    d.d = pl.d; d.rows = (int32_t)pl.rows; d.cols = (int32_t)pl.cols; d.ldy = pl.ldy;
+    d.kind = pl.kind; d.wdtype = pl.wdtype; d.gdtype = pl.gdtype;
+    d.word_off = pl.word_off; d.n_words = pl.n_words; d.chunks_per_worker = pl.chunks_per_worker;
+    const bool eq2 = c->cfg.update_scale == 1 ||
+                     (pl.kind == SIGNMUON_PARAM_MATRIX && c->cfg.local_polar && c->cfg.ns_steps == 0);
+    d.upd_scale = eq2 ? (float)(1.0 / std::sqrt((double)pl.rows * (double)pl.cols)) : 1.f;
+    d.vec_ok = (pl.d % 8 == 0 && pl.ldy == pl.cols) ? 1 : 0;
+  }
+  c->paramdev_uploaded = false;
+  ok = ok && up(c->off_list_matrix, c->matrix_list.data(), c->matrix_list.size() * 4);
+  ok = ok && up(c->off_list_plain, c->plain_list.data(), c->plain_list.size() * 4);
+  ok = ok && up(c->off_list_packfb, c->packfb_list.data(), c->packfb_list.size() * 4);
+  ok = ok && up(c->off_starts_mom, c->mom_starts.data(), c->mom_starts.size() * 4);
+  ok = ok && up(c->off_starts_plain, c->plain_starts.data(), c->plain_starts.size() * 4);
+  ok = ok && up(c->off_starts_vote, c->vote_starts.data(), c->vote_starts.size() * 4);
+  ok = ok && up(c->off_starts_packfb, c->packfb_starts.data(), c->packfb_starts.size() * 4);
+  if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+
+  // tile tables (need the SM count) and tensor maps (need the device addresses)
+  const size_t nm = c->matrix_list.size();
+  for (int t = 0; t < 4; ++t) {
+    TileTable& tt = c->tables[t];
+    const std::vector<LaunchPlan>& ls = (t < 2) ? c->ns_launches : c->lp_launches;
+    tt.tiles.clear();
+    if (ls.empty()) continue;
+    build_tile_table(tt, c->problems, ls[t & 1].problem_base, (t < 2) ? nm * M : nm, tt.bn, c->num_sms);
+    ok = ok && up(tt.tiles_off, tt.tiles.data(), tt.tiles.size() * sizeof(TileEntry));
+    ok = ok && up(tt.cta_off, tt.cta_start.data(), tt.cta_start.size() * 4);
+  }
+  std::vector<CUtensorMap> maps((size_t)c->num_tmaps);
+  const bool need_maps = !(c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) && c->cfg.ns_steps > 0;
+  if (need_maps) {
+    for (int32_t p : c->matrix_list) {
+      const ParamPlan& pl = c->plan[p];
+      CUtensorMap* mp = maps.data() + pl.tmap_base;
+      const uint32_t bn = 128;   // box rows of a K-major B operand = tile width
+      const uint64_t slots = (uint64_t)M + (c->cfg.local_polar ? 1 : 0);
+      for (int buf = 0; buf < 2; ++buf) {
+        void* y = c->d_ws + pl.y_off[buf];
+        const uint64_t yb = (uint64_t)pl.rows * pl.ldy;
+        ok = ok && encode_map(mp + buf * 3 + 0, y, pl.cols, pl.rows, slots, pl.ldy, yb, 128);
+        ok = ok && encode_map(mp + buf * 3 + 1, y, pl.cols, pl.rows, slots, pl.ldy, yb, bn);
+        ok = ok && encode_map(mp + buf * 3 + 2, y, pl.cols, pl.rows, slots, pl.ldy, yb, 64);
+      }
+      void* q = c->d_ws + pl.q_off;
+      const uint64_t qb = (uint64_t)pl.s * pl.ldq;
+      ok = ok && encode_map(mp + TM_Q_K128, q, pl.s, pl.s, slots, pl.ldq, qb, 128);
+      ok = ok && encode_map(mp + TM_Q_KBN, q, pl.s, pl.s, slots, pl.ldq, qb, bn);
+    }
+    if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+    ok = ok && up(c->off_tmaps, maps.data(), maps.size() * sizeof(CUtensorMap));
+  }
+  // resolve workspace-relative pointers of the problems
+  std::vector<GemmProblem> probs = c->problems;
+  for (GemmProblem& pr : probs) {
+    pr.A = reinterpret_cast<const bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.A));
+    pr.B = reinterpret_cast<const bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.B));
+    pr.out = c->d_ws + reinterpret_cast<size_t>(pr.out);
+    if (pr.epi != EPI_GRAM) {
+      uint8_t* cbase = (pr.c_mode == C_F32) ? c->d_state : c->d_ws;
+      pr.C = cbase + reinterpret_cast<size_t>(pr.C);
+      if (pr.C_lo) pr.C_lo = reinterpret_cast<const bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.C_lo));
+      pr.out_lo = reinterpret_cast<bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.out_lo));
+    }
+    if (pr.scale_ptr) pr.scale_ptr = reinterpret_cast<const float*>(c->d_ws + reinterpret_cast<size_t>(pr.scale_ptr));
+    if (pr.epi == EPI_APPLY_PACK)
+      pr.bits_out = reinterpret_cast<uint32_t*>(c->d_ws + c->off_bits + reinterpret_cast<size_t>(pr.bits_out));
+  }
+  ok = ok && up(c->off_problems, probs.data(), probs.size() * sizeof(GemmProblem));
+  // the uploads above read host vectors that die with this call: make sure they are consumed
+  ok = ok && cudaStreamSynchronize(s) == cudaSuccess;
+  if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+  c->bound = true;
+  c->sticky = SIGNMUON_OK;
+  return SIGNMUON_OK;
+}
+
+int signmuon_step(signmuon_ctx* c, void* const* weights, const void* const* grads, float lr, void* cuda_stream) {
+  return run_stages_impl(c, SIGNMUON_STAGE_ALL, weights, grads, lr, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int signmuon_run_stages(signmuon_ctx* c, int32_t stage_mask, void* const* weights, const void* const* grads, float lr,
+                        void* cuda_stream) {
+  if (stage_mask & ~SIGNMUON_STAGE_ALL) return SIGNMUON_ERR_INVALID_ARG;
+  return run_stages_impl(c, stage_mask, weights, grads, lr, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int signmuon_step_host(signmuon_ctx* c, void* const* host_weights, const void* const* host_grads, float lr,
+                       void* cuda_stream) {
+  if (!c || !host_weights || !host_grads) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound || !c->d_staging) return SIGNMUON_ERR_NOT_BOUND;
+  if (c->sticky != SIGNMUON_OK) return c->sticky;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const int M = c->cfg.num_workers;
+  const size_t n = c->params.size();
+  std::vector<void*> w(n);
+  std::vector<const void*> g(n);
+  for (size_t p = 0; p < n; ++p) {
+    if (!host_weights[p] || !host_grads[p]) return SIGNMUON_ERR_INVALID_ARG;
+    const ParamPlan& pl = c->plan[p];
+    w[p] = c->d_staging + pl.stage_w_off;
+    g[p] = c->d_staging + pl.stage_g_off;
+    bool ok = cudaMemcpyAsync(w[p], host_weights[p], (size_t)pl.d * dtype_size(pl.wdtype), cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(const_cast<void*>(g[p]), host_grads[p], (size_t)M * pl.d * dtype_size(pl.gdtype),
+                               cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+  }
+  int rc = run_stages_impl(c, SIGNMUON_STAGE_ALL, w.data(), g.data(), lr, s);
+  if (rc != SIGNMUON_OK) return rc;
+  for (size_t p = 0; p < n; ++p) {
+    const ParamPlan& pl = c->plan[p];
+    if (cudaMemcpyAsync(host_weights[p], w[p], (size_t)pl.d * dtype_size(pl.wdtype), cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+      c->sticky = SIGNMUON_ERR_CUDA;
+      return c->sticky;
+    }
+  }
+  return SIGNMUON_OK;
+}
+
+int signmuon_packed_payload(const signmuon_ctx* c, int32_t worker, const uint32_t** dev_ptr, size_t* bytes,
+                            size_t* entries) {
+  if (!c || worker < 0 || worker >= c->cfg.num_workers) return SIGNMUON_ERR_INVALID_ARG;
+  if (bytes) *bytes = (size_t)c->words_per_worker * 4;
+  if (entries) *entries = (size_t)c->entries;
+  if (dev_ptr) {
+    if (!c->bound) { *dev_ptr = nullptr; return SIGNMUON_ERR_NOT_BOUND; }
+    *dev_ptr = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_bits) + (size_t)worker * c->words_per_worker;
+  }
+  return SIGNMUON_OK;
+}
+
+int signmuon_payload_segment(const signmuon_ctx* c, int32_t param, size_t* word_offset, size_t* words) {
+  if (!c || param < 0 || param >= (int32_t)c->params.size()) return SIGNMUON_ERR_INVALID_ARG;
+  if (word_offset) *word_offset = c->plan[param].word_off;
+  if (words) *words = c->plan[param].n_words;
+  return SIGNMUON_OK;
+}
+
+int signmuon_debug_tap(const signmuon_ctx* c, int32_t what, int32_t param, int32_t worker, const void** dev_ptr,
+                       size_t* bytes, int64_t* ld) {
+  if (!c || !dev_ptr || param < 0 || param >= (int32_t)c->params.size()) return SIGNMUON_ERR_INVALID_ARG;
+  if (worker < 0 || worker >= c->cfg.num_workers) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  const ParamPlan& pl = c->plan[param];
+  size_t nbytes = 0;
+  int64_t pitch = pl.cols;
+  const void* ptr = nullptr;
+  switch (what) {
+    case SIGNMUON_TAP_MOMENTUM:
+      ptr = c->d_state + pl.mom_off + (size_t)worker * pl.d * 4; nbytes = (size_t)pl.d * 4; break;
+    case SIGNMUON_TAP_POLAR: {
+      if (pl.kind != SIGNMUON_PARAM_MATRIX) return SIGNMUON_ERR_INVALID_ARG;
+      if (!(c->cfg.flags & SIGNMUON_FLAG_KEEP_POLAR) && pl.fused_pack) return SIGNMUON_ERR_INVALID_ARG;
+      const size_t yb = (size_t)pl.rows * pl.ldy * 2;
+      ptr = c->d_ws + pl.y_off[c->cfg.ns_steps & 1] + (size_t)worker * yb; nbytes = yb; pitch = pl.ldy; break;
+    }
+    case SIGNMUON_TAP_VOTE_BITS:
+      ptr = c->d_ws + c->off_vote + (size_t)pl.word_off * 4; nbytes = (size_t)pl.n_words * 4; break;
+    case SIGNMUON_TAP_WORKER_BITS:
+      ptr = c->d_ws + c->off_bits + ((size_t)worker * c->words_per_worker + pl.word_off) * 4;
+      nbytes = (size_t)pl.n_words * 4; break;
+    case SIGNMUON_TAP_NORM:
+      if (pl.kind != SIGNMUON_PARAM_MATRIX) return SIGNMUON_ERR_INVALID_ARG;
+      ptr = c->d_ws + pl.scales_off + (size_t)worker * 8; nbytes = 8; break;
+    default: return SIGNMUON_ERR_INVALID_ARG;
+  }
+  *dev_ptr = ptr;
+  if (bytes) *bytes = nbytes;
+  if (ld) *ld = pitch;
+  return SIGNMUON_OK;
+}
+
+int signmuon_status(signmuon_ctx* c, void* cuda_stream) {
+  if (!c) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0;
+  if (cudaMemcpyAsync(&word, c->d_ws + c->off_status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess) {
+    c->sticky = SIGNMUON_ERR_CUDA;
+    return c->sticky;
+  }
+  if (c->sticky != SIGNMUON_OK) return c->sticky;
+  return word == STATUS_OK ? SIGNMUON_OK : SIGNMUON_ERR_TIMEOUT;
+}
+
+int signmuon_launches_per_step(const signmuon_ctx* c, int32_t* launches) {
+  if (!c || !launches) return SIGNMUON_ERR_INVALID_ARG;
+  int n = 0;
+  const bool nm = !c->matrix_list.empty();
+  if (nm) n += 2;                                   // momentum + norms
+  if (!c->plain_list.empty()) n += 1;
+  if (nm) n += (int)c->ns_launches.size() + (c->packfb_blocks ? 1 : 0) + 1;   // NS, fallback pack, vote
+  if (nm && c->cfg.local_polar && c->cfg.ns_steps > 0) n += (int)c->lp_launches.size();
+  *launches = n;
+  return SIGNMUON_OK;
+}
+
+int signmuon_ns_flops_per_step(const signmuon_ctx* c, double* flops) {
+  if (!c || !flops) return SIGNMUON_ERR_INVALID_ARG;
+  double f = 0;
+  for (int32_t p : c->matrix_list) {
+    const ParamPlan& pl = c->plan[p];
+    f += 4.0 * (double)pl.s * (double)pl.s * (double)pl.l * c->cfg.ns_steps *
+         (c->cfg.num_workers + (c->cfg.local_polar ? 1 : 0));
+  }
+  *flops = f;
+  return SIGNMUON_OK;
+}
+
+void signmuon_destroy(signmuon_ctx* c) { delete c; }
+
+const char* signmuon_error_string(int code) {
+  switch (code) {
+    case SIGNMUON_OK: return "ok";
+    case SIGNMUON_ERR_INVALID_ARG: return "invalid argument";
+    case SIGNMUON_ERR_BAD_SHAPE: return "bad parameter shape";
+    case SIGNMUON_ERR_NOT_BOUND: return "context has no device buffers bound";
+    case SIGNMUON_ERR_BUFFER_TOO_SMALL: return "state, workspace or staging buffer too small";
+    case SIGNMUON_ERR_CUDA: return "CUDA call or kernel launch failed";
+    case SIGNMUON_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case SIGNMUON_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
+    case SIGNMUON_ERR_MISALIGNED: return "device pointer is not sufficiently aligned";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

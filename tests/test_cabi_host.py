@@ -1,0 +1,106 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, validates its arguments and reports sizes that follow from the payload format."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2605_16311_b200 import binding as B
+from paper_2605_16311_b200 import build as build_mod
+from paper_2605_16311_b200 import workloads as wlmod
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built_library():
+    build_mod.build()
+    return B.load_library()
+
+
+def test_library_exports_every_declared_symbol(built_library):
+    header = open(os.path.join(ROOT, "include", "signmuon.h")).read()
+    declared = set(re.findall(r"\b(signmuon_[a-z_]+)\s*\(", header))
+    assert declared == set(B.EXPORTS)
+    for name in declared:
+        assert hasattr(built_library, name)
+
+
+def _cfg(params, **kw):
+    arr = (B.ParamStruct * len(params))(*[B.ParamStruct(*p) for p in params])
+    vals = dict(num_workers=4, momentum=0.9, lr=1e-3, ns_steps=5, local_polar=0, weight_decay=0.0, eps=1e-12,
+                update_scale=0, flags=0)
+    vals.update(kw)
+    cfg = B.ConfigStruct(len(params), arr, vals["num_workers"], vals["momentum"], vals["lr"], vals["ns_steps"],
+                         vals["local_polar"], vals["weight_decay"], vals["eps"], vals["update_scale"], vals["flags"])
+    cfg._keep = arr
+    return cfg
+
+
+def test_create_rejects_bad_arguments():
+    good = [(64, 64, 0, 0, 0)]
+    assert B.signmuon_create_raw(None)[0] == -1
+    for kw in (dict(num_workers=0), dict(num_workers=256), dict(momentum=1.0), dict(momentum=-0.1),
+               dict(ns_steps=-1), dict(weight_decay=-1.0), dict(update_scale=2), dict(local_polar=3),
+               dict(lr=float("nan"))):
+        code, h = B.signmuon_create_raw(_cfg(good, **kw))
+        assert code == -1 and h is None, kw
+    for bad in ([(0, 64, 0, 0, 0)], [(64, -1, 0, 0, 0)], [(1 << 25, 4, 0, 0, 0)]):
+        assert B.signmuon_create_raw(_cfg(bad))[0] == -2
+    assert B.signmuon_create_raw(_cfg([(64, 64, 7, 0, 0)]))[0] == -1
+    assert B.signmuon_create_raw(_cfg([(64, 64, 0, 5, 0)]))[0] == -1
+    empty = _cfg(good)
+    empty.num_params = 0
+    assert B.signmuon_create_raw(empty)[0] == -1
+    assert B.load_library().signmuon_create(C.byref(_cfg(good)), None) == -1
+
+
+def test_unbound_context_refuses_device_calls():
+    ctx = B.signmuon_create([(64, 64, 0, 0, 0)], 2, 0.9, 1e-3, 5, False)
+    lib = B.load_library()
+    arr = (C.c_void_p * 1)(C.c_void_p(256))
+    assert lib.signmuon_step(ctx, arr, arr, 0.1, None) == -3
+    assert lib.signmuon_status(ctx, None) == -3
+    p = C.c_void_p()
+    assert lib.signmuon_packed_payload(ctx, 0, C.byref(p), None, None) == -3
+    assert lib.signmuon_packed_payload(ctx, 2, None, None, None) == -1      # worker out of range
+    assert lib.signmuon_bind(ctx, None, 0, None, 0, None, 0, 1, None) == -1
+    assert lib.signmuon_bind(ctx, C.c_void_p(1024), 16, C.c_void_p(1024), 16, None, 0, 1, None) == -4
+    B.signmuon_destroy(ctx)
+    assert B.load_library().signmuon_error_string(-6).decode().startswith("a bounded")
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
+def test_payload_is_one_bit_per_entry(name):
+    wl = wlmod.by_name(name)
+    tuples = [(p.rows, p.cols, B._KIND[p.kind], B._DT[p.dtype], B._DT[p.dtype]) for p in wl.params]
+    ctx = B.signmuon_create(tuples, wl.num_workers, wl.momentum, wl.lr, wl.ns_steps, wl.local_polar)
+    _, nbytes, entries = B.signmuon_packed_payload(ctx, 0, want_ptr=False)
+    assert entries == wl.numel
+    assert nbytes * 8 == entries                      # exactly one bit per entry at these shapes
+    assert 4 * entries / nbytes == 32                 # 32x smaller than float32
+    off = 0
+    for i, p in enumerate(wl.params):
+        o, w = B.signmuon_payload_segment(ctx, i)
+        assert o == off and w == (p.numel + 31) // 32
+        off += w
+    state, ws, staging = B.signmuon_state_bytes(ctx)
+    assert state >= 4 * wl.num_workers * wl.numel     # one float32 momentum per worker and entry
+    assert state < 4 * wl.num_workers * wl.numel + 256 * len(wl.params) + 1
+    assert ws > wl.num_workers * nbytes
+    flops = B.signmuon_ns_flops_per_step(ctx)
+    expect = sum(4.0 * min(p.rows, p.cols) ** 2 * max(p.rows, p.cols) * wl.ns_steps *
+                 (wl.num_workers + (1 if wl.local_polar else 0)) for p in wl.params if p.kind == "matrix")
+    assert flops == pytest.approx(expect, rel=1e-12)
+    B.signmuon_destroy(ctx)
+
+
+def test_ragged_parameter_pads_to_words():
+    ctx = B.signmuon_create([(3, 11, 0, 0, 0), (1, 5, 1, 0, 0)], 3, 0.9, 1e-3, 2, False)
+    _, nbytes, entries = B.signmuon_packed_payload(ctx, 1, want_ptr=False)
+    assert entries == 38 and nbytes == 4 * (2 + 1)
+    assert B.signmuon_payload_segment(ctx, 1) == (2, 1)
+    # momentum, norms, 2x2 NS products, fallback pack (11 columns do not fill words), vote, plain kernel
+    assert B.signmuon_launches_per_step(ctx) == 2 + 1 + 4 + 1 + 1
+    B.signmuon_destroy(ctx)

@@ -1,0 +1,179 @@
+"""GPU parity tests: the CUDA path through the C ABI against the float64 oracle, stage by stage."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_16311_b200 import binding as B
+from paper_2605_16311_b200 import workloads as wlmod
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    from paper_2605_16311_b200 import build as build_mod
+    build_mod.build()
+    assert torch.cuda.is_available()
+    B.load_library()
+
+
+def _wl(shapes, M, dtype="f32", K=5, local_polar=False, kinds=None, **kw):
+    kinds = kinds or ["matrix"] * len(shapes)
+    ps = [wlmod.Param(r, c, k, dtype, f"p{i}") for i, ((r, c), k) in enumerate(zip(shapes, kinds))]
+    base = dict(momentum=0.9, lr=1e-3, ns_steps=K, local_polar=local_polar, steps=2, signal_std=1e-3,
+                noise_std=3e-3, config_id=77)
+    base.update(kw)
+    return wlmod.Workload("t", ps, num_workers=M, **base)
+
+
+def test_config1_simt_diagnostic_path():
+    from parity_utils import run_and_check
+    rep = run_and_check(wlmod.config1(), steps=2, flags=B.FLAG_KEEP_POLAR | B.FLAG_SIMT_GEMM)
+    assert rep["sign_match_min"] >= 0.999
+
+
+def test_config1_ten_steps():
+    from parity_utils import run_and_check
+    rep = run_and_check(wlmod.config1(), steps=10)
+    print(rep)
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 8])
+def test_ragged_shapes_wide_tall_and_stem(M):
+    from parity_utils import run_and_check
+    wl = _wl([(200, 328), (328, 200), (64, 147), (130, 64), (96, 96), (1, 160), (300, 1)], M)
+    run_and_check(wl, steps=2)
+
+
+def test_local_polar_ragged_and_eq2_scale():
+    from parity_utils import run_and_check
+    run_and_check(_wl([(200, 328), (328, 200), (64, 147), (256, 256)], 4, local_polar=True, lr=0.01), steps=2)
+
+
+@pytest.mark.parametrize("K", [0, 1, 2, 3])
+def test_ns_step_counts(K):
+    from parity_utils import run_and_check
+    run_and_check(_wl([(128, 384), (384, 128), (64, 147)], 2, K=K), steps=1)
+    run_and_check(_wl([(128, 384), (64, 147)], 2, K=K, local_polar=True), steps=1)
+
+
+def test_bf16_weights_matrix_and_plain_student_t():
+    from parity_utils import run_and_check
+    wl = _wl([(256, 768), (768, 256), (1000, 33), (1, 768), (515, 64)], 16, dtype="bf16", local_polar=True,
+             kinds=["matrix", "matrix", "plain", "plain", "plain"], noise="student_t4", signal_std=5e-4,
+             noise_std=1e-3)
+    run_and_check(wl, steps=3)
+    wl.local_polar = False
+    run_and_check(wl, steps=2)
+
+
+@pytest.mark.parametrize("M", [1, 5, 16, 32, 33, 100])
+def test_vote_worker_counts(M):
+    from parity_utils import run_and_check
+    run_and_check(_wl([(64, 96), (40, 7)], M, K=1, kinds=["matrix", "plain"]), steps=1, check_polar=(M <= 16))
+
+
+def test_resnet50_prefix_and_large_tiles():
+    from parity_utils import run_and_check
+    c2 = wlmod.config2()
+    wl = wlmod.scaled_down(c2, 9)
+    run_and_check(wl, steps=2)
+    run_and_check(_wl([(512, 1152), (1024, 512)], 2), steps=1)
+
+
+def test_gpt2_and_llama_like_shapes_bf16():
+    from parity_utils import run_and_check
+    run_and_check(_wl([(768, 2304), (3072, 768)], 2, dtype="bf16", local_polar=True, signal_std=5e-4,
+                      noise_std=1e-3, noise="student_t4"), steps=1)
+    run_and_check(_wl([(1024, 4096)], 2, dtype="bf16", signal_std=1e-4, noise_std=5e-4), steps=1)
+
+
+def test_full_resnet50_config_sampled():
+    """The benchmark's configuration at full size, parameters sampled for the oracle."""
+    from parity_utils import run_and_check
+    wl = wlmod.config2()
+    names = [p.name for p in wl.params]
+    sample = [0, 1, names.index("s0b0.conv3"), names.index("s1b0.conv2"), names.index("s2b0.down"),
+              names.index("s3b2.conv2"), names.index("fc")]
+    rep = run_and_check(wl, steps=2, sample=sample)
+    print(rep)
+
+
+def test_weight_decay_and_step_lr_override():
+    from parity_utils import check_param_step, make_optimizer
+    import numpy as np
+    wl = _wl([(96, 160)], 3)
+    opt = B.SignMuon(wl.params, 3, momentum=0.8, lr=123.0, ns_steps=5, weight_decay=0.05, flags=B.FLAG_KEEP_POLAR)
+    wl.momentum = 0.8
+    w = wlmod.make_weights(wl, "cuda:0")
+    sig = wlmod.make_signal(wl, "cuda:0")
+    g = wlmod.make_grads(wl, sig, 0, "cuda:0")
+    before = w[0].clone()
+    opt.step(w, g, 0.004)                     # per-step learning rate overrides the configured one
+    torch.cuda.synchronize()
+    check_param_step(opt, wl, 0, before, w[0], g[0], None, 0.004, weight_decay=0.05)
+    opt.close()
+
+
+def test_stage_calls_equal_one_step_and_determinism():
+    wl = _wl([(256, 320), (320, 256), (64, 147), (1, 99)], 4, local_polar=True,
+             kinds=["matrix", "matrix", "matrix", "plain"])
+    sig = wlmod.make_signal(wl, "cuda:0")
+    g = wlmod.make_grads(wl, sig, 0, "cuda:0")
+    outs = []
+    for mode in range(3):
+        opt = B.SignMuon(wl.params, 4, lr=0.01, local_polar=True)
+        w = wlmod.make_weights(wl, "cuda:0")
+        if mode == 1:
+            for st in (B.STAGE_MOMENTUM, B.STAGE_NS, B.STAGE_VOTE, B.STAGE_LOCAL_POLAR):
+                opt.step(w, g, stages=st)
+        else:
+            opt.step(w, g)
+        torch.cuda.synchronize()
+        assert opt.status() == B.OK
+        outs.append(([x.clone() for x in w], opt.payload(0).clone(), opt.payload(3).clone()))
+        opt.close()
+    for other in outs[1:]:
+        for a, b in zip(outs[0][0], other[0]):
+            assert torch.equal(a, b)                       # bit-identical weights
+        assert torch.equal(outs[0][1], other[1]) and torch.equal(outs[0][2], other[2])
+
+
+def test_garbage_worker_is_outvoted():
+    """One worker sending NaN gradients maps to -1 everywhere; the vote still equals the popcount rule."""
+    from parity_utils import check_param_step
+    wl = _wl([(64, 128), (1, 64)], 5, kinds=["matrix", "plain"])
+    opt = B.SignMuon(wl.params, 5, flags=B.FLAG_KEEP_POLAR)
+    w = wlmod.make_weights(wl, "cuda:0")
+    sig = wlmod.make_signal(wl, "cuda:0")
+    g = wlmod.make_grads(wl, sig, 0, "cuda:0")
+    for t in g:
+        t[2].fill_(float("nan"))
+    opt.step(w, g)
+    torch.cuda.synchronize()
+    for p in range(2):
+        bits = opt.tap(B.TAP_WORKER_BITS, p, 2).cpu().numpy()
+        assert not bits.any()                              # NaN >= 0 is false -> bit 0
+        import oracle as O
+        d = wl.params[p].numel
+        packed = [opt.tap(B.TAP_WORKER_BITS, p, m).cpu().numpy()[: (d + 7) // 8] for m in range(5)]
+        vote = O.unpack_bits(opt.tap(B.TAP_VOTE_BITS, p, 0).cpu().numpy(), d)
+        assert np.array_equal(vote, O.majority_vote_popcount(packed, d))
+    opt.close()
+
+
+def test_host_resident_step_matches_device_step():
+    wl = _wl([(128, 256), (64, 147), (1, 40)], 3, kinds=["matrix", "matrix", "plain"])
+    sig = wlmod.make_signal(wl, "cuda:0")
+    g = wlmod.make_grads(wl, sig, 0, "cuda:0")
+    w_dev = wlmod.make_weights(wl, "cuda:0")
+    w_host = [x.cpu().pin_memory() for x in w_dev]
+    g_host = [x.cpu().pin_memory() for x in g]
+    a = B.SignMuon(wl.params, 3)
+    a.step(w_dev, g)
+    b = B.SignMuon(wl.params, 3, host_staging=True)
+    b.step_host(w_host, g_host)
+    torch.cuda.synchronize()
+    for x, y in zip(w_dev, w_host):
+        assert torch.equal(x.cpu(), y)
+    a.close(); b.close()
