@@ -56,7 +56,8 @@ enum {
   SIGNMUON_ERR_CUDA = -5,             /* a CUDA call or launch failed (sticky) */
   SIGNMUON_ERR_TIMEOUT = -6,          /* a bounded device-side wait ran out (see signmuon_status) */
   SIGNMUON_ERR_UNSUPPORTED_ARCH = -7, /* current device is not compute capability 10.x */
-  SIGNMUON_ERR_MISALIGNED = -8        /* a device pointer is not 16-byte aligned */
+  SIGNMUON_ERR_MISALIGNED = -8,       /* a device pointer is not 16-byte aligned */
+  SIGNMUON_ERR_TOO_LARGE = -9         /* problem exceeds a fixed capacity (signmuon_momentum_norm_noalloc) */
 };
 
 typedef enum { SIGNMUON_F32 = 0, SIGNMUON_BF16 = 1 } signmuon_dtype;
@@ -178,6 +179,41 @@ int signmuon_launches_per_step(const signmuon_ctx* ctx, int32_t* launches);
 /* Newton-Schulz floating-point operations of one step: 4 s^2 l K per matrix and worker (plus one
  * more "worker" for the local polar step), s = min(rows, cols), l = max(rows, cols). */
 int signmuon_ns_flops_per_step(const signmuon_ctx* ctx, double* flops);
+
+/* Capacity of the built-in scratch of signmuon_momentum_norm_noalloc: one float per 8192 entries per
+ * worker, i.e. num_workers * ceil(rows*cols / 8192) must not exceed it (about 5.4e8 entries over all
+ * workers; e.g. 4096 x 4096 with 32 workers just fits). */
+#define SIGNMUON_NOALLOC_MAX_PARTIALS 65536
+
+/* Momentum + Frobenius-norm stage for ONE matrix, usable where device memory cannot be allocated.
+ * (The paper has no counterpart: it is the first stage of signmuon_step - weight decay, momentum,
+ * bf16 operand, 1/max(||Mom||_F, eps) - repackaged for a class of callers.)
+ *
+ * Some hosts of this library may not call cudaMalloc around an optimizer step: a step recorded into a
+ * pipeline whose memory plan is already frozen, a plugin that must not grow its host framework's memory
+ * pool, a latency-critical loop that cannot take the allocator lock.  signmuon_step serves them only if
+ * they can still hand over a workspace; this call needs none.  Its only scratch - the per-block partial
+ * sums of the norm reduction - lives in a fixed 256 KB array inside the library image, present on every
+ * GPU that loads the library until the process exits.  The call itself allocates nothing and calls
+ * nothing that allocates.
+ *
+ *   dev_grads        DEVICE [M][rows*cols] grad_dtype, read only
+ *   dev_weights      DEVICE [rows*cols] weight_dtype, read only; may be NULL when weight_decay == 0
+ *   dev_momentum     DEVICE [M][rows*cols] float32, updated in place
+ *   dev_operand_bf16 DEVICE [M][rows*cols] bf16, written: bf16(momentum), the Newton-Schulz operand
+ *   dev_scales       DEVICE [M][2] float32, written: 1/max(sigma,eps)^2 and 1/max(sigma,eps)
+ * rows*cols must be a multiple of 8 and all array pointers 16-byte aligned.
+ *
+ * Limits and sharing: problems larger than SIGNMUON_NOALLOC_MAX_PARTIALS allows are refused with
+ * SIGNMUON_ERR_TOO_LARGE before anything is launched.  Every call on a device uses the same array; a
+ * call overwrites the part it uses before reading it, so no clearing is needed between calls, but calls
+ * that may run concurrently on one GPU (different streams without ordering) race - keep them ordered.
+ * The first call on each device resolves the array's device address; make that call outside any stream
+ * capture.  Other errors: INVALID_ARG, BAD_SHAPE, MISALIGNED, CUDA. */
+int signmuon_momentum_norm_noalloc(const void* dev_grads, int32_t grad_dtype, const void* dev_weights,
+                                   int32_t weight_dtype, float* dev_momentum, void* dev_operand_bf16,
+                                   float* dev_scales, int64_t rows, int64_t cols, int32_t num_workers,
+                                   float momentum, float weight_decay, float eps, void* cuda_stream);
 
 void signmuon_destroy(signmuon_ctx* ctx);
 

@@ -26,9 +26,11 @@ TAP_MOMENTUM, TAP_POLAR, TAP_VOTE_BITS, TAP_WORKER_BITS, TAP_NORM = 0, 1, 2, 3, 
 EXPORTS = [
     "signmuon_create", "signmuon_state_bytes", "signmuon_bind", "signmuon_step", "signmuon_run_stages",
     "signmuon_step_host", "signmuon_packed_payload", "signmuon_payload_segment", "signmuon_debug_tap",
-    "signmuon_status", "signmuon_launches_per_step", "signmuon_ns_flops_per_step", "signmuon_destroy",
-    "signmuon_error_string",
+    "signmuon_status", "signmuon_launches_per_step", "signmuon_ns_flops_per_step",
+    "signmuon_momentum_norm_noalloc", "signmuon_destroy", "signmuon_error_string",
 ]
+NOALLOC_MAX_PARTIALS = 65536
+ERR_TOO_LARGE = -9
 
 
 class ParamStruct(C.Structure):
@@ -68,6 +70,8 @@ def load_library() -> C.CDLL:
     lib.signmuon_status.argtypes = [vp, vp]
     lib.signmuon_launches_per_step.argtypes = [vp, C.POINTER(i32)]
     lib.signmuon_ns_flops_per_step.argtypes = [vp, C.POINTER(C.c_double)]
+    lib.signmuon_momentum_norm_noalloc.argtypes = [vp, i32, vp, i32, vp, vp, vp, C.c_int64, C.c_int64, i32,
+                                                   f32, f32, f32, vp]
     lib.signmuon_destroy.argtypes = [vp]
     lib.signmuon_destroy.restype = None
     lib.signmuon_error_string.argtypes = [C.c_int]
@@ -184,6 +188,18 @@ def signmuon_ns_flops_per_step(ctx: int) -> float:
     f = C.c_double()
     _check(load_library().signmuon_ns_flops_per_step(ctx, C.byref(f)), "signmuon_ns_flops_per_step")
     return f.value
+
+
+def signmuon_momentum_norm_noalloc(grads_ptr: int, grad_dtype: int, weights_ptr: int, weight_dtype: int,
+                                   momentum_ptr: int, operand_ptr: int, scales_ptr: int, rows: int, cols: int,
+                                   num_workers: int, momentum: float, weight_decay: float, eps: float,
+                                   stream: int) -> int:
+    """Momentum + Frobenius-norm stage of one matrix with the library's built-in scratch: for callers
+    that may not allocate device memory. Returns the C error code (0 = ok) instead of raising, so that
+    the capacity refusal can be inspected."""
+    return load_library().signmuon_momentum_norm_noalloc(
+        grads_ptr, grad_dtype, weights_ptr or None, weight_dtype, momentum_ptr, operand_ptr, scales_ptr,
+        rows, cols, num_workers, momentum, weight_decay, eps, stream or None)
 
 
 def signmuon_destroy(ctx: int):

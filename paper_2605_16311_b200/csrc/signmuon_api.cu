@@ -823,6 +823,7 @@ const char* signmuon_error_string(int code) {
     case SIGNMUON_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case SIGNMUON_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
     case SIGNMUON_ERR_MISALIGNED: return "device pointer is not sufficiently aligned";
+    case SIGNMUON_ERR_TOO_LARGE: return "problem exceeds the fixed capacity of this entry point";
     default: return "unknown error";
   }
 }
