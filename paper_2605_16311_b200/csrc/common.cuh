@@ -75,6 +75,11 @@ struct GemmProblem {
   int32_t store_out;      // APPLY_PACK: also write hi(y)
   int32_t param;          // APPLY_UPDATE: index into the ParamDev table
   uint32_t* bits_out;     // APPLY_PACK: first payload word of this (param, worker)
+  // TMA-staged epilogue (tensor-core kernel): tensor maps with {64 x 128} bf16 or {32 x 128} fp32 boxes
+  int32_t tma_c, tma_out; // 1: C arrives / results leave through TMA, 0: direct global accesses
+  int32_t tmapC0, tmapC1; // C hi (or fp32 momentum) and C lo
+  int32_t tmapO0, tmapO1; // out hi and out lo
+  int32_t batch_c, batch_o;
 };
 
 struct TileEntry {
@@ -103,31 +108,25 @@ __device__ __forceinline__ void store_hi_lo(bf16* o, bf16* olo, const float (&v)
       if (olo) reinterpret_cast<uint4*>(olo)[q] = make_uint4(wl[0], wl[1], wl[2], wl[3]);
     }
   } else {
-    for (int j = 0; j < n_valid; ++j) {
-      const bf16 h = __float2bfloat16_rn(v[j]);
-      o[j] = h;
-      if (olo) olo[j] = __float2bfloat16_rn(v[j] - __bfloat162float(h));
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      if (j < n_valid) {
+        const bf16 h = __float2bfloat16_rn(v[j]);
+        o[j] = h;
+        if (olo) olo[j] = __float2bfloat16_rn(v[j] - __bfloat162float(h));
+      }
     }
   }
 }
 
-// Applies one epilogue to 32 consecutive columns [col0, col0+32) of output row `row`.
-// `v` holds the fp32 accumulators.  Rows/columns outside the problem are skipped.
-__device__ __forceinline__ void epilogue_row32(const GemmProblem& pr, const ParamDev* params, float lr,
-                                               int row, int col0, float (&v)[32]) {
+// ---- epilogue building blocks, each over 32 consecutive columns [col0, col0+32) of output row `row`;
+// rows/columns outside the problem are skipped.
+
+// v <- scale * (v + 1.5 * C) with C read directly from global memory.
+__device__ __forceinline__ void apply_c_direct(const GemmProblem& pr, float scale, int row, int col0, float* v) {
   if (row >= pr.M || col0 >= pr.N) return;
-  const float scale = pr.scale_ptr ? __ldg(pr.scale_ptr) : pr.scale_imm;
   const bool full = (col0 + 32 <= pr.N);
   const int n_valid = full ? 32 : pr.N - col0;
-  if (pr.epi == EPI_GRAM) {
-    const float f = -0.5f * scale;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] *= f;
-    bf16* o = reinterpret_cast<bf16*>(pr.out) + (int64_t)row * pr.ld_out + col0;
-    store_hi_lo(o, nullptr, v, full && ((pr.ld_out & 7) == 0), n_valid);
-    return;
-  }
-  // APPLY family: y = scale * (acc + 1.5 * C)
   if (pr.c_mode == C_F32) {
     const float* c = reinterpret_cast<const float*>(pr.C) + (int64_t)row * pr.ldc + col0;
     if (full && ((pr.ldc & 3) == 0)) {
@@ -141,6 +140,7 @@ __device__ __forceinline__ void epilogue_row32(const GemmProblem& pr, const Para
         v[4 * q + 3] = scale * fmaf(1.5f, t.w, v[4 * q + 3]);
       }
     } else {
+#pragma unroll
       for (int j = 0; j < 32; ++j) v[j] = (j < n_valid) ? scale * fmaf(1.5f, __ldg(c + j), v[j]) : 0.f;
     }
   } else {
@@ -163,6 +163,7 @@ __device__ __forceinline__ void epilogue_row32(const GemmProblem& pr, const Para
         }
       }
     } else {
+#pragma unroll
       for (int j = 0; j < 32; ++j) {
         float cv = 0.f;
         if (j < n_valid) cv = __bfloat162float(c[j]) + (cl ? __bfloat162float(cl[j]) : 0.f);
@@ -170,41 +171,92 @@ __device__ __forceinline__ void epilogue_row32(const GemmProblem& pr, const Para
       }
     }
   }
-  if (pr.epi == EPI_APPLY || (pr.epi == EPI_APPLY_PACK && pr.store_out)) {
-    bf16* o = reinterpret_cast<bf16*>(pr.out) + (int64_t)row * pr.ld_out + col0;
-    bf16* ol = (pr.epi == EPI_APPLY && pr.out_lo) ? pr.out_lo + (int64_t)row * pr.ld_out + col0 : nullptr;
-    store_hi_lo(o, ol, v, full && ((pr.ld_out & 7) == 0), n_valid);
-  }
-  if (pr.epi == EPI_APPLY_PACK) {
-    // Only issued for parameters with cols % 32 == 0: the 32 columns are one payload word.
-    uint32_t word = 0;
+}
+
+// out <- hi(v) (and out_lo <- lo(v)) written directly to global memory.
+__device__ __forceinline__ void store_out_direct(const GemmProblem& pr, int row, int col0, const float* v, bool with_lo) {
+  if (row >= pr.M || col0 >= pr.N) return;
+  const bool full = (col0 + 32 <= pr.N);
+  const int n_valid = full ? 32 : pr.N - col0;
+  bf16* o = reinterpret_cast<bf16*>(pr.out) + (int64_t)row * pr.ld_out + col0;
+  bf16* ol = (with_lo && pr.out_lo) ? pr.out_lo + (int64_t)row * pr.ld_out + col0 : nullptr;
+  const float(&vv)[32] = *reinterpret_cast<const float(*)[32]>(v);
+  store_hi_lo(o, ol, vv, full && ((pr.ld_out & 7) == 0), n_valid);
+}
+
+// One payload word from 32 consecutive columns (only issued for parameters with cols % 32 == 0).
+__device__ __forceinline__ void pack_bits_direct(const GemmProblem& pr, int row, int col0, const float* v) {
+  if (row >= pr.M || col0 + 32 > pr.N) return;
+  uint32_t word = 0;
 #pragma unroll
-    for (int j = 0; j < 32; ++j) word |= (v[j] >= 0.f ? 1u : 0u) << j;
-    pr.bits_out[((int64_t)row * pr.N + col0) >> 5] = word;
-  } else if (pr.epi == EPI_APPLY_UPDATE) {
-    const ParamDev& pd = params[pr.param];
-    const float step = lr;
-    if (pd.wdtype == 0) {
-      float* w = reinterpret_cast<float*>(pd.W) + (int64_t)row * pr.N + col0;
-      if (full && ((pr.N & 3) == 0)) {
-        float4* w4 = reinterpret_cast<float4*>(w);
+  for (int j = 0; j < 32; ++j) word |= (v[j] >= 0.f ? 1u : 0u) << j;
+  pr.bits_out[((int64_t)row * pr.N + col0) >> 5] = word;
+}
+
+// W <- W - lr * v (local polar step's last epilogue).
+__device__ __forceinline__ void update_weights_direct(const GemmProblem& pr, const ParamDev* params, float lr, int row,
+                                                      int col0, const float* v) {
+  if (row >= pr.M || col0 >= pr.N) return;
+  const bool full = (col0 + 32 <= pr.N);
+  const int n_valid = full ? 32 : pr.N - col0;
+  const ParamDev& pd = params[pr.param];
+  if (pd.wdtype == 0) {
+    float* w = reinterpret_cast<float*>(pd.W) + (int64_t)row * pr.N + col0;
+    if (full && ((pr.N & 3) == 0)) {
+      float4* w4 = reinterpret_cast<float4*>(w);
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          float4 t = w4[q];
-          t.x = fmaf(-step, v[4 * q], t.x);
-          t.y = fmaf(-step, v[4 * q + 1], t.y);
-          t.z = fmaf(-step, v[4 * q + 2], t.z);
-          t.w = fmaf(-step, v[4 * q + 3], t.w);
-          w4[q] = t;
-        }
-      } else {
-        for (int j = 0; j < n_valid; ++j) w[j] = fmaf(-step, v[j], w[j]);
+      for (int q = 0; q < 8; ++q) {
+        float4 t = w4[q];
+        t.x = fmaf(-lr, v[4 * q], t.x);
+        t.y = fmaf(-lr, v[4 * q + 1], t.y);
+        t.z = fmaf(-lr, v[4 * q + 2], t.z);
+        t.w = fmaf(-lr, v[4 * q + 3], t.w);
+        w4[q] = t;
       }
     } else {
-      bf16* w = reinterpret_cast<bf16*>(pd.W) + (int64_t)row * pr.N + col0;
-      for (int j = 0; j < n_valid; ++j) w[j] = __float2bfloat16_rn(fmaf(-step, v[j], __bfloat162float(w[j])));
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < n_valid) w[j] = fmaf(-lr, v[j], w[j]);
+    }
+  } else {
+    bf16* w = reinterpret_cast<bf16*>(pd.W) + (int64_t)row * pr.N + col0;
+    if (full && ((pr.N & 7) == 0)) {
+      uint4* w4 = reinterpret_cast<uint4*>(w);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 t = w4[q];
+        const uint32_t in[4] = {t.x, t.y, t.z, t.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          o[e] = pack_bf16x2(fmaf(-lr, v[q * 8 + 2 * e], __uint_as_float(in[e] << 16)),
+                             fmaf(-lr, v[q * 8 + 2 * e + 1], __uint_as_float(in[e] & 0xffff0000u)));
+        w4[q] = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < n_valid) w[j] = __float2bfloat16_rn(fmaf(-lr, v[j], __bfloat162float(w[j])));
     }
   }
+}
+
+// Whole epilogue of 32 columns with direct global accesses (diagnostic kernel and ragged fallbacks).
+__device__ __forceinline__ void epilogue_row32(const GemmProblem& pr, const ParamDev* params, float lr,
+                                               int row, int col0, float (&v)[32]) {
+  if (row >= pr.M || col0 >= pr.N) return;
+  const float scale = pr.scale_ptr ? __ldg(pr.scale_ptr) : pr.scale_imm;
+  if (pr.epi == EPI_GRAM) {
+    const float f = -0.5f * scale;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] *= f;
+    store_out_direct(pr, row, col0, v, false);
+    return;
+  }
+  apply_c_direct(pr, scale, row, col0, v);
+  if (pr.epi == EPI_APPLY || (pr.epi == EPI_APPLY_PACK && pr.store_out)) store_out_direct(pr, row, col0, v, pr.epi == EPI_APPLY);
+  if (pr.epi == EPI_APPLY_PACK) pack_bits_direct(pr, row, col0, v);
+  else if (pr.epi == EPI_APPLY_UPDATE) update_weights_direct(pr, params, lr, row, col0, v);
 }
 
 }  // namespace signmuon

@@ -15,6 +15,10 @@
 //   MN-major (contiguous along M/N): per 64 rows of M/N one 8 KB chunk = 64 k-rows of 128 bytes,
 //            TMA box {64 mn, 64 k}; descriptor LBO = 8192 (next chunk), SBO = 1024 (next 8 k-rows),
 //            a 16-element K step advances the start by 2048 bytes.
+// Epilogue traffic also goes through TMA: the Y_k tile that enters as 1.5*C is prefetched into a ring
+// of 64-column chunk buffers (128-byte swizzle; hi half and lo half, or two fp32 halves for the first
+// iteration's momentum), the results overwrite the chunk in place and leave with a TMA store, so the
+// epilogue warps touch global memory directly only for payload words and the final weight update.
 // Every wait is bounded: after about two seconds a waiting thread records STATUS_TIMEOUT in the
 // status word, raises a CTA-wide abort flag and the CTA drains and exits (TMEM is freed).
 #pragma once
@@ -112,21 +116,52 @@ __device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, int x, int y, int z, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+               ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Barrier over the 128 epilogue threads that also ANDs a flag, so that all of them take the same exit.
+__device__ __forceinline__ bool epi_bar_and(bool flag) {
+  uint32_t out;
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, 128, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out)
+      : "r"((uint32_t)flag)
+      : "memory");
+  return out != 0;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// Loads 64 consecutive fp32 columns of this thread's TMEM lane and waits for them.  Load and wait sit in
+// one asm statement so that no use of the destination registers can be scheduled before the wait.
+__device__ __forceinline__ void tc_ld64(uint32_t taddr, float (&v)[64]) {
+  uint32_t r[64];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+  for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // Shared-memory matrix descriptor (128-byte swizzle).  Bits: [0,14) start >> 4, [16,30) LBO >> 4,
@@ -156,23 +191,46 @@ __device__ __forceinline__ uint32_t instr_desc(int n, int a_mn, int b_mn) {
 }
 
 // ------------------------------------------------------------------------------------------ kernel
-template <int BN, int STAGES>
+constexpr uint32_t EPI_HALF_BYTES = 128 * 128;        // 128 rows x 128 bytes (one swizzled half)
+constexpr uint32_t EPI_BUF_BYTES = 2 * EPI_HALF_BYTES;
+
+// Issues the TMA loads of the C chunk (64 columns from column `col0`) of a tile into an epilogue buffer.
+__device__ __forceinline__ void epi_issue_c_load(const GemmLaunchArgs& args, const GemmProblem& pr, int row0, int col0,
+                                                 uint32_t buf, uint32_t bar) {
+  if (pr.c_mode == C_F32) {
+    mbar_expect_tx(bar, EPI_BUF_BYTES);
+    tma_load_3d(buf, args.tmaps + pr.tmapC0, col0, row0, pr.batch_c, bar);
+    tma_load_3d(buf + EPI_HALF_BYTES, args.tmaps + pr.tmapC0, col0 + 32, row0, pr.batch_c, bar);
+  } else if (pr.c_mode == C_HILO) {
+    mbar_expect_tx(bar, EPI_BUF_BYTES);
+    tma_load_3d(buf, args.tmaps + pr.tmapC0, col0, row0, pr.batch_c, bar);
+    tma_load_3d(buf + EPI_HALF_BYTES, args.tmaps + pr.tmapC1, col0, row0, pr.batch_c, bar);
+  } else {
+    mbar_expect_tx(bar, EPI_HALF_BYTES);
+    tma_load_3d(buf, args.tmaps + pr.tmapC0, col0, row0, pr.batch_c, bar);
+  }
+}
+
+template <int BN, int STAGES, int EPI_BUFS>
 __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmLaunchArgs args) {
   constexpr uint32_t A_BYTES = GEMM_BM * GEMM_BK * 2;          // 16 KB
   constexpr uint32_t B_BYTES = BN * GEMM_BK * 2;
   constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
   constexpr uint32_t TMEM_COLS = 2 * BN;                       // two accumulator buffers
   static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM columns: power of two");
+  static_assert(EPI_BUFS == 3, "the chunk ring is written for three buffers");
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[STAGES];
   __shared__ uint64_t empty_bar[STAGES];
   __shared__ uint64_t tmem_full_bar[2];
   __shared__ uint64_t tmem_empty_bar[2];
+  __shared__ uint64_t c_full_bar[EPI_BUFS];
   __shared__ uint32_t tmem_slot;
   __shared__ uint32_t abort_word;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   volatile uint32_t* abort_flag = &abort_word;
@@ -187,6 +245,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
       mbar_init(smem_u32(&tmem_full_bar[a]), 1);
       mbar_init(smem_u32(&tmem_empty_bar[a]), 4);
     }
+    for (int b = 0; b < EPI_BUFS; ++b) mbar_init(smem_u32(&c_full_bar[b]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -286,29 +345,167 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
   } else {
     // ===================================================================== epilogue (warps 2..5)
     const int q = warp & 3;                      // TMEM lane quarter this warp may read
+    const bool leader = (threadIdx.x == 64);     // issues the chunk loads and stores
+    const int r_in = q * 32 + lane;              // row of the tile this thread owns
+    const uint32_t row_off = (uint32_t)r_in * 128u;
+    const uint32_t sw = (uint32_t)(r_in & 7);
+    uint32_t g = 0;                              // running chunk counter (ring position)
+    uint32_t c_phase = 0;                        // bit b: parity of the next C load landing in buffer b
+    uint32_t pending_bar = 0, pending_par = 0;   // leader: the prefetch in flight (for the abort path)
     uint32_t tcount = 0;
-    for (uint32_t t = tile_begin; t < tile_end; ++t, ++tcount) {
+    bool ok = true;
+    // first chunk of the first tile
+    if (leader && tile_begin < tile_end) {
+      const TileEntry te = args.tiles[tile_begin];
+      const GemmProblem& pr = args.problems[te.problem];
+      if (pr.tma_c) {
+        epi_issue_c_load(args, pr, te.tm * GEMM_BM, te.tn * BN, epi_base, smem_u32(&c_full_bar[0]));
+        pending_bar = smem_u32(&c_full_bar[0]); pending_par = 0;
+      }
+    }
+    for (uint32_t t = tile_begin; t < tile_end && ok; ++t, ++tcount) {
       const TileEntry te = args.tiles[t];
       const GemmProblem& pr = args.problems[te.problem];
       const uint32_t acc = tcount & 1u;
       const uint32_t acc_round = tcount >> 1;
-      bool ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_round & 1u, abort_flag, args.status);
-      ok = __all_sync(0xffffffffu, ok);
+      ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_round & 1u, abort_flag, args.status);
+      ok = epi_bar_and(ok);                      // uniform over the four epilogue warps
       if (!ok) break;
       tc_fence_after();
-      const int row = te.tm * GEMM_BM + q * 32 + lane;
+      const int row0 = te.tm * GEMM_BM;
+      const int row = row0 + r_in;
       const int n0 = te.tn * BN;
       const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
+      int n_chunks = (pr.N - n0 + 63) / 64;
+      if (n_chunks > BN / 64) n_chunks = BN / 64;
+      const float scale = pr.scale_ptr ? __ldg(pr.scale_ptr) : pr.scale_imm;
+      const bool tma_c = pr.tma_c != 0, tma_out = pr.tma_out != 0;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        if (n0 + c * 32 >= pr.N) break;          // warp-uniform
-        float v[32];
-        tc_ld32(taddr + c * 32, v);
-        epilogue_row32(pr, args.params, args.lr, row, n0 + c * 32, v);
+      for (int ch = 0; ch < n_chunks; ++ch, ++g) {
+        const uint32_t b = g % EPI_BUFS;
+        const uint32_t buf = epi_base + b * EPI_BUF_BYTES;
+        const int col0 = n0 + ch * 64;
+        if (leader) {
+          // buffer (g+1)%3 was last stored from two chunks ago: at most the latest store may be pending
+          bulk_wait_read<1>();
+          const GemmProblem* npr = nullptr;
+          int nrow0 = 0, ncol0 = 0;
+          if (ch + 1 < n_chunks) { npr = &pr; nrow0 = row0; ncol0 = col0 + 64; }
+          else if (t + 1 < tile_end) {
+            const TileEntry ne = args.tiles[t + 1];
+            npr = &args.problems[ne.problem]; nrow0 = ne.tm * GEMM_BM; ncol0 = ne.tn * BN;
+          }
+          if (npr && npr->tma_c) {
+            const uint32_t nb = (g + 1) % EPI_BUFS;
+            epi_issue_c_load(args, *npr, nrow0, ncol0, epi_base + nb * EPI_BUF_BYTES, smem_u32(&c_full_bar[nb]));
+            // this chunk's own load (if any) flips bit b before the next one is waited on
+            pending_bar = smem_u32(&c_full_bar[nb]);
+            pending_par = ((c_phase ^ (tma_c ? (1u << b) : 0u)) >> nb) & 1u;
+          }
+        }
+        __syncwarp();
+        epi_bar_sync();                          // the buffer of this chunk is free for everyone from here
+        float v[64];
+        tc_ld64(taddr + ch * 64, v);
+        bool c_ok = true;                        // folded into the barrier below: nobody leaves the chunk early
+        if (tma_c) {
+          c_ok = mbar_wait(smem_u32(&c_full_bar[b]), (c_phase >> b) & 1u, abort_flag, args.status);
+          c_phase ^= 1u << b;
+        }
+        if (pr.epi == EPI_GRAM) {
+          const float f = -0.5f * scale;
+#pragma unroll
+          for (int j = 0; j < 64; ++j) v[j] *= f;
+        } else if (tma_c) {
+          if (pr.c_mode == C_F32) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+#pragma unroll
+              for (int c16 = 0; c16 < 8; ++c16) {
+                const uint4 u = lds128(buf + h * EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4));
+                float* o = v + h * 32 + c16 * 4;
+                o[0] = scale * fmaf(1.5f, __uint_as_float(u.x), o[0]);
+                o[1] = scale * fmaf(1.5f, __uint_as_float(u.y), o[1]);
+                o[2] = scale * fmaf(1.5f, __uint_as_float(u.z), o[2]);
+                o[3] = scale * fmaf(1.5f, __uint_as_float(u.w), o[3]);
+              }
+            }
+          } else {
+            const bool has_lo = pr.c_mode == C_HILO;
+#pragma unroll
+            for (int c16 = 0; c16 < 8; ++c16) {
+              const uint4 uh = lds128(buf + row_off + ((c16 ^ sw) << 4));
+              uint4 ul = make_uint4(0, 0, 0, 0);
+              if (has_lo) ul = lds128(buf + EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4));
+              const uint32_t wh[4] = {uh.x, uh.y, uh.z, uh.w};
+              const uint32_t wl[4] = {ul.x, ul.y, ul.z, ul.w};
+              float* o = v + c16 * 8;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float c0 = __uint_as_float(wh[e] << 16) + __uint_as_float(wl[e] << 16);
+                const float c1 = __uint_as_float(wh[e] & 0xffff0000u) + __uint_as_float(wl[e] & 0xffff0000u);
+                o[2 * e] = scale * fmaf(1.5f, c0, o[2 * e]);
+                o[2 * e + 1] = scale * fmaf(1.5f, c1, o[2 * e + 1]);
+              }
+            }
+          }
+        } else {
+          apply_c_direct(pr, scale, row, col0, v);
+          apply_c_direct(pr, scale, row, col0 + 32, v + 32);
+        }
+        // ---- outputs
+        const bool store_hi = pr.epi == EPI_GRAM || pr.epi == EPI_APPLY || (pr.epi == EPI_APPLY_PACK && pr.store_out);
+        const bool store_lo = pr.epi == EPI_APPLY;
+        if (store_hi) {
+          if (tma_out) {
+#pragma unroll
+            for (int c16 = 0; c16 < 8; ++c16) {
+              const float* o = v + c16 * 8;
+              uint32_t wh[4], wl[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                wh[e] = pack_bf16x2(o[2 * e], o[2 * e + 1]);
+                wl[e] = pack_bf16x2(o[2 * e] - __uint_as_float(wh[e] << 16),
+                                    o[2 * e + 1] - __uint_as_float(wh[e] & 0xffff0000u));
+              }
+              sts128(buf + row_off + ((c16 ^ sw) << 4), make_uint4(wh[0], wh[1], wh[2], wh[3]));
+              if (store_lo) sts128(buf + EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4), make_uint4(wl[0], wl[1], wl[2], wl[3]));
+            }
+            fence_async_smem();
+          } else {
+            store_out_direct(pr, row, col0, v, store_lo);
+            store_out_direct(pr, row, col0 + 32, v + 32, store_lo);
+          }
+        }
+        if (pr.epi == EPI_APPLY_PACK) {
+          pack_bits_direct(pr, row, col0, v);
+          pack_bits_direct(pr, row, col0 + 32, v + 32);
+        } else if (pr.epi == EPI_APPLY_UPDATE) {
+          update_weights_direct(pr, args.params, args.lr, row, col0, v);
+          update_weights_direct(pr, args.params, args.lr, row, col0 + 32, v + 32);
+        }
+        ok = epi_bar_and(c_ok);                  // every thread's part of the chunk is in shared memory
+        if (!ok) break;
+        if (leader) {
+          if (store_hi && tma_out) {
+            tma_store_3d(args.tmaps + pr.tmapO0, col0, row0, pr.batch_o, buf);
+            if (store_lo) tma_store_3d(args.tmaps + pr.tmapO1, col0, row0, pr.batch_o, buf + EPI_HALF_BYTES);
+          }
+          bulk_commit();                         // one group per chunk (possibly empty) keeps the ring arithmetic fixed
+        }
+        __syncwarp();
       }
+      if (!ok) break;
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+    }
+    if (leader) {
+      if (!ok && pending_bar) {                  // abort path: let a prefetch in flight land (bounded)
+        uint32_t spins = 0;
+        while (!mbar_try_wait(pending_bar, pending_par) && ++spins < (1u << 22)) {}
+      }
+      bulk_wait_all();                           // stores must be complete before the CTA retires
     }
   }
 
@@ -319,9 +516,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
   }
 }
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, int EPI_BUFS>
 constexpr size_t ns_gemm_tc_smem_bytes() {
-  return (size_t)STAGES * (GEMM_BM * GEMM_BK * 2 + BN * GEMM_BK * 2) + 1024;
+  return (size_t)STAGES * (GEMM_BM * GEMM_BK * 2 + BN * GEMM_BK * 2) + (size_t)EPI_BUFS * EPI_BUF_BYTES + 1024;
 }
 
 }  // namespace signmuon

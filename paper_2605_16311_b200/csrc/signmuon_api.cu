@@ -36,12 +36,13 @@ struct ParamPlan {
   bool fused_pack;       // sign+pack happens in the last apply epilogue
   size_t mom_off;        // bytes into the state buffer
   size_t y_off[2], lo_off, q_off, scales_off, partials_off;   // bytes into the workspace (matrix params)
-  int tmap_base;         // first of this parameter's 8 tensor maps
+  int tmap_base;         // first of this parameter's TM_PER_PARAM tensor maps
   size_t stage_w_off, stage_g_off;                    // bytes into the host-staging buffer
 };
 
 // indices of a parameter's tensor maps relative to tmap_base
-enum { TM_Y0_K128 = 0, TM_Y0_KBN, TM_Y0_MN, TM_Y1_K128, TM_Y1_KBN, TM_Y1_MN, TM_Q_K128, TM_Q_KBN, TM_PER_PARAM };
+enum { TM_Y0_K128 = 0, TM_Y0_KBN, TM_Y0_MN, TM_Y1_K128, TM_Y1_KBN, TM_Y1_MN, TM_Q_K128, TM_Q_KBN, TM_LO_K128, TM_MOM_F32,
+       TM_PER_PARAM };
 
 struct LaunchPlan {        // one grouped GEMM launch
   size_t problem_base;     // index of its first problem in the problem array
@@ -174,6 +175,7 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         pr.epi = EPI_GRAM;
         pr.out = reinterpret_cast<void*>(q);
         pr.ld_out = pl.ldq;
+        pr.tma_out = 1; pr.tmapO0 = pl.tmap_base + TM_Q_K128; pr.batch_o = m;
         if (k == 0) {
           if (local_polar_phase) pr.scale_imm = (float)(1.0 / ((double)pl.rows * (double)pl.cols));
           else pr.scale_ptr = reinterpret_cast<const float*>(pl.scales_off + (size_t)m * 8);
@@ -205,6 +207,20 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         pr.out = reinterpret_cast<void*>(ydst);
         pr.out_lo = reinterpret_cast<bf16*>(lo);
         pr.ld_out = pl.ldy;
+        // TMA-staged epilogue: possible whenever the row pitches are multiples of 16 bytes
+        pr.tma_out = 1;
+        pr.tmapO0 = pl.tmap_base + (dst ? TM_Y1_K128 : TM_Y0_K128);
+        pr.tmapO1 = pl.tmap_base + TM_LO_K128;
+        pr.batch_o = m;
+        pr.batch_c = m;
+        if (pr.c_mode == C_F32) {
+          pr.tma_c = (pl.cols % 4 == 0) ? 1 : 0;
+          pr.tmapC0 = pl.tmap_base + TM_MOM_F32;
+        } else {
+          pr.tma_c = 1;
+          pr.tmapC0 = pl.tmap_base + ty;
+          pr.tmapC1 = pl.tmap_base + TM_LO_K128;
+        }
         if (k == 0) {
           if (local_polar_phase) pr.scale_imm = (float)(1.0 / std::sqrt((double)pl.rows * (double)pl.cols));
           else pr.scale_ptr = reinterpret_cast<const float*>(pl.scales_off + (size_t)m * 8 + 4);
@@ -374,14 +390,16 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
 
 // 3-D bf16 tensor {inner, rows, batch} with a {64, box_rows, 1} box and 128-byte swizzle.
 bool encode_map(CUtensorMap* map, void* base, uint64_t inner, uint64_t rows, uint64_t batch, uint64_t pitch_elems,
-                uint64_t batch_elems, uint32_t box_rows) {
+                uint64_t batch_elems, uint32_t box_rows, bool f32 = false) {
   PFN_cuTensorMapEncodeTiled_v12000 fn = get_encode_fn();
   if (!fn) return false;
+  const uint64_t es = f32 ? 4 : 2;
   cuuint64_t gdim[3] = {inner, rows, batch};
-  cuuint64_t gstr[2] = {pitch_elems * 2, batch_elems * 2};
-  cuuint32_t box[3] = {64, box_rows, 1};
+  cuuint64_t gstr[2] = {pitch_elems * es, batch_elems * es};
+  cuuint32_t box[3] = {f32 ? 32u : 64u, box_rows, 1};     // 128 bytes wide either way
   cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+  return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -391,15 +409,16 @@ int check_launch(signmuon_ctx* c) {
   return c->sticky;
 }
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, int EPI_BUFS>
 void launch_tc(const GemmLaunchArgs& a, int grid, cudaStream_t s) {
-  static bool configured = false;
-  constexpr size_t smem = ns_gemm_tc_smem_bytes<BN, STAGES>();
-  if (!configured) {
-    cudaFuncSetAttribute(ns_gemm_tc_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    configured = true;
-  }
-  ns_gemm_tc_kernel<BN, STAGES><<<grid, GEMM_THREADS, smem, s>>>(a);
+  constexpr size_t smem = ns_gemm_tc_smem_bytes<BN, STAGES, EPI_BUFS>();
+  ns_gemm_tc_kernel<BN, STAGES, EPI_BUFS><<<grid, GEMM_THREADS, smem, s>>>(a);
+}
+
+// Opt in to the large dynamic shared memory of the tensor-core kernel (per device, at bind).
+bool configure_kernels() {
+  return cudaFuncSetAttribute(ns_gemm_tc_kernel<128, 4, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)ns_gemm_tc_smem_bytes<128, 4, 3>()) == cudaSuccess;
 }
 
 void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s) {
@@ -420,8 +439,7 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
   a.params = pd;
   a.status = reinterpret_cast<uint32_t*>(c->d_ws + c->off_status);
   a.lr = lr;
-  if (tt.bn == 256) launch_tc<256, 4>(a, tt.grid, s);
-  else launch_tc<128, 6>(a, tt.grid, s);
+  launch_tc<128, 4, 3>(a, tt.grid, s);
 }
 
 template <int PLANES>
@@ -629,6 +647,7 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     ok = ok && up(tt.tiles_off, tt.tiles.data(), tt.tiles.size() * sizeof(TileEntry));
     ok = ok && up(tt.cta_off, tt.cta_start.data(), tt.cta_start.size() * 4);
   }
+  ok = ok && configure_kernels();
   std::vector<CUtensorMap> maps((size_t)c->num_tmaps);
   const bool need_maps = !(c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) && c->cfg.ns_steps > 0;
   if (need_maps) {
@@ -648,6 +667,11 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
       const uint64_t qb = (uint64_t)pl.s * pl.ldq;
       ok = ok && encode_map(mp + TM_Q_K128, q, pl.s, pl.s, slots, pl.ldq, qb, 128);
       ok = ok && encode_map(mp + TM_Q_KBN, q, pl.s, pl.s, slots, pl.ldq, qb, bn);
+      ok = ok && encode_map(mp + TM_LO_K128, c->d_ws + pl.lo_off, pl.cols, pl.rows, slots, pl.ldy,
+                            (uint64_t)pl.rows * pl.ldy, 128);
+      if (pl.cols % 4 == 0)   // float32 momentum as the first iteration's C operand
+        ok = ok && encode_map(mp + TM_MOM_F32, c->d_state + pl.mom_off, pl.cols, pl.rows, M, pl.cols, (uint64_t)pl.d, 128,
+                              true);
     }
     if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
     ok = ok && up(c->off_tmaps, maps.data(), maps.size() * sizeof(CUtensorMap));
