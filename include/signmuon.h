@@ -92,8 +92,10 @@ typedef struct {
 
 enum {
   SIGNMUON_FLAG_KEEP_POLAR = 1,   /* also store U_m = Y_K (bf16) so that signmuon_debug_tap can return it */
-  SIGNMUON_FLAG_SIMT_GEMM = 2     /* diagnostic: run the Newton-Schulz products on a plain CUDA-core
+  SIGNMUON_FLAG_SIMT_GEMM = 2,    /* diagnostic: run the Newton-Schulz products on a plain CUDA-core
                                      kernel instead of the tensor-core kernel (slow; for fault isolation) */
+  SIGNMUON_FLAG_GEMM_1CTA = 4     /* run the tensor-core kernel with one CTA per 128 x 128 tile instead of
+                                     CTA pairs on 256 x 256 tiles (same results; for comparison) */
 };
 
 /* Stages of one step, for signmuon_run_stages (bit mask). A full step is all of them in this order. */

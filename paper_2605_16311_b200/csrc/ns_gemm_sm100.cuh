@@ -7,7 +7,19 @@
 //   - epilogue warps read TMEM with tcgen05.ld and apply the fused Newton-Schulz epilogues
 //     (Gram scaling, 1.5 Y + Q Y, sign + pack, weight update).
 // One launch covers every (parameter, worker) product of one Newton-Schulz half-iteration: each
-// CTA walks a host-built list of tiles (problem, tile_m, tile_n).
+// CTA (or CTA pair) walks a host-built list of tiles (problem, tile_m, tile_n).
+//
+// Two shapes of the same kernel (template parameter CTAS):
+//   CTAS = 1: one CTA per 128 x BN tile, tcgen05.mma.cta_group::1.
+//   CTAS = 2: a cluster of two CTAs on neighbouring SMs shares a 256 x BN tile (cta_group::2): CTA r
+//             stages rows [128 r, 128 r + 128) of A and columns [BN/2 r, BN/2 (r+1)) of B, the MMA is
+//             issued by CTA 0 alone and reads both shared memories, and each CTA keeps and drains the
+//             accumulator of its own 128 rows.  Per flop this halves the operand bytes every SM has
+//             to pull from L2, which is what bounds the 128 x 128 shape.  Barriers that cross the
+//             pair: the "stage full" barrier lives in CTA 0 and counts the TMA bytes of both CTAs;
+//             "stage empty" and "accumulator full" are signalled in both CTAs by a multicast
+//             tcgen05.commit; "accumulator empty" lives in CTA 0 and collects the epilogue warps of both.
+//             No TMA load uses cluster multicast.
 //
 // Operand layouts in shared memory (one 64-wide K block per stage):
 //   K-major  (contiguous along K):  rows of 128 bytes, TMA box {64 k, R rows}, 8-row swizzle atoms
@@ -101,6 +113,34 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// Same load inside a CTA pair: the completion bytes may be credited to a barrier of the peer CTA.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
+                                                 uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar_cluster_addr)
+      : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// Barrier over every thread of every CTA of the cluster (all threads of a warp must arrive together).
+__device__ __forceinline__ void cluster_sync_all() {
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -115,6 +155,22 @@ __device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint
 }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// CTA-pair forms: the MMA spans both CTAs; the commit arrives on the barrier at the same offset in both.
+__device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask)
+               : "memory");
 }
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, int x, int y, int z, uint32_t src) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
@@ -177,8 +233,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 }
 
 // Instruction descriptor, kind::f16: D fp32 (bits [4,6) = 1), A/B bf16 (bits [7,10) = [10,13) = 1),
-// bit 15 / 16: A / B contiguous along M / N, bits [17,23) N >> 3, bits [24,29) M >> 4.
-__device__ __forceinline__ uint32_t instr_desc(int n, int a_mn, int b_mn) {
+// bit 15 / 16: A / B contiguous along M / N, bits [17,23) N >> 3, bits [24,29) M >> 4
+// (M = 128 for one CTA, 256 for a CTA pair).
+__device__ __forceinline__ uint32_t instr_desc(int m, int n, int a_mn, int b_mn) {
   uint32_t d = 0;
   d |= 1u << 4;
   d |= 1u << 7;
@@ -186,7 +243,7 @@ __device__ __forceinline__ uint32_t instr_desc(int n, int a_mn, int b_mn) {
   d |= (uint32_t)(a_mn & 1) << 15;
   d |= (uint32_t)(b_mn & 1) << 16;
   d |= (uint32_t)(n >> 3) << 17;
-  d |= (uint32_t)(GEMM_BM >> 4) << 24;
+  d |= (uint32_t)(m >> 4) << 24;
   return d;
 }
 
@@ -211,12 +268,16 @@ __device__ __forceinline__ void epi_issue_c_load(const GemmLaunchArgs& args, con
   }
 }
 
-template <int BN, int STAGES, int EPI_BUFS>
+template <int BN, int STAGES, int EPI_BUFS, int CTAS>
 __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmLaunchArgs args) {
+  constexpr int B_ROWS = BN / CTAS;                            // rows of the B operand this CTA stages
+  constexpr int TILE_M = GEMM_BM * CTAS;                       // rows of the output tile of the CTA (pair)
   constexpr uint32_t A_BYTES = GEMM_BM * GEMM_BK * 2;          // 16 KB
-  constexpr uint32_t B_BYTES = BN * GEMM_BK * 2;
+  constexpr uint32_t B_BYTES = B_ROWS * GEMM_BK * 2;
   constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
   constexpr uint32_t TMEM_COLS = 2 * BN;                       // two accumulator buffers
+  static_assert(CTAS == 1 || CTAS == 2, "one CTA or a CTA pair");
+  static_assert(B_ROWS % 64 == 0, "B rows per CTA: whole 64-row chunks");
   static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM columns: power of two");
   static_assert(EPI_BUFS == 3, "the chunk ring is written for three buffers");
 
@@ -234,6 +295,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   volatile uint32_t* abort_flag = &abort_word;
+  const uint32_t cta_rank = (CTAS == 2) ? cluster_cta_rank() : 0u;     // 0 issues the MMAs of the pair
+  const uint32_t work_id = (CTAS == 2) ? (blockIdx.x >> 1) : blockIdx.x;
 
   if (threadIdx.x == 0) {
     abort_word = 0;
@@ -243,24 +306,38 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&tmem_full_bar[a]), 1);
-      mbar_init(smem_u32(&tmem_empty_bar[a]), 4);
+      mbar_init(smem_u32(&tmem_empty_bar[a]), 4 * CTAS);
     }
     for (int b = 0; b < EPI_BUFS; ++b) mbar_init(smem_u32(&c_full_bar[b]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
-                 "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CTAS == 2) {   // the same warp of both CTAs allocates the pair's columns
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync_all();   // the peer's barriers are initialised before anything signals them
+  else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_slot;
 
-  const uint32_t tile_begin = args.cta_tile_start[blockIdx.x];
-  const uint32_t tile_end = args.cta_tile_start[blockIdx.x + 1];
+  const uint32_t tile_begin = args.cta_tile_start[work_id];
+  const uint32_t tile_end = args.cta_tile_start[work_id + 1];
+
+  auto load_operand = [&](uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+    if (CTAS == 2) tma_load_3d_pair(dst, map, x, y, z, bar);
+    else tma_load_3d(dst, map, x, y, z, bar);
+  };
+  const int row_shift = (int)cta_rank * GEMM_BM;   // this CTA's rows inside the tile of the pair
 
   if (warp == 0) {
     // ===================================================================== TMA producer
@@ -272,45 +349,54 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         const GemmProblem& pr = args.problems[te.problem];
         const CUtensorMap* mapA = args.tmaps + pr.tmapA;
         const CUtensorMap* mapB = args.tmaps + pr.tmapB;
-        const int m0 = te.tm * GEMM_BM, n0 = te.tn * BN, batch = pr.batch;
+        const int m0 = te.tm * TILE_M + (int)cta_rank * GEMM_BM;       // this CTA's rows of A
+        const int n0 = te.tn * BN + (int)cta_rank * B_ROWS;            // this CTA's rows of B
+        const int batch = pr.batch;
         const int a_mn = pr.a_mn, b_mn = pr.b_mn;
         const int nk = (pr.K + GEMM_BK - 1) / GEMM_BK;
         for (int kb = 0; kb < nk; ++kb, ++it) {
           const uint32_t s = it % STAGES;
           const uint32_t round = it / STAGES;
           if (!mbar_wait(smem_u32(&empty_bar[s]), (round & 1u) ^ 1u, abort_flag, args.status)) { ok = false; break; }
-          const uint32_t fb = smem_u32(&full_bar[s]);
-          mbar_expect_tx(fb, STAGE_BYTES);
+          // the "full" barrier of the pair is CTA 0's: it expects the bytes of both CTAs
+          const uint32_t fb = (CTAS == 2) ? map_to_cta(smem_u32(&full_bar[s]), 0) : smem_u32(&full_bar[s]);
+          if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[s]), CTAS * STAGE_BYTES);
           const uint32_t sa = smem_base + s * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
           const int k0 = kb * GEMM_BK;
           if (!a_mn) {
-            tma_load_3d(sa, mapA, k0, m0, batch, fb);
+            load_operand(sa, mapA, k0, m0, batch, fb);
           } else {
 #pragma unroll
-            for (int c = 0; c < GEMM_BM / 64; ++c) tma_load_3d(sa + c * 8192, mapA, m0 + 64 * c, k0, batch, fb);
+            for (int c = 0; c < GEMM_BM / 64; ++c) load_operand(sa + c * 8192, mapA, m0 + 64 * c, k0, batch, fb);
           }
           if (!b_mn) {
-            tma_load_3d(sb, mapB, k0, n0, batch, fb);
+            load_operand(sb, mapB, k0, n0, batch, fb);
           } else {
 #pragma unroll
-            for (int c = 0; c < BN / 64; ++c) tma_load_3d(sb + c * 8192, mapB, n0 + 64 * c, k0, batch, fb);
+            for (int c = 0; c < B_ROWS / 64; ++c) load_operand(sb + c * 8192, mapB, n0 + 64 * c, k0, batch, fb);
           }
         }
       }
       if (!ok) {
         // Abort path: let the copies already issued land before the CTA's shared memory goes away.
-        const uint32_t pending = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
-        for (uint32_t j = 0; j < pending; ++j) {
-          const uint32_t i2 = it - 1 - j;
-          uint32_t spins = 0;
-          while (!mbar_try_wait(smem_u32(&full_bar[i2 % STAGES]), (i2 / STAGES) & 1u) && ++spins < (1u << 22)) {}
+        if (cta_rank == 0) {
+          const uint32_t pending = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+          for (uint32_t j = 0; j < pending; ++j) {
+            const uint32_t i2 = it - 1 - j;
+            uint32_t spins = 0;
+            while (!mbar_try_wait(smem_u32(&full_bar[i2 % STAGES]), (i2 / STAGES) & 1u) && ++spins < (1u << 22)) {}
+          }
+        } else {
+          // the peer's barrier cannot be polled from here: give the copies a fixed 100 us
+          const uint64_t t0 = global_timer_ns();
+          while (global_timer_ns() - t0 < 100000ull) {}
         }
       }
     }
   } else if (warp == 1) {
-    // ===================================================================== MMA issuer
-    if (lane == 0) {
+    // ===================================================================== MMA issuer (CTA 0 of a pair)
+    if (lane == 0 && cta_rank == 0) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (uint32_t t = tile_begin; t < tile_end && ok; ++t, ++tcount) {
@@ -318,7 +404,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         const GemmProblem& pr = args.problems[te.problem];
         const int a_mn = pr.a_mn, b_mn = pr.b_mn;
         const int nk = (pr.K + GEMM_BK - 1) / GEMM_BK;
-        const uint32_t idesc = instr_desc(BN, a_mn, b_mn);
+        const uint32_t idesc = instr_desc(TILE_M, BN, a_mn, b_mn);
         const uint32_t acc = tcount & 1u;
         const uint32_t acc_round = tcount >> 1;
         if (!mbar_wait(smem_u32(&tmem_empty_bar[acc]), (acc_round & 1u) ^ 1u, abort_flag, args.status)) { ok = false; break; }
@@ -335,11 +421,15 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
           for (int kk = 0; kk < GEMM_BK / 16; ++kk) {
             const uint64_t adesc = a_mn ? smem_desc(sa + kk * 2048, 8192, 1024) : smem_desc(sa + kk * 32, 16, 1024);
             const uint64_t bdesc = b_mn ? smem_desc(sb + kk * 2048, 8192, 1024) : smem_desc(sb + kk * 32, 16, 1024);
-            tc_mma_f16(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
+            if (CTAS == 2) tc_mma_f16_pair(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
+            else tc_mma_f16(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
           }
-          tc_commit(smem_u32(&empty_bar[s]));        // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if (CTAS == 2) tc_commit_pair(smem_u32(&empty_bar[s])); else tc_commit(smem_u32(&empty_bar[s]));
         }
-        if (ok) tc_commit(smem_u32(&tmem_full_bar[acc]));   // accumulator complete
+        if (ok) {                                    // accumulator complete
+          if (CTAS == 2) tc_commit_pair(smem_u32(&tmem_full_bar[acc])); else tc_commit(smem_u32(&tmem_full_bar[acc]));
+        }
       }
     }
   } else {
@@ -358,8 +448,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
     if (leader && tile_begin < tile_end) {
       const TileEntry te = args.tiles[tile_begin];
       const GemmProblem& pr = args.problems[te.problem];
-      if (pr.tma_c) {
-        epi_issue_c_load(args, pr, te.tm * GEMM_BM, te.tn * BN, epi_base, smem_u32(&c_full_bar[0]));
+      if (pr.tma_c && te.tm * TILE_M + row_shift < pr.M) {
+        epi_issue_c_load(args, pr, te.tm * TILE_M + row_shift, te.tn * BN, epi_base, smem_u32(&c_full_bar[0]));
         pending_bar = smem_u32(&c_full_bar[0]); pending_par = 0;
       }
     }
@@ -372,14 +462,16 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
       ok = epi_bar_and(ok);                      // uniform over the four epilogue warps
       if (!ok) break;
       tc_fence_after();
-      const int row0 = te.tm * GEMM_BM;
+      const int row0 = te.tm * TILE_M + row_shift;
       const int row = row0 + r_in;
       const int n0 = te.tn * BN;
       const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
       int n_chunks = (pr.N - n0 + 63) / 64;
       if (n_chunks > BN / 64) n_chunks = BN / 64;
       const float scale = pr.scale_ptr ? __ldg(pr.scale_ptr) : pr.scale_imm;
-      const bool tma_c = pr.tma_c != 0, tma_out = pr.tma_out != 0;
+      // a CTA whose 128 rows lie wholly below the matrix moves nothing through TMA (it still drains TMEM)
+      const bool rows_live = row0 < pr.M;
+      const bool tma_c = pr.tma_c != 0 && rows_live, tma_out = pr.tma_out != 0;
 #pragma unroll 1
       for (int ch = 0; ch < n_chunks; ++ch, ++g) {
         const uint32_t b = g % EPI_BUFS;
@@ -393,9 +485,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
           if (ch + 1 < n_chunks) { npr = &pr; nrow0 = row0; ncol0 = col0 + 64; }
           else if (t + 1 < tile_end) {
             const TileEntry ne = args.tiles[t + 1];
-            npr = &args.problems[ne.problem]; nrow0 = ne.tm * GEMM_BM; ncol0 = ne.tn * BN;
+            npr = &args.problems[ne.problem]; nrow0 = ne.tm * TILE_M + row_shift; ncol0 = ne.tn * BN;
           }
-          if (npr && npr->tma_c) {
+          if (npr && npr->tma_c && nrow0 < npr->M) {
             const uint32_t nb = (g + 1) % EPI_BUFS;
             epi_issue_c_load(args, *npr, nrow0, ncol0, epi_base + nb * EPI_BUF_BYTES, smem_u32(&c_full_bar[nb]));
             // this chunk's own load (if any) flips bit b before the next one is waited on
@@ -487,7 +579,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         ok = epi_bar_and(c_ok);                  // every thread's part of the chunk is in shared memory
         if (!ok) break;
         if (leader) {
-          if (store_hi && tma_out) {
+          if (store_hi && tma_out && rows_live) {
             tma_store_3d(args.tmaps + pr.tmapO0, col0, row0, pr.batch_o, buf);
             if (store_lo) tma_store_3d(args.tmaps + pr.tmapO1, col0, row0, pr.batch_o, buf + EPI_HALF_BYTES);
           }
@@ -498,7 +590,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
       if (!ok) break;
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+      if (lane == 0) {                           // the accumulator may be overwritten (barrier of CTA 0)
+        if (CTAS == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
+        else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+      }
     }
     if (leader) {
       if (!ok && pending_bar) {                  // abort path: let a prefetch in flight land (bounded)
@@ -510,15 +605,21 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
   }
 
   tc_fence_before();
-  __syncthreads();
-  if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  if (CTAS == 2) {
+    // neither CTA may retire (or free TMEM) while the peer can still signal its barriers or read its operands
+    cluster_sync_all();
+    if (warp == 1)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  } else {
+    __syncthreads();
+    if (warp == 1)
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
-template <int BN, int STAGES, int EPI_BUFS>
+template <int BN, int STAGES, int EPI_BUFS, int CTAS>
 constexpr size_t ns_gemm_tc_smem_bytes() {
-  return (size_t)STAGES * (GEMM_BM * GEMM_BK * 2 + BN * GEMM_BK * 2) + (size_t)EPI_BUFS * EPI_BUF_BYTES + 1024;
+  return (size_t)STAGES * (GEMM_BM * GEMM_BK * 2 + (BN / CTAS) * GEMM_BK * 2) + (size_t)EPI_BUFS * EPI_BUF_BYTES + 1024;
 }
 
 }  // namespace signmuon

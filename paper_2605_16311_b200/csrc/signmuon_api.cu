@@ -52,8 +52,9 @@ struct LaunchPlan {        // one grouped GEMM launch
 struct TileTable {
   std::vector<TileEntry> tiles;         // ordered by CTA
   std::vector<uint32_t> cta_start;      // [grid + 1]
-  int grid = 0;
-  int bn = 128;
+  int grid = 0;            // number of tile lists = CTAs (one-CTA kernel) or CTA pairs
+  int bm = 128, bn = 128;  // tile shape
+  int ctas = 1;            // CTAs that share a tile
   size_t tiles_off = 0, cta_off = 0;    // bytes into the workspace
 };
 
@@ -98,18 +99,18 @@ size_t dtype_size(int32_t t) { return t == SIGNMUON_F32 ? 4 : 2; }
 // ------------------------------------------------------------------ tile scheduling (host)
 // Longest-processing-time-first assignment of tiles to `grid` persistent CTAs; cost = K blocks
 // of the main loop plus a constant for the epilogue.
-void build_tile_table(TileTable& tt, const std::vector<GemmProblem>& probs, size_t pbase, size_t pcount, int bn,
+void build_tile_table(TileTable& tt, const std::vector<GemmProblem>& probs, size_t pbase, size_t pcount,
                       int grid_limit) {
+  const int bm = tt.bm, bn = tt.bn;
   struct T { TileEntry e; int cost; };
   std::vector<T> all;
   for (size_t i = 0; i < pcount; ++i) {
     const GemmProblem& pr = probs[pbase + i];
-    const int tm = (pr.M + GEMM_BM - 1) / GEMM_BM, tn = (pr.N + bn - 1) / bn;
+    const int tm = (pr.M + bm - 1) / bm, tn = (pr.N + bn - 1) / bn;
     const int cost = (pr.K + GEMM_BK - 1) / GEMM_BK + 2;
     for (int a = 0; a < tm; ++a)
       for (int b = 0; b < tn; ++b) all.push_back({{(uint32_t)i, (uint16_t)a, (uint16_t)b}, cost});
   }
-  tt.bn = bn;
   tt.grid = (int)std::min<size_t>((size_t)grid_limit, std::max<size_t>(all.size(), 1));
   std::stable_sort(all.begin(), all.end(), [](const T& x, const T& y) { return x.cost > y.cost; });
   std::vector<std::vector<TileEntry>> per(tt.grid);
@@ -131,11 +132,11 @@ void build_tile_table(TileTable& tt, const std::vector<GemmProblem>& probs, size
   tt.cta_start[tt.grid] = (uint32_t)tt.tiles.size();
 }
 
-size_t count_tiles(const std::vector<GemmProblem>& probs, size_t pbase, size_t pcount, int bn) {
+size_t count_tiles(const std::vector<GemmProblem>& probs, size_t pbase, size_t pcount, int bm, int bn) {
   size_t n = 0;
   for (size_t i = 0; i < pcount; ++i) {
     const GemmProblem& pr = probs[pbase + i];
-    n += (size_t)((pr.M + GEMM_BM - 1) / GEMM_BM) * ((pr.N + bn - 1) / bn);
+    n += (size_t)((pr.M + bm - 1) / bm) * ((pr.N + bn - 1) / bn);
   }
   return n;
 }
@@ -355,11 +356,14 @@ int plan_layout(signmuon_ctx* c) {
   const size_t nm = c->matrix_list.size();
   for (int t = 0; t < 4; ++t) {
     TileTable& tt = c->tables[t];
-    tt.bn = 128;
+    const bool pair = !(c->cfg.flags & (SIGNMUON_FLAG_GEMM_1CTA | SIGNMUON_FLAG_SIMT_GEMM));
+    tt.ctas = pair ? 2 : 1;
+    tt.bm = pair ? 256 : 128;
+    tt.bn = pair ? 256 : 128;
     size_t ntiles = 0;
     const std::vector<LaunchPlan>& ls = (t < 2) ? c->ns_launches : c->lp_launches;
     const size_t per = (t < 2) ? nm * M : nm;
-    if (!ls.empty()) ntiles = count_tiles(c->problems, ls[t & 1].problem_base, per, tt.bn);
+    if (!ls.empty()) ntiles = count_tiles(c->problems, ls[t & 1].problem_base, per, tt.bm, tt.bn);
     tt.tiles_off = off; off += round_up(std::max<size_t>(ntiles, 1) * sizeof(TileEntry), ALIGN);
     tt.cta_off = off; off += round_up((MAX_CTAS + 1) * 4, ALIGN);
   }
@@ -409,16 +413,54 @@ int check_launch(signmuon_ctx* c) {
   return c->sticky;
 }
 
-template <int BN, int STAGES, int EPI_BUFS>
-void launch_tc(const GemmLaunchArgs& a, int grid, cudaStream_t s) {
-  constexpr size_t smem = ns_gemm_tc_smem_bytes<BN, STAGES, EPI_BUFS>();
-  ns_gemm_tc_kernel<BN, STAGES, EPI_BUFS><<<grid, GEMM_THREADS, smem, s>>>(a);
+// One-CTA tiles: `lists` CTAs.  CTA pairs: a cluster of two CTAs per tile list.
+template <int BN, int STAGES, int EPI_BUFS, int CTAS>
+void launch_tc(const GemmLaunchArgs& a, int lists, cudaStream_t s) {
+  constexpr size_t smem = ns_gemm_tc_smem_bytes<BN, STAGES, EPI_BUFS, CTAS>();
+  if (CTAS == 1) {
+    ns_gemm_tc_kernel<BN, STAGES, EPI_BUFS, CTAS><<<lists, GEMM_THREADS, smem, s>>>(a);
+    return;
+  }
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)lists * CTAS, 1, 1);
+  cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = CTAS;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, ns_gemm_tc_kernel<BN, STAGES, EPI_BUFS, CTAS>, a);
 }
 
-// Opt in to the large dynamic shared memory of the tensor-core kernel (per device, at bind).
-bool configure_kernels() {
-  return cudaFuncSetAttribute(ns_gemm_tc_kernel<128, 4, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)ns_gemm_tc_smem_bytes<128, 4, 3>()) == cudaSuccess;
+// Opt in to the large dynamic shared memory of the tensor-core kernels (per device, at bind) and ask how
+// many CTA pairs the device can hold at once.
+bool configure_kernels(int* max_pairs) {
+  bool ok = cudaFuncSetAttribute(ns_gemm_tc_kernel<128, 4, 3, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)ns_gemm_tc_smem_bytes<128, 4, 3, 1>()) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(ns_gemm_tc_kernel<256, 4, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)ns_gemm_tc_smem_bytes<256, 4, 3, 2>()) == cudaSuccess;
+  if (!ok) return false;
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(2, 1, 1);
+  cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = ns_gemm_tc_smem_bytes<256, 4, 3, 2>();
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, ns_gemm_tc_kernel<256, 4, 3, 2>, &cfg) != cudaSuccess || n < 1) return false;
+  *max_pairs = n;
+  return true;
 }
 
 void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s) {
@@ -439,7 +481,8 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
   a.params = pd;
   a.status = reinterpret_cast<uint32_t*>(c->d_ws + c->off_status);
   a.lr = lr;
-  launch_tc<128, 4, 3>(a, tt.grid, s);
+  if (tt.ctas == 2) launch_tc<256, 4, 3, 2>(a, tt.grid, s);
+  else launch_tc<128, 4, 3, 1>(a, tt.grid, s);
 }
 
 template <int PLANES>
@@ -638,16 +681,20 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
 
   // tile tables (need the SM count) and tensor maps (need the device addresses)
   const size_t nm = c->matrix_list.size();
+  int max_pairs = 1;
+  if (!configure_kernels(&max_pairs)) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+  max_pairs = std::min(max_pairs, MAX_CTAS);
   for (int t = 0; t < 4; ++t) {
     TileTable& tt = c->tables[t];
     const std::vector<LaunchPlan>& ls = (t < 2) ? c->ns_launches : c->lp_launches;
     tt.tiles.clear();
     if (ls.empty()) continue;
-    build_tile_table(tt, c->problems, ls[t & 1].problem_base, (t < 2) ? nm * M : nm, tt.bn, c->num_sms);
+    build_tile_table(tt, c->problems, ls[t & 1].problem_base, (t < 2) ? nm * M : nm,
+                     tt.ctas == 2 ? max_pairs : c->num_sms);
     ok = ok && up(tt.tiles_off, tt.tiles.data(), tt.tiles.size() * sizeof(TileEntry));
     ok = ok && up(tt.cta_off, tt.cta_start.data(), tt.cta_start.size() * 4);
   }
-  ok = ok && configure_kernels();
+  // (moved up) kernels configured before the tile tables are split
   std::vector<CUtensorMap> maps((size_t)c->num_tmaps);
   const bool need_maps = !(c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) && c->cfg.ns_steps > 0;
   if (need_maps) {

@@ -32,6 +32,14 @@ def test_config1_simt_diagnostic_path():
     assert rep["sign_match_min"] >= 0.999
 
 
+def test_one_cta_tile_variant_ragged_and_local_polar():
+    """The 128 x 128 one-CTA shape of the tensor-core kernel (the default is CTA pairs on 256 x 256 tiles)."""
+    from parity_utils import run_and_check
+    flags = B.FLAG_KEEP_POLAR | B.FLAG_GEMM_1CTA
+    run_and_check(_wl([(200, 328), (328, 200), (64, 147), (512, 640)], 3), steps=2, flags=flags)
+    run_and_check(_wl([(200, 328), (328, 200), (256, 256)], 2, local_polar=True, lr=0.01), steps=1, flags=flags)
+
+
 def test_config1_ten_steps():
     from parity_utils import run_and_check
     rep = run_and_check(wlmod.config1(), steps=10)
