@@ -268,7 +268,7 @@ __device__ __forceinline__ void epi_issue_c_load(const GemmLaunchArgs& args, con
   }
 }
 
-template <int BN, int STAGES, int EPI_BUFS, int CTAS>
+template <int BN, int STAGES, int EPI_BUFS, int CTAS, int KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmLaunchArgs args) {
   constexpr int B_ROWS = BN / CTAS;                            // rows of the B operand this CTA stages
   constexpr int TILE_M = GEMM_BM * CTAS;                       // rows of the output tile of the CTA (pair)
@@ -276,10 +276,14 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
   constexpr uint32_t B_BYTES = B_ROWS * GEMM_BK * 2;
   constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
   constexpr uint32_t TMEM_COLS = 2 * BN;                       // two accumulator buffers
+  // KIND 0: a launch of Gram products only (no C operand, bf16 output: ring buffers of one half);
+  // KIND 1: a launch of apply products (C operand, hi/lo output, pack or weight update).
+  constexpr uint32_t BUF_BYTES = (KIND == 0) ? EPI_HALF_BYTES : EPI_BUF_BYTES;
+  static_assert(KIND == 0 || KIND == 1, "Gram or apply launch");
   static_assert(CTAS == 1 || CTAS == 2, "one CTA or a CTA pair");
   static_assert(B_ROWS % 64 == 0, "B rows per CTA: whole 64-row chunks");
   static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM columns: power of two");
-  static_assert(EPI_BUFS == 3, "the chunk ring is written for three buffers");
+  static_assert(EPI_BUFS >= 2 && EPI_BUFS <= 8, "chunk ring: 2 to 8 buffers (2 = no prefetch of C)");
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[STAGES];
@@ -434,6 +438,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
     }
   } else {
     // ===================================================================== epilogue (warps 2..5)
+    // Chunks (64 output columns of this CTA's 128 rows) are numbered g = 0, 1, ... across the CTA's tiles;
+    // chunk g lives in ring buffer g % EPI_BUFS: its C operand lands there by TMA, the results overwrite it
+    // in place and leave by a TMA store.  The leader thread runs a cursor PREFETCH chunks ahead of the
+    // chunk being computed and issues the C loads from there, so that PREFETCH loads are in flight while
+    // one chunk is computed and the previous one drains.
+    constexpr uint32_t PREFETCH = EPI_BUFS - 2;
     const int q = warp & 3;                      // TMEM lane quarter this warp may read
     const bool leader = (threadIdx.x == 64);     // issues the chunk loads and stores
     const int r_in = q * 32 + lane;              // row of the tile this thread owns
@@ -441,18 +451,39 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
     const uint32_t sw = (uint32_t)(r_in & 7);
     uint32_t g = 0;                              // running chunk counter (ring position)
     uint32_t c_phase = 0;                        // bit b: parity of the next C load landing in buffer b
-    uint32_t pending_bar = 0, pending_par = 0;   // leader: the prefetch in flight (for the abort path)
     uint32_t tcount = 0;
     bool ok = true;
-    // first chunk of the first tile
-    if (leader && tile_begin < tile_end) {
-      const TileEntry te = args.tiles[tile_begin];
-      const GemmProblem& pr = args.problems[te.problem];
-      if (pr.tma_c && te.tm * TILE_M + row_shift < pr.M) {
-        epi_issue_c_load(args, pr, te.tm * TILE_M + row_shift, te.tn * BN, epi_base, smem_u32(&c_full_bar[0]));
-        pending_bar = smem_u32(&c_full_bar[0]); pending_par = 0;
+    // ---- leader's prefetch cursor
+    uint32_t pf_t = tile_begin;                  // tile of the next chunk to prefetch
+    int pf_ch = 0, pf_n = 0, pf_row0 = 0, pf_n0 = 0;
+    const GemmProblem* pf_pr = nullptr;
+    bool pf_live = false;
+    uint32_t pf_issued = 0;                      // loads issued so far (for the abort path)
+    auto pf_enter_tile = [&]() {
+      if (pf_t >= tile_end) return;
+      const TileEntry te = args.tiles[pf_t];
+      pf_pr = &args.problems[te.problem];
+      pf_row0 = te.tm * TILE_M + row_shift;
+      pf_n0 = te.tn * BN;
+      pf_n = (pf_pr->N - pf_n0 + 63) / 64;
+      if (pf_n > BN / 64) pf_n = BN / 64;
+      pf_live = KIND == 1 && pf_pr->tma_c != 0 && pf_row0 < pf_pr->M;
+      pf_ch = 0;
+    };
+    auto pf_issue = [&](uint32_t ring_pos) {     // C load of the cursor's chunk into buffer ring_pos % EPI_BUFS
+      if (pf_t >= tile_end) return;
+      if (pf_live) {
+        const uint32_t nb = ring_pos % EPI_BUFS;
+        epi_issue_c_load(args, *pf_pr, pf_row0, pf_n0 + pf_ch * 64, epi_base + nb * BUF_BYTES, smem_u32(&c_full_bar[nb]));
+        ++pf_issued;
       }
+      if (++pf_ch == pf_n) { ++pf_t; pf_enter_tile(); }
+    };
+    if (leader) {
+      pf_enter_tile();
+      for (uint32_t j = 0; j + 1 <= PREFETCH; ++j) pf_issue(j);
     }
+    uint32_t waited = 0;                         // C loads consumed by this thread
     for (uint32_t t = tile_begin; t < tile_end && ok; ++t, ++tcount) {
       const TileEntry te = args.tiles[t];
       const GemmProblem& pr = args.problems[te.problem];
@@ -471,29 +502,18 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
       const float scale = pr.scale_ptr ? __ldg(pr.scale_ptr) : pr.scale_imm;
       // a CTA whose 128 rows lie wholly below the matrix moves nothing through TMA (it still drains TMEM)
       const bool rows_live = row0 < pr.M;
-      const bool tma_c = pr.tma_c != 0 && rows_live, tma_out = pr.tma_out != 0;
+      const bool tma_c = KIND == 1 && pr.tma_c != 0 && rows_live, tma_out = pr.tma_out != 0;
+      const int epi = (KIND == 0) ? (int)EPI_GRAM : pr.epi;
 #pragma unroll 1
       for (int ch = 0; ch < n_chunks; ++ch, ++g) {
         const uint32_t b = g % EPI_BUFS;
-        const uint32_t buf = epi_base + b * EPI_BUF_BYTES;
+        const uint32_t buf = epi_base + b * BUF_BYTES;
         const int col0 = n0 + ch * 64;
         if (leader) {
-          // buffer (g+1)%3 was last stored from two chunks ago: at most the latest store may be pending
+          // buffer (g + PREFETCH) % EPI_BUFS was last stored from two chunks ago: at most the latest
+          // store may still be reading shared memory
           bulk_wait_read<1>();
-          const GemmProblem* npr = nullptr;
-          int nrow0 = 0, ncol0 = 0;
-          if (ch + 1 < n_chunks) { npr = &pr; nrow0 = row0; ncol0 = col0 + 64; }
-          else if (t + 1 < tile_end) {
-            const TileEntry ne = args.tiles[t + 1];
-            npr = &args.problems[ne.problem]; nrow0 = ne.tm * TILE_M + row_shift; ncol0 = ne.tn * BN;
-          }
-          if (npr && npr->tma_c && nrow0 < npr->M) {
-            const uint32_t nb = (g + 1) % EPI_BUFS;
-            epi_issue_c_load(args, *npr, nrow0, ncol0, epi_base + nb * EPI_BUF_BYTES, smem_u32(&c_full_bar[nb]));
-            // this chunk's own load (if any) flips bit b before the next one is waited on
-            pending_bar = smem_u32(&c_full_bar[nb]);
-            pending_par = ((c_phase ^ (tma_c ? (1u << b) : 0u)) >> nb) & 1u;
-          }
+          pf_issue(g + PREFETCH);
         }
         __syncwarp();
         epi_bar_sync();                          // the buffer of this chunk is free for everyone from here
@@ -503,8 +523,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         if (tma_c) {
           c_ok = mbar_wait(smem_u32(&c_full_bar[b]), (c_phase >> b) & 1u, abort_flag, args.status);
           c_phase ^= 1u << b;
+          ++waited;
         }
-        if (pr.epi == EPI_GRAM) {
+        if (KIND == 0) {
           const float f = -0.5f * scale;
 #pragma unroll
           for (int j = 0; j < 64; ++j) v[j] *= f;
@@ -541,13 +562,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
               }
             }
           }
-        } else {
+        } else if (KIND == 1) {
           apply_c_direct(pr, scale, row, col0, v);
           apply_c_direct(pr, scale, row, col0 + 32, v + 32);
         }
         // ---- outputs
-        const bool store_hi = pr.epi == EPI_GRAM || pr.epi == EPI_APPLY || (pr.epi == EPI_APPLY_PACK && pr.store_out);
-        const bool store_lo = pr.epi == EPI_APPLY;
+        const bool store_hi = KIND == 0 || epi == EPI_APPLY || (epi == EPI_APPLY_PACK && pr.store_out);
+        const bool store_lo = KIND == 1 && epi == EPI_APPLY;
         if (store_hi) {
           if (tma_out) {
 #pragma unroll
@@ -569,10 +590,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
             store_out_direct(pr, row, col0 + 32, v + 32, store_lo);
           }
         }
-        if (pr.epi == EPI_APPLY_PACK) {
+        if (KIND == 1 && epi == EPI_APPLY_PACK) {
           pack_bits_direct(pr, row, col0, v);
           pack_bits_direct(pr, row, col0 + 32, v + 32);
-        } else if (pr.epi == EPI_APPLY_UPDATE) {
+        } else if (KIND == 1 && epi == EPI_APPLY_UPDATE) {
           update_weights_direct(pr, args.params, args.lr, row, col0, v);
           update_weights_direct(pr, args.params, args.lr, row, col0 + 32, v + 32);
         }
@@ -596,9 +617,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
       }
     }
     if (leader) {
-      if (!ok && pending_bar) {                  // abort path: let a prefetch in flight land (bounded)
-        uint32_t spins = 0;
-        while (!mbar_try_wait(pending_bar, pending_par) && ++spins < (1u << 22)) {}
+      if (!ok && pf_issued > waited) {           // abort path: give the prefetches in flight a fixed 100 us to land
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 100000ull) {}
       }
       bulk_wait_all();                           // stores must be complete before the CTA retires
     }
@@ -617,9 +638,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
   }
 }
 
-template <int BN, int STAGES, int EPI_BUFS, int CTAS>
+template <int BN, int STAGES, int EPI_BUFS, int CTAS, int KIND>
 constexpr size_t ns_gemm_tc_smem_bytes() {
-  return (size_t)STAGES * (GEMM_BM * GEMM_BK * 2 + (BN / CTAS) * GEMM_BK * 2) + (size_t)EPI_BUFS * EPI_BUF_BYTES + 1024;
+  return (size_t)STAGES * (GEMM_BM * GEMM_BK * 2 + (BN / CTAS) * GEMM_BK * 2) +
+         (size_t)EPI_BUFS * (KIND == 0 ? EPI_HALF_BYTES : EPI_BUF_BYTES) + 1024;
 }
 
 }  // namespace signmuon

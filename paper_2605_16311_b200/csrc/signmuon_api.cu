@@ -414,11 +414,11 @@ int check_launch(signmuon_ctx* c) {
 }
 
 // One-CTA tiles: `lists` CTAs.  CTA pairs: a cluster of two CTAs per tile list.
-template <int BN, int STAGES, int EPI_BUFS, int CTAS>
+template <int BN, int STAGES, int EPI_BUFS, int CTAS, int KIND>
 void launch_tc(const GemmLaunchArgs& a, int lists, cudaStream_t s) {
-  constexpr size_t smem = ns_gemm_tc_smem_bytes<BN, STAGES, EPI_BUFS, CTAS>();
+  constexpr size_t smem = ns_gemm_tc_smem_bytes<BN, STAGES, EPI_BUFS, CTAS, KIND>();
   if (CTAS == 1) {
-    ns_gemm_tc_kernel<BN, STAGES, EPI_BUFS, CTAS><<<lists, GEMM_THREADS, smem, s>>>(a);
+    ns_gemm_tc_kernel<BN, STAGES, EPI_BUFS, CTAS, KIND><<<lists, GEMM_THREADS, smem, s>>>(a);
     return;
   }
   cudaLaunchConfig_t cfg;
@@ -434,22 +434,49 @@ void launch_tc(const GemmLaunchArgs& a, int lists, cudaStream_t s) {
   attr.val.clusterDim.z = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  cudaLaunchKernelEx(&cfg, ns_gemm_tc_kernel<BN, STAGES, EPI_BUFS, CTAS>, a);
+  cudaLaunchKernelEx(&cfg, ns_gemm_tc_kernel<BN, STAGES, EPI_BUFS, CTAS, KIND>, a);
+}
+
+// Shapes of the tensor-core kernel in use.  Gram launches have a long K loop and a small bf16 output:
+// deep operand ring, two half-size output buffers.  Apply launches have a short K loop and move 8 bytes
+// per entry through the epilogue: shallower operand ring, four chunk buffers (two C loads in flight).
+// Operand stages / chunk buffers of each shape; overridable at compile time for tuning runs.
+#ifndef NS_GRAM_STAGES
+#define NS_GRAM_STAGES 6
+#endif
+#ifndef NS_GRAM_BUFS
+#define NS_GRAM_BUFS 2
+#endif
+#ifndef NS_APPLY_STAGES
+#define NS_APPLY_STAGES 3
+#endif
+#ifndef NS_APPLY_BUFS
+#define NS_APPLY_BUFS 4
+#endif
+// (BN, operand stages, chunk buffers, CTAs per tile, kind)
+#define NS_GEMM_PAIR_GRAM 256, NS_GRAM_STAGES, NS_GRAM_BUFS, 2, 0
+#define NS_GEMM_PAIR_APPLY 256, NS_APPLY_STAGES, NS_APPLY_BUFS, 2, 1
+#define NS_GEMM_ONE_GRAM 128, NS_GRAM_STAGES, NS_GRAM_BUFS, 1, 0
+#define NS_GEMM_ONE_APPLY 128, NS_APPLY_STAGES, NS_APPLY_BUFS, 1, 1
+
+template <int BN, int STAGES, int EPI_BUFS, int CTAS, int KIND>
+bool opt_in_smem() {
+  return cudaFuncSetAttribute(ns_gemm_tc_kernel<BN, STAGES, EPI_BUFS, CTAS, KIND>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)ns_gemm_tc_smem_bytes<BN, STAGES, EPI_BUFS, CTAS, KIND>()) == cudaSuccess;
 }
 
 // Opt in to the large dynamic shared memory of the tensor-core kernels (per device, at bind) and ask how
 // many CTA pairs the device can hold at once.
 bool configure_kernels(int* max_pairs) {
-  bool ok = cudaFuncSetAttribute(ns_gemm_tc_kernel<128, 4, 3, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)ns_gemm_tc_smem_bytes<128, 4, 3, 1>()) == cudaSuccess;
-  ok = ok && cudaFuncSetAttribute(ns_gemm_tc_kernel<256, 4, 3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)ns_gemm_tc_smem_bytes<256, 4, 3, 2>()) == cudaSuccess;
+  bool ok = opt_in_smem<NS_GEMM_PAIR_GRAM>() && opt_in_smem<NS_GEMM_PAIR_APPLY>() && opt_in_smem<NS_GEMM_ONE_GRAM>() &&
+            opt_in_smem<NS_GEMM_ONE_APPLY>();
   if (!ok) return false;
   cudaLaunchConfig_t cfg;
   std::memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(2, 1, 1);
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = ns_gemm_tc_smem_bytes<256, 4, 3, 2>();
+  cfg.dynamicSmemBytes = ns_gemm_tc_smem_bytes<NS_GEMM_PAIR_APPLY>();
   cudaLaunchAttribute attr;
   attr.id = cudaLaunchAttributeClusterDimension;
   attr.val.clusterDim.x = 2;
@@ -458,7 +485,7 @@ bool configure_kernels(int* max_pairs) {
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, ns_gemm_tc_kernel<256, 4, 3, 2>, &cfg) != cudaSuccess || n < 1) return false;
+  if (cudaOccupancyMaxActiveClusters(&n, ns_gemm_tc_kernel<NS_GEMM_PAIR_APPLY>, &cfg) != cudaSuccess || n < 1) return false;
   *max_pairs = n;
   return true;
 }
@@ -481,8 +508,12 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
   a.params = pd;
   a.status = reinterpret_cast<uint32_t*>(c->d_ws + c->off_status);
   a.lr = lr;
-  if (tt.ctas == 2) launch_tc<256, 4, 3, 2>(a, tt.grid, s);
-  else launch_tc<128, 4, 3, 1>(a, tt.grid, s);
+  const bool gram = (lp.tile_table & 1) == 0;
+  if (tt.ctas == 2) {
+    if (gram) launch_tc<NS_GEMM_PAIR_GRAM>(a, tt.grid, s); else launch_tc<NS_GEMM_PAIR_APPLY>(a, tt.grid, s);
+  } else {
+    if (gram) launch_tc<NS_GEMM_ONE_GRAM>(a, tt.grid, s); else launch_tc<NS_GEMM_ONE_APPLY>(a, tt.grid, s);
+  }
 }
 
 template <int PLANES>
