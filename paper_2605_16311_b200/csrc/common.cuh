@@ -80,6 +80,9 @@ struct GemmProblem {
   int32_t tmapC0, tmapC1; // C hi (or fp32 momentum) and C lo
   int32_t tmapO0, tmapO1; // out hi and out lo
   int32_t batch_c, batch_o;
+  // Gram products (tensor-core kernel): the result is symmetric, so only tiles on or above the diagonal are
+  // scheduled and every off-diagonal tile is also written transposed through the {64 x 64}-box map tmapOT
+  int32_t sym, tmapOT;
 };
 
 struct TileEntry {

@@ -278,7 +278,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
   constexpr uint32_t TMEM_COLS = 2 * BN;                       // two accumulator buffers
   // KIND 0: a launch of Gram products only (no C operand, bf16 output: ring buffers of one half);
   // KIND 1: a launch of apply products (C operand, hi/lo output, pack or weight update).
-  constexpr uint32_t BUF_BYTES = (KIND == 0) ? EPI_HALF_BYTES : EPI_BUF_BYTES;
+  // (a Gram chunk buffer holds the bf16 chunk and, in its second half, the transposed copy for the mirror tile)
+  constexpr uint32_t BUF_BYTES = EPI_BUF_BYTES;
   static_assert(KIND == 0 || KIND == 1, "Gram or apply launch");
   static_assert(CTAS == 1 || CTAS == 2, "one CTA or a CTA pair");
   static_assert(B_ROWS % 64 == 0, "B rows per CTA: whole 64-row chunks");
@@ -504,6 +505,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
       const bool rows_live = row0 < pr.M;
       const bool tma_c = KIND == 1 && pr.tma_c != 0 && rows_live, tma_out = pr.tma_out != 0;
       const int epi = (KIND == 0) ? (int)EPI_GRAM : pr.epi;
+      const bool mirror = KIND == 0 && pr.sym != 0 && te.tn != te.tm && rows_live;   // off-diagonal Gram tile
 #pragma unroll 1
       for (int ch = 0; ch < n_chunks; ++ch, ++g) {
         const uint32_t b = g % EPI_BUFS;
@@ -584,6 +586,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
               sts128(buf + row_off + ((c16 ^ sw) << 4), make_uint4(wh[0], wh[1], wh[2], wh[3]));
               if (store_lo) sts128(buf + EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4), make_uint4(wl[0], wl[1], wl[2], wl[3]));
             }
+            if (mirror) {
+              // transposed copy: element (j, r) of a 64 x 128 chunk kept as two {64 x 64} swizzled boxes
+              const uint32_t tb = buf + EPI_HALF_BYTES + (uint32_t)(r_in >> 6) * 8192u + (uint32_t)(r_in & 7) * 2u;
+              const uint32_t unit = (uint32_t)(r_in & 63) >> 3;
+#pragma unroll
+              for (int j = 0; j < 64; ++j) {
+                const uint16_t h = __bfloat16_as_ushort(__float2bfloat16_rn(v[j]));
+                asm volatile("st.shared.u16 [%0], %1;" ::"r"(tb + (uint32_t)j * 128u + ((unit ^ (uint32_t)(j & 7)) << 4)), "h"(h)
+                             : "memory");
+              }
+            }
             fence_async_smem();
           } else {
             store_out_direct(pr, row, col0, v, store_lo);
@@ -603,6 +616,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
           if (store_hi && tma_out && rows_live) {
             tma_store_3d(args.tmaps + pr.tmapO0, col0, row0, pr.batch_o, buf);
             if (store_lo) tma_store_3d(args.tmaps + pr.tmapO1, col0, row0, pr.batch_o, buf + EPI_HALF_BYTES);
+            if (mirror) {                        // rows col0.. of the output, columns row0.. (two 64-column boxes)
+              tma_store_3d(args.tmaps + pr.tmapOT, row0, col0, pr.batch_o, buf + EPI_HALF_BYTES);
+              if (row0 + 64 < pr.M)
+                tma_store_3d(args.tmaps + pr.tmapOT, row0 + 64, col0, pr.batch_o, buf + EPI_HALF_BYTES + 8192u);
+            }
           }
           bulk_commit();                         // one group per chunk (possibly empty) keeps the ring arithmetic fixed
         }
@@ -641,7 +659,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
 template <int BN, int STAGES, int EPI_BUFS, int CTAS, int KIND>
 constexpr size_t ns_gemm_tc_smem_bytes() {
   return (size_t)STAGES * (GEMM_BM * GEMM_BK * 2 + (BN / CTAS) * GEMM_BK * 2) +
-         (size_t)EPI_BUFS * (KIND == 0 ? EPI_HALF_BYTES : EPI_BUF_BYTES) + 1024;
+         (size_t)EPI_BUFS * EPI_BUF_BYTES + 1024;
 }
 
 }  // namespace signmuon

@@ -42,7 +42,7 @@ struct ParamPlan {
 
 // indices of a parameter's tensor maps relative to tmap_base
 enum { TM_Y0_K128 = 0, TM_Y0_KBN, TM_Y0_MN, TM_Y1_K128, TM_Y1_KBN, TM_Y1_MN, TM_Q_K128, TM_Q_KBN, TM_LO_K128, TM_MOM_F32,
-       TM_PER_PARAM };
+       TM_Q_BOX64, TM_PER_PARAM };
 
 struct LaunchPlan {        // one grouped GEMM launch
   size_t problem_base;     // index of its first problem in the problem array
@@ -109,7 +109,8 @@ void build_tile_table(TileTable& tt, const std::vector<GemmProblem>& probs, size
     const int tm = (pr.M + bm - 1) / bm, tn = (pr.N + bn - 1) / bn;
     const int cost = (pr.K + GEMM_BK - 1) / GEMM_BK + 2;
     for (int a = 0; a < tm; ++a)
-      for (int b = 0; b < tn; ++b) all.push_back({{(uint32_t)i, (uint16_t)a, (uint16_t)b}, cost});
+      for (int b = (pr.sym ? a : 0); b < tn; ++b)     // symmetric results: tiles on or above the diagonal
+        all.push_back({{(uint32_t)i, (uint16_t)a, (uint16_t)b}, cost});
   }
   tt.grid = (int)std::min<size_t>((size_t)grid_limit, std::max<size_t>(all.size(), 1));
   std::stable_sort(all.begin(), all.end(), [](const T& x, const T& y) { return x.cost > y.cost; });
@@ -177,6 +178,8 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         pr.out = reinterpret_cast<void*>(q);
         pr.ld_out = pl.ldq;
         pr.tma_out = 1; pr.tmapO0 = pl.tmap_base + TM_Q_K128; pr.batch_o = m;
+        pr.sym = (c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) ? 0 : 1;   // square tiles only (bm == bn in every shape)
+        pr.tmapOT = pl.tmap_base + TM_Q_BOX64;
         if (k == 0) {
           if (local_polar_phase) pr.scale_imm = (float)(1.0 / ((double)pl.rows * (double)pl.cols));
           else pr.scale_ptr = reinterpret_cast<const float*>(pl.scales_off + (size_t)m * 8);
@@ -442,7 +445,7 @@ void launch_tc(const GemmLaunchArgs& a, int lists, cudaStream_t s) {
 // per entry through the epilogue: shallower operand ring, four chunk buffers (two C loads in flight).
 // Operand stages / chunk buffers of each shape; overridable at compile time for tuning runs.
 #ifndef NS_GRAM_STAGES
-#define NS_GRAM_STAGES 6
+#define NS_GRAM_STAGES 5
 #endif
 #ifndef NS_GRAM_BUFS
 #define NS_GRAM_BUFS 2
@@ -745,6 +748,7 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
       const uint64_t qb = (uint64_t)pl.s * pl.ldq;
       ok = ok && encode_map(mp + TM_Q_K128, q, pl.s, pl.s, slots, pl.ldq, qb, 128);
       ok = ok && encode_map(mp + TM_Q_KBN, q, pl.s, pl.s, slots, pl.ldq, qb, bn);
+      ok = ok && encode_map(mp + TM_Q_BOX64, q, pl.s, pl.s, slots, pl.ldq, qb, 64);
       ok = ok && encode_map(mp + TM_LO_K128, c->d_ws + pl.lo_off, pl.cols, pl.rows, slots, pl.ldy,
                             (uint64_t)pl.rows * pl.ldy, 128);
       if (pl.cols % 4 == 0)   // float32 momentum as the first iteration's C operand
