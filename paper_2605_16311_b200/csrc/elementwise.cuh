@@ -338,6 +338,49 @@ __device__ __forceinline__ void vote_block(const ParamDev& pd, uint32_t chunk, i
   }
   WT* w = reinterpret_cast<WT*>(pd.W);
   bf16* sbar = pd.y0 + (int64_t)M * pd.rows * pd.ldy;   // slot M of operand buffer 0: input of the local polar step
+  const int64_t e0 = wbase * 32;                        // first entry of this warp's 1024
+  if (pd.vec_ok && e0 + 1024 <= pd.d) {
+    // 128-bit path: the warp's 1024 entries are 256 float4 (fp32 weights) or 128 uint4 (bf16 weights or the
+    // +-1 matrix); a lane's vector lies inside one vote word, fetched from its owner lane by shuffle.
+    if (!write_sbar && sizeof(WT) == 4) {
+      float4* w4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(w) + e0);
+      float4 x[8];
+#pragma unroll
+      for (int it = 0; it < 8; ++it) x[it] = __ldcs(w4 + it * 32 + lane);
+#pragma unroll
+      for (int it = 0; it < 8; ++it) {
+        const uint32_t bits4 = __shfl_sync(0xffffffffu, v, it * 4 + (lane >> 3)) >> ((lane & 7) * 4);
+        x[it].x -= (bits4 & 1u) ? step : -step;
+        x[it].y -= (bits4 & 2u) ? step : -step;
+        x[it].z -= (bits4 & 4u) ? step : -step;
+        x[it].w -= (bits4 & 8u) ? step : -step;
+        __stcs(w4 + it * 32 + lane, x[it]);
+      }
+    } else {
+      uint4* w8 = write_sbar ? reinterpret_cast<uint4*>(sbar + e0) : reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(w) + e0);
+      uint4 x[4];
+#pragma unroll
+      for (int it = 0; it < 4; ++it) x[it] = write_sbar ? make_uint4(0, 0, 0, 0) : __ldcs(w8 + it * 32 + lane);
+#pragma unroll
+      for (int it = 0; it < 4; ++it) {
+        const uint32_t bits8 = __shfl_sync(0xffffffffu, v, it * 8 + (lane >> 2)) >> ((lane & 3) * 8);
+        const uint32_t in[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
+        uint32_t o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const bool p0 = (bits8 >> (2 * e)) & 1u, p1 = (bits8 >> (2 * e + 1)) & 1u;
+          if (write_sbar) {
+            o[e] = pack_bf16x2(p0 ? 1.f : -1.f, p1 ? 1.f : -1.f);
+          } else {
+            o[e] = pack_bf16x2(__uint_as_float(in[e] << 16) - (p0 ? step : -step),
+                               __uint_as_float(in[e] & 0xffff0000u) - (p1 ? step : -step));
+          }
+        }
+        __stcs(w8 + it * 32 + lane, make_uint4(o[0], o[1], o[2], o[3]));
+      }
+    }
+    return;
+  }
 #pragma unroll 4
   for (int k = 0; k < 32; ++k) {
     const uint32_t vk = __shfl_sync(0xffffffffu, v, k);
