@@ -334,6 +334,62 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Kernel sweep (BASELINE config 5): squares and 1:4 rectangles from 512 to 8192 per side, bf16,
+    M in {1..32}, K in {3, 5}; Newton-Schulz timed separately from momentum and vote+update.
+    Prints one JSON line per point (this mode is not the one-line benchmark contract)."""
+    import torch
+    from paper_2605_16311_b200 import binding as B
+    from paper_2605_16311_b200 import build as build_mod
+    from paper_2605_16311_b200 import workloads as wlmod
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the SignMuon step has no CPU fallback")
+    build_mod.build()
+    B.load_library()
+    peaks = load_peaks()
+    sides = [512, 1024, 2048, 4096, 8192]
+    shapes = [(n, n) for n in sides] + [(512, 2048), (2048, 512), (1024, 4096), (4096, 1024), (2048, 8192), (8192, 2048)]
+    workers = [int(x) for x in args.sweep_workers.split(",")]
+    for (r, c) in shapes:
+        for M in workers:
+            for K in (3, 5):
+                wl = wlmod.config5(r, c, M, K)
+                opt = B.SignMuon(wl.params, M, momentum=wl.momentum, lr=wl.lr, ns_steps=K, local_polar=False,
+                                 device="cuda:0")
+                weights = wlmod.make_weights(wl, "cuda:0")
+                signal = wlmod.make_signal(wl, "cuda:0")
+                grads = wlmod.make_grads(wl, signal, 0, "cuda:0")
+                for _ in range(3):
+                    opt.step(weights, grads, wl.lr)
+                torch.cuda.synchronize()
+                reps = 5
+                masks = [B.STAGE_MOMENTUM, B.STAGE_NS, B.STAGE_VOTE]
+                ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(reps)]
+                for t in range(reps):
+                    ev[t][0].record()
+                    for i, mask in enumerate(masks):
+                        opt.step(weights, grads, wl.lr, stages=mask)
+                        ev[t][i + 1].record()
+                torch.cuda.synchronize()
+                if opt.status() != B.OK:
+                    raise RuntimeError("device status word set during the sweep")
+                ms = [statistics.median(ev[t][i].elapsed_time(ev[t][i + 1]) for t in range(reps)) for i in range(3)]
+                d = r * c
+                ns_flops = opt.ns_flops_per_step
+                mom_bytes = M * d * (2 + 4 + 4 + 2)
+                vote_bytes = d * (M / 8 + 1 / 8 + 4)
+                line = {"workload": f"c5:{r}x{c}:{M}:{K}", "rows": r, "cols": c, "num_workers": M, "ns_steps": K,
+                        "ns_ms": ms[1], "ns_tflops": ns_flops / ms[1] / 1e9,
+                        "ns_frac_of_sustained_peak": ns_flops / ms[1] / 1e9 / peaks["bf16_tflops_sustained"],
+                        "momentum_ms": ms[0], "momentum_gbs": mom_bytes / ms[0] / 1e6,
+                        "vote_update_ms": ms[2], "vote_update_gbs": vote_bytes / ms[2] / 1e6,
+                        "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"]}
+                print(json.dumps(line), flush=True)
+                opt.close()
+                del opt, weights, signal, grads
+                torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -347,7 +403,12 @@ def main():
                     help="float64 operation budget of one oracle sample step")
     ap.add_argument("--cpu-baseline-flops", type=float, default=8e11,
                     help="float64 operation budget of the oracle sample timed beside the GPU run")
+    ap.add_argument("--sweep", action="store_true", help="run the kernel sweep (config 5) and print one line per point")
+    ap.add_argument("--sweep-workers", default="1,2,4,8,16,32")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2605_16311_b200 import workloads as wlmod
     wl = wlmod.by_name(args.workload)

@@ -55,6 +55,7 @@ struct TileTable {
   int grid = 0;            // number of tile lists = CTAs (one-CTA kernel) or CTA pairs
   int bm = 128, bn = 128;  // tile shape
   int ctas = 1;            // CTAs that share a tile
+  bool long_k = false;     // tile-weighted mean contraction length >= 1536 (chooses the apply kernel's rings)
   size_t tiles_off = 0, cta_off = 0;    // bytes into the workspace
 };
 
@@ -124,6 +125,9 @@ void build_tile_table(TileTable& tt, const std::vector<GemmProblem>& probs, size
     per[top.second].push_back(t.e);
     heap.push({top.first + t.cost, top.second});
   }
+  long long ksum = 0;
+  for (const T& t : all) ksum += probs[pbase + t.e.problem].K;
+  tt.long_k = !all.empty() && ksum / (long long)all.size() >= 1536;
   tt.tiles.clear();
   tt.cta_start.assign(tt.grid + 1, 0);
   for (int c = 0; c < tt.grid; ++c) {
@@ -459,6 +463,7 @@ void launch_tc(const GemmLaunchArgs& a, int lists, cudaStream_t s) {
 // (BN, operand stages, chunk buffers, CTAs per tile, kind)
 #define NS_GEMM_PAIR_GRAM 256, NS_GRAM_STAGES, NS_GRAM_BUFS, 2, 0
 #define NS_GEMM_PAIR_APPLY 256, NS_APPLY_STAGES, NS_APPLY_BUFS, 2, 1
+#define NS_GEMM_PAIR_APPLY_LONGK 256, 4, 3, 2, 1   /* long contraction: the operand ring matters more than the chunk ring */
 #define NS_GEMM_ONE_GRAM 128, NS_GRAM_STAGES, NS_GRAM_BUFS, 1, 0
 #define NS_GEMM_ONE_APPLY 128, NS_APPLY_STAGES, NS_APPLY_BUFS, 1, 1
 
@@ -473,7 +478,7 @@ bool opt_in_smem() {
 // many CTA pairs the device can hold at once.
 bool configure_kernels(int* max_pairs) {
   bool ok = opt_in_smem<NS_GEMM_PAIR_GRAM>() && opt_in_smem<NS_GEMM_PAIR_APPLY>() && opt_in_smem<NS_GEMM_ONE_GRAM>() &&
-            opt_in_smem<NS_GEMM_ONE_APPLY>();
+            opt_in_smem<NS_GEMM_ONE_APPLY>() && opt_in_smem<NS_GEMM_PAIR_APPLY_LONGK>();
   if (!ok) return false;
   cudaLaunchConfig_t cfg;
   std::memset(&cfg, 0, sizeof(cfg));
@@ -513,7 +518,9 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
   a.lr = lr;
   const bool gram = (lp.tile_table & 1) == 0;
   if (tt.ctas == 2) {
-    if (gram) launch_tc<NS_GEMM_PAIR_GRAM>(a, tt.grid, s); else launch_tc<NS_GEMM_PAIR_APPLY>(a, tt.grid, s);
+    if (gram) launch_tc<NS_GEMM_PAIR_GRAM>(a, tt.grid, s);
+    else if (tt.long_k) launch_tc<NS_GEMM_PAIR_APPLY_LONGK>(a, tt.grid, s);
+    else launch_tc<NS_GEMM_PAIR_APPLY>(a, tt.grid, s);
   } else {
     if (gram) launch_tc<NS_GEMM_ONE_GRAM>(a, tt.grid, s); else launch_tc<NS_GEMM_ONE_APPLY>(a, tt.grid, s);
   }
