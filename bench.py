@@ -152,6 +152,29 @@ def time_oracle(wl, steps, warmup, budget_flops):
             "sample_seconds_per_step": per_sample_step}
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the ncu
+# captures summarised under profiles/; None for workloads without a capture of the current kernel.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {
+    ("c2_resnet50", "ns_gemm_tc_kernel"): 525.2e6,   # mean of 5 Gram (230.8 MB) and 5 apply (819.5 MB) launches
+}
+
+
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group):
+    multi-GPU times are the slowest rank's."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_value(ms_step, world):
+    """Replicas only: every rank runs one full step per `ms_step`, so the job does `world` steps in that time."""
+    return world * 1e3 / ms_step
+
+
 def describe(wl):
     return {"workload": wl.name, "params": len(wl.params), "entries": wl.numel, "num_workers": wl.num_workers,
             "ns_steps": wl.ns_steps, "local_polar": bool(wl.local_polar), "momentum": wl.momentum, "lr": wl.lr,
@@ -258,11 +281,7 @@ def run_ours(args, wl):
     e2e_ms = h0.elapsed_time(h1) / e2e_steps if e2e_steps else float("nan")
 
     # ---------------------------------------------------------------- reduce over ranks
-    ms_step = ms_total / args.steps
-    if dist is not None:
-        t = torch.tensor([ms_step, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step, e2e_ms = float(t[0]), float(t[1])
+    ms_step, e2e_ms = max_over_ranks([ms_total / args.steps, e2e_ms], dist, dev)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -300,7 +319,8 @@ def run_ours(args, wl):
         achieved = kd["achieved_tflops"]
         peak = peaks["bf16_tflops_sustained"]
         roof = {"kernel": "ns_gemm_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                "unit": "TFLOP/s", "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((wl.name, "ns_gemm_tc_kernel")),
                 "flops_per_launch": ns_flops / launches, "ms_per_launch": per_launch_ms,
                 "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0}
@@ -317,12 +337,12 @@ def run_ours(args, wl):
         cpu = time_oracle(wl, 1, 0, args.cpu_baseline_flops)
         cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
 
-    line = {"metric": METRIC, "value": world * 1e3 / ms_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+    line = {"metric": METRIC, "value": whole_job_value(ms_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": describe(wl),
             "clocks": clocks,
             "e2e": (None if args.no_e2e else
-                    {"value": world * 1e3 / e2e_ms, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    {"value": whole_job_value(e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                      "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms}),
             "gpu_launches": opt.launches_per_step * args.steps,
             "roofline": roof, "cpu_baseline": cpu,
