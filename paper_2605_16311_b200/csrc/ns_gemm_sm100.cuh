@@ -29,8 +29,11 @@
 //            a 16-element K step advances the start by 2048 bytes.
 // Epilogue traffic also goes through TMA: the Y_k tile that enters as 1.5*C is prefetched into a ring
 // of 64-column chunk buffers (128-byte swizzle; hi half and lo half, or two fp32 halves for the first
-// iteration's momentum), the results overwrite the chunk in place and leave with a TMA store, so the
-// epilogue warps touch global memory directly only for payload words and the final weight update.
+// iteration's momentum) by a dedicated thread, eight math warps (two per TMEM lane quarter) overwrite the
+// chunk in place, and the same dedicated thread sends it off with TMA stores; the math warps touch global
+// memory directly only for payload words and the final weight update.  The math warps never wait for each
+// other: per chunk they wait on the buffer's "C landed / buffer free" mbarrier and arrive on its "results
+// written" mbarrier.
 // Every wait is bounded: after about two seconds a waiting thread records STATUS_TIMEOUT in the
 // status word, raises a CTA-wide abort flag and the CTA drains and exits (TMEM is freed).
 #pragma once
@@ -43,7 +46,9 @@ namespace signmuon {
 
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;
-constexpr int GEMM_THREADS = 192;            // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr int EPI_WARPS = 8;                 // two warps per TMEM lane quarter, 32 of a chunk's 64 columns each
+constexpr int GEMM_THREADS = 32 * (3 + EPI_WARPS);   // warp 0: operand TMA, warp 1: MMA, warps 2-9: epilogue math,
+                                                     // warp 10: epilogue TMA (C loads, result stores)
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
 struct GemmLaunchArgs {
@@ -182,20 +187,6 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-// Barrier over the 128 epilogue threads that also ANDs a flag, so that all of them take the same exit.
-__device__ __forceinline__ bool epi_bar_and(bool flag) {
-  uint32_t out;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.and.pred p, 1, 128, q;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(out)
-      : "r"((uint32_t)flag)
-      : "memory");
-  return out != 0;
-}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
@@ -205,19 +196,19 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
   asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-// Loads 64 consecutive fp32 columns of this thread's TMEM lane and waits for them.  Load and wait sit in
+// Loads 32 consecutive fp32 columns of this thread's TMEM lane and waits for them.  Load and wait sit in
 // one asm statement so that no use of the destination registers can be scheduled before the wait.
-__device__ __forceinline__ void tc_ld64(uint32_t taddr, float (&v)[64]) {
-  uint32_t r[64];
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
       "tcgen05.wait::ld.sync.aligned;"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
 #pragma unroll
-  for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // Shared-memory matrix descriptor (128-byte swizzle).  Bits: [0,14) start >> 4, [16,30) LBO >> 4,
@@ -291,7 +282,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
   __shared__ uint64_t empty_bar[STAGES];
   __shared__ uint64_t tmem_full_bar[2];
   __shared__ uint64_t tmem_empty_bar[2];
-  __shared__ uint64_t c_full_bar[EPI_BUFS];
+  __shared__ uint64_t c_full_bar[EPI_BUFS];      // chunk buffer holds its C operand / may be overwritten
+  __shared__ uint64_t buf_ready_bar[EPI_BUFS];   // the eight math warps have written their results into it
+  __shared__ uint64_t row_pair_bar[4];           // the two math warps of a lane quarter (fp32 C chunks only)
   __shared__ uint32_t tmem_slot;
   __shared__ uint32_t abort_word;
 
@@ -311,9 +304,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&tmem_full_bar[a]), 1);
-      mbar_init(smem_u32(&tmem_empty_bar[a]), 4 * CTAS);
+      mbar_init(smem_u32(&tmem_empty_bar[a]), EPI_WARPS * CTAS);
     }
-    for (int b = 0; b < EPI_BUFS; ++b) mbar_init(smem_u32(&c_full_bar[b]), 1);
+    for (int b = 0; b < EPI_BUFS; ++b) {
+      mbar_init(smem_u32(&c_full_bar[b]), 1);
+      mbar_init(smem_u32(&buf_ready_bar[b]), EPI_WARPS);
+    }
+    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&row_pair_bar[i]), 2);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -438,208 +435,231 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
       }
     }
   } else {
-    // ===================================================================== epilogue (warps 2..5)
+    // ===================================================================== epilogue
     // Chunks (64 output columns of this CTA's 128 rows) are numbered g = 0, 1, ... across the CTA's tiles;
-    // chunk g lives in ring buffer g % EPI_BUFS: its C operand lands there by TMA, the results overwrite it
-    // in place and leave by a TMA store.  The leader thread runs a cursor PREFETCH chunks ahead of the
-    // chunk being computed and issues the C loads from there, so that PREFETCH loads are in flight while
-    // one chunk is computed and the previous one drains.
+    // chunk g lives in ring buffer g % EPI_BUFS.  For every chunk the TMA thread (warp 10) first makes the
+    // buffer available - it waits until the store that last used the buffer has left shared memory, then
+    // either starts the C loads on c_full_bar (bytes expected) or just arrives on it - and it does so
+    // PREFETCH chunks ahead of the chunk whose results it sends off.  A math warp waits on c_full_bar,
+    // reads its accumulator columns, combines, writes the results in place and arrives on buf_ready_bar;
+    // the TMA thread waits on that and issues the stores.
     constexpr uint32_t PREFETCH = EPI_BUFS - 2;
-    const int q = warp & 3;                      // TMEM lane quarter this warp may read
-    const bool leader = (threadIdx.x == 64);     // issues the chunk loads and stores
-    const int r_in = q * 32 + lane;              // row of the tile this thread owns
-    const uint32_t row_off = (uint32_t)r_in * 128u;
-    const uint32_t sw = (uint32_t)(r_in & 7);
-    uint32_t g = 0;                              // running chunk counter (ring position)
-    uint32_t c_phase = 0;                        // bit b: parity of the next C load landing in buffer b
-    uint32_t tcount = 0;
-    bool ok = true;
-    // ---- leader's prefetch cursor
-    uint32_t pf_t = tile_begin;                  // tile of the next chunk to prefetch
-    int pf_ch = 0, pf_n = 0, pf_row0 = 0, pf_n0 = 0;
-    const GemmProblem* pf_pr = nullptr;
-    bool pf_live = false;
-    uint32_t pf_issued = 0;                      // loads issued so far (for the abort path)
-    auto pf_enter_tile = [&]() {
-      if (pf_t >= tile_end) return;
-      const TileEntry te = args.tiles[pf_t];
-      pf_pr = &args.problems[te.problem];
-      pf_row0 = te.tm * TILE_M + row_shift;
-      pf_n0 = te.tn * BN;
-      pf_n = (pf_pr->N - pf_n0 + 63) / 64;
-      if (pf_n > BN / 64) pf_n = BN / 64;
-      pf_live = KIND == 1 && pf_pr->tma_c != 0 && pf_row0 < pf_pr->M;
-      pf_ch = 0;
-    };
-    auto pf_issue = [&](uint32_t ring_pos) {     // C load of the cursor's chunk into buffer ring_pos % EPI_BUFS
-      if (pf_t >= tile_end) return;
-      if (pf_live) {
-        const uint32_t nb = ring_pos % EPI_BUFS;
-        epi_issue_c_load(args, *pf_pr, pf_row0, pf_n0 + pf_ch * 64, epi_base + nb * BUF_BYTES, smem_u32(&c_full_bar[nb]));
-        ++pf_issued;
+    if (warp == 2 + EPI_WARPS) {
+      // ------------------------------------------------------------------- epilogue TMA thread
+      if (lane == 0) {
+        bool ok = true;
+        // load-side cursor
+        uint32_t pf_t = tile_begin, pf_g = 0;
+        int pf_ch = 0, pf_n = 0, pf_row0 = 0, pf_n0 = 0;
+        const GemmProblem* pf_pr = nullptr;
+        bool pf_live = false;
+        uint32_t pf_issued = 0;
+        auto pf_enter_tile = [&]() {
+          if (pf_t >= tile_end) return;
+          const TileEntry te = args.tiles[pf_t];
+          pf_pr = &args.problems[te.problem];
+          pf_row0 = te.tm * TILE_M + row_shift;
+          pf_n0 = te.tn * BN;
+          pf_n = (pf_pr->N - pf_n0 + 63) / 64;
+          if (pf_n > BN / 64) pf_n = BN / 64;
+          pf_live = KIND == 1 && pf_pr->tma_c != 0 && pf_row0 < pf_pr->M;
+          pf_ch = 0;
+        };
+        auto pf_step = [&]() {                   // makes the buffer of chunk pf_g available to the math warps
+          if (pf_t >= tile_end) return;
+          const uint32_t nb = pf_g % EPI_BUFS;
+          if (pf_live) {
+            epi_issue_c_load(args, *pf_pr, pf_row0, pf_n0 + pf_ch * 64, epi_base + nb * BUF_BYTES, smem_u32(&c_full_bar[nb]));
+            ++pf_issued;
+          } else {
+            mbar_arrive(smem_u32(&c_full_bar[nb]));
+          }
+          ++pf_g;
+          if (++pf_ch == pf_n) { ++pf_t; pf_enter_tile(); }
+        };
+        pf_enter_tile();
+        for (uint32_t j = 0; j + 1 <= PREFETCH; ++j) pf_step();
+        uint32_t g = 0;
+        for (uint32_t t = tile_begin; t < tile_end && ok; ++t) {
+          const TileEntry te = args.tiles[t];
+          const GemmProblem& pr = args.problems[te.problem];
+          const int row0 = te.tm * TILE_M + row_shift;
+          const int n0 = te.tn * BN;
+          int n_chunks = (pr.N - n0 + 63) / 64;
+          if (n_chunks > BN / 64) n_chunks = BN / 64;
+          const bool rows_live = row0 < pr.M;
+          const int epi = (KIND == 0) ? (int)EPI_GRAM : pr.epi;
+          const bool store_hi = (KIND == 0 || epi == EPI_APPLY || (epi == EPI_APPLY_PACK && pr.store_out)) &&
+                                pr.tma_out != 0 && rows_live;
+          const bool store_lo = KIND == 1 && epi == EPI_APPLY;
+          const bool mirror = KIND == 0 && pr.sym != 0 && te.tn != te.tm && rows_live;
+          const CUtensorMap* mapO0 = args.tmaps + pr.tmapO0;
+          const CUtensorMap* mapO1 = args.tmaps + pr.tmapO1;
+          const CUtensorMap* mapOT = args.tmaps + pr.tmapOT;
+          const int batch_o = pr.batch_o, prM = pr.M;
+          for (int ch = 0; ch < n_chunks; ++ch, ++g) {
+            const uint32_t b = g % EPI_BUFS;
+            const uint32_t buf = epi_base + b * BUF_BYTES;
+            const int col0 = n0 + ch * 64;
+            // buffer (g + PREFETCH) % EPI_BUFS was last stored from two chunks ago: at most the latest store
+            // may still be reading shared memory
+            bulk_wait_read<1>();
+            pf_step();
+            if (!mbar_wait(smem_u32(&buf_ready_bar[b]), (g / EPI_BUFS) & 1u, abort_flag, args.status)) { ok = false; break; }
+            if (store_hi) {
+              tma_store_3d(mapO0, col0, row0, batch_o, buf);
+              if (store_lo) tma_store_3d(mapO1, col0, row0, batch_o, buf + EPI_HALF_BYTES);
+              if (mirror) {                      // rows col0.. of the output, columns row0.. (two 64-column boxes)
+                tma_store_3d(mapOT, row0, col0, batch_o, buf + EPI_HALF_BYTES);
+                if (row0 + 64 < prM) tma_store_3d(mapOT, row0 + 64, col0, batch_o, buf + EPI_HALF_BYTES + 8192u);
+              }
+            }
+            bulk_commit();                       // one group per chunk (possibly empty) keeps the ring arithmetic fixed
+          }
+        }
+        if (!ok && pf_issued) {                  // abort path: give the loads in flight a fixed 100 us to land
+          const uint64_t t0 = global_timer_ns();
+          while (global_timer_ns() - t0 < 100000ull) {}
+        }
+        bulk_wait_all();                         // stores must be complete before the CTA retires
       }
-      if (++pf_ch == pf_n) { ++pf_t; pf_enter_tile(); }
-    };
-    if (leader) {
-      pf_enter_tile();
-      for (uint32_t j = 0; j + 1 <= PREFETCH; ++j) pf_issue(j);
-    }
-    uint32_t waited = 0;                         // C loads consumed by this thread
-    for (uint32_t t = tile_begin; t < tile_end && ok; ++t, ++tcount) {
-      const TileEntry te = args.tiles[t];
-      const GemmProblem& pr = args.problems[te.problem];
-      const uint32_t acc = tcount & 1u;
-      const uint32_t acc_round = tcount >> 1;
-      ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_round & 1u, abort_flag, args.status);
-      ok = epi_bar_and(ok);                      // uniform over the four epilogue warps
-      if (!ok) break;
-      tc_fence_after();
-      const int row0 = te.tm * TILE_M + row_shift;
-      const int row = row0 + r_in;
-      const int n0 = te.tn * BN;
-      const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
-      int n_chunks = (pr.N - n0 + 63) / 64;
-      if (n_chunks > BN / 64) n_chunks = BN / 64;
-      const float scale = pr.scale_ptr ? __ldg(pr.scale_ptr) : pr.scale_imm;
-      // a CTA whose 128 rows lie wholly below the matrix moves nothing through TMA (it still drains TMEM)
-      const bool rows_live = row0 < pr.M;
-      const bool tma_c = KIND == 1 && pr.tma_c != 0 && rows_live, tma_out = pr.tma_out != 0;
-      const int epi = (KIND == 0) ? (int)EPI_GRAM : pr.epi;
-      const bool mirror = KIND == 0 && pr.sym != 0 && te.tn != te.tm && rows_live;   // off-diagonal Gram tile
+    } else {
+      // ------------------------------------------------------------------- epilogue math warps (2 .. 9)
+      const int q = warp & 3;                    // TMEM lane quarter this warp may read
+      const int half = (warp - 2) >> 2;          // which 32 of a chunk's 64 columns
+      const int r_in = q * 32 + lane;            // row of the tile this thread owns
+      const uint32_t row_off = (uint32_t)r_in * 128u;
+      const uint32_t sw = (uint32_t)(r_in & 7);
+      uint32_t g = 0, tcount = 0, f32_chunks = 0;
+      bool ok = true;
+      for (uint32_t t = tile_begin; t < tile_end && ok; ++t, ++tcount) {
+        const TileEntry te = args.tiles[t];
+        const GemmProblem& pr = args.problems[te.problem];
+        // the fields used per chunk, read once per tile
+        const int prM = pr.M, prN = pr.N, c_mode = pr.c_mode;
+        const int epi = (KIND == 0) ? (int)EPI_GRAM : pr.epi;
+        const int row0 = te.tm * TILE_M + row_shift;
+        const int row = row0 + r_in;
+        const int n0 = te.tn * BN;
+        int n_chunks = (prN - n0 + 63) / 64;
+        if (n_chunks > BN / 64) n_chunks = BN / 64;
+        const float scale = pr.scale_ptr ? __ldg(pr.scale_ptr) : pr.scale_imm;
+        // a CTA whose 128 rows lie wholly below the matrix moves nothing through TMA (it still drains TMEM)
+        const bool rows_live = row0 < prM;
+        const bool tma_c = KIND == 1 && pr.tma_c != 0 && rows_live, tma_out = pr.tma_out != 0;
+        const bool store_hi = KIND == 0 || epi == EPI_APPLY || (epi == EPI_APPLY_PACK && pr.store_out);
+        const bool store_lo = KIND == 1 && epi == EPI_APPLY;
+        const bool mirror = KIND == 0 && pr.sym != 0 && te.tn != te.tm && rows_live;   // off-diagonal Gram tile
+        const uint32_t acc = tcount & 1u;
+        const uint32_t acc_round = tcount >> 1;
+        ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_round & 1u, abort_flag, args.status);
+        ok = __all_sync(0xffffffffu, ok);        // the whole warp takes the same exit
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)half * 32u;
 #pragma unroll 1
-      for (int ch = 0; ch < n_chunks; ++ch, ++g) {
-        const uint32_t b = g % EPI_BUFS;
-        const uint32_t buf = epi_base + b * BUF_BYTES;
-        const int col0 = n0 + ch * 64;
-        if (leader) {
-          // buffer (g + PREFETCH) % EPI_BUFS was last stored from two chunks ago: at most the latest
-          // store may still be reading shared memory
-          bulk_wait_read<1>();
-          pf_issue(g + PREFETCH);
-        }
-        __syncwarp();
-        epi_bar_sync();                          // the buffer of this chunk is free for everyone from here
-        float v[64];
-        tc_ld64(taddr + ch * 64, v);
-        bool c_ok = true;                        // folded into the barrier below: nobody leaves the chunk early
-        if (tma_c) {
-          c_ok = mbar_wait(smem_u32(&c_full_bar[b]), (c_phase >> b) & 1u, abort_flag, args.status);
-          c_phase ^= 1u << b;
-          ++waited;
-        }
-        if (KIND == 0) {
-          const float f = -0.5f * scale;
+        for (int ch = 0; ch < n_chunks; ++ch, ++g) {
+          const uint32_t b = g % EPI_BUFS;
+          const uint32_t buf = epi_base + b * BUF_BYTES;
+          const int col0 = n0 + ch * 64 + half * 32;   // first of this thread's 32 columns
+          ok = mbar_wait(smem_u32(&c_full_bar[b]), (g / EPI_BUFS) & 1u, abort_flag, args.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          float v[32];
+          tc_ld32(taddr + ch * 64, v);
+          if (ch == n_chunks - 1) {              // last read of this accumulator: hand it back to the MMA issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+              if (CTAS == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
+              else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+            }
+          }
+          if (KIND == 0) {
+            const float f = -0.5f * scale;
 #pragma unroll
-          for (int j = 0; j < 64; ++j) v[j] *= f;
-        } else if (tma_c) {
-          if (pr.c_mode == C_F32) {
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
+            for (int j = 0; j < 32; ++j) v[j] *= f;
+          } else if (tma_c) {
+            if (c_mode == C_F32) {               // half h of the buffer = fp32 columns 32 h .. 32 h + 31
 #pragma unroll
               for (int c16 = 0; c16 < 8; ++c16) {
-                const uint4 u = lds128(buf + h * EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4));
-                float* o = v + h * 32 + c16 * 4;
+                const uint4 u = lds128(buf + half * EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4));
+                float* o = v + c16 * 4;
                 o[0] = scale * fmaf(1.5f, __uint_as_float(u.x), o[0]);
                 o[1] = scale * fmaf(1.5f, __uint_as_float(u.y), o[1]);
                 o[2] = scale * fmaf(1.5f, __uint_as_float(u.z), o[2]);
                 o[3] = scale * fmaf(1.5f, __uint_as_float(u.w), o[3]);
               }
-            }
-          } else {
-            const bool has_lo = pr.c_mode == C_HILO;
+              // The bf16 results go to units 4h..4h+3 of BOTH halves, i.e. into the fp32 columns of the warp
+              // that owns the other 32 columns of these rows: both warps finish reading before either writes.
+              __syncwarp();
+              if (lane == 0) mbar_arrive(smem_u32(&row_pair_bar[q]));
+              ok = mbar_wait(smem_u32(&row_pair_bar[q]), f32_chunks & 1u, abort_flag, args.status);
+              ++f32_chunks;
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+            } else {
+              const bool has_lo = c_mode == C_HILO;
 #pragma unroll
-            for (int c16 = 0; c16 < 8; ++c16) {
-              const uint4 uh = lds128(buf + row_off + ((c16 ^ sw) << 4));
-              uint4 ul = make_uint4(0, 0, 0, 0);
-              if (has_lo) ul = lds128(buf + EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4));
-              const uint32_t wh[4] = {uh.x, uh.y, uh.z, uh.w};
-              const uint32_t wl[4] = {ul.x, ul.y, ul.z, ul.w};
-              float* o = v + c16 * 8;
+              for (int c = 0; c < 4; ++c) {
+                const uint32_t c16 = (uint32_t)(half * 4 + c);
+                const uint4 uh = lds128(buf + row_off + ((c16 ^ sw) << 4));
+                uint4 ul = make_uint4(0, 0, 0, 0);
+                if (has_lo) ul = lds128(buf + EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4));
+                const uint32_t wh[4] = {uh.x, uh.y, uh.z, uh.w};
+                const uint32_t wl[4] = {ul.x, ul.y, ul.z, ul.w};
+                float* o = v + c * 8;
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float c0 = __uint_as_float(wh[e] << 16) + __uint_as_float(wl[e] << 16);
-                const float c1 = __uint_as_float(wh[e] & 0xffff0000u) + __uint_as_float(wl[e] & 0xffff0000u);
-                o[2 * e] = scale * fmaf(1.5f, c0, o[2 * e]);
-                o[2 * e + 1] = scale * fmaf(1.5f, c1, o[2 * e + 1]);
+                for (int e = 0; e < 4; ++e) {
+                  const float c0 = __uint_as_float(wh[e] << 16) + __uint_as_float(wl[e] << 16);
+                  const float c1 = __uint_as_float(wh[e] & 0xffff0000u) + __uint_as_float(wl[e] & 0xffff0000u);
+                  o[2 * e] = scale * fmaf(1.5f, c0, o[2 * e]);
+                  o[2 * e + 1] = scale * fmaf(1.5f, c1, o[2 * e + 1]);
+                }
               }
             }
+          } else if (KIND == 1) {
+            apply_c_direct(pr, scale, row, col0, v);
           }
-        } else if (KIND == 1) {
-          apply_c_direct(pr, scale, row, col0, v);
-          apply_c_direct(pr, scale, row, col0 + 32, v + 32);
-        }
-        // ---- outputs
-        const bool store_hi = KIND == 0 || epi == EPI_APPLY || (epi == EPI_APPLY_PACK && pr.store_out);
-        const bool store_lo = KIND == 1 && epi == EPI_APPLY;
-        if (store_hi) {
-          if (tma_out) {
+          // ---- outputs
+          if (store_hi) {
+            if (tma_out) {
 #pragma unroll
-            for (int c16 = 0; c16 < 8; ++c16) {
-              const float* o = v + c16 * 8;
-              uint32_t wh[4], wl[4];
+              for (int c = 0; c < 4; ++c) {
+                const uint32_t c16 = (uint32_t)(half * 4 + c);
+                const float* o = v + c * 8;
+                uint32_t wh[4], wl[4];
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                wh[e] = pack_bf16x2(o[2 * e], o[2 * e + 1]);
-                wl[e] = pack_bf16x2(o[2 * e] - __uint_as_float(wh[e] << 16),
-                                    o[2 * e + 1] - __uint_as_float(wh[e] & 0xffff0000u));
+                for (int e = 0; e < 4; ++e) {
+                  wh[e] = pack_bf16x2(o[2 * e], o[2 * e + 1]);
+                  wl[e] = pack_bf16x2(o[2 * e] - __uint_as_float(wh[e] << 16),
+                                      o[2 * e + 1] - __uint_as_float(wh[e] & 0xffff0000u));
+                }
+                sts128(buf + row_off + ((c16 ^ sw) << 4), make_uint4(wh[0], wh[1], wh[2], wh[3]));
+                if (store_lo) sts128(buf + EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4), make_uint4(wl[0], wl[1], wl[2], wl[3]));
               }
-              sts128(buf + row_off + ((c16 ^ sw) << 4), make_uint4(wh[0], wh[1], wh[2], wh[3]));
-              if (store_lo) sts128(buf + EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4), make_uint4(wl[0], wl[1], wl[2], wl[3]));
-            }
-            if (mirror) {
-              // transposed copy: element (j, r) of a 64 x 128 chunk kept as two {64 x 64} swizzled boxes
-              const uint32_t tb = buf + EPI_HALF_BYTES + (uint32_t)(r_in >> 6) * 8192u + (uint32_t)(r_in & 7) * 2u;
-              const uint32_t unit = (uint32_t)(r_in & 63) >> 3;
+              if (mirror) {
+                // transposed copy: element (j, r) of a 64 x 128 chunk kept as two {64 x 64} swizzled boxes
+                const uint32_t tb = buf + EPI_HALF_BYTES + (uint32_t)(r_in >> 6) * 8192u + (uint32_t)(r_in & 7) * 2u;
+                const uint32_t unit = (uint32_t)(r_in & 63) >> 3;
 #pragma unroll
-              for (int j = 0; j < 64; ++j) {
-                const uint16_t h = __bfloat16_as_ushort(__float2bfloat16_rn(v[j]));
-                asm volatile("st.shared.u16 [%0], %1;" ::"r"(tb + (uint32_t)j * 128u + ((unit ^ (uint32_t)(j & 7)) << 4)), "h"(h)
-                             : "memory");
+                for (int j = 0; j < 32; ++j) {
+                  const uint16_t h = __bfloat16_as_ushort(__float2bfloat16_rn(v[j]));
+                  const uint32_t jj = (uint32_t)(half * 32 + j);
+                  asm volatile("st.shared.u16 [%0], %1;" ::"r"(tb + jj * 128u + ((unit ^ (jj & 7u)) << 4)), "h"(h) : "memory");
+                }
               }
-            }
-            fence_async_smem();
-          } else {
-            store_out_direct(pr, row, col0, v, store_lo);
-            store_out_direct(pr, row, col0 + 32, v + 32, store_lo);
-          }
-        }
-        if (KIND == 1 && epi == EPI_APPLY_PACK) {
-          pack_bits_direct(pr, row, col0, v);
-          pack_bits_direct(pr, row, col0 + 32, v + 32);
-        } else if (KIND == 1 && epi == EPI_APPLY_UPDATE) {
-          update_weights_direct(pr, args.params, args.lr, row, col0, v);
-          update_weights_direct(pr, args.params, args.lr, row, col0 + 32, v + 32);
-        }
-        ok = epi_bar_and(c_ok);                  // every thread's part of the chunk is in shared memory
-        if (!ok) break;
-        if (leader) {
-          if (store_hi && tma_out && rows_live) {
-            tma_store_3d(args.tmaps + pr.tmapO0, col0, row0, pr.batch_o, buf);
-            if (store_lo) tma_store_3d(args.tmaps + pr.tmapO1, col0, row0, pr.batch_o, buf + EPI_HALF_BYTES);
-            if (mirror) {                        // rows col0.. of the output, columns row0.. (two 64-column boxes)
-              tma_store_3d(args.tmaps + pr.tmapOT, row0, col0, pr.batch_o, buf + EPI_HALF_BYTES);
-              if (row0 + 64 < pr.M)
-                tma_store_3d(args.tmaps + pr.tmapOT, row0 + 64, col0, pr.batch_o, buf + EPI_HALF_BYTES + 8192u);
+              fence_async_smem();
+            } else {
+              store_out_direct(pr, row, col0, v, store_lo);
             }
           }
-          bulk_commit();                         // one group per chunk (possibly empty) keeps the ring arithmetic fixed
+          if (KIND == 1 && epi == EPI_APPLY_PACK) pack_bits_direct(pr, row, col0, v);
+          else if (KIND == 1 && epi == EPI_APPLY_UPDATE) update_weights_direct(pr, args.params, args.lr, row, col0, v);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&buf_ready_bar[b]));   // this warp's part of the chunk is in shared memory
         }
-        __syncwarp();
       }
-      if (!ok) break;
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {                           // the accumulator may be overwritten (barrier of CTA 0)
-        if (CTAS == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
-        else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
-      }
-    }
-    if (leader) {
-      if (!ok && pf_issued > waited) {           // abort path: give the prefetches in flight a fixed 100 us to land
-        const uint64_t t0 = global_timer_ns();
-        while (global_timer_ns() - t0 < 100000ull) {}
-      }
-      bulk_wait_all();                           // stores must be complete before the CTA retires
     }
   }
 
