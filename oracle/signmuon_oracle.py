@@ -10,7 +10,8 @@ Notation (the paper uses M for both the momentum and the worker count; here
 `num_workers` is the worker count and `mom` the momentum buffer):
 
     Alg. 1  single-worker SignMuon          Alg. 2  distributed, int8 SUM all-reduce
-    Alg. 3  distributed, 1-bit all-gather   Alg. 4  PolarNS (scale = fro)
+    Alg. 3  distributed, 1-bit all-gather   Alg. 4  PolarNS (scale = fro or spectral)
+    Alg. 5  PowerIter (spectral-norm estimate; the sampled start vector is an input)
     Alg. 6  bare Newton-Schulz loop          Eq. 1   majority vote
     Eq. 2   normalised update S/sqrt(mn)     App. B  packed 1-bit representation
 
@@ -18,7 +19,9 @@ Pins (tests/test_oracle_pins.py): SVD closed form of the K-step map, the
 polar-factor error bound of the Newton-Schulz theorem, literal-vs-short-side
 equality, brute-force vote counting, int8-sum vs popcount vote, the packed size
 s1 = ceil(d/8) and the 32x ratio, the ResNet-50 worked example of App. B, and
-the closed form of the momentum recursion.  The end-to-end multi-step weight
+the closed form of the momentum recursion; for PowerIter: rank-one matrices
+(exact after one round), the diagonal closed form, the sigma_max lower bound and
+its limit against numpy's SVD, P = 0.  The end-to-end multi-step weight
 trajectory has no printed example in the paper: beyond the per-stage pins it is
 "parity unpinned".
 """
@@ -32,7 +35,7 @@ import numpy as np
 
 __all__ = [
     "OracleConfig", "ParamSpec", "OracleState",
-    "momentum_update", "frobenius_norm", "newton_schulz", "polar_ns",
+    "momentum_update", "frobenius_norm", "power_iter", "newton_schulz", "polar_ns",
     "polar_ns_short_side", "sign_pm1", "encode_bits", "decode_bits",
     "pack_bits", "unpack_bits", "bytes_to_words", "words_to_bytes",
     "majority_vote_sum", "majority_vote_popcount", "local_polar",
@@ -62,6 +65,9 @@ class OracleConfig:
     weight_decay: float = 0.0      # lambda
     eps: float = 1e-12             # epsilon of Alg. 4
     update_scale: int = 0          # 0: W -= eta*S (Alg. 2); 1: W -= eta*S/sqrt(rc) (Eq. 2)
+    ns_scale: str = "fro"          # Alg. 4 scale: "fro" or "spectral" (the workers' PolarNS; the local polar
+                                   # step keeps "fro": ||S_bar||_F = sqrt(rc) needs no sampled vector)
+    power_iters: int = 2           # P of Alg. 5 (the paper's experiments fix 2)
 
 
 @dataclass
@@ -100,6 +106,26 @@ def frobenius_norm(x):
     return math.sqrt(float(np.sum(x * x)))
 
 
+def power_iter(x, num_rounds, eps, v0):
+    """Alg. 5: estimate of ||X||_op by `num_rounds` rounds of power iteration on X^T X.
+
+    v0 is the "sampled" start vector of length c (an input here, so that runs are reproducible):
+        v <- v0 / (||v0|| + eps)
+        repeat P times:  u <- X v,  u <- u / (||u|| + eps);  v <- X^T u,  v <- v / (||v|| + eps)
+        return ||X v||
+    """
+    x = np.asarray(x, dtype=np.float64)
+    v = np.asarray(v0, dtype=np.float64).reshape(-1)
+    v = v / (math.sqrt(float(np.sum(v * v))) + eps)
+    for _ in range(num_rounds):
+        u = x @ v
+        u = u / (math.sqrt(float(np.sum(u * u))) + eps)
+        v = x.T @ u
+        v = v / (math.sqrt(float(np.sum(v * v))) + eps)
+    w = x @ v
+    return math.sqrt(float(np.sum(w * w)))
+
+
 def newton_schulz(y0, num_iters):
     """Alg. 6: Y_{k+1} = 1/2 Y_k (3 I - Y_k^T Y_k), K times, I the c x c identity."""
     y = np.array(y0, dtype=np.float64, copy=True)
@@ -110,15 +136,17 @@ def newton_schulz(y0, num_iters):
     return y
 
 
-def polar_ns(x, num_iters, eps=1e-12):
-    """Alg. 4 with scale = fro: sigma = ||X||_F ; Y = X / max(sigma, eps) ; K Newton-Schulz steps."""
+def polar_ns(x, num_iters, eps=1e-12, sigma=None):
+    """Alg. 4: sigma = ||X||_F (scale = fro; the default) or the caller's PowerIter estimate (scale =
+    spectral, passed as `sigma`); Y = X / max(sigma, eps); K Newton-Schulz steps."""
     x = np.asarray(x, dtype=np.float64)
-    sigma = frobenius_norm(x)
+    if sigma is None:
+        sigma = frobenius_norm(x)
     y = x / max(sigma, eps)
     return newton_schulz(y, num_iters)
 
 
-def polar_ns_short_side(x, num_iters, eps=1e-12):
+def polar_ns_short_side(x, num_iters, eps=1e-12, sigma=None):
     """Same map as polar_ns, with the Gram matrix taken on the shorter side.
 
     For r < c,  Y (3 I_c - Y^T Y) = (3 I_r - Y Y^T) Y, so the iteration may use the
@@ -128,8 +156,9 @@ def polar_ns_short_side(x, num_iters, eps=1e-12):
     x = np.asarray(x, dtype=np.float64)
     r, c = x.shape
     if r >= c:
-        return polar_ns(x, num_iters, eps)
-    sigma = frobenius_norm(x)
+        return polar_ns(x, num_iters, eps, sigma)
+    if sigma is None:
+        sigma = frobenius_norm(x)
     y = x / max(sigma, eps)
     eye = np.eye(r, dtype=np.float64)
     for _ in range(num_iters):
@@ -269,7 +298,7 @@ def init_state(params: Sequence[ParamSpec], cfg: OracleConfig) -> OracleState:
 
 
 def step_param(spec: ParamSpec, cfg: OracleConfig, mom, weight, grads, lr=None,
-               short_side=False, vote_bits_override=None) -> StepTrace:
+               short_side=False, vote_bits_override=None, power_start=None) -> StepTrace:
     """One SignMuon step for one parameter block.
 
     mom    [M, r, c] float64 momentum of every worker (input state)
@@ -278,6 +307,7 @@ def step_param(spec: ParamSpec, cfg: OracleConfig, mom, weight, grads, lr=None,
     vote_bits_override: if given (flat 0/1 array of d entries), stages after the vote
         use these bits instead of the oracle's own (staged parity: feed the oracle the
         vote another implementation produced).
+    power_start: [M, c] start vectors of PowerIter (needed when cfg.ns_scale == "spectral").
     """
     lr = cfg.lr if lr is None else lr
     M = cfg.num_workers
@@ -294,7 +324,10 @@ def step_param(spec: ParamSpec, cfg: OracleConfig, mom, weight, grads, lr=None,
     for m in range(M):                                     # "each worker m independently"
         new_mom[m] = momentum_update(mom[m], grads[m], weight64, cfg.momentum, cfg.weight_decay)
         if spec.kind == "matrix":
-            polar[m] = ns(new_mom[m], cfg.ns_steps, cfg.eps)   # U = PolarNS(Mom)
+            sigma = None
+            if cfg.ns_scale == "spectral":
+                sigma = power_iter(new_mom[m], cfg.power_iters, cfg.eps, np.asarray(power_start)[m])
+            polar[m] = ns(new_mom[m], cfg.ns_steps, cfg.eps, sigma)   # U = PolarNS(Mom)
         else:
             polar[m] = new_mom[m]                              # vector-like params: sign of the momentum
         bits[m] = encode_bits(polar[m]).reshape(-1)            # S = sign(U), encoded
@@ -317,7 +350,7 @@ def step_param(spec: ParamSpec, cfg: OracleConfig, mom, weight, grads, lr=None,
 
 
 def step(params: Sequence[ParamSpec], cfg: OracleConfig, state: OracleState, weights, grads,
-         lr=None, short_side=False):
+         lr=None, short_side=False, power_starts=None):
     """One optimizer step over all parameter blocks.
 
     weights: list of [r, c] arrays; grads: list of [M, r, c] arrays.  Returns
@@ -325,7 +358,8 @@ def step(params: Sequence[ParamSpec], cfg: OracleConfig, state: OracleState, wei
     """
     new_weights, traces = [], []
     for p, spec in enumerate(params):
-        tr = step_param(spec, cfg, state.mom[p], weights[p], grads[p], lr=lr, short_side=short_side)
+        tr = step_param(spec, cfg, state.mom[p], weights[p], grads[p], lr=lr, short_side=short_side,
+                        power_start=None if power_starts is None else power_starts[p])
         state.mom[p] = tr.mom
         new_weights.append(tr.new_weight)
         traces.append(tr)

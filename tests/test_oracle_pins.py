@@ -327,3 +327,72 @@ def test_step_local_polar_direction():
     flipped = 1 - tr[0].vote_bits
     tr2 = O.step_param(spec, cfg, np.zeros((4, 8, 5)), w, g, vote_bits_override=flipped)
     assert np.allclose(tr2.direction, -expect_d, rtol=1e-10, atol=1e-13)
+
+
+# --------------------------------------------------------------------------- #
+# Alg. 5 (PowerIter) and Alg. 4 with scale = spectral
+# --------------------------------------------------------------------------- #
+def test_power_iter_rank_one_is_exact_after_one_round():
+    # X = a b^T has one non-zero singular value ||a|| ||b||; X^T X v is parallel to b for any v not orthogonal to b.
+    rng = np.random.default_rng(3)
+    a, b, v0 = rng.standard_normal(7), rng.standard_normal(11), rng.standard_normal(11)
+    x = np.outer(a, b)
+    want = np.linalg.norm(a) * np.linalg.norm(b)
+    assert abs(O.power_iter(x, 1, 1e-300, v0) - want) <= 1e-12 * want
+    assert abs(O.power_iter(x, 4, 1e-300, v0) - want) <= 1e-12 * want
+    # P = 0: just ||X v0 / ||v0|| || = ||a|| |b . v0| / ||v0||
+    want0 = np.linalg.norm(a) * abs(b @ v0) / np.linalg.norm(v0)
+    assert abs(O.power_iter(x, 0, 1e-300, v0) - want0) <= 1e-12 * want0
+
+
+def test_power_iter_diagonal_closed_form():
+    # X = diag(s): after P rounds v is proportional to s^(2P) * v0, so the estimate is ||s^(2P+1) v0|| / ||s^(2P) v0||.
+    s = np.array([3.0, 2.0, 1.0, 0.5])
+    v0 = np.array([0.2, -0.7, 1.1, 0.4])
+    for P in (0, 1, 2, 5):
+        want = np.linalg.norm(s ** (2 * P + 1) * v0) / np.linalg.norm(s ** (2 * P) * v0)
+        assert abs(O.power_iter(np.diag(s), P, 1e-300, v0) - want) <= 1e-12 * want
+
+
+def test_power_iter_is_a_lower_bound_that_rises_to_sigma_max():
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((9, 14))
+    v0 = rng.standard_normal(14)
+    smax = np.linalg.svd(x, compute_uv=False)[0]
+    est = [O.power_iter(x, P, 1e-300, v0) for P in (0, 1, 2, 4, 8, 400)]
+    assert all(e <= smax * (1 + 1e-12) for e in est)                    # ||X v|| <= sigma_max for ||v|| <= 1
+    assert all(b >= a * (1 - 1e-12) for a, b in zip(est, est[1:]))      # Rayleigh quotients of (X^T X)^P v0 rise
+    assert abs(est[-1] - smax) <= 1e-9 * smax                           # and converge (spectral gap)
+    # a transposed operand or a missing normalisation would break either the bound or the limit
+    assert abs(O.power_iter(x.T, 400, 1e-300, rng.standard_normal(9)) - smax) <= 1e-9 * smax
+
+
+def test_power_iter_eps_enters_as_a_sum_and_zero_matrix_is_safe():
+    v0 = np.array([3.0, 4.0])
+    x = np.eye(2)
+    # v <- v0 / (5 + eps): with eps = 5 the start vector has norm 1/2; one round renormalises with (1/2 + 5)
+    got = O.power_iter(x, 0, 5.0, v0)
+    assert abs(got - 0.5) <= 1e-15
+    assert O.power_iter(np.zeros((3, 2)), 2, 1e-12, v0) == 0.0
+    assert np.all(O.polar_ns(np.zeros((3, 2)), 3, 1e-12, sigma=0.0) == 0.0)
+
+
+def test_spectral_scaling_reaches_the_polar_factor():
+    # With sigma ~ ||X||_op the singular values of Y0 lie in (0, ~1]; for a well-conditioned matrix K = 5
+    # cubic steps bring all of them to 1 within the theorem's bound.
+    rng = np.random.default_rng(5)
+    u, _ = np.linalg.qr(rng.standard_normal((6, 6)))
+    v, _ = np.linalg.qr(rng.standard_normal((10, 10)))
+    sv = np.array([1.0, 0.95, 0.9, 0.85, 0.8, 0.75])
+    x = 3.7 * (u * sv) @ v[:, :6].T
+    sigma = O.power_iter(x, 200, 1e-12, rng.standard_normal(10))
+    assert abs(sigma - 3.7) <= 1e-9
+    y = O.polar_ns(x, 5, 1e-12, sigma=sigma)
+    polar = u @ v[:, :6].T
+    rho = 1.0 - 0.75 ** 2                                               # ||I - Y0^T Y0||_op on the row space
+    assert np.linalg.norm(y - polar, 2) <= rho ** (2 ** 5) + 1e-12
+    # the step routes sigma through PowerIter when asked to
+    cfg = O.OracleConfig(num_workers=1, ns_steps=5, ns_scale="spectral", power_iters=200)
+    tr = O.step_param(O.ParamSpec(6, 10), cfg, np.zeros((1, 6, 10)), np.zeros((6, 10)), x[None] / (1 - cfg.momentum),
+                      power_start=rng.standard_normal((1, 10)))
+    assert np.linalg.norm(tr.polar[0] - polar, 2) <= 1e-6
