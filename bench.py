@@ -219,7 +219,15 @@ def run_ours(args, wl):
     B.load_library()
 
     opt = B.SignMuon(wl.params, wl.num_workers, momentum=wl.momentum, lr=wl.lr, ns_steps=wl.ns_steps,
-                     local_polar=wl.local_polar, device=dev, host_staging=True)
+                     local_polar=wl.local_polar, device=dev, host_staging=True, ns_scale=args.ns_scale,
+                     power_iters=args.power_iters)
+    if args.ns_scale == "spectral":     # seeded start vectors of the power iteration, reused by every step
+        flat = torch.zeros(opt.power_start_size, dtype=torch.float32, device=dev)
+        for p, v in enumerate(wlmod.make_power_start(wl, 0, dev)):
+            if v is not None:
+                off, _ = opt.power_start_segment(p)
+                flat[off: off + v.numel()] = v.reshape(-1)
+        opt.set_power_start(flat)
     weights = wlmod.make_weights(wl, dev)
     signal = wlmod.make_signal(wl, dev)
     n_sets = 2                                           # fresh noise per step, rotating pre-drawn sets
@@ -298,6 +306,8 @@ def run_ours(args, wl):
         sum(p.numel * (M * (gb[p.dtype] + 8) + 2 * gb[p.dtype] + M / 8 + 1 / 8) for p in plain)
     vote_bytes = sum(p.numel * (M / 8 + 1 / 8 + (2 if wl.local_polar else 2 * gb[p.dtype])) for p in mat)
     n_ns_launches = 2 * wl.ns_steps
+    if args.ns_scale == "spectral":      # the power iteration reads the float32 momentum 2P + 1 more times
+        mom_bytes += sum(M * p.numel * 4 * (2 * args.power_iters + 1) for p in mat)
     kernels = {}
     if stage_ms["momentum"] > 0:
         kernels["momentum+plain"] = {"ms": stage_ms["momentum"], "bound": "hbm", "algorithmic_bytes": mom_bytes,
@@ -339,7 +349,9 @@ def run_ours(args, wl):
 
     line = {"metric": METRIC, "value": whole_job_value(ms_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": describe(wl),
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": dict(describe(wl), ns_scale=args.ns_scale,
+                           **({"power_iters": args.power_iters} if args.ns_scale == "spectral" else {})),
             "clocks": clocks,
             "e2e": (None if args.no_e2e else
                     {"value": whole_job_value(e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -423,6 +435,9 @@ def main():
                     help="float64 operation budget of one oracle sample step")
     ap.add_argument("--cpu-baseline-flops", type=float, default=8e11,
                     help="float64 operation budget of the oracle sample timed beside the GPU run")
+    ap.add_argument("--ns-scale", default="fro", choices=["fro", "spectral"],
+                    help="Alg. 4 scale: Frobenius norm (default, the benchmark configuration) or power iteration")
+    ap.add_argument("--power-iters", type=int, default=2)
     ap.add_argument("--sweep", action="store_true", help="run the kernel sweep (config 5) and print one line per point")
     ap.add_argument("--sweep-workers", default="1,2,4,8,16,32")
     args = ap.parse_args()

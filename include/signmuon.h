@@ -88,7 +88,13 @@ typedef struct {
   float eps;                    /* Alg. 4 stability constant; <= 0 selects 1e-12 */
   int32_t update_scale;         /* 0: W -= eta S (Alg. 2)   1: W -= eta S / sqrt(rows cols) (Eq. 2) */
   int32_t flags;                /* SIGNMUON_FLAG_* */
+  int32_t ns_scale;             /* Alg. 4 "scale" of the workers' PolarNS: SIGNMUON_SCALE_FRO (sigma = ||Mom||_F) or
+                                   SIGNMUON_SCALE_SPECTRAL (sigma = PowerIter(Mom, power_iters, eps), Alg. 5).  The
+                                   local polar step always uses ||S||_F = sqrt(rows cols). */
+  int32_t power_iters;          /* P of Alg. 5, 0..64 (the paper's experiments use 2); ignored for SCALE_FRO */
 } signmuon_config;
+
+enum { SIGNMUON_SCALE_FRO = 0, SIGNMUON_SCALE_SPECTRAL = 1 };
 
 enum {
   SIGNMUON_FLAG_KEEP_POLAR = 1,   /* also store U_m = Y_K (bf16) so that signmuon_debug_tap can return it */
@@ -174,6 +180,20 @@ int signmuon_debug_tap(const signmuon_ctx* ctx, int32_t what, int32_t param, int
 /* Synchronises `cuda_stream`, then reads the device status word: OK, TIMEOUT (a bounded wait in a
  * kernel gave up; results of that step are invalid) or CUDA. */
 int signmuon_status(signmuon_ctx* ctx, void* cuda_stream);
+
+/* Start vectors of the power iteration (Alg. 5, "Sample v in R^c"), needed when ns_scale is
+ * SIGNMUON_SCALE_SPECTRAL: the method draws them at random, so the caller passes them in.
+ *   signmuon_power_start_size:    length in floats of the whole array (0 when the scale is FRO)
+ *   signmuon_power_start_segment: where the vectors of matrix parameter `param` start inside it; worker m's
+ *                                 vector (cols floats) follows at float_offset + m * floats_per_worker
+ *   signmuon_set_power_start:     DEVICE array (16-byte aligned, owned by the caller, read by every following
+ *                                 step until replaced; fill it with fresh draws between steps as desired).
+ * Errors: INVALID_ARG (scale is FRO, plain parameter, null), NOT_BOUND, BUFFER_TOO_SMALL, MISALIGNED;
+ * signmuon_step returns NOT_BOUND when the scale is SPECTRAL and no start vectors were set. */
+int signmuon_power_start_size(const signmuon_ctx* ctx, size_t* floats);
+int signmuon_power_start_segment(const signmuon_ctx* ctx, int32_t param, size_t* float_offset,
+                                 size_t* floats_per_worker);
+int signmuon_set_power_start(signmuon_ctx* ctx, const float* dev_vectors, size_t floats);
 
 /* Number of kernels signmuon_step launches per call with the current configuration. */
 int signmuon_launches_per_step(const signmuon_ctx* ctx, int32_t* launches);

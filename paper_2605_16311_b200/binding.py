@@ -27,6 +27,7 @@ EXPORTS = [
     "signmuon_create", "signmuon_state_bytes", "signmuon_bind", "signmuon_step", "signmuon_run_stages",
     "signmuon_step_host", "signmuon_packed_payload", "signmuon_payload_segment", "signmuon_debug_tap",
     "signmuon_status", "signmuon_launches_per_step", "signmuon_ns_flops_per_step",
+    "signmuon_power_start_size", "signmuon_power_start_segment", "signmuon_set_power_start",
     "signmuon_momentum_norm_noalloc", "signmuon_destroy", "signmuon_error_string",
 ]
 NOALLOC_MAX_PARTIALS = 65536
@@ -42,7 +43,8 @@ class ConfigStruct(C.Structure):
     _fields_ = [("num_params", C.c_int32), ("params", C.POINTER(ParamStruct)),
                 ("num_workers", C.c_int32), ("momentum", C.c_float), ("lr", C.c_float),
                 ("ns_steps", C.c_int32), ("local_polar", C.c_int32), ("weight_decay", C.c_float),
-                ("eps", C.c_float), ("update_scale", C.c_int32), ("flags", C.c_int32)]
+                ("eps", C.c_float), ("update_scale", C.c_int32), ("flags", C.c_int32),
+                ("ns_scale", C.c_int32), ("power_iters", C.c_int32)]
 
 
 _lib = None
@@ -70,6 +72,9 @@ def load_library() -> C.CDLL:
     lib.signmuon_status.argtypes = [vp, vp]
     lib.signmuon_launches_per_step.argtypes = [vp, C.POINTER(i32)]
     lib.signmuon_ns_flops_per_step.argtypes = [vp, C.POINTER(C.c_double)]
+    lib.signmuon_power_start_size.argtypes = [vp, C.POINTER(sz)]
+    lib.signmuon_power_start_segment.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
+    lib.signmuon_set_power_start.argtypes = [vp, vp, sz]
     lib.signmuon_momentum_norm_noalloc.argtypes = [vp, i32, vp, i32, vp, vp, vp, C.c_int64, C.c_int64, i32,
                                                    f32, f32, f32, vp]
     lib.signmuon_destroy.argtypes = [vp]
@@ -97,14 +102,14 @@ def _check(code: int, where: str):
 # ------------------------------------------------------------------------- C-ABI mirrors
 def signmuon_create(params: Sequence[tuple], num_workers: int, momentum: float, lr: float, ns_steps: int,
                     local_polar: bool, weight_decay: float = 0.0, eps: float = 1e-12, update_scale: int = 0,
-                    flags: int = 0) -> int:
+                    flags: int = 0, ns_scale: int = 0, power_iters: int = 2) -> int:
     """params: (rows, cols, kind, weight_dtype, grad_dtype) tuples. Returns the context handle."""
     lib = load_library()
     arr = (ParamStruct * max(len(params), 1))()
     for i, (r, c, k, wd, gd) in enumerate(params):
         arr[i] = ParamStruct(r, c, k, wd, gd)
     cfg = ConfigStruct(len(params), arr, num_workers, momentum, lr, ns_steps, int(local_polar), weight_decay,
-                       eps, update_scale, flags)
+                       eps, update_scale, flags, ns_scale, power_iters)
     out = C.c_void_p()
     _check(lib.signmuon_create(C.byref(cfg), C.byref(out)), "signmuon_create")
     return out.value
@@ -190,6 +195,23 @@ def signmuon_ns_flops_per_step(ctx: int) -> float:
     return f.value
 
 
+def signmuon_power_start_size(ctx: int) -> int:
+    n = C.c_size_t()
+    _check(load_library().signmuon_power_start_size(ctx, C.byref(n)), "signmuon_power_start_size")
+    return n.value
+
+
+def signmuon_power_start_segment(ctx: int, param: int):
+    o, n = C.c_size_t(), C.c_size_t()
+    _check(load_library().signmuon_power_start_segment(ctx, param, C.byref(o), C.byref(n)),
+           "signmuon_power_start_segment")
+    return o.value, n.value
+
+
+def signmuon_set_power_start(ctx: int, ptr: int, floats: int):
+    _check(load_library().signmuon_set_power_start(ctx, ptr, floats), "signmuon_set_power_start")
+
+
 def signmuon_momentum_norm_noalloc(grads_ptr: int, grad_dtype: int, weights_ptr: int, weight_dtype: int,
                                    momentum_ptr: int, operand_ptr: int, scales_ptr: int, rows: int, cols: int,
                                    num_workers: int, momentum: float, weight_decay: float, eps: float,
@@ -209,6 +231,7 @@ def signmuon_destroy(ctx: int):
 # ------------------------------------------------------------------------- convenience wrapper
 _DT = {"f32": F32, "bf16": BF16}
 _KIND = {"matrix": PARAM_MATRIX, "plain": PARAM_PLAIN}
+SCALES = {"fro": 0, "spectral": 1}
 
 
 def _view_device(ptr: int, nbytes: int, dtype: torch.dtype, owner: torch.Tensor, base_ptr: int) -> torch.Tensor:
@@ -223,14 +246,15 @@ class SignMuon:
 
     def __init__(self, params, num_workers: int, momentum: float = 0.9, lr: float = 1e-3, ns_steps: int = 5,
                  local_polar: bool = False, weight_decay: float = 0.0, eps: float = 1e-12, update_scale: int = 0,
-                 flags: int = 0, device: str = "cuda:0", host_staging: bool = False):
+                 flags: int = 0, device: str = "cuda:0", host_staging: bool = False, ns_scale: str = "fro",
+                 power_iters: int = 2):
         self.params = list(params)
         self.num_workers = num_workers
         self.ns_steps = ns_steps
         self.device = torch.device(device)
         tuples = [(p.rows, p.cols, _KIND[p.kind], _DT[p.dtype], _DT[p.dtype]) for p in self.params]
         self.ctx = signmuon_create(tuples, num_workers, momentum, lr, ns_steps, local_polar, weight_decay, eps,
-                                   update_scale, flags)
+                                   update_scale, flags, SCALES[ns_scale], power_iters)
         self.state_bytes, self.workspace_bytes, self.staging_bytes = signmuon_state_bytes(self.ctx)
         with torch.cuda.device(self.device):
             self.state = torch.empty(self.state_bytes, dtype=torch.uint8, device=self.device)
@@ -296,6 +320,20 @@ class SignMuon:
         if what == TAP_NORM:
             return _view_device(ptr, nbytes, torch.float32, self.workspace, base)
         raise ValueError(what)
+
+    def power_start_segment(self, param: int):
+        """(offset, floats per worker) of a matrix parameter's start vectors inside the start-vector array."""
+        return signmuon_power_start_segment(self.ctx, param)
+
+    @property
+    def power_start_size(self) -> int:
+        return signmuon_power_start_size(self.ctx)
+
+    def set_power_start(self, vectors: torch.Tensor):
+        """float32 device tensor of power_start_size floats: the sampled start vectors of Alg. 5; the caller keeps it alive."""
+        assert vectors.dtype == torch.float32 and vectors.is_cuda and vectors.is_contiguous()
+        self._power_start = vectors
+        signmuon_set_power_start(self.ctx, vectors.data_ptr(), vectors.numel())
 
     @property
     def launches_per_step(self) -> int:

@@ -30,6 +30,11 @@ struct ParamDev {
   uint32_t chunks_per_worker;  // momentum-kernel blocks (= norm partials) per worker
   float upd_scale;      // 1, or 1/sqrt(rows*cols) for the Eq. 2 normalisation
   int32_t vec_ok;       // 16-byte vector path allowed (d % 8 == 0 and ldy == cols)
+  // power iteration (scale = spectral): un-normalised vectors and their norms
+  float* pi_v;          // [M][cols]
+  float* pi_u;          // [M][rows]
+  float* pi_scal;       // [M][2] = {||v||, ||u||}
+  const float* pi_start;// [M][cols] the caller's start vectors
 };
 
 // Epilogues of the Newton-Schulz products.

@@ -15,6 +15,7 @@
 #include "common.cuh"
 #include "elementwise.cuh"
 #include "ns_gemm_simt.cuh"
+#include "power_iter.cuh"
 #include "ns_gemm_sm100.cuh"
 
 using namespace signmuon;
@@ -38,6 +39,8 @@ struct ParamPlan {
   size_t y_off[2], lo_off, q_off, scales_off, partials_off;   // bytes into the workspace (matrix params)
   int tmap_base;         // first of this parameter's TM_PER_PARAM tensor maps
   size_t stage_w_off, stage_g_off;                    // bytes into the host-staging buffer
+  size_t pi_v_off, pi_u_off, pi_scal_off;             // power iteration (scale = spectral), bytes into the workspace
+  size_t pi_start_off;                                // floats into the caller's start-vector array
 };
 
 // indices of a parameter's tensor maps relative to tmap_base
@@ -66,8 +69,10 @@ struct signmuon_ctx {
   std::vector<signmuon_param> params;
   std::vector<ParamPlan> plan;
   std::vector<int32_t> matrix_list, plain_list, packfb_list;
-  std::vector<uint32_t> mom_starts, plain_starts, vote_starts, packfb_starts;
-  uint32_t mom_blocks = 0, plain_blocks = 0, vote_blocks = 0, packfb_blocks = 0;
+  std::vector<uint32_t> mom_starts, plain_starts, vote_starts, packfb_starts, xv_starts, xtu_starts;
+  uint32_t mom_blocks = 0, plain_blocks = 0, vote_blocks = 0, packfb_blocks = 0, xv_blocks = 0, xtu_blocks = 0;
+  size_t power_start_floats = 0;          // length of the start-vector array (scale = spectral)
+  const float* d_power_start = nullptr;   // caller's start vectors (device)
   uint64_t words_per_worker = 0;
   int64_t entries = 0;
   size_t state_bytes = 0, workspace_bytes = 0, staging_bytes = 0;
@@ -75,7 +80,7 @@ struct signmuon_ctx {
   size_t off_status = 0, off_paramdev = 0, off_lists = 0, off_bits = 0, off_vote = 0, off_tmaps = 0,
          off_problems = 0, off_tables_end = 0;
   size_t off_list_matrix = 0, off_list_plain = 0, off_list_packfb = 0, off_starts_mom = 0, off_starts_plain = 0,
-         off_starts_vote = 0, off_starts_packfb = 0;
+         off_starts_vote = 0, off_starts_packfb = 0, off_starts_xv = 0, off_starts_xtu = 0;
   // GEMM plans
   std::vector<GemmProblem> problems;      // pointers filled at bind
   std::vector<LaunchPlan> ns_launches, lp_launches;
@@ -302,6 +307,24 @@ int plan_layout(signmuon_ctx* c) {
   }
   if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
   c->packfb_blocks = (uint32_t)b;
+  const bool spectral = c->cfg.ns_scale == SIGNMUON_SCALE_SPECTRAL && K > 0;
+  if (spectral) {
+    uint64_t bx = 0, bt = 0;
+    size_t nf = 0;
+    for (int32_t p : c->matrix_list) {
+      ParamPlan& pl = c->plan[p];
+      c->xv_starts.push_back((uint32_t)bx);
+      c->xtu_starts.push_back((uint32_t)bt);
+      bx += (uint64_t)M * ((pl.rows + PI_ROWS_PER_BLOCK - 1) / PI_ROWS_PER_BLOCK);
+      bt += (uint64_t)M * ((pl.cols + PI_COLS_PER_BLOCK - 1) / PI_COLS_PER_BLOCK);
+      pl.pi_start_off = nf;
+      nf += (size_t)M * pl.cols;
+    }
+    if (bx >= (1ull << 31) || bt >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
+    c->xv_blocks = (uint32_t)bx;
+    c->xtu_blocks = (uint32_t)bt;
+    c->power_start_floats = nf;
+  }
 
   // workspace layout: small tables first, then the large buffers
   size_t off = 0;
@@ -315,10 +338,17 @@ int plan_layout(signmuon_ctx* c) {
   place(c->off_starts_plain, c->plain_starts.size() * 4);
   place(c->off_starts_vote, c->vote_starts.size() * 4);
   place(c->off_starts_packfb, c->packfb_starts.size() * 4);
+  place(c->off_starts_xv, c->xv_starts.size() * 4);
+  place(c->off_starts_xtu, c->xtu_starts.size() * 4);
   for (int32_t p : c->matrix_list) {
     ParamPlan& pl = c->plan[p];
     pl.scales_off = off; off += round_up((size_t)M * 8, ALIGN);
     pl.partials_off = off; off += round_up((size_t)M * pl.chunks_per_worker * 4, ALIGN);
+    if (spectral) {
+      pl.pi_v_off = off; off += round_up((size_t)M * pl.cols * 4, ALIGN);
+      pl.pi_u_off = off; off += round_up((size_t)M * pl.rows * 4, ALIGN);
+      pl.pi_scal_off = off; off += round_up((size_t)M * 8, ALIGN);
+    }
   }
   c->off_bits = off; off += round_up((size_t)M * words * 4, ALIGN);
   c->off_vote = off; off += round_up((size_t)words * 4, ALIGN);
@@ -566,6 +596,7 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
   if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
   if (c->sticky != SIGNMUON_OK) return c->sticky;
   if (!weights || !grads) return SIGNMUON_ERR_INVALID_ARG;
+  if ((mask & SIGNMUON_STAGE_MOMENTUM) && c->power_start_floats && !c->d_power_start) return SIGNMUON_ERR_NOT_BOUND;
   if (lr < 0.f) lr = c->cfg.lr;
   int rc = upload_params(c, weights, grads, s);
   if (rc != SIGNMUON_OK) return rc;
@@ -581,9 +612,24 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
       momentum_kernel<<<c->mom_blocks, EW_THREADS, 0, s>>>(
           pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_matrix),
           reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_mom), nm, c->cfg.momentum, c->cfg.weight_decay);
-      const int warps = nm * M;
-      finalize_norms_kernel<<<(warps * 32 + 255) / 256, 256, 0, s>>>(
-          pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_matrix), nm, M, eps);
+      const int32_t* mlist = reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_matrix);
+      if (c->power_start_floats) {
+        // scale = spectral (Alg. 4): sigma from P rounds of power iteration on the momentum (Alg. 5)
+        const uint32_t* xs = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_xv);
+        const uint32_t* ts = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_xtu);
+        pi_norm_kernel<<<nm * M, EW_THREADS, 0, s>>>(pd, mlist, M, PI_NORM_START, eps);
+        for (int it = 0; it < c->cfg.power_iters; ++it) {
+          pi_xv_kernel<<<c->xv_blocks, EW_THREADS, 0, s>>>(pd, mlist, xs, nm, eps);
+          pi_norm_kernel<<<nm * M, EW_THREADS, 0, s>>>(pd, mlist, M, PI_NORM_U, eps);
+          pi_xtu_kernel<<<c->xtu_blocks, EW_THREADS, 0, s>>>(pd, mlist, ts, nm, eps);
+          pi_norm_kernel<<<nm * M, EW_THREADS, 0, s>>>(pd, mlist, M, PI_NORM_V, eps);
+        }
+        pi_xv_kernel<<<c->xv_blocks, EW_THREADS, 0, s>>>(pd, mlist, xs, nm, eps);
+        pi_norm_kernel<<<nm * M, EW_THREADS, 0, s>>>(pd, mlist, M, PI_NORM_SIGMA, eps);
+      } else {
+        const int warps = nm * M;
+        finalize_norms_kernel<<<(warps * 32 + 255) / 256, 256, 0, s>>>(pd, mlist, nm, M, eps);
+      }
     }
     if (np) {
       plain_params_kernel<<<c->plain_blocks, EW_THREADS, 0, s>>>(
@@ -631,6 +677,8 @@ int signmuon_create(const signmuon_config* config, signmuon_ctx** out) {
   if (!(config->lr == config->lr)) return SIGNMUON_ERR_INVALID_ARG;
   if (config->update_scale != 0 && config->update_scale != 1) return SIGNMUON_ERR_INVALID_ARG;
   if (config->local_polar != 0 && config->local_polar != 1) return SIGNMUON_ERR_INVALID_ARG;
+  if (config->ns_scale != SIGNMUON_SCALE_FRO && config->ns_scale != SIGNMUON_SCALE_SPECTRAL) return SIGNMUON_ERR_INVALID_ARG;
+  if (config->power_iters < 0 || config->power_iters > 64) return SIGNMUON_ERR_INVALID_ARG;
   for (int i = 0; i < config->num_params; ++i) {
     const signmuon_param& p = config->params[i];
     if (p.rows < 1 || p.cols < 1 || p.rows > (1 << 24) || p.cols > (1 << 24)) return SIGNMUON_ERR_BAD_SHAPE;
@@ -701,6 +749,12 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
       d.y1 = reinterpret_cast<bf16*>(c->d_ws + pl.y_off[1]);
       d.scales = reinterpret_cast<float*>(c->d_ws + pl.scales_off);
       d.partials = reinterpret_cast<float*>(c->d_ws + pl.partials_off);
+      if (c->power_start_floats) {
+        d.pi_v = reinterpret_cast<float*>(c->d_ws + pl.pi_v_off);
+        d.pi_u = reinterpret_cast<float*>(c->d_ws + pl.pi_u_off);
+        d.pi_scal = reinterpret_cast<float*>(c->d_ws + pl.pi_scal_off);
+        d.pi_start = c->d_power_start ? c->d_power_start + pl.pi_start_off : nullptr;
+      }
     }
     d.d = pl.d; d.rows = (int32_t)pl.rows; d.cols = (int32_t)pl.cols; d.ldy = pl.ldy;
     d.kind = pl.kind; d.wdtype = pl.wdtype; d.gdtype = pl.gdtype;
@@ -718,6 +772,8 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
   ok = ok && up(c->off_starts_plain, c->plain_starts.data(), c->plain_starts.size() * 4);
   ok = ok && up(c->off_starts_vote, c->vote_starts.data(), c->vote_starts.size() * 4);
   ok = ok && up(c->off_starts_packfb, c->packfb_starts.data(), c->packfb_starts.size() * 4);
+  ok = ok && up(c->off_starts_xv, c->xv_starts.data(), c->xv_starts.size() * 4);
+  ok = ok && up(c->off_starts_xtu, c->xtu_starts.data(), c->xtu_starts.size() * 4);
   if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
 
   // tile tables (need the SM count) and tensor maps (need the device addresses)
@@ -899,11 +955,40 @@ int signmuon_status(signmuon_ctx* c, void* cuda_stream) {
   return word == STATUS_OK ? SIGNMUON_OK : SIGNMUON_ERR_TIMEOUT;
 }
 
+int signmuon_power_start_size(const signmuon_ctx* c, size_t* floats) {
+  if (!c || !floats) return SIGNMUON_ERR_INVALID_ARG;
+  *floats = c->power_start_floats;
+  return SIGNMUON_OK;
+}
+
+int signmuon_power_start_segment(const signmuon_ctx* c, int32_t param, size_t* float_offset, size_t* floats_per_worker) {
+  if (!c || param < 0 || param >= (int32_t)c->params.size()) return SIGNMUON_ERR_INVALID_ARG;
+  if (c->plan[param].kind != SIGNMUON_PARAM_MATRIX || c->power_start_floats == 0) return SIGNMUON_ERR_INVALID_ARG;
+  if (float_offset) *float_offset = c->plan[param].pi_start_off;
+  if (floats_per_worker) *floats_per_worker = (size_t)c->plan[param].cols;
+  return SIGNMUON_OK;
+}
+
+int signmuon_set_power_start(signmuon_ctx* c, const float* dev_vectors, size_t floats) {
+  if (!c) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  if (c->power_start_floats == 0) return SIGNMUON_ERR_INVALID_ARG;
+  if (!dev_vectors) return SIGNMUON_ERR_INVALID_ARG;
+  if (floats < c->power_start_floats) return SIGNMUON_ERR_BUFFER_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(dev_vectors) & 15) return SIGNMUON_ERR_MISALIGNED;
+  if (c->d_power_start != dev_vectors) {
+    c->d_power_start = dev_vectors;
+    for (int32_t p : c->matrix_list) c->paramdev[p].pi_start = dev_vectors + c->plan[p].pi_start_off;
+    c->paramdev_uploaded = false;     // the table goes to the device again with the next step
+  }
+  return SIGNMUON_OK;
+}
+
 int signmuon_launches_per_step(const signmuon_ctx* c, int32_t* launches) {
   if (!c || !launches) return SIGNMUON_ERR_INVALID_ARG;
   int n = 0;
   const bool nm = !c->matrix_list.empty();
-  if (nm) n += 2;                                   // momentum + norms
+  if (nm) n += 1 + (c->power_start_floats ? 3 + 4 * c->cfg.power_iters : 1);   // momentum + norms (or power iteration)
   if (!c->plain_list.empty()) n += 1;
   if (nm) n += (int)c->ns_launches.size() + (c->packfb_blocks ? 1 : 0) + 1;   // NS, fallback pack, vote
   if (nm && c->cfg.local_polar && c->cfg.ns_steps > 0) n += (int)c->lp_launches.size();

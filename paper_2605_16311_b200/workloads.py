@@ -221,3 +221,16 @@ def make_grads(wl: Workload, signal: List[torch.Tensor], step: int, device="cpu"
             t = out[p_idx]
         res.append(t)
     return res
+
+
+def make_power_start(wl: Workload, step: int, device="cpu") -> List[Optional[torch.Tensor]]:
+    """Start vectors of the power iteration (the method "samples" them: here seeded standard normals),
+    one [num_workers, cols] float32 tensor per matrix parameter, None for plain parameters."""
+    out: List[Optional[torch.Tensor]] = []
+    for p_idx, p in enumerate(wl.params):
+        if p.kind != "matrix":
+            out.append(None)
+            continue
+        g = _generator(device, wl.config_id, 404, step, p_idx)
+        out.append(torch.randn((wl.num_workers, p.cols), generator=g, device=device, dtype=torch.float32))
+    return out

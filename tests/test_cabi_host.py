@@ -104,3 +104,28 @@ def test_ragged_parameter_pads_to_words():
     # momentum, norms, 2x2 NS products, fallback pack (11 columns do not fill words), vote, plain kernel
     assert B.signmuon_launches_per_step(ctx) == 2 + 1 + 4 + 1 + 1
     B.signmuon_destroy(ctx)
+
+
+def test_power_start_layout_and_errors():
+    lib = B.load_library()
+    # Frobenius scale: no start vectors
+    ctx = B.signmuon_create([(8, 12, 0, 0, 0)], 2, 0.9, 1e-3, 5, False)
+    assert B.signmuon_power_start_size(ctx) == 0
+    assert lib.signmuon_power_start_segment(ctx, 0, None, None) == -1
+    B.signmuon_destroy(ctx)
+    # spectral scale: [M][cols] floats per matrix parameter, in creation order; plain parameters have none
+    params = [(8, 12, 0, 0, 0), (1, 40, 1, 0, 0), (20, 6, 0, 0, 0)]
+    ctx = B.signmuon_create(params, 3, 0.9, 1e-3, 5, False, ns_scale=1, power_iters=2)
+    assert B.signmuon_power_start_size(ctx) == 3 * 12 + 3 * 6
+    assert B.signmuon_power_start_segment(ctx, 0) == (0, 12)
+    assert B.signmuon_power_start_segment(ctx, 2) == (36, 6)
+    assert lib.signmuon_power_start_segment(ctx, 1, None, None) == -1      # plain parameter
+    assert lib.signmuon_set_power_start(ctx, C.c_void_p(4096), 54) == -3     # not bound yet
+    # momentum, start norm + 2 rounds x 4 + final matvec + sigma, 5 x 2 NS products, fallback pack, vote, plain kernel
+    assert B.signmuon_launches_per_step(ctx) == 1 + (3 + 8) + 10 + 1 + 1 + 1
+    B.signmuon_destroy(ctx)
+    for kw in (dict(ns_scale=2), dict(ns_scale=-1), dict(power_iters=-1), dict(power_iters=65)):
+        cfg = _cfg([(64, 64, 0, 0, 0)])
+        for k, v in kw.items():
+            setattr(cfg, k, v)
+        assert B.signmuon_create_raw(cfg)[0] == -1, kw

@@ -40,6 +40,36 @@ def test_one_cta_tile_variant_ragged_and_local_polar():
     run_and_check(_wl([(200, 328), (328, 200), (256, 256)], 2, local_polar=True, lr=0.01), steps=1, flags=flags)
 
 
+@pytest.mark.parametrize("P,K", [(0, 1), (1, 1), (2, 5), (3, 5), (2, 3)])
+def test_spectral_scaling_power_iteration(P, K):
+    """Alg. 4 with scale = spectral: sigma from P rounds of Alg. 5 on the momentum, start vectors passed in.
+    With P < 2 the estimate can lie so far below the spectral norm that the cubic iteration leaves its
+    basin (singular values of Y_0 above sqrt 3) and the result is decided by cancellation: those cases check
+    sigma, the pack, the vote and the update, not the Newton-Schulz values."""
+    from parity_utils import run_and_check
+    shapes = [(200, 328), (328, 200), (64, 147), (256, 256), (1, 160)]
+    wl = _wl(shapes, 3, K=K, extra={"ns_scale": "spectral", "power_iters": P})
+    rep = run_and_check(wl, steps=2, check_polar=P >= 2)
+    assert "sigma_rel" in rep
+    print(rep)
+    if P >= 2:
+        wl = _wl([(128, 384), (384, 128)], 2, K=K, local_polar=True, lr=0.01,
+                 extra={"ns_scale": "spectral", "power_iters": P})
+        run_and_check(wl, steps=1)
+
+
+def test_spectral_scaling_needs_start_vectors():
+    wl = _wl([(64, 64)], 2, extra={"ns_scale": "spectral"})
+    from parity_utils import make_optimizer
+    opt = make_optimizer(wl)
+    w = wlmod.make_weights(wl, "cuda:0")
+    g = wlmod.make_grads(wl, wlmod.make_signal(wl, "cuda:0"), 0, "cuda:0")
+    with pytest.raises(B.SignMuonError) as e:
+        opt.step(w, g, 1e-3)
+    assert e.value.code == -3
+    opt.close()
+
+
 def test_config1_ten_steps():
     from parity_utils import run_and_check
     rep = run_and_check(wlmod.config1(), steps=10)
