@@ -42,9 +42,11 @@ def _np64(t: torch.Tensor) -> np.ndarray:
 
 def check_param_step(opt: B.SignMuon, wl, p_idx: int, w_before: torch.Tensor, w_after: torch.Tensor,
                      grads: torch.Tensor, mom_before: Optional[np.ndarray], lr: float, weight_decay: float = 0.0,
-                     check_polar: bool = True, report: Optional[dict] = None, power_start=None, power_iters: int = 2):
+                     check_polar: bool = True, report: Optional[dict] = None, power_start=None, power_iters: int = 2,
+                     ns_workers: Optional[Sequence[int]] = None):
     """Checks every stage of parameter p_idx for the step just run. Returns the oracle momentum
-    (float64, [M, r, c]) evolved from `mom_before` (None = zeros)."""
+    (float64, [M, r, c]) evolved from `mom_before` (None = zeros).  `ns_workers` restricts the Newton-Schulz
+    comparison (the costly part of the oracle) to those workers; every other stage covers all workers."""
     p = wl.params[p_idx]
     M, r, c, d = wl.num_workers, p.rows, p.cols, p.rows * p.cols
     K = wl.ns_steps
@@ -71,7 +73,7 @@ def check_param_step(opt: B.SignMuon, wl, p_idx: int, w_before: torch.Tensor, w_
             assert last >> (d % 32) == 0
 
     if p.kind == "matrix":
-        for m in range(M):
+        for m in (range(M) if ns_workers is None else ns_workers):
             # ---- norm
             scales = opt.tap(B.TAP_NORM, p_idx, m).cpu().numpy().astype(np.float64)
             if power_start is None:
@@ -161,7 +163,8 @@ def check_param_step(opt: B.SignMuon, wl, p_idx: int, w_before: torch.Tensor, w_
 
 
 def run_and_check(wl, steps: int, flags: int = B.FLAG_KEEP_POLAR, sample: Optional[Sequence[int]] = None,
-                  device: str = "cuda:0", check_polar: bool = True, report: Optional[dict] = None):
+                  device: str = "cuda:0", check_polar: bool = True, report: Optional[dict] = None,
+                  ns_workers: Optional[Sequence[int]] = None):
     """Runs `steps` optimizer steps of workload `wl` on the GPU and checks the sampled parameters
     (default: all) against the oracle after every step."""
     opt = make_optimizer(wl, flags=flags)
@@ -192,7 +195,7 @@ def run_and_check(wl, steps: int, flags: int = B.FLAG_KEEP_POLAR, sample: Option
             mom_or[p] = check_param_step(opt, wl, p, before[p], weights[p], grads[p], mom_or[p], wl.lr,
                                          check_polar=check_polar, report=rep,
                                          power_start=None if starts is None else starts[p],
-                                         power_iters=wl.extra.get("power_iters", 2))
+                                         power_iters=wl.extra.get("power_iters", 2), ns_workers=ns_workers)
             mom_or[p] = np.stack([_np64(opt.tap(B.TAP_MOMENTUM, p, m)) for m in range(wl.num_workers)])
     opt.close()
     return rep

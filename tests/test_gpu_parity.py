@@ -137,6 +137,28 @@ def test_full_resnet50_config_sampled():
     print(rep)
 
 
+def test_full_gpt2_config_sampled():
+    """Config 3 at full size (12 layers, embeddings and norm gains as plain parameters, M = 16, Student-t noise,
+    local polar on): sampled parameters, Newton-Schulz compared for two of the sixteen workers."""
+    from parity_utils import run_and_check
+    wl = wlmod.config3()
+    names = [p.name for p in wl.params]
+    sample = [names.index("h0.qkv"), names.index("h5.attn_proj"), names.index("h11.mlp_proj"), names.index("wpe"),
+              names.index("ln7")]
+    rep = run_and_check(wl, steps=1, sample=sample, ns_workers=[0, 15])
+    print(rep)
+
+
+def test_full_llama_layer_config_sampled():
+    """Config 4 at full size (4096 x 4096 x 4, 4096 x 11008, 11008 x 4096; M = 8; local polar on): a square and
+    a rectangular matrix, Newton-Schulz compared for one worker each, plus the local polar direction."""
+    from parity_utils import run_and_check
+    wl = wlmod.config4()
+    rep = run_and_check(wl, steps=1, sample=[1], ns_workers=[3])
+    rep2 = run_and_check(wl, steps=1, sample=[5], ns_workers=[6])
+    print(rep, rep2)
+
+
 def test_weight_decay_and_step_lr_override():
     from parity_utils import check_param_step, make_optimizer
     import numpy as np
