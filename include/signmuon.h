@@ -130,7 +130,8 @@ int signmuon_create(const signmuon_config* config, signmuon_ctx** out);
 /* Bytes the caller must provide: `state` = momenta of all workers (float32 [M][d] per parameter,
  * parameters in creation order) - the only persistent optimizer state; `workspace` = scratch
  * (bf16 Newton-Schulz operands, Gram matrices, packed bits, norms, tile tables);
- * `host_staging` = extra device bytes needed only by signmuon_step_host (may be queried as NULL). */
+ * `host_staging` = extra device bytes needed only by signmuon_step_host: the weights once and the gradients
+ * twice (may be queried as NULL). */
 int signmuon_state_bytes(const signmuon_ctx* ctx, size_t* state, size_t* workspace, size_t* host_staging);
 
 /* Attaches DEVICE buffers (owned by the caller, must outlive the context's use of them) and
@@ -157,9 +158,15 @@ int signmuon_run_stages(signmuon_ctx* ctx, int32_t stage_mask, void* const* weig
                         const void* const* grads, float lr, void* cuda_stream);
 
 /* Same step with HOST-resident weights and gradients (same layouts as signmuon_step, but HOST
- * pointers inside the HOST arrays; pinned memory recommended): copies them to the staging
- * buffer bound by signmuon_bind, runs the step, copies the weights back, all on `cuda_stream`,
- * without synchronising.  Errors as signmuon_step, plus NOT_BOUND when no staging was bound. */
+ * pointers inside the HOST arrays; pinned memory recommended): copies them to the staging buffer
+ * bound by signmuon_bind, runs the step, copies the weights back, without synchronising the host.
+ * The weights travel on `cuda_stream`; the gradients travel on a stream of the library's own into one of
+ * two staging sets, so that, when calls follow one another without a synchronisation in between, the
+ * gradient copy of a call overlaps the compute and the weight copy-back of the call before it.  As with
+ * any asynchronous copy, the host arrays of a call must stay unchanged until that call's work has run
+ * (synchronise `cuda_stream`, whose work waits for the gradient copy).  signmuon_bind creates that stream
+ * and four events when a staging buffer is given; signmuon_destroy releases them.
+ * Errors as signmuon_step, plus NOT_BOUND when no staging was bound. */
 int signmuon_step_host(signmuon_ctx* ctx, void* const* host_weights, const void* const* host_grads,
                        float lr, void* cuda_stream);
 

@@ -91,6 +91,11 @@ struct signmuon_ctx {
   uint8_t* d_state = nullptr;
   uint8_t* d_ws = nullptr;
   uint8_t* d_staging = nullptr;
+  size_t stage_g_base = 0, stage_g_set_bytes = 0;
+  // signmuon_step_host: gradients are copied on an internal stream, one step ahead of the compute
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_loaded[2] = {nullptr, nullptr}, ev_consumed[2] = {nullptr, nullptr};
+  uint64_t host_steps = 0;
   int num_sms = 0;
   std::vector<ParamDev> paramdev;         // host copy of the device table
   bool paramdev_uploaded = false;
@@ -407,13 +412,15 @@ int plan_layout(signmuon_ctx* c) {
   c->off_tables_end = off;
   c->workspace_bytes = off;
 
-  // host staging: W and G of every parameter
+  // host staging: W of every parameter once, G of every parameter twice (two sets, so that the copy of the
+  // next step's gradients can run while this step computes)
   size_t st = 0;
-  for (ParamPlan& pl : c->plan) {
-    pl.stage_w_off = st; st += round_up((size_t)pl.d * dtype_size(pl.wdtype), ALIGN);
-    pl.stage_g_off = st; st += round_up((size_t)M * pl.d * dtype_size(pl.gdtype), ALIGN);
-  }
-  c->staging_bytes = st;
+  for (ParamPlan& pl : c->plan) { pl.stage_w_off = st; st += round_up((size_t)pl.d * dtype_size(pl.wdtype), ALIGN); }
+  c->stage_g_base = st;
+  size_t gs = 0;
+  for (ParamPlan& pl : c->plan) { pl.stage_g_off = gs; gs += round_up((size_t)M * pl.d * dtype_size(pl.gdtype), ALIGN); }
+  c->stage_g_set_bytes = gs;
+  c->staging_bytes = st + 2 * gs;
   return SIGNMUON_OK;
 }
 
@@ -725,6 +732,15 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
   c->d_state = static_cast<uint8_t*>(dev_state);
   c->d_ws = static_cast<uint8_t*>(dev_workspace);
   c->d_staging = static_cast<uint8_t*>(dev_staging);
+  if (dev_staging && !c->copy_stream) {
+    bool sok = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < 2 && sok; ++i) {
+      sok = cudaEventCreateWithFlags(&c->ev_loaded[i], cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&c->ev_consumed[i], cudaEventDisableTiming) == cudaSuccess;
+    }
+    if (!sok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+  }
+  c->host_steps = 0;
   const int M = c->cfg.num_workers;
 
   // host image of the table area [0, off_tables_end) minus the big buffers: assemble piecewise
@@ -864,27 +880,39 @@ int signmuon_step_host(signmuon_ctx* c, void* const* host_weights, const void* c
   cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
   const int M = c->cfg.num_workers;
   const size_t n = c->params.size();
+  for (size_t p = 0; p < n; ++p)
+    if (!host_weights[p] || !host_grads[p]) return SIGNMUON_ERR_INVALID_ARG;
+  const int set = (int)(c->host_steps & 1);
+  uint8_t* gbase = c->d_staging + c->stage_g_base + (size_t)set * c->stage_g_set_bytes;
   std::vector<void*> w(n);
   std::vector<const void*> g(n);
-  for (size_t p = 0; p < n; ++p) {
-    if (!host_weights[p] || !host_grads[p]) return SIGNMUON_ERR_INVALID_ARG;
+  bool ok = true;
+  // gradients: internal stream, as soon as the step that last used this set (two calls ago) has finished
+  if (c->host_steps >= 2) ok = cudaStreamWaitEvent(c->copy_stream, c->ev_consumed[set], 0) == cudaSuccess;
+  for (size_t p = 0; p < n && ok; ++p) {
+    const ParamPlan& pl = c->plan[p];
+    g[p] = gbase + pl.stage_g_off;
+    ok = cudaMemcpyAsync(const_cast<void*>(g[p]), host_grads[p], (size_t)M * pl.d * dtype_size(pl.gdtype),
+                         cudaMemcpyHostToDevice, c->copy_stream) == cudaSuccess;
+  }
+  ok = ok && cudaEventRecord(c->ev_loaded[set], c->copy_stream) == cudaSuccess;
+  // weights: the caller's stream, behind the previous call's copy back to the same host arrays
+  for (size_t p = 0; p < n && ok; ++p) {
     const ParamPlan& pl = c->plan[p];
     w[p] = c->d_staging + pl.stage_w_off;
-    g[p] = c->d_staging + pl.stage_g_off;
-    bool ok = cudaMemcpyAsync(w[p], host_weights[p], (size_t)pl.d * dtype_size(pl.wdtype), cudaMemcpyHostToDevice, s) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(const_cast<void*>(g[p]), host_grads[p], (size_t)M * pl.d * dtype_size(pl.gdtype),
-                               cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+    ok = cudaMemcpyAsync(w[p], host_weights[p], (size_t)pl.d * dtype_size(pl.wdtype), cudaMemcpyHostToDevice, s) == cudaSuccess;
   }
+  ok = ok && cudaStreamWaitEvent(s, c->ev_loaded[set], 0) == cudaSuccess;
+  if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
   int rc = run_stages_impl(c, SIGNMUON_STAGE_ALL, w.data(), g.data(), lr, s);
   if (rc != SIGNMUON_OK) return rc;
-  for (size_t p = 0; p < n; ++p) {
+  for (size_t p = 0; p < n && ok; ++p) {
     const ParamPlan& pl = c->plan[p];
-    if (cudaMemcpyAsync(host_weights[p], w[p], (size_t)pl.d * dtype_size(pl.wdtype), cudaMemcpyDeviceToHost, s) != cudaSuccess) {
-      c->sticky = SIGNMUON_ERR_CUDA;
-      return c->sticky;
-    }
+    ok = cudaMemcpyAsync(host_weights[p], w[p], (size_t)pl.d * dtype_size(pl.wdtype), cudaMemcpyDeviceToHost, s) == cudaSuccess;
   }
+  ok = ok && cudaEventRecord(c->ev_consumed[set], s) == cudaSuccess;
+  if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+  ++c->host_steps;
   return SIGNMUON_OK;
 }
 
@@ -1008,7 +1036,18 @@ int signmuon_ns_flops_per_step(const signmuon_ctx* c, double* flops) {
   return SIGNMUON_OK;
 }
 
-void signmuon_destroy(signmuon_ctx* c) { delete c; }
+void signmuon_destroy(signmuon_ctx* c) {
+  if (!c) return;
+  if (c->copy_stream) {
+    cudaStreamSynchronize(c->copy_stream);
+    for (int i = 0; i < 2; ++i) {
+      if (c->ev_loaded[i]) cudaEventDestroy(c->ev_loaded[i]);
+      if (c->ev_consumed[i]) cudaEventDestroy(c->ev_consumed[i]);
+    }
+    cudaStreamDestroy(c->copy_stream);
+  }
+  delete c;
+}
 
 const char* signmuon_error_string(int code) {
   switch (code) {

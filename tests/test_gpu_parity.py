@@ -223,17 +223,22 @@ def test_garbage_worker_is_outvoted():
 
 
 def test_host_resident_step_matches_device_step():
+    """Four host-buffer steps issued back to back (the gradient copies run one step ahead on the library's
+    own stream) against four device-buffer steps on the same inputs: bit-identical weights."""
     wl = _wl([(128, 256), (64, 147), (1, 40)], 3, kinds=["matrix", "matrix", "plain"])
     sig = wlmod.make_signal(wl, "cuda:0")
-    g = wlmod.make_grads(wl, sig, 0, "cuda:0")
+    gs = [wlmod.make_grads(wl, sig, t, "cuda:0") for t in range(4)]
     w_dev = wlmod.make_weights(wl, "cuda:0")
     w_host = [x.cpu().pin_memory() for x in w_dev]
-    g_host = [x.cpu().pin_memory() for x in g]
+    g_host = [[x.cpu().pin_memory() for x in g] for g in gs]
     a = B.SignMuon(wl.params, 3)
-    a.step(w_dev, g)
+    for g in gs:
+        a.step(w_dev, g)
     b = B.SignMuon(wl.params, 3, host_staging=True)
-    b.step_host(w_host, g_host)
+    for g in g_host:
+        b.step_host(w_host, g)
     torch.cuda.synchronize()
+    assert b.status() == B.OK
     for x, y in zip(w_dev, w_host):
         assert torch.equal(x.cpu(), y)
     a.close(); b.close()
