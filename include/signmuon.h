@@ -100,8 +100,10 @@ enum {
   SIGNMUON_FLAG_KEEP_POLAR = 1,   /* also store U_m = Y_K (bf16) so that signmuon_debug_tap can return it */
   SIGNMUON_FLAG_SIMT_GEMM = 2,    /* diagnostic: run the Newton-Schulz products on a plain CUDA-core
                                      kernel instead of the tensor-core kernel (slow; for fault isolation) */
-  SIGNMUON_FLAG_GEMM_1CTA = 4     /* run the tensor-core kernel with one CTA per 128 x 128 tile instead of
+  SIGNMUON_FLAG_GEMM_1CTA = 4,    /* run the tensor-core kernel with one CTA per 128 x 128 tile instead of
                                      CTA pairs on 256 x 256 tiles (same results; for comparison) */
+  SIGNMUON_FLAG_SIGN_AGREEMENT = 16 /* count, every step, how many of each worker's sign bits equal the vote
+                                     (one more small kernel; read with signmuon_sign_agreement) */
 };
 
 /* Stages of one step, for signmuon_run_stages (bit mask). A full step is all of them in this order. */
@@ -201,6 +203,12 @@ int signmuon_power_start_size(const signmuon_ctx* ctx, size_t* floats);
 int signmuon_power_start_segment(const signmuon_ctx* ctx, int32_t param, size_t* float_offset,
                                  size_t* floats_per_worker);
 int signmuon_set_power_start(signmuon_ctx* ctx, const float* dev_vectors, size_t floats);
+
+/* Sign agreement of the last step (Sec. 5.3 logs "sign agreement ratios" next to the communication volume):
+ * host_agree[m] (HOST, num_workers entries) = number of entries whose sign bit of worker m equals the
+ * majority vote; *host_entries (may be NULL) = entries per worker, so the ratio is agree / entries.
+ * Needs SIGNMUON_FLAG_SIGN_AGREEMENT; synchronises `cuda_stream`.  Errors: INVALID_ARG, NOT_BOUND, CUDA. */
+int signmuon_sign_agreement(signmuon_ctx* ctx, uint64_t* host_agree, uint64_t* host_entries, void* cuda_stream);
 
 /* Number of kernels signmuon_step launches per call with the current configuration. */
 int signmuon_launches_per_step(const signmuon_ctx* ctx, int32_t* launches);

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libsignmuon.so")
 OK = 0
 F32, BF16 = 0, 1
 PARAM_MATRIX, PARAM_PLAIN = 0, 1
-FLAG_KEEP_POLAR, FLAG_SIMT_GEMM, FLAG_GEMM_1CTA = 1, 2, 4
+FLAG_KEEP_POLAR, FLAG_SIMT_GEMM, FLAG_GEMM_1CTA, FLAG_SIGN_AGREEMENT = 1, 2, 4, 16
 STAGE_MOMENTUM, STAGE_NS, STAGE_VOTE, STAGE_LOCAL_POLAR, STAGE_ALL = 1, 2, 4, 8, 15
 TAP_MOMENTUM, TAP_POLAR, TAP_VOTE_BITS, TAP_WORKER_BITS, TAP_NORM = 0, 1, 2, 3, 4
 
@@ -28,6 +28,7 @@ EXPORTS = [
     "signmuon_step_host", "signmuon_packed_payload", "signmuon_payload_segment", "signmuon_debug_tap",
     "signmuon_status", "signmuon_launches_per_step", "signmuon_ns_flops_per_step",
     "signmuon_power_start_size", "signmuon_power_start_segment", "signmuon_set_power_start",
+    "signmuon_sign_agreement",
     "signmuon_momentum_norm_noalloc", "signmuon_destroy", "signmuon_error_string",
 ]
 NOALLOC_MAX_PARTIALS = 65536
@@ -75,6 +76,7 @@ def load_library() -> C.CDLL:
     lib.signmuon_power_start_size.argtypes = [vp, C.POINTER(sz)]
     lib.signmuon_power_start_segment.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
     lib.signmuon_set_power_start.argtypes = [vp, vp, sz]
+    lib.signmuon_sign_agreement.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), vp]
     lib.signmuon_momentum_norm_noalloc.argtypes = [vp, i32, vp, i32, vp, vp, vp, C.c_int64, C.c_int64, i32,
                                                    f32, f32, f32, vp]
     lib.signmuon_destroy.argtypes = [vp]
@@ -212,6 +214,15 @@ def signmuon_set_power_start(ctx: int, ptr: int, floats: int):
     _check(load_library().signmuon_set_power_start(ctx, ptr, floats), "signmuon_set_power_start")
 
 
+def signmuon_sign_agreement(ctx: int, num_workers: int, stream: int):
+    """(per-worker counts of sign bits equal to the vote, entries per worker) of the last step."""
+    agree = (C.c_uint64 * num_workers)()
+    entries = C.c_uint64()
+    _check(load_library().signmuon_sign_agreement(ctx, agree, C.byref(entries), stream or None),
+           "signmuon_sign_agreement")
+    return list(agree), entries.value
+
+
 def signmuon_momentum_norm_noalloc(grads_ptr: int, grad_dtype: int, weights_ptr: int, weight_dtype: int,
                                    momentum_ptr: int, operand_ptr: int, scales_ptr: int, rows: int, cols: int,
                                    num_workers: int, momentum: float, weight_decay: float, eps: float,
@@ -324,6 +335,9 @@ class SignMuon:
     def power_start_segment(self, param: int):
         """(offset, floats per worker) of a matrix parameter's start vectors inside the start-vector array."""
         return signmuon_power_start_segment(self.ctx, param)
+
+    def sign_agreement(self):
+        return signmuon_sign_agreement(self.ctx, self.num_workers, torch.cuda.current_stream(self.device).cuda_stream)
 
     @property
     def power_start_size(self) -> int:

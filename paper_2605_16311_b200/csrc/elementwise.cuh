@@ -419,4 +419,31 @@ __global__ void __launch_bounds__(EW_THREADS) vote_update_kernel(const ParamDev*
   else vote_block<PLANES, bf16>(pd, chunk, M, step, write_sbar, bits, vote_words, words_per_worker);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Sign agreement (the quantity the paper's training scripts log next to the communication volume):
+// per worker, the number of payload bits equal to the vote.  blockIdx.y = worker; pad bits are zero in
+// every payload and in the vote, so they count as agreeing and the host subtracts them.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) sign_agreement_kernel(const uint32_t* __restrict__ bits,
+                                                                    const uint32_t* __restrict__ vote_words,
+                                                                    int64_t words_per_worker,
+                                                                    unsigned long long* __restrict__ agree) {
+  const int m = blockIdx.y;
+  const uint32_t* mine = bits + (int64_t)m * words_per_worker;
+  unsigned int acc = 0;   // at most 32 bits x (words / threads) per thread: far below 2^32
+  for (int64_t i = (int64_t)blockIdx.x * EW_THREADS + threadIdx.x; i < words_per_worker; i += (int64_t)gridDim.x * EW_THREADS)
+    acc += __popc(~(__ldg(mine + i) ^ __ldg(vote_words + i)));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  __shared__ unsigned int red[EW_THREADS / 32];
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long t = 0;
+#pragma unroll
+    for (int i = 0; i < EW_THREADS / 32; ++i) t += red[i];
+    atomicAdd(agree + m, t);    // integer: the result does not depend on the order
+  }
+}
+
 }  // namespace signmuon

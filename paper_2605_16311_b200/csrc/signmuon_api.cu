@@ -80,7 +80,7 @@ struct signmuon_ctx {
   size_t off_status = 0, off_paramdev = 0, off_lists = 0, off_bits = 0, off_vote = 0, off_tmaps = 0,
          off_problems = 0, off_tables_end = 0;
   size_t off_list_matrix = 0, off_list_plain = 0, off_list_packfb = 0, off_starts_mom = 0, off_starts_plain = 0,
-         off_starts_vote = 0, off_starts_packfb = 0, off_starts_xv = 0, off_starts_xtu = 0;
+         off_starts_vote = 0, off_starts_packfb = 0, off_starts_xv = 0, off_starts_xtu = 0, off_agree = 0;
   // GEMM plans
   std::vector<GemmProblem> problems;      // pointers filled at bind
   std::vector<LaunchPlan> ns_launches, lp_launches;
@@ -343,6 +343,7 @@ int plan_layout(signmuon_ctx* c) {
   place(c->off_starts_plain, c->plain_starts.size() * 4);
   place(c->off_starts_vote, c->vote_starts.size() * 4);
   place(c->off_starts_packfb, c->packfb_starts.size() * 4);
+  place(c->off_agree, (size_t)M * 8);
   place(c->off_starts_xv, c->xv_starts.size() * 4);
   place(c->off_starts_xtu, c->xtu_starts.size() * 4);
   for (int32_t p : c->matrix_list) {
@@ -661,6 +662,13 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
     if (M <= 7) launch_vote<3>(c, lr, write_sbar, s);
     else if (M <= 63) launch_vote<6>(c, lr, write_sbar, s);
     else launch_vote<8>(c, lr, write_sbar, s);
+  }
+  if ((mask & SIGNMUON_STAGE_VOTE) && (c->cfg.flags & SIGNMUON_FLAG_SIGN_AGREEMENT)) {
+    // after the vote of the matrix parameters (the plain parameters voted in the momentum stage)
+    unsigned long long* agree = reinterpret_cast<unsigned long long*>(c->d_ws + c->off_agree);
+    if (cudaMemsetAsync(agree, 0, (size_t)M * 8, s) != cudaSuccess) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+    const unsigned gx = (unsigned)std::min<uint64_t>((c->words_per_worker + EW_THREADS - 1) / EW_THREADS, 1024);
+    sign_agreement_kernel<<<dim3(gx, (unsigned)M), EW_THREADS, 0, s>>>(bits, vote, (int64_t)c->words_per_worker, agree);
   }
   if ((mask & SIGNMUON_STAGE_LOCAL_POLAR) && nm && lp_ns) {
     for (const LaunchPlan& lp : c->lp_launches) launch_gemm(c, lp, lr, s);
@@ -1012,6 +1020,24 @@ int signmuon_set_power_start(signmuon_ctx* c, const float* dev_vectors, size_t f
   return SIGNMUON_OK;
 }
 
+int signmuon_sign_agreement(signmuon_ctx* c, uint64_t* host_agree, uint64_t* host_entries, void* cuda_stream) {
+  if (!c || !host_agree) return SIGNMUON_ERR_INVALID_ARG;
+  if (!(c->cfg.flags & SIGNMUON_FLAG_SIGN_AGREEMENT)) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const int M = c->cfg.num_workers;
+  std::vector<unsigned long long> raw((size_t)M);
+  if (cudaMemcpyAsync(raw.data(), c->d_ws + c->off_agree, (size_t)M * 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess) {
+    c->sticky = SIGNMUON_ERR_CUDA;
+    return c->sticky;
+  }
+  const uint64_t pads = c->words_per_worker * 32 - (uint64_t)c->entries;   // zero in every payload and in the vote
+  for (int m = 0; m < M; ++m) host_agree[m] = (uint64_t)raw[m] - pads;
+  if (host_entries) *host_entries = (uint64_t)c->entries;
+  return SIGNMUON_OK;
+}
+
 int signmuon_launches_per_step(const signmuon_ctx* c, int32_t* launches) {
   if (!c || !launches) return SIGNMUON_ERR_INVALID_ARG;
   int n = 0;
@@ -1020,6 +1046,7 @@ int signmuon_launches_per_step(const signmuon_ctx* c, int32_t* launches) {
   if (!c->plain_list.empty()) n += 1;
   if (nm) n += (int)c->ns_launches.size() + (c->packfb_blocks ? 1 : 0) + 1;   // NS, fallback pack, vote
   if (nm && c->cfg.local_polar && c->cfg.ns_steps > 0) n += (int)c->lp_launches.size();
+  if (c->cfg.flags & SIGNMUON_FLAG_SIGN_AGREEMENT) n += 1;
   *launches = n;
   return SIGNMUON_OK;
 }

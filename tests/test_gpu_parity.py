@@ -222,6 +222,33 @@ def test_garbage_worker_is_outvoted():
     opt.close()
 
 
+def test_sign_agreement_counts_match_the_payload():
+    """Per worker, the number of sign bits equal to the vote, against plain counting on the GPU's own bits
+    (ragged parameters: pad bits must not be counted)."""
+    import oracle as O
+    wl = _wl([(64, 147), (200, 328), (1, 37), (5, 9)], 5, kinds=["matrix", "matrix", "plain", "plain"])
+    opt = B.SignMuon(wl.params, 5, flags=B.FLAG_KEEP_POLAR | B.FLAG_SIGN_AGREEMENT)
+    w = wlmod.make_weights(wl, "cuda:0")
+    sig = wlmod.make_signal(wl, "cuda:0")
+    for t in range(2):
+        opt.step(w, wlmod.make_grads(wl, sig, t, "cuda:0"))
+    agree, entries = opt.sign_agreement()
+    assert entries == wl.numel
+    want = [0] * 5
+    for p, prm in enumerate(wl.params):
+        vote = O.unpack_bits(opt.tap(B.TAP_VOTE_BITS, p, 0).cpu().numpy(), prm.numel)
+        for m in range(5):
+            mine = O.unpack_bits(opt.tap(B.TAP_WORKER_BITS, p, m).cpu().numpy(), prm.numel)
+            want[m] += int((mine == vote).sum())
+    assert agree == want
+    assert all(a > entries // 2 for a in agree)       # a majority vote agrees with most workers on most entries
+    opt.close()
+    plain = B.SignMuon(wl.params, 5)
+    with pytest.raises(B.SignMuonError):
+        plain.sign_agreement()
+    plain.close()
+
+
 def test_host_resident_step_matches_device_step():
     """Four host-buffer steps issued back to back (the gradient copies run one step ahead on the library's
     own stream) against four device-buffer steps on the same inputs: bit-identical weights."""
