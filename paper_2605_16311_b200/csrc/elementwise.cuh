@@ -8,9 +8,9 @@ namespace signmuon {
 
 constexpr int EW_THREADS = 256;
 constexpr int MOM_CHUNK = 8192;        // entries per block of the momentum kernel (256 threads x 8 x 4)
-constexpr int PLAIN_CHUNK = 1024;      // entries per block of the plain-parameter kernel (8 warps x 128)
+constexpr int PLAIN_CHUNK = 2048;      // entries per block of the plain-parameter kernel (8 warps x 256)
 constexpr int VOTE_WORDS = 256;        // payload words per block of the vote kernel (8 warps x 32)
-constexpr int PACK_CHUNK = 8192;       // entries per block of the stand-alone pack kernel
+constexpr int PACK_CHUNK = 1024;       // entries per block of the stand-alone pack kernel (small: it only sees small, ragged matrices)
 
 // Finds the list slot whose block range contains `block` (`starts` is ascending, one entry per slot).
 __device__ __forceinline__ int find_slot(const uint32_t* __restrict__ starts, int n, uint32_t block) {
@@ -167,6 +167,86 @@ __global__ void finalize_norms_kernel(const ParamDev* __restrict__ params, const
 // Each warp owns 128 consecutive entries; lane l holds entries base + 32 k + l, k = 0..3, so that
 // one __ballot_sync per (worker, k) yields one payload word.
 // ---------------------------------------------------------------------------------------------
+// Stores 8 consecutive elements.
+__device__ __forceinline__ void store8(float* p, const float (&x)[8]) {
+  __stcs(reinterpret_cast<float4*>(p), make_float4(x[0], x[1], x[2], x[3]));
+  __stcs(reinterpret_cast<float4*>(p) + 1, make_float4(x[4], x[5], x[6], x[7]));
+}
+__device__ __forceinline__ void store8(bf16* p, const float (&x)[8]) {
+  __stcs(reinterpret_cast<uint4*>(p), make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]),
+                                                 pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7])));
+}
+
+// Vector form of the plain-parameter step for a warp whose 256 entries are all inside the parameter and
+// 16-byte aligned: lane l owns entries base + 8 l .. + 7 (128-bit accesses), its 8 sign bits form one byte
+// and four neighbouring lanes' bytes one payload word (OR within the 4-lane group).  Two workers are in
+// flight at a time so that a lane keeps 6 vector loads outstanding.
+template <typename GT, typename WT>
+__device__ __forceinline__ void plain_warp_vec(const ParamDev& pd, int64_t base, int M, float beta, float lambda,
+                                               float step, uint32_t* __restrict__ bits,
+                                               uint32_t* __restrict__ vote_words, int64_t words_per_worker) {
+  const int lane = threadIdx.x & 31;
+  const int64_t d = pd.d;
+  const int64_t i0 = base + 8 * lane;
+  const GT* __restrict__ g = reinterpret_cast<const GT*>(pd.G) + i0;
+  float* __restrict__ mom = pd.mom + i0;
+  WT* w = reinterpret_cast<WT*>(pd.W) + i0;
+  const float omb = 1.f - beta;
+  const unsigned group = 0xfu << (lane & ~3);            // this lane's 4-lane group
+  const int shift = (lane & 3) * 8;
+  const int64_t word = (base >> 5) + (lane >> 2);        // the payload word this group builds
+  uint32_t* out = bits + pd.word_off + word;
+  float wv[8];
+  load8(w, wv);
+  int count[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) count[e] = 0;
+  auto finish = [&](float (&gv)[8], float (&mv)[8], int m) {
+    uint32_t byte = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      mv[e] = fmaf(beta, mv[e], omb * fmaf(lambda, wv[e], gv[e]));
+      const bool b = mv[e] >= 0.f;
+      count[e] += b ? 1 : 0;
+      byte |= (b ? 1u : 0u) << e;
+    }
+    store8(mom + (int64_t)m * d, mv);
+    const uint32_t wordv = __reduce_or_sync(group, byte << shift);
+    if ((lane & 3) == 0) out[(int64_t)m * words_per_worker] = wordv;
+  };
+  int m = 0;
+  for (; m + 1 < M; m += 2) {
+    float g0[8], m0[8], g1[8], m1[8];
+    load8(g + (int64_t)m * d, g0);
+    load8(mom + (int64_t)m * d, m0);
+    load8(g + (int64_t)(m + 1) * d, g1);
+    load8(mom + (int64_t)(m + 1) * d, m1);
+    finish(g0, m0, m);
+    finish(g1, m1, m + 1);
+  }
+  if (m < M) {
+    float g0[8], m0[8];
+    load8(g + (int64_t)m * d, g0);
+    load8(mom + (int64_t)m * d, m0);
+    finish(g0, m0, m);
+  }
+  uint32_t vbyte = 0;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const bool plus = 2 * count[e] >= M;
+    vbyte |= (plus ? 1u : 0u) << e;
+    wv[e] -= plus ? step : -step;
+  }
+  store8(w, wv);
+  const uint32_t vword = __reduce_or_sync(group, vbyte << shift);
+  if ((lane & 3) == 0) vote_words[pd.word_off + word] = vword;
+}
+
+template <typename GT, typename WT>
+__device__ __forceinline__ void plain_warp_scalar(const ParamDev& pd, int64_t base, int M, float beta, float lambda,
+                                                  float step, uint32_t* __restrict__ bits,
+                                                  uint32_t* __restrict__ vote_words, int64_t words_per_worker);
+
 template <typename GT, typename WT>
 __device__ __forceinline__ void plain_block(const ParamDev& pd, uint32_t chunk, int M, float beta,
                                             float lambda, float step, uint32_t* __restrict__ bits,
@@ -174,7 +254,23 @@ __device__ __forceinline__ void plain_block(const ParamDev& pd, uint32_t chunk, 
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int64_t d = pd.d;
-  const int64_t base = (int64_t)chunk * PLAIN_CHUNK + warp * 128;
+  if ((d & 7) == 0 && (int64_t)chunk * PLAIN_CHUNK + (warp + 1) * 256 <= d) {
+    plain_warp_vec<GT, WT>(pd, (int64_t)chunk * PLAIN_CHUNK + warp * 256, M, beta, lambda, step, bits, vote_words,
+                           words_per_worker);
+    return;
+  }
+  // ragged tail (or an unaligned parameter): the warp's 256 entries as two scalar passes of 128
+  for (int pass = 0; pass < 2; ++pass)
+    plain_warp_scalar<GT, WT>(pd, (int64_t)chunk * PLAIN_CHUNK + warp * 256 + pass * 128, M, beta, lambda, step, bits,
+                              vote_words, words_per_worker);
+}
+
+template <typename GT, typename WT>
+__device__ __forceinline__ void plain_warp_scalar(const ParamDev& pd, int64_t base, int M, float beta,
+                                                  float lambda, float step, uint32_t* __restrict__ bits,
+                                                  uint32_t* __restrict__ vote_words, int64_t words_per_worker) {
+  const int lane = threadIdx.x & 31;
+  const int64_t d = pd.d;
   if (base >= d) return;
   const GT* g = reinterpret_cast<const GT*>(pd.G);
   WT* w = reinterpret_cast<WT*>(pd.W);

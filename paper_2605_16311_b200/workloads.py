@@ -146,6 +146,12 @@ def by_name(name: str) -> Workload:
              "c4_nolp": lambda: config4(False)}
     if name in table:
         return table[name]()
+    if name in ("c3_plain", "c3_matrix"):   # the plain-sign / Newton-Schulz halves of config 3 (profiling cases)
+        wl = config3()
+        kind = "plain" if name == "c3_plain" else "matrix"
+        wl.params = [p for p in wl.params if p.kind == kind]
+        wl.name = name
+        return wl
     if name.startswith("c5:"):           # c5:ROWSxCOLS:M[:K]
         parts = name.split(":")
         r, c = (int(v) for v in parts[1].split("x"))
