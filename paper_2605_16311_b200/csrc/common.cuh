@@ -19,6 +19,8 @@ struct ParamDev {
   float* mom;           // [M][rows*cols] float32 momentum (state buffer)
   bf16* y0;             // matrix params: Newton-Schulz operand buffer 0, [M][rows][ldy]
   bf16* y1;             // matrix params: operand buffer 1 (ping-pong partner)
+  bf16* ylo;            // optional: receives bf16(Mom - bf16(Mom)), the lo part of the first operand (same layout
+                        // as y0); set when the Newton-Schulz products run in split precision
   float* scales;        // matrix params: [M][2] = {1/max(sigma,eps)^2, 1/max(sigma,eps)}
   float* partials;      // matrix params: [M][chunks_per_worker] per-block sums of squares
   int64_t d;            // rows*cols
@@ -88,6 +90,11 @@ struct GemmProblem {
   // Gram products (tensor-core kernel): the result is symmetric, so only tiles on or above the diagonal are
   // scheduled and every off-diagonal tile is also written transposed through the {64 x 64}-box map tmapOT
   int32_t sym, tmapOT;
+  // Split-precision products: up to three operand pairs (hi hi, lo hi, hi lo) accumulated into the same
+  // tile, every segment contracting over the same K.
+  int32_t nseg;           // 0 or 1: one pair
+  int32_t tmapA2, tmapB2, tmapA3, tmapB3;
+  int32_t gram_lo;        // EPI_GRAM: also store lo(-A/2) through tmapO1 (then the tile is not mirrored)
 };
 
 struct TileEntry {

@@ -63,6 +63,7 @@ __device__ __forceinline__ void momentum_block(const ParamDev& pd, int m, uint32
   const WT* w = reinterpret_cast<const WT*>(pd.W);
   float* mom = pd.mom + (int64_t)m * d;
   bf16* y = pd.y0 + (int64_t)m * pd.rows * pd.ldy;
+  bf16* ylo = pd.ylo ? pd.ylo + (int64_t)m * pd.rows * pd.ldy : nullptr;
   const int64_t base = (int64_t)chunk * MOM_CHUNK;
   const float omb = 1.f - beta;
   if (pd.vec_ok) {
@@ -94,6 +95,14 @@ __device__ __forceinline__ void momentum_block(const ParamDev& pd, int m, uint32
         mo[0] = make_float4(mv[0], mv[1], mv[2], mv[3]);
         mo[1] = make_float4(mv[4], mv[5], mv[6], mv[7]);
         *reinterpret_cast<uint4*>(y + i) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        if (ylo) {
+          uint32_t lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            lo[e] = pack_bf16x2(mv[2 * e] - __uint_as_float(packed[e] << 16),
+                                mv[2 * e + 1] - __uint_as_float(packed[e] & 0xffff0000u));
+          *reinterpret_cast<uint4*>(ylo + i) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
       }
     }
   } else {
@@ -106,7 +115,9 @@ __device__ __forceinline__ void momentum_block(const ParamDev& pd, int m, uint32
       sumsq = fmaf(mv, mv, sumsq);
       const int64_t r = i / pd.cols;
       const int64_t c = i - r * pd.cols;
-      y[r * pd.ldy + c] = __float2bfloat16_rn(mv);
+      const bf16 h = __float2bfloat16_rn(mv);
+      y[r * pd.ldy + c] = h;
+      if (ylo) ylo[r * pd.ldy + c] = __float2bfloat16_rn(mv - __bfloat162float(h));
     }
   }
 }
@@ -399,15 +410,24 @@ __device__ __forceinline__ uint32_t vote_word(const uint32_t* __restrict__ bits,
   uint32_t c[PLANES];
 #pragma unroll
   for (int b = 0; b < PLANES; ++b) c[b] = 0;
-  for (int m = 0; m < M; ++m) {
-    uint32_t carry = __ldcs(bits + (int64_t)m * words_per_worker + word_index);
+  auto add_word = [&](uint32_t carry) {
 #pragma unroll
     for (int b = 0; b < PLANES; ++b) {
       const uint32_t t = c[b] & carry;
       c[b] ^= carry;
       carry = t;
     }
+  };
+  const uint32_t* col = bits + word_index;
+  int m = 0;
+  for (; m + 3 < M; m += 4) {          // four workers' words in flight
+    uint32_t w4[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) w4[k] = __ldcs(col + (int64_t)(m + k) * words_per_worker);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) add_word(w4[k]);
   }
+  for (; m < M; ++m) add_word(__ldcs(col + (int64_t)m * words_per_worker));
   const uint32_t add = (1u << PLANES) - (uint32_t)((M + 1) >> 1);
   uint32_t carry = 0;
 #pragma unroll

@@ -356,27 +356,32 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         const int batch = pr.batch;
         const int a_mn = pr.a_mn, b_mn = pr.b_mn;
         const int nk = (pr.K + GEMM_BK - 1) / GEMM_BK;
-        for (int kb = 0; kb < nk; ++kb, ++it) {
-          const uint32_t s = it % STAGES;
-          const uint32_t round = it / STAGES;
-          if (!mbar_wait(smem_u32(&empty_bar[s]), (round & 1u) ^ 1u, abort_flag, args.status)) { ok = false; break; }
-          // the "full" barrier of the pair is CTA 0's: it expects the bytes of both CTAs
-          const uint32_t fb = (CTAS == 2) ? map_to_cta(smem_u32(&full_bar[s]), 0) : smem_u32(&full_bar[s]);
-          if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[s]), CTAS * STAGE_BYTES);
-          const uint32_t sa = smem_base + s * STAGE_BYTES;
-          const uint32_t sb = sa + A_BYTES;
-          const int k0 = kb * GEMM_BK;
-          if (!a_mn) {
-            load_operand(sa, mapA, k0, m0, batch, fb);
-          } else {
+        const int nseg = pr.nseg > 1 ? pr.nseg : 1;           // split-precision products: segments along K
+        for (int seg = 0; seg < nseg && ok; ++seg) {
+          if (seg == 1) { mapA = args.tmaps + pr.tmapA2; mapB = args.tmaps + pr.tmapB2; }
+          else if (seg == 2) { mapA = args.tmaps + pr.tmapA3; mapB = args.tmaps + pr.tmapB3; }
+          for (int kb = 0; kb < nk; ++kb, ++it) {
+            const uint32_t s = it % STAGES;
+            const uint32_t round = it / STAGES;
+            if (!mbar_wait(smem_u32(&empty_bar[s]), (round & 1u) ^ 1u, abort_flag, args.status)) { ok = false; break; }
+            // the "full" barrier of the pair is CTA 0's: it expects the bytes of both CTAs
+            const uint32_t fb = (CTAS == 2) ? map_to_cta(smem_u32(&full_bar[s]), 0) : smem_u32(&full_bar[s]);
+            if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[s]), CTAS * STAGE_BYTES);
+            const uint32_t sa = smem_base + s * STAGE_BYTES;
+            const uint32_t sb = sa + A_BYTES;
+            const int k0 = kb * GEMM_BK;
+            if (!a_mn) {
+              load_operand(sa, mapA, k0, m0, batch, fb);
+            } else {
 #pragma unroll
-            for (int c = 0; c < GEMM_BM / 64; ++c) load_operand(sa + c * 8192, mapA, m0 + 64 * c, k0, batch, fb);
-          }
-          if (!b_mn) {
-            load_operand(sb, mapB, k0, n0, batch, fb);
-          } else {
+              for (int c = 0; c < GEMM_BM / 64; ++c) load_operand(sa + c * 8192, mapA, m0 + 64 * c, k0, batch, fb);
+            }
+            if (!b_mn) {
+              load_operand(sb, mapB, k0, n0, batch, fb);
+            } else {
 #pragma unroll
-            for (int c = 0; c < B_ROWS / 64; ++c) load_operand(sb + c * 8192, mapB, n0 + 64 * c, k0, batch, fb);
+              for (int c = 0; c < B_ROWS / 64; ++c) load_operand(sb + c * 8192, mapB, n0 + 64 * c, k0, batch, fb);
+            }
           }
         }
       }
@@ -405,7 +410,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         const TileEntry te = args.tiles[t];
         const GemmProblem& pr = args.problems[te.problem];
         const int a_mn = pr.a_mn, b_mn = pr.b_mn;
-        const int nk = (pr.K + GEMM_BK - 1) / GEMM_BK;
+        const int nk = ((pr.K + GEMM_BK - 1) / GEMM_BK) * (pr.nseg > 1 ? pr.nseg : 1);
         const uint32_t idesc = instr_desc(TILE_M, BN, a_mn, b_mn);
         const uint32_t acc = tcount & 1u;
         const uint32_t acc_round = tcount >> 1;
@@ -491,8 +496,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
           const int epi = (KIND == 0) ? (int)EPI_GRAM : pr.epi;
           const bool store_hi = (KIND == 0 || epi == EPI_APPLY || (epi == EPI_APPLY_PACK && pr.store_out)) &&
                                 pr.tma_out != 0 && rows_live;
-          const bool store_lo = KIND == 1 && epi == EPI_APPLY;
-          const bool mirror = KIND == 0 && pr.sym != 0 && te.tn != te.tm && rows_live;
+          const bool store_lo = (KIND == 1 && epi == EPI_APPLY) || (KIND == 0 && pr.gram_lo != 0);
+          const bool mirror = KIND == 0 && pr.sym != 0 && pr.gram_lo == 0 && te.tn != te.tm && rows_live;
           const CUtensorMap* mapO0 = args.tmaps + pr.tmapO0;
           const CUtensorMap* mapO1 = args.tmaps + pr.tmapO1;
           const CUtensorMap* mapOT = args.tmaps + pr.tmapOT;
@@ -548,8 +553,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         const bool rows_live = row0 < prM;
         const bool tma_c = KIND == 1 && pr.tma_c != 0 && rows_live, tma_out = pr.tma_out != 0;
         const bool store_hi = KIND == 0 || epi == EPI_APPLY || (epi == EPI_APPLY_PACK && pr.store_out);
-        const bool store_lo = KIND == 1 && epi == EPI_APPLY;
-        const bool mirror = KIND == 0 && pr.sym != 0 && te.tn != te.tm && rows_live;   // off-diagonal Gram tile
+        const bool store_lo = (KIND == 1 && epi == EPI_APPLY) || (KIND == 0 && pr.gram_lo != 0);
+        const bool mirror = KIND == 0 && pr.sym != 0 && pr.gram_lo == 0 && te.tn != te.tm && rows_live;   // off-diagonal Gram tile
         const uint32_t acc = tcount & 1u;
         const uint32_t acc_round = tcount >> 1;
         ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_round & 1u, abort_flag, args.status);

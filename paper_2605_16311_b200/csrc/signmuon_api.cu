@@ -36,7 +36,8 @@ struct ParamPlan {
   uint32_t chunks_per_worker;
   bool fused_pack;       // sign+pack happens in the last apply epilogue
   size_t mom_off;        // bytes into the state buffer
-  size_t y_off[2], lo_off, q_off, scales_off, partials_off;   // bytes into the workspace (matrix params)
+  size_t y_off[2], lo_off[2], q_off, qlo_off, scales_off, partials_off;   // bytes into the workspace (matrix params)
+                         // lo_off[0] == lo_off[1] (updated in place) unless the products run in split precision
   int tmap_base;         // first of this parameter's TM_PER_PARAM tensor maps
   size_t stage_w_off, stage_g_off;                    // bytes into the host-staging buffer
   size_t pi_v_off, pi_u_off, pi_scal_off;             // power iteration (scale = spectral), bytes into the workspace
@@ -44,8 +45,8 @@ struct ParamPlan {
 };
 
 // indices of a parameter's tensor maps relative to tmap_base
-enum { TM_Y0_K128 = 0, TM_Y0_KBN, TM_Y0_MN, TM_Y1_K128, TM_Y1_KBN, TM_Y1_MN, TM_Q_K128, TM_Q_KBN, TM_LO_K128, TM_MOM_F32,
-       TM_Q_BOX64, TM_PER_PARAM };
+enum { TM_Y0_K128 = 0, TM_Y0_KBN, TM_Y0_MN, TM_Y1_K128, TM_Y1_KBN, TM_Y1_MN, TM_Q_K128, TM_Q_KBN, TM_LO0_K128, TM_MOM_F32,
+       TM_Q_BOX64, TM_LO1_K128, TM_LO0_MN, TM_LO1_MN, TM_QLO_K128, TM_QLO_KBN, TM_PER_PARAM };
 
 struct LaunchPlan {        // one grouped GEMM launch
   size_t problem_base;     // index of its first problem in the problem array
@@ -87,6 +88,7 @@ struct signmuon_ctx {
   TileTable tables[4];
   int num_tmaps = 0;
   // binding
+  bool split = false;      // Newton-Schulz products of the workers in split precision (scale = spectral)
   bool bound = false;
   uint8_t* d_state = nullptr;
   uint8_t* d_ws = nullptr;
@@ -194,6 +196,23 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         pr.tma_out = 1; pr.tmapO0 = pl.tmap_base + TM_Q_K128; pr.batch_o = m;
         pr.sym = (c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) ? 0 : 1;   // square tiles only (bm == bn in every shape)
         pr.tmapOT = pl.tmap_base + TM_Q_BOX64;
+        if (c->split && !local_polar_phase) {       // -A/2 as a hi/lo pair, both triangles computed
+          pr.gram_lo = 1;
+          pr.sym = 0;
+          pr.out_lo = reinterpret_cast<bf16*>(pl.qlo_off + m * qbytes);
+          pr.tmapO1 = pl.tmap_base + TM_QLO_K128;
+          // Y Y^T ~ Yhi Yhi^T + Yhi Ylo^T + Ylo Yhi^T: the off-diagonal entries of the Gram matrix are small sums of
+          // products, and dropping the lo part would leave them with the operands' 2^-9 relative rounding
+          pr.nseg = 3;
+          const int lk = src ? TM_LO1_K128 : TM_LO0_K128, lmn = src ? TM_LO1_MN : TM_LO0_MN;
+          if (pl.wide) {
+            pr.tmapA2 = pr.tmapA;             pr.tmapB2 = pl.tmap_base + lk;     // (a K-major box of 128 rows serves as B)
+            pr.tmapA3 = pl.tmap_base + lk;    pr.tmapB3 = pr.tmapB;
+          } else {
+            pr.tmapA2 = pr.tmapA;             pr.tmapB2 = pl.tmap_base + lmn;
+            pr.tmapA3 = pl.tmap_base + lmn;   pr.tmapB3 = pr.tmapB;
+          }
+        }
         if (k == 0) {
           if (local_polar_phase) pr.scale_imm = (float)(1.0 / ((double)pl.rows * (double)pl.cols));
           else pr.scale_ptr = reinterpret_cast<const float*>(pl.scales_off + (size_t)m * 8);
@@ -211,7 +230,21 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
           pr.B = reinterpret_cast<const bf16*>(q); pr.b_sn = pl.ldq; pr.b_sk = 1;
           pr.tmapA = pl.tmap_base + ty; pr.tmapB = pl.tmap_base + TM_Q_KBN;
         }
-        const size_t lo = pl.lo_off + m * ybytes;
+        const bool split = c->split && !local_polar_phase;
+        const size_t lo = pl.lo_off[split ? src : 0] + m * ybytes;       // lo part of Y_k
+        const size_t lo_dst = pl.lo_off[split ? dst : 0] + m * ybytes;   // lo part of Y_{k+1}
+        const int tlo = split && src ? TM_LO1_K128 : TM_LO0_K128, tlo_dst = split && dst ? TM_LO1_K128 : TM_LO0_K128;
+        if (split) {      // Q Y ~ Qhi Yhi + Qlo Yhi + Qhi Ylo (three operand segments along K)
+          pr.nseg = 3;
+          const int tlo_mn = src ? TM_LO1_MN : TM_LO0_MN;
+          if (pl.wide) {
+            pr.tmapA2 = pl.tmap_base + TM_QLO_K128; pr.tmapB2 = pr.tmapB;
+            pr.tmapA3 = pr.tmapA;                   pr.tmapB3 = pl.tmap_base + tlo_mn;
+          } else {
+            pr.tmapA2 = pr.tmapA;                   pr.tmapB2 = pl.tmap_base + TM_QLO_KBN;
+            pr.tmapA3 = pl.tmap_base + tlo;         pr.tmapB3 = pr.tmapB;
+          }
+        }
         if (k == 0 && !local_polar_phase) {          // own term from the float32 momentum itself
           pr.c_mode = C_F32;
           pr.C = reinterpret_cast<const void*>(pl.mom_off + (size_t)m * pl.d * 4);   // offset into the state buffer
@@ -223,12 +256,12 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
           pr.ldc = pl.ldy;
         }
         pr.out = reinterpret_cast<void*>(ydst);
-        pr.out_lo = reinterpret_cast<bf16*>(lo);
+        pr.out_lo = reinterpret_cast<bf16*>(lo_dst);
         pr.ld_out = pl.ldy;
         // TMA-staged epilogue: possible whenever the row pitches are multiples of 16 bytes
         pr.tma_out = 1;
         pr.tmapO0 = pl.tmap_base + (dst ? TM_Y1_K128 : TM_Y0_K128);
-        pr.tmapO1 = pl.tmap_base + TM_LO_K128;
+        pr.tmapO1 = pl.tmap_base + tlo_dst;
         pr.batch_o = m;
         pr.batch_c = m;
         if (pr.c_mode == C_F32) {
@@ -237,7 +270,7 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         } else {
           pr.tma_c = 1;
           pr.tmapC0 = pl.tmap_base + ty;
-          pr.tmapC1 = pl.tmap_base + TM_LO_K128;
+          pr.tmapC1 = pl.tmap_base + tlo;
         }
         if (k == 0) {
           if (local_polar_phase) pr.scale_imm = (float)(1.0 / std::sqrt((double)pl.rows * (double)pl.cols));
@@ -313,6 +346,9 @@ int plan_layout(signmuon_ctx* c) {
   if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
   c->packfb_blocks = (uint32_t)b;
   const bool spectral = c->cfg.ns_scale == SIGNMUON_SCALE_SPECTRAL && K > 0;
+  // With sigma ~ ||Mom||_op the product term of the iteration is as large as the own term: the products then
+  // run in split precision (not on the diagnostic CUDA-core kernel, which has no operand segments).
+  c->split = spectral && !(c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM);
   if (spectral) {
     uint64_t bx = 0, bt = 0;
     size_t nf = 0;
@@ -371,8 +407,12 @@ int plan_layout(signmuon_ctx* c) {
     const size_t ybytes = round_up(slots * pl.rows * pl.ldy * 2, 1024);
     pl.y_off[0] = off; off += ybytes;
     pl.y_off[1] = off; off += ybytes;
-    pl.lo_off = off; off += ybytes;
+    pl.lo_off[0] = pl.lo_off[1] = off; off += ybytes;
     pl.q_off = off; off += round_up(slots * pl.s * pl.ldq * 2, 1024);
+    if (c->split) {
+      pl.lo_off[1] = off; off += ybytes;
+      pl.qlo_off = off; off += round_up(slots * pl.s * pl.ldq * 2, 1024);
+    }
   }
   // GEMM problems: K x (gram, apply) for the workers, and again for the local polar step
   c->problems.clear();
@@ -771,6 +811,7 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     if (pl.kind == SIGNMUON_PARAM_MATRIX) {
       d.y0 = reinterpret_cast<bf16*>(c->d_ws + pl.y_off[0]);
       d.y1 = reinterpret_cast<bf16*>(c->d_ws + pl.y_off[1]);
+      d.ylo = c->split ? reinterpret_cast<bf16*>(c->d_ws + pl.lo_off[0]) : nullptr;
       d.scales = reinterpret_cast<float*>(c->d_ws + pl.scales_off);
       d.partials = reinterpret_cast<float*>(c->d_ws + pl.partials_off);
       if (c->power_start_floats) {
@@ -836,8 +877,16 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
       ok = ok && encode_map(mp + TM_Q_K128, q, pl.s, pl.s, slots, pl.ldq, qb, 128);
       ok = ok && encode_map(mp + TM_Q_KBN, q, pl.s, pl.s, slots, pl.ldq, qb, bn);
       ok = ok && encode_map(mp + TM_Q_BOX64, q, pl.s, pl.s, slots, pl.ldq, qb, 64);
-      ok = ok && encode_map(mp + TM_LO_K128, c->d_ws + pl.lo_off, pl.cols, pl.rows, slots, pl.ldy,
-                            (uint64_t)pl.rows * pl.ldy, 128);
+      for (int b2 = 0; b2 < 2; ++b2) {
+        ok = ok && encode_map(mp + (b2 ? TM_LO1_K128 : TM_LO0_K128), c->d_ws + pl.lo_off[b2], pl.cols, pl.rows, slots,
+                              pl.ldy, (uint64_t)pl.rows * pl.ldy, 128);
+        ok = ok && encode_map(mp + (b2 ? TM_LO1_MN : TM_LO0_MN), c->d_ws + pl.lo_off[b2], pl.cols, pl.rows, slots,
+                              pl.ldy, (uint64_t)pl.rows * pl.ldy, 64);
+      }
+      if (c->split) {
+        ok = ok && encode_map(mp + TM_QLO_K128, c->d_ws + pl.qlo_off, pl.s, pl.s, slots, pl.ldq, qb, 128);
+        ok = ok && encode_map(mp + TM_QLO_KBN, c->d_ws + pl.qlo_off, pl.s, pl.s, slots, pl.ldq, qb, bn);
+      }
       if (pl.cols % 4 == 0)   // float32 momentum as the first iteration's C operand
         ok = ok && encode_map(mp + TM_MOM_F32, c->d_state + pl.mom_off, pl.cols, pl.rows, M, pl.cols, (uint64_t)pl.d, 128,
                               true);
@@ -855,6 +904,8 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
       uint8_t* cbase = (pr.c_mode == C_F32) ? c->d_state : c->d_ws;
       pr.C = cbase + reinterpret_cast<size_t>(pr.C);
       if (pr.C_lo) pr.C_lo = reinterpret_cast<const bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.C_lo));
+      pr.out_lo = reinterpret_cast<bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.out_lo));
+    } else if (pr.gram_lo) {
       pr.out_lo = reinterpret_cast<bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.out_lo));
     }
     if (pr.scale_ptr) pr.scale_ptr = reinterpret_cast<const float*>(c->d_ws + reinterpret_cast<size_t>(pr.scale_ptr));
