@@ -345,6 +345,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
     // ===================================================================== TMA producer
     if (lane == 0) {
       uint32_t it = 0;   // running k-block counter across tiles
+      uint32_t s = 0, par = 1;   // ring position and the parity to wait for on its "empty" barrier
+      const uint32_t full0 = (CTAS == 2) ? map_to_cta(smem_u32(&full_bar[0]), 0) : smem_u32(&full_bar[0]);
       bool ok = true;
       for (uint32_t t = tile_begin; t < tile_end && ok; ++t) {
         const TileEntry te = args.tiles[t];
@@ -361,12 +363,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
           if (seg == 1) { mapA = args.tmaps + pr.tmapA2; mapB = args.tmaps + pr.tmapB2; }
           else if (seg == 2) { mapA = args.tmaps + pr.tmapA3; mapB = args.tmaps + pr.tmapB3; }
           for (int kb = 0; kb < nk; ++kb, ++it) {
-            const uint32_t s = it % STAGES;
-            const uint32_t round = it / STAGES;
-            if (!mbar_wait(smem_u32(&empty_bar[s]), (round & 1u) ^ 1u, abort_flag, args.status)) { ok = false; break; }
+            if (!mbar_wait(smem_u32(&empty_bar[0]) + 8u * s, par, abort_flag, args.status)) { ok = false; break; }
             // the "full" barrier of the pair is CTA 0's: it expects the bytes of both CTAs
-            const uint32_t fb = (CTAS == 2) ? map_to_cta(smem_u32(&full_bar[s]), 0) : smem_u32(&full_bar[s]);
-            if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[s]), CTAS * STAGE_BYTES);
+            const uint32_t fb = full0 + 8u * s;
+            if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[0]) + 8u * s, CTAS * STAGE_BYTES);
             const uint32_t sa = smem_base + s * STAGE_BYTES;
             const uint32_t sb = sa + A_BYTES;
             const int k0 = kb * GEMM_BK;
@@ -382,6 +382,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
 #pragma unroll
               for (int c = 0; c < B_ROWS / 64; ++c) load_operand(sb + c * 8192, mapB, n0 + 64 * c, k0, batch, fb);
             }
+            if (++s == STAGES) { s = 0; par ^= 1u; }
           }
         }
       }
@@ -404,7 +405,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
   } else if (warp == 1) {
     // ===================================================================== MMA issuer (CTA 0 of a pair)
     if (lane == 0 && cta_rank == 0) {
-      uint32_t it = 0, tcount = 0;
+      uint32_t tcount = 0;
+      uint32_t s = 0, par = 0;   // ring position and the parity to wait for on its "full" barrier
       bool ok = true;
       for (uint32_t t = tile_begin; t < tile_end && ok; ++t, ++tcount) {
         const TileEntry te = args.tiles[t];
@@ -417,10 +419,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         if (!mbar_wait(smem_u32(&tmem_empty_bar[acc]), (acc_round & 1u) ^ 1u, abort_flag, args.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb = 0; kb < nk; ++kb, ++it) {
-          const uint32_t s = it % STAGES;
-          const uint32_t round = it / STAGES;
-          if (!mbar_wait(smem_u32(&full_bar[s]), round & 1u, abort_flag, args.status)) { ok = false; break; }
+        for (int kb = 0; kb < nk; ++kb) {
+          if (!mbar_wait(smem_u32(&full_bar[0]) + 8u * s, par, abort_flag, args.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + s * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
@@ -432,7 +432,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
             else tc_mma_f16(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
-          if (CTAS == 2) tc_commit_pair(smem_u32(&empty_bar[s])); else tc_commit(smem_u32(&empty_bar[s]));
+          if (CTAS == 2) tc_commit_pair(smem_u32(&empty_bar[0]) + 8u * s); else tc_commit(smem_u32(&empty_bar[0]) + 8u * s);
+          if (++s == STAGES) { s = 0; par ^= 1u; }
         }
         if (ok) {                                    // accumulator complete
           if (CTAS == 2) tc_commit_pair(smem_u32(&tmem_full_bar[acc])); else tc_commit(smem_u32(&tmem_full_bar[acc]));
