@@ -129,3 +129,30 @@ def test_power_start_layout_and_errors():
         for k, v in kw.items():
             setattr(cfg, k, v)
         assert B.signmuon_create_raw(cfg)[0] == -1, kw
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/signmuon.h must compile as C (no C++ in the boundary) and a C caller must link against the library."""
+    import subprocess
+    src = tmp_path / "use.c"
+    src.write_text('#include "signmuon.h"\n'
+                   '#include <stdio.h>\n'
+                   'int main(void) {\n'
+                   '  signmuon_param p = {64, 64, SIGNMUON_PARAM_MATRIX, SIGNMUON_F32, SIGNMUON_F32};\n'
+                   '  signmuon_config c = {0};\n'
+                   '  signmuon_ctx* ctx = NULL;\n'
+                   '  size_t bytes = 0, entries = 0;\n'
+                   '  c.num_params = 1; c.params = &p; c.num_workers = 4; c.momentum = 0.9f; c.lr = 1e-3f; c.ns_steps = 5;\n'
+                   '  if (signmuon_create(&c, &ctx) != SIGNMUON_OK) return 1;\n'
+                   '  if (signmuon_packed_payload(ctx, 0, NULL, &bytes, &entries) != SIGNMUON_OK) return 2;\n'
+                   '  printf("%zu %zu %s\\n", bytes, entries, signmuon_error_string(SIGNMUON_ERR_TIMEOUT));\n'
+                   '  signmuon_destroy(ctx);\n'
+                   '  return 0;\n'
+                   '}\n')
+    exe = tmp_path / "use"
+    libdir = os.path.dirname(B.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe),
+                    "-L", libdir, "-l:libsignmuon.so", "-Wl,-rpath," + libdir], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split(maxsplit=2)
+    assert out[0] == "512" and out[1] == "4096"          # 64 x 64 entries, one bit each
+    assert out[2].startswith("a bounded")
