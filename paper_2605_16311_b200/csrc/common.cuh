@@ -107,11 +107,12 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// Stores 32 floats as bf16 (hi) and optionally the bf16 remainders (lo) at row pointer offsets.
-__device__ __forceinline__ void store_hi_lo(bf16* o, bf16* olo, const float (&v)[32], bool vec, int n_valid) {
+// Stores NC floats as bf16 (hi) and optionally the bf16 remainders (lo) at row pointer offsets.
+template <int NC>
+__device__ __forceinline__ void store_hi_lo(bf16* o, bf16* olo, const float (&v)[NC], bool vec, int n_valid) {
   if (vec) {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < NC / 8; ++q) {
       uint32_t w[4], wl[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -124,7 +125,7 @@ __device__ __forceinline__ void store_hi_lo(bf16* o, bf16* olo, const float (&v)
     }
   } else {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
+    for (int j = 0; j < NC; ++j) {
       if (j < n_valid) {
         const bf16 h = __float2bfloat16_rn(v[j]);
         o[j] = h;
@@ -138,16 +139,17 @@ __device__ __forceinline__ void store_hi_lo(bf16* o, bf16* olo, const float (&v)
 // rows/columns outside the problem are skipped.
 
 // v <- scale * (v + 1.5 * C) with C read directly from global memory.
+template <int NC = 32>
 __device__ __forceinline__ void apply_c_direct(const GemmProblem& pr, float scale, int row, int col0, float* v) {
   if (row >= pr.M || col0 >= pr.N) return;
-  const bool full = (col0 + 32 <= pr.N);
-  const int n_valid = full ? 32 : pr.N - col0;
+  const bool full = (col0 + NC <= pr.N);
+  const int n_valid = full ? NC : pr.N - col0;
   if (pr.c_mode == C_F32) {
     const float* c = reinterpret_cast<const float*>(pr.C) + (int64_t)row * pr.ldc + col0;
     if (full && ((pr.ldc & 3) == 0)) {
       const float4* c4 = reinterpret_cast<const float4*>(c);
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
+      for (int q = 0; q < NC / 4; ++q) {
         const float4 t = __ldg(c4 + q);
         v[4 * q] = scale * fmaf(1.5f, t.x, v[4 * q]);
         v[4 * q + 1] = scale * fmaf(1.5f, t.y, v[4 * q + 1]);
@@ -156,14 +158,14 @@ __device__ __forceinline__ void apply_c_direct(const GemmProblem& pr, float scal
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = (j < n_valid) ? scale * fmaf(1.5f, __ldg(c + j), v[j]) : 0.f;
+      for (int j = 0; j < NC; ++j) v[j] = (j < n_valid) ? scale * fmaf(1.5f, __ldg(c + j), v[j]) : 0.f;
     }
   } else {
     const bf16* c = reinterpret_cast<const bf16*>(pr.C) + (int64_t)row * pr.ldc + col0;
     const bf16* cl = pr.c_mode == C_HILO ? pr.C_lo + (int64_t)row * pr.ldc + col0 : nullptr;
     if (full && ((pr.ldc & 7) == 0)) {
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < NC / 8; ++q) {
         const uint4 t = __ldg(reinterpret_cast<const uint4*>(c) + q);
         uint4 u = make_uint4(0, 0, 0, 0);
         if (cl) u = *(reinterpret_cast<const uint4*>(cl) + q);
@@ -179,7 +181,7 @@ __device__ __forceinline__ void apply_c_direct(const GemmProblem& pr, float scal
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
+      for (int j = 0; j < NC; ++j) {
         float cv = 0.f;
         if (j < n_valid) cv = __bfloat162float(c[j]) + (cl ? __bfloat162float(cl[j]) : 0.f);
         v[j] = (j < n_valid) ? scale * fmaf(1.5f, cv, v[j]) : 0.f;
@@ -189,14 +191,15 @@ __device__ __forceinline__ void apply_c_direct(const GemmProblem& pr, float scal
 }
 
 // out <- hi(v) (and out_lo <- lo(v)) written directly to global memory.
+template <int NC = 32>
 __device__ __forceinline__ void store_out_direct(const GemmProblem& pr, int row, int col0, const float* v, bool with_lo) {
   if (row >= pr.M || col0 >= pr.N) return;
-  const bool full = (col0 + 32 <= pr.N);
-  const int n_valid = full ? 32 : pr.N - col0;
+  const bool full = (col0 + NC <= pr.N);
+  const int n_valid = full ? NC : pr.N - col0;
   bf16* o = reinterpret_cast<bf16*>(pr.out) + (int64_t)row * pr.ld_out + col0;
   bf16* ol = (with_lo && pr.out_lo) ? pr.out_lo + (int64_t)row * pr.ld_out + col0 : nullptr;
-  const float(&vv)[32] = *reinterpret_cast<const float(*)[32]>(v);
-  store_hi_lo(o, ol, vv, full && ((pr.ld_out & 7) == 0), n_valid);
+  const float(&vv)[NC] = *reinterpret_cast<const float(*)[NC]>(v);
+  store_hi_lo<NC>(o, ol, vv, full && ((pr.ld_out & 7) == 0), n_valid);
 }
 
 // One payload word from 32 consecutive columns (only issued for parameters with cols % 32 == 0).
@@ -207,20 +210,30 @@ __device__ __forceinline__ void pack_bits_direct(const GemmProblem& pr, int row,
   for (int j = 0; j < 32; ++j) word |= (v[j] >= 0.f ? 1u : 0u) << j;
   pr.bits_out[((int64_t)row * pr.N + col0) >> 5] = word;
 }
+// Half a payload word from 16 consecutive columns (col0 a multiple of 16; little-endian words: the lower
+// columns are the lower half).
+__device__ __forceinline__ void pack_bits16_direct(const GemmProblem& pr, int row, int col0, const float* v) {
+  if (row >= pr.M || col0 + 16 > pr.N) return;
+  uint32_t half = 0;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) half |= (v[j] >= 0.f ? 1u : 0u) << j;
+  reinterpret_cast<uint16_t*>(pr.bits_out)[((int64_t)row * pr.N + col0) >> 4] = (uint16_t)half;
+}
 
 // W <- W - lr * v (local polar step's last epilogue).
+template <int NC = 32>
 __device__ __forceinline__ void update_weights_direct(const GemmProblem& pr, const ParamDev* params, float lr, int row,
                                                       int col0, const float* v) {
   if (row >= pr.M || col0 >= pr.N) return;
-  const bool full = (col0 + 32 <= pr.N);
-  const int n_valid = full ? 32 : pr.N - col0;
+  const bool full = (col0 + NC <= pr.N);
+  const int n_valid = full ? NC : pr.N - col0;
   const ParamDev& pd = params[pr.param];
   if (pd.wdtype == 0) {
     float* w = reinterpret_cast<float*>(pd.W) + (int64_t)row * pr.N + col0;
     if (full && ((pr.N & 3) == 0)) {
       float4* w4 = reinterpret_cast<float4*>(w);
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
+      for (int q = 0; q < NC / 4; ++q) {
         float4 t = w4[q];
         t.x = fmaf(-lr, v[4 * q], t.x);
         t.y = fmaf(-lr, v[4 * q + 1], t.y);
@@ -230,7 +243,7 @@ __device__ __forceinline__ void update_weights_direct(const GemmProblem& pr, con
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
+      for (int j = 0; j < NC; ++j)
         if (j < n_valid) w[j] = fmaf(-lr, v[j], w[j]);
     }
   } else {
@@ -238,7 +251,7 @@ __device__ __forceinline__ void update_weights_direct(const GemmProblem& pr, con
     if (full && ((pr.N & 7) == 0)) {
       uint4* w4 = reinterpret_cast<uint4*>(w);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < NC / 8; ++q) {
         const uint4 t = w4[q];
         const uint32_t in[4] = {t.x, t.y, t.z, t.w};
         uint32_t o[4];
@@ -250,7 +263,7 @@ __device__ __forceinline__ void update_weights_direct(const GemmProblem& pr, con
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
+      for (int j = 0; j < NC; ++j)
         if (j < n_valid) w[j] = __float2bfloat16_rn(fmaf(-lr, v[j], __bfloat162float(w[j])));
     }
   }

@@ -46,9 +46,14 @@ namespace signmuon {
 
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;
-constexpr int EPI_WARPS = 8;                 // two warps per TMEM lane quarter, 32 of a chunk's 64 columns each
-constexpr int GEMM_THREADS = 32 * (3 + EPI_WARPS);   // warp 0: operand TMA, warp 1: MMA, warps 2-9: epilogue math,
-                                                     // warp 10: epilogue TMA (C loads, result stores)
+#ifndef NS_EPI_WARPS
+#define NS_EPI_WARPS 8
+#endif
+constexpr int EPI_WARPS = NS_EPI_WARPS;      // EPI_WARPS / 4 warps per TMEM lane quarter, each NCOL of a chunk's 64 columns
+constexpr int EPI_NCOL = 256 / EPI_WARPS;    // columns of a chunk one math thread owns (32 or 16)
+static_assert(EPI_WARPS == 8 || EPI_WARPS == 16, "8 or 16 epilogue math warps");
+constexpr int GEMM_THREADS = 32 * (3 + EPI_WARPS);   // warp 0: operand TMA, warp 1: MMA, then the epilogue math warps,
+                                                     // last warp: epilogue TMA (C loads, result stores)
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
 struct GemmLaunchArgs {
@@ -211,6 +216,21 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_ld_cols(uint32_t taddr, float (&v)[32]) { tc_ld32(taddr, v); }
+__device__ __forceinline__ void tc_ld_cols(uint32_t taddr, float (&v)[16]) { tc_ld16(taddr, v); }
+
 // Shared-memory matrix descriptor (128-byte swizzle).  Bits: [0,14) start >> 4, [16,30) LBO >> 4,
 // [32,46) SBO >> 4, [46,48) = 1 (descriptor version), [61,64) = 2 (SWIZZLE_128B).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -284,7 +304,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
   __shared__ uint64_t tmem_empty_bar[2];
   __shared__ uint64_t c_full_bar[EPI_BUFS];      // chunk buffer holds its C operand / may be overwritten
   __shared__ uint64_t buf_ready_bar[EPI_BUFS];   // the eight math warps have written their results into it
-  __shared__ uint64_t row_pair_bar[4];           // the two math warps of a lane quarter (fp32 C chunks only)
+  __shared__ uint64_t row_pair_bar[4];           // the math warps of a lane quarter (fp32 C chunks only)
   __shared__ uint32_t tmem_slot;
   __shared__ uint32_t abort_word;
 
@@ -310,7 +330,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
       mbar_init(smem_u32(&c_full_bar[b]), 1);
       mbar_init(smem_u32(&buf_ready_bar[b]), EPI_WARPS);
     }
-    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&row_pair_bar[i]), 2);
+    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&row_pair_bar[i]), EPI_WARPS / 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -532,7 +552,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
     } else {
       // ------------------------------------------------------------------- epilogue math warps (2 .. 9)
       const int q = warp & 3;                    // TMEM lane quarter this warp may read
-      const int half = (warp - 2) >> 2;          // which 32 of a chunk's 64 columns
+      constexpr int NC = EPI_NCOL;               // columns per thread
+      constexpr int UNITS = NC / 8;              // 16-byte units of bf16 per thread
+      const int sub = (warp - 2) >> 2;           // which NC of a chunk's 64 columns
       const int r_in = q * 32 + lane;            // row of the tile this thread owns
       const uint32_t row_off = (uint32_t)r_in * 128u;
       const uint32_t sw = (uint32_t)(r_in & 7);
@@ -562,17 +584,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         ok = __all_sync(0xffffffffu, ok);        // the whole warp takes the same exit
         if (!ok) break;
         tc_fence_after();
-        const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)half * 32u;
+        const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)(sub * NC);
 #pragma unroll 1
         for (int ch = 0; ch < n_chunks; ++ch, ++g) {
           const uint32_t b = g % EPI_BUFS;
           const uint32_t buf = epi_base + b * BUF_BYTES;
-          const int col0 = n0 + ch * 64 + half * 32;   // first of this thread's 32 columns
+          const int col0 = n0 + ch * 64 + sub * NC;    // first of this thread's columns
           ok = mbar_wait(smem_u32(&c_full_bar[b]), (g / EPI_BUFS) & 1u, abort_flag, args.status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          float v[32];
-          tc_ld32(taddr + ch * 64, v);
+          float v[NC];
+          tc_ld_cols(taddr + ch * 64, v);
           if (ch == n_chunks - 1) {              // last read of this accumulator: hand it back to the MMA issuer
             tc_fence_before();
             __syncwarp();
@@ -584,20 +606,22 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
           if (KIND == 0) {
             const float f = -0.5f * scale;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] *= f;
+            for (int j = 0; j < NC; ++j) v[j] *= f;
           } else if (tma_c) {
             if (c_mode == C_F32) {               // half h of the buffer = fp32 columns 32 h .. 32 h + 31
+              const uint32_t fhalf = (uint32_t)(sub * NC) >> 5, funit0 = ((uint32_t)(sub * NC) & 31u) >> 2;
 #pragma unroll
-              for (int c16 = 0; c16 < 8; ++c16) {
-                const uint4 u = lds128(buf + half * EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4));
-                float* o = v + c16 * 4;
+              for (int cc = 0; cc < NC / 4; ++cc) {
+                const uint32_t c16 = funit0 + (uint32_t)cc;
+                const uint4 u = lds128(buf + fhalf * EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4));
+                float* o = v + cc * 4;
                 o[0] = scale * fmaf(1.5f, __uint_as_float(u.x), o[0]);
                 o[1] = scale * fmaf(1.5f, __uint_as_float(u.y), o[1]);
                 o[2] = scale * fmaf(1.5f, __uint_as_float(u.z), o[2]);
                 o[3] = scale * fmaf(1.5f, __uint_as_float(u.w), o[3]);
               }
-              // The bf16 results go to units 4h..4h+3 of BOTH halves, i.e. into the fp32 columns of the warp
-              // that owns the other 32 columns of these rows: both warps finish reading before either writes.
+              // The bf16 results go to this thread's units of BOTH halves, i.e. into fp32 columns that other warps
+              // of this lane quarter still have to read: all of them finish reading before any writes.
               __syncwarp();
               if (lane == 0) mbar_arrive(smem_u32(&row_pair_bar[q]));
               ok = mbar_wait(smem_u32(&row_pair_bar[q]), f32_chunks & 1u, abort_flag, args.status);
@@ -607,8 +631,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
             } else {
               const bool has_lo = c_mode == C_HILO;
 #pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                const uint32_t c16 = (uint32_t)(half * 4 + c);
+              for (int c = 0; c < UNITS; ++c) {
+                const uint32_t c16 = (uint32_t)(sub * UNITS + c);
                 const uint4 uh = lds128(buf + row_off + ((c16 ^ sw) << 4));
                 uint4 ul = make_uint4(0, 0, 0, 0);
                 if (has_lo) ul = lds128(buf + EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4));
@@ -625,14 +649,14 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
               }
             }
           } else if (KIND == 1) {
-            apply_c_direct(pr, scale, row, col0, v);
+            apply_c_direct<NC>(pr, scale, row, col0, v);
           }
           // ---- outputs
           if (store_hi) {
             if (tma_out) {
 #pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                const uint32_t c16 = (uint32_t)(half * 4 + c);
+              for (int c = 0; c < UNITS; ++c) {
+                const uint32_t c16 = (uint32_t)(sub * UNITS + c);
                 const float* o = v + c * 8;
                 uint32_t wh[4], wl[4];
 #pragma unroll
@@ -649,19 +673,22 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
                 const uint32_t tb = buf + EPI_HALF_BYTES + (uint32_t)(r_in >> 6) * 8192u + (uint32_t)(r_in & 7) * 2u;
                 const uint32_t unit = (uint32_t)(r_in & 63) >> 3;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
+                for (int j = 0; j < NC; ++j) {
                   const uint16_t h = __bfloat16_as_ushort(__float2bfloat16_rn(v[j]));
-                  const uint32_t jj = (uint32_t)(half * 32 + j);
+                  const uint32_t jj = (uint32_t)(sub * NC + j);
                   asm volatile("st.shared.u16 [%0], %1;" ::"r"(tb + jj * 128u + ((unit ^ (jj & 7u)) << 4)), "h"(h) : "memory");
                 }
               }
               fence_async_smem();
             } else {
-              store_out_direct(pr, row, col0, v, store_lo);
+              store_out_direct<NC>(pr, row, col0, v, store_lo);
             }
           }
-          if (KIND == 1 && epi == EPI_APPLY_PACK) pack_bits_direct(pr, row, col0, v);
-          else if (KIND == 1 && epi == EPI_APPLY_UPDATE) update_weights_direct(pr, args.params, args.lr, row, col0, v);
+          if (KIND == 1 && epi == EPI_APPLY_PACK) {
+            if (NC == 32) pack_bits_direct(pr, row, col0, v); else pack_bits16_direct(pr, row, col0, v);
+          } else if (KIND == 1 && epi == EPI_APPLY_UPDATE) {
+            update_weights_direct<NC>(pr, args.params, args.lr, row, col0, v);
+          }
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&buf_ready_bar[b]));   // this warp's part of the chunk is in shared memory
         }
