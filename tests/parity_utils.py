@@ -168,7 +168,8 @@ def run_and_check(wl, steps: int, flags: int = B.FLAG_KEEP_POLAR, sample: Option
     sample = list(range(len(wl.params))) if sample is None else list(sample)
     mom_or = {p: None for p in sample}
     rep = report if report is not None else {}
-    spectral = wl.extra.get("ns_scale", "fro") == "spectral"
+    # (with K = 0 no scale is needed at all: the library then asks for no start vectors)
+    spectral = wl.extra.get("ns_scale", "fro") == "spectral" and opt.power_start_size > 0
     for t in range(steps):
         grads = wlmod.make_grads(wl, signal, t, device)
         before = {p: weights[p].clone() for p in sample}

@@ -58,6 +58,15 @@ def test_spectral_scaling_power_iteration(P, K):
         run_and_check(wl, steps=1)
 
 
+def test_spectral_scaling_one_cta_variant_and_k0():
+    """Split-precision products on the one-CTA tile shape, and the degenerate K = 0 (sign of the momentum)."""
+    from parity_utils import run_and_check
+    wl = _wl([(200, 328), (328, 200), (64, 147)], 2, extra={"ns_scale": "spectral", "power_iters": 2})
+    run_and_check(wl, steps=1, flags=B.FLAG_KEEP_POLAR | B.FLAG_GEMM_1CTA)
+    wl0 = _wl([(128, 384), (64, 147)], 2, K=0, extra={"ns_scale": "spectral", "power_iters": 2})
+    run_and_check(wl0, steps=1)
+
+
 def test_spectral_scaling_needs_start_vectors():
     wl = _wl([(64, 64)], 2, extra={"ns_scale": "spectral"})
     from parity_utils import make_optimizer
