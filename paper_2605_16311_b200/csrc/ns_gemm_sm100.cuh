@@ -34,6 +34,9 @@
 // memory directly only for payload words and the final weight update.  The math warps never wait for each
 // other: per chunk they wait on the buffer's "C landed / buffer free" mbarrier and arrive on its "results
 // written" mbarrier.
+// Gram products are symmetric: only tiles on or above the diagonal are scheduled and an off-diagonal tile is
+// also stored transposed.  A problem may carry up to three operand pairs ("segments") that are accumulated
+// into the same tile along K: split-precision products (hi hi + lo hi + hi lo) of the spectral scale.
 // Every wait is bounded: after about two seconds a waiting thread records STATUS_TIMEOUT in the
 // status word, raises a CTA-wide abort flag and the CTA drains and exits (TMEM is freed).
 #pragma once
