@@ -95,6 +95,7 @@ struct GemmProblem {
   int32_t nseg;           // 0 or 1: one pair
   int32_t tmapA2, tmapB2, tmapA3, tmapB3;
   int32_t gram_lo;        // EPI_GRAM: also store lo(-A/2) through tmapO1 (then the tile is not mirrored)
+  int32_t diag_share;     // EPI_GRAM, one segment: on diagonal tiles the B operand is the A tile (not loaded twice)
 };
 
 struct TileEntry {

@@ -382,6 +382,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         const int a_mn = pr.a_mn, b_mn = pr.b_mn;
         const int nk = (pr.K + GEMM_BK - 1) / GEMM_BK;
         const int nseg = pr.nseg > 1 ? pr.nseg : 1;           // split-precision products: segments along K
+        // Diagonal tile of a one-segment Gram product: this CTA's B rows are its A rows, so B is not loaded
+        // and the MMA reads the A tile for both operands (B_ROWS == GEMM_BM and equal box shapes).
+        const bool share_ab = KIND == 0 && B_ROWS == GEMM_BM && pr.diag_share != 0 && te.tm == te.tn;
+        const uint32_t stage_tx = share_ab ? CTAS * A_BYTES : CTAS * STAGE_BYTES;
         for (int seg = 0; seg < nseg && ok; ++seg) {
           if (seg == 1) { mapA = args.tmaps + pr.tmapA2; mapB = args.tmaps + pr.tmapB2; }
           else if (seg == 2) { mapA = args.tmaps + pr.tmapA3; mapB = args.tmaps + pr.tmapB3; }
@@ -389,7 +393,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
             if (!mbar_wait(smem_u32(&empty_bar[0]) + 8u * s, par, abort_flag, args.status)) { ok = false; break; }
             // the "full" barrier of the pair is CTA 0's: it expects the bytes of both CTAs
             const uint32_t fb = full0 + 8u * s;
-            if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[0]) + 8u * s, CTAS * STAGE_BYTES);
+            if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[0]) + 8u * s, stage_tx);
             const uint32_t sa = smem_base + s * STAGE_BYTES;
             const uint32_t sb = sa + A_BYTES;
             const int k0 = kb * GEMM_BK;
@@ -399,7 +403,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
 #pragma unroll
               for (int c = 0; c < GEMM_BM / 64; ++c) load_operand(sa + c * 8192, mapA, m0 + 64 * c, k0, batch, fb);
             }
-            if (!b_mn) {
+            if (share_ab) {
+            } else if (!b_mn) {
               load_operand(sb, mapB, k0, n0, batch, fb);
             } else {
 #pragma unroll
@@ -437,6 +442,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         const int a_mn = pr.a_mn, b_mn = pr.b_mn;
         const int nk = ((pr.K + GEMM_BK - 1) / GEMM_BK) * (pr.nseg > 1 ? pr.nseg : 1);
         const uint32_t idesc = instr_desc(TILE_M, BN, a_mn, b_mn);
+        const bool share_ab = KIND == 0 && B_ROWS == GEMM_BM && pr.diag_share != 0 && te.tm == te.tn;
         const uint32_t acc = tcount & 1u;
         const uint32_t acc_round = tcount >> 1;
         if (!mbar_wait(smem_u32(&tmem_empty_bar[acc]), (acc_round & 1u) ^ 1u, abort_flag, args.status)) { ok = false; break; }
@@ -446,7 +452,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
           if (!mbar_wait(smem_u32(&full_bar[0]) + 8u * s, par, abort_flag, args.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + s * STAGE_BYTES;
-          const uint32_t sb = sa + A_BYTES;
+          const uint32_t sb = share_ab ? sa : sa + A_BYTES;
 #pragma unroll
           for (int kk = 0; kk < GEMM_BK / 16; ++kk) {
             const uint64_t adesc = a_mn ? smem_desc(sa + kk * 2048, 8192, 1024) : smem_desc(sa + kk * 32, 16, 1024);

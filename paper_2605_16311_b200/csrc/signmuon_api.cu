@@ -196,9 +196,11 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         pr.tma_out = 1; pr.tmapO0 = pl.tmap_base + TM_Q_K128; pr.batch_o = m;
         pr.sym = (c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) ? 0 : 1;   // square tiles only (bm == bn in every shape)
         pr.tmapOT = pl.tmap_base + TM_Q_BOX64;
+        pr.diag_share = 1;                          // A and B are the same rows of the same matrix on diagonal tiles
         if (c->split && !local_polar_phase) {       // -A/2 as a hi/lo pair, both triangles computed
           pr.gram_lo = 1;
           pr.sym = 0;
+          pr.diag_share = 0;                        // the segments pair different operands
           pr.out_lo = reinterpret_cast<bf16*>(pl.qlo_off + m * qbytes);
           pr.tmapO1 = pl.tmap_base + TM_QLO_K128;
           // Y Y^T ~ Yhi Yhi^T + Yhi Ylo^T + Ylo Yhi^T: the off-diagonal entries of the Gram matrix are small sums of
