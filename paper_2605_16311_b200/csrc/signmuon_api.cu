@@ -120,10 +120,18 @@ void build_tile_table(TileTable& tt, const std::vector<GemmProblem>& probs, size
   for (size_t i = 0; i < pcount; ++i) {
     const GemmProblem& pr = probs[pbase + i];
     const int tm = (pr.M + bm - 1) / bm, tn = (pr.N + bn - 1) / bn;
-    const int cost = (pr.K + GEMM_BK - 1) / GEMM_BK + 2;
+    // Cost in units of one K block of the main loop (about 512 cycles on a CTA pair).  Main loop and epilogue of
+    // consecutive tiles overlap, so a tile costs the longer of the two; a 64-column chunk of an apply epilogue
+    // (C in, combine, hi/lo out) takes about five such units, a chunk of a Gram epilogue about one (measured
+    // per-chunk cycle counts).
+    const int nk = ((pr.K + GEMM_BK - 1) / GEMM_BK) * (pr.nseg > 1 ? pr.nseg : 1);
+    const int per_chunk = (pr.epi == EPI_GRAM) ? 1 : 5;
     for (int a = 0; a < tm; ++a)
-      for (int b = (pr.sym ? a : 0); b < tn; ++b)     // symmetric results: tiles on or above the diagonal
+      for (int b = (pr.sym ? a : 0); b < tn; ++b) {   // symmetric results: tiles on or above the diagonal
+        const int cols = std::min(bn, pr.N - b * bn);
+        const int cost = std::max(nk, per_chunk * ((cols + 63) / 64)) + 2;
         all.push_back({{(uint32_t)i, (uint16_t)a, (uint16_t)b}, cost});
+      }
   }
   tt.grid = (int)std::min<size_t>((size_t)grid_limit, std::max<size_t>(all.size(), 1));
   std::stable_sort(all.begin(), all.end(), [](const T& x, const T& y) { return x.cost > y.cost; });
