@@ -168,6 +168,16 @@ def test_full_llama_layer_config_sampled():
     print(rep, rep2)
 
 
+def test_llama_layer_without_local_polar_and_sweep_extremes():
+    """Config 4 with the local polar step off (vote + update fused), and the corners of the kernel sweep:
+    the largest square (8192 x 8192, K = 3) and a 1:4 rectangle with 32 workers (Newton-Schulz of the last worker)."""
+    from parity_utils import run_and_check
+    rep = run_and_check(wlmod.config4(False), steps=1, sample=[4], ns_workers=[0])
+    rep2 = run_and_check(wlmod.config5(8192, 8192, 1, 3), steps=1)
+    rep3 = run_and_check(wlmod.config5(2048, 8192, 32, 5), steps=1, ns_workers=[31])
+    print(rep, rep2, rep3)
+
+
 def test_weight_decay_and_step_lr_override():
     from parity_utils import check_param_step, make_optimizer
     import numpy as np
