@@ -266,19 +266,20 @@ constexpr uint32_t EPI_HALF_BYTES = 128 * 128;        // 128 rows x 128 bytes (o
 constexpr uint32_t EPI_BUF_BYTES = 2 * EPI_HALF_BYTES;
 
 // Issues the TMA loads of the C chunk (64 columns from column `col0`) of a tile into an epilogue buffer.
-__device__ __forceinline__ void epi_issue_c_load(const GemmLaunchArgs& args, const GemmProblem& pr, int row0, int col0,
-                                                 uint32_t buf, uint32_t bar) {
-  if (pr.c_mode == C_F32) {
+// (c_mode, the two tensor maps and the batch slot are the problem's, read once per tile by the caller)
+__device__ __forceinline__ void epi_issue_c_load(int c_mode, const CUtensorMap* map0, const CUtensorMap* map1, int batch_c,
+                                                 int row0, int col0, uint32_t buf, uint32_t bar) {
+  if (c_mode == C_F32) {
     mbar_expect_tx(bar, EPI_BUF_BYTES);
-    tma_load_3d(buf, args.tmaps + pr.tmapC0, col0, row0, pr.batch_c, bar);
-    tma_load_3d(buf + EPI_HALF_BYTES, args.tmaps + pr.tmapC0, col0 + 32, row0, pr.batch_c, bar);
-  } else if (pr.c_mode == C_HILO) {
+    tma_load_3d(buf, map0, col0, row0, batch_c, bar);
+    tma_load_3d(buf + EPI_HALF_BYTES, map0, col0 + 32, row0, batch_c, bar);
+  } else if (c_mode == C_HILO) {
     mbar_expect_tx(bar, EPI_BUF_BYTES);
-    tma_load_3d(buf, args.tmaps + pr.tmapC0, col0, row0, pr.batch_c, bar);
-    tma_load_3d(buf + EPI_HALF_BYTES, args.tmaps + pr.tmapC1, col0, row0, pr.batch_c, bar);
+    tma_load_3d(buf, map0, col0, row0, batch_c, bar);
+    tma_load_3d(buf + EPI_HALF_BYTES, map1, col0, row0, batch_c, bar);
   } else {
     mbar_expect_tx(bar, EPI_HALF_BYTES);
-    tma_load_3d(buf, args.tmaps + pr.tmapC0, col0, row0, pr.batch_c, bar);
+    tma_load_3d(buf, map0, col0, row0, batch_c, bar);
   }
 }
 
@@ -487,6 +488,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         uint32_t pf_t = tile_begin, pf_g = 0;
         int pf_ch = 0, pf_n = 0, pf_row0 = 0, pf_n0 = 0;
         const GemmProblem* pf_pr = nullptr;
+        const CUtensorMap* pf_map0 = nullptr;
+        const CUtensorMap* pf_map1 = nullptr;
+        int pf_cmode = 0, pf_batch = 0;
         bool pf_live = false;
         uint32_t pf_issued = 0;
         auto pf_enter_tile = [&]() {
@@ -498,13 +502,16 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
           pf_n = (pf_pr->N - pf_n0 + 63) / 64;
           if (pf_n > BN / 64) pf_n = BN / 64;
           pf_live = KIND == 1 && pf_pr->tma_c != 0 && pf_row0 < pf_pr->M;
+          pf_cmode = pf_pr->c_mode; pf_batch = pf_pr->batch_c;
+          pf_map0 = args.tmaps + pf_pr->tmapC0; pf_map1 = args.tmaps + pf_pr->tmapC1;
           pf_ch = 0;
         };
         auto pf_step = [&]() {                   // makes the buffer of chunk pf_g available to the math warps
           if (pf_t >= tile_end) return;
           const uint32_t nb = pf_g % EPI_BUFS;
           if (pf_live) {
-            epi_issue_c_load(args, *pf_pr, pf_row0, pf_n0 + pf_ch * 64, epi_base + nb * BUF_BYTES, smem_u32(&c_full_bar[nb]));
+            epi_issue_c_load(pf_cmode, pf_map0, pf_map1, pf_batch, pf_row0, pf_n0 + pf_ch * 64, epi_base + nb * BUF_BYTES,
+                             smem_u32(&c_full_bar[nb]));
             ++pf_issued;
           } else {
             mbar_arrive(smem_u32(&c_full_bar[nb]));
