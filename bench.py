@@ -367,7 +367,7 @@ def run_ours(args, wl):
 
 
 def run_sweep(args):
-    """Kernel sweep (BASELINE config 5): squares and 1:4 rectangles from 512 to 8192 per side, bf16,
+    """Kernel sweep: squares and 1:4 rectangles from 512 to 8192 per side, bf16,
     M in {1..32}, K in {3, 5}; Newton-Schulz timed separately from momentum and vote+update.
     Prints one JSON line per point (this mode is not the one-line benchmark contract)."""
     import torch
