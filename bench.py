@@ -433,7 +433,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--oracle-flops", type=float, default=1.2e11,
                     help="float64 operation budget of one oracle sample step")
-    ap.add_argument("--cpu-baseline-flops", type=float, default=8e11,
+    ap.add_argument("--cpu-baseline-flops", type=float, default=2.5e12,
                     help="float64 operation budget of the oracle sample timed beside the GPU run")
     ap.add_argument("--ns-scale", default="fro", choices=["fro", "spectral"],
                     help="Alg. 4 scale: Frobenius norm (default, the benchmark configuration) or power iteration")
