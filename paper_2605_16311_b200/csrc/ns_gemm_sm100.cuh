@@ -479,7 +479,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
     // PREFETCH chunks ahead of the chunk whose results it sends off.  A math warp waits on c_full_bar,
     // reads its accumulator columns, combines, writes the results in place and arrives on buf_ready_bar;
     // the TMA thread waits on that and issues the stores.
-    constexpr uint32_t PREFETCH = EPI_BUFS - 2;
+    constexpr uint32_t PREFETCH = EPI_BUFS;      // every buffer is handed out again as soon as its store has left it
     if (warp == 2 + EPI_WARPS) {
       // ------------------------------------------------------------------- epilogue TMA thread
       if (lane == 0) {
@@ -543,10 +543,6 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
             const uint32_t b = g % EPI_BUFS;
             const uint32_t buf = epi_base + b * BUF_BYTES;
             const int col0 = n0 + ch * 64;
-            // buffer (g + PREFETCH) % EPI_BUFS was last stored from two chunks ago: at most the latest store
-            // may still be reading shared memory
-            bulk_wait_read<1>();
-            pf_step();
             if (!mbar_wait(smem_u32(&buf_ready_bar[b]), (g / EPI_BUFS) & 1u, abort_flag, args.status)) { ok = false; break; }
             if (store_hi) {
               tma_store_3d(mapO0, col0, row0, batch_o, buf);
@@ -556,7 +552,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
                 if (row0 + 64 < prM) tma_store_3d(mapOT, row0 + 64, col0, batch_o, buf + EPI_HALF_BYTES + 8192u);
               }
             }
-            bulk_commit();                       // one group per chunk (possibly empty) keeps the ring arithmetic fixed
+            bulk_commit();
+            // The buffer goes straight to chunk g + EPI_BUFS: wait until this store has read it out of shared
+            // memory (a few hundred cycles), then start that chunk's C loads (or just release the buffer).
+            bulk_wait_read<0>();
+            pf_step();
           }
         }
         if (!ok && pf_issued) {                  // abort path: give the loads in flight a fixed 100 us to land
