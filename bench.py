@@ -155,7 +155,7 @@ def time_oracle(wl, steps, warmup, budget_flops):
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the ncu
 # captures summarised under profiles/; None for workloads without a capture of the current kernel.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    ("c2_resnet50", "ns_gemm_tc_kernel"): 523.8e6,   # mean of 5 Gram (230.3 MB) and 5 apply (817.4 MB) launches
+    ("c2_resnet50", "ns_gemm_tc_kernel"): 525.7e6,   # mean of 5 Gram (230.5 MB) and 5 apply (820.8 MB) launches
 }
 
 
