@@ -317,6 +317,12 @@ def run_ours(args, wl):
         kernels["ns_gemm_tc"] = {"ms": ns_ms, "bound": "tensor", "algorithmic_flops": ns_flops,
                                  "launches": n_ns_launches * (2 if wl.local_polar else 1),
                                  "achieved_tflops": ns_flops / ns_ms / 1e9}
+    if "ns_gemm_tc" in kernels:
+        # the iteration's own memory traffic: per entry, worker and iteration the Gram product reads the bf16 iterate
+        # (2 B), the apply product reads it again as an operand (2 B) and moves hi + lo in and out (8 B)
+        ns_bytes = sum(12.0 * p.numel * wl.ns_steps * (M + (1 if wl.local_polar else 0)) for p in mat)
+        kernels["ns_gemm_tc"].update({"hbm_algorithmic_bytes": ns_bytes, "hbm_achieved_gbs": ns_bytes / ns_ms / 1e6,
+                                      "hbm_frac_of_measured": ns_bytes / ns_ms / 1e6 / peaks["hbm_gbs"]})
     if stage_ms["vote_update"] > 0 and vote_bytes > 0:
         kernels["vote_update"] = {"ms": stage_ms["vote_update"], "bound": "hbm", "algorithmic_bytes": vote_bytes,
                                   "achieved_gbs": vote_bytes / stage_ms["vote_update"] / 1e6}
