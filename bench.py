@@ -1,15 +1,20 @@
 #!/usr/bin/env python
 """Benchmark of the SignMuon optimizer step on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl ours|reference]
 
-A "step" is one full optimizer step (momentum, Newton-Schulz, sign+pack, vote, update) over one
-set of synthetic per-worker gradients.  Default workload: the ResNet-50-shaped parameter set
-(54 matrices, fp32, M = 4 workers, K = 5 Newton-Schulz steps).  Prints ONE JSON line.
+A "step" is one full optimizer step (momentum, Newton-Schulz, sign + pack, vote, local polar step,
+update) over one set of synthetic per-worker gradients.  Default workload: the Llama-7B-layer-shaped
+parameter set (six matrices, bf16 weights, M = 8 workers, K = 5 Newton-Schulz steps, local polar on) -
+the largest of the configurations that fits one GPU, and a timed region of seconds.  The ResNet-50- and
+GPT-2-small-shaped sets are timed in the same run as secondary blocks (`secondary`), without the
+host-buffer and CPU legs.  Prints ONE JSON line.
 
-With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs an independent
-replica of the same step ("replicas only": the worker axis is simulated on each GPU, there is no
-exchange step to shard); the value is the sum over ranks, timed as the max over ranks.
+With N > 1 (launched by torch.distributed.run, one rank per GPU) the M workers are sharded over the ranks
+(Alg. 3 of the paper: every rank computes momentum, Newton-Schulz and the 1-bit pack of its own workers,
+the packed words are all-gathered, every rank then runs the identical vote / local polar / update on its
+replica of the weights); total work is fixed, so the scaling is "strong".  When M is not a multiple of N
+every rank runs an independent replica instead ("weak").
 
 --impl reference times the float64 CPU oracle on a bounded sample of the same workload.
 """
@@ -30,6 +35,8 @@ if ROOT not in sys.path:
 
 METRIC = "signmuon_optimizer_steps_per_sec"
 UNIT = "steps/s"
+NOMINAL_BF16_TFLOPS = 2250.0     # dense bf16, B200 data sheet
+NOMINAL_HBM_GBS = 8000.0
 
 
 def load_peaks():
@@ -81,81 +88,122 @@ class ClockSampler:
             self.proc.wait(timeout=2)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         for r in self.rows:
             try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
             except ValueError:
                 continue
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
-# ------------------------------------------------------------------------------------------------
-def oracle_sample_plan(wl, budget_flops=1.2e11):
-    """Chooses a prefix-by-cost sample of the workload's parameters whose literal float64
-    Newton-Schulz work stays near `budget_flops`, and returns (indices, sample_cost, total_cost)."""
-    def cost(p):
-        base = 10.0 * p.numel * wl.num_workers
-        if p.kind != "matrix":
-            return base
-        c = 4.0 * p.cols * p.cols * p.rows * wl.ns_steps * (wl.num_workers + (1 if wl.local_polar else 0))
-        return base + c
-    costs = [cost(p) for p in wl.params]
-    total = sum(costs)
-    order = sorted(range(len(costs)), key=lambda i: costs[i])
+# ------------------------------------------------------------------------------------------------ oracle timing
+def _oracle_costs(wl):
+    """Float64 operation counts of the oracle's step per parameter: (per worker, shared) - momentum, Newton-Schulz
+    on the short side, sign + pack per worker; vote, optional local polar step, update once."""
+    out = []
+    for p in wl.params:
+        s, l = min(p.rows, p.cols), max(p.rows, p.cols)
+        ns = 4.0 * s * s * l * wl.ns_steps if p.kind == "matrix" else 0.0
+        per_worker = 12.0 * p.numel + ns
+        shared = 6.0 * p.numel * wl.num_workers + 4.0 * p.numel + (ns if (wl.local_polar and p.kind == "matrix") else 0.0)
+        out.append((per_worker, shared))
+    return out
+
+
+def oracle_sample_plan(wl, budget_flops):
+    """The ONE sample plan both the reference arm and the cpu_baseline leg use: one parameter per distinct shape,
+    cheapest first, while the float64 work of (one worker's share + the shared part) stays inside `budget_flops`;
+    at least one matrix parameter.  Returns (indices, sample_cost, total_cost)."""
+    costs = _oracle_costs(wl)
+    total = sum(w * wl.num_workers + s for (w, s) in costs)
+    seen, firsts = set(), []
+    for i, p in enumerate(wl.params):
+        key = (p.rows, p.cols, p.kind)
+        if key not in seen:
+            seen.add(key)
+            firsts.append(i)
+    firsts.sort(key=lambda i: sum(costs[i]))
     chosen, acc = [], 0.0
-    # spread over the size range: walk from cheap to expensive, taking every other parameter
-    for i in order[::2]:
-        if acc + costs[i] > budget_flops and chosen:
+    for i in firsts:
+        c = sum(costs[i])
+        if chosen and acc + c > budget_flops:
             continue
         chosen.append(i)
-        acc += costs[i]
+        acc += c
+    if not any(wl.params[i].kind == "matrix" for i in chosen):
+        mats = [i for i in firsts if wl.params[i].kind == "matrix"]
+        if mats:
+            chosen.append(mats[0])
+            acc += sum(costs[mats[0]])
     return sorted(chosen), acc, total
 
 
-def time_oracle(wl, steps, warmup, budget_flops):
+def time_oracle(wl, steps, warmup, budget_flops, min_seconds=0.0):
+    """Times the oracle's functions, as they stand, on the sample plan: for every sampled parameter ONE worker's
+    share (momentum, PolarNS on the short side, sign, pack) and the shared part (vote over M payloads, local polar
+    step, update).  A sample step costs sum(worker share + shared part); the whole-workload step time is that,
+    scaled by the float64 operation count of the full step over that of the sample (labelled extrapolated)."""
     import numpy as np
-    import torch
     import oracle as O
     from threadpoolctl import threadpool_info
     from paper_2605_16311_b200 import workloads as wlmod
 
     idx, c_sample, c_total = oracle_sample_plan(wl, budget_flops)
-    sub = wlmod.Workload(wl.name + "_oracle_sample", [wl.params[i] for i in idx], wl.num_workers, wl.momentum, wl.lr,
+    sub = wlmod.Workload(wl.name + "_oracle_sample", [wl.params[i] for i in idx], 1, wl.momentum, wl.lr,
                          wl.ns_steps, wl.local_polar, wl.steps, wl.signal_std, wl.noise_std, wl.noise,
                          wl.weight_std, wl.config_id)
-    specs = [O.ParamSpec(p.rows, p.cols, p.kind, p.dtype) for p in sub.params]
-    cfg = O.OracleConfig(num_workers=wl.num_workers, momentum=wl.momentum, lr=wl.lr, ns_steps=wl.ns_steps,
-                         local_polar=wl.local_polar)
-    st = O.init_state(specs, cfg)
     weights = [w.float().numpy().astype(np.float64) for w in wlmod.make_weights(sub)]
     signal = wlmod.make_signal(sub)
-    grads = [g.float().numpy() for g in wlmod.make_grads(sub, signal, 0)]
+    grads = [g.float().numpy().astype(np.float64)[0] for g in wlmod.make_grads(sub, signal, 0)]
+    moms = [np.zeros_like(g) for g in grads]
+    M, K = wl.num_workers, wl.ns_steps
+
+    def sample_step():
+        for j, p in enumerate(sub.params):
+            d = p.numel
+            moms[j] = O.momentum_update(moms[j], grads[j], weights[j], wl.momentum, 0.0)          # one worker's share
+            u = O.polar_ns_short_side(moms[j], K, 1e-12) if p.kind == "matrix" else moms[j]
+            packed = O.pack_bits(O.encode_bits(u).reshape(-1))
+            vote = O.majority_vote_popcount([packed] * M, d)                                       # shared part
+            s_bar = O.decode_bits(vote).reshape(p.rows, p.cols).astype(np.float64)
+            direction = O.local_polar(s_bar, K, 1e-12, short_side=True) if (wl.local_polar and p.kind == "matrix") else s_bar
+            weights[j] = O.apply_update(weights[j], direction, wl.lr)
+
     times = []
-    for t in range(warmup + steps):
+    t_begin = time.perf_counter()
+    n = 0
+    while n < warmup + steps or (time.perf_counter() - t_begin < min_seconds and n < warmup + 50):
         t0 = time.perf_counter()
-        weights, _ = O.step(specs, cfg, st, weights, grads)
+        sample_step()
         dt = time.perf_counter() - t0
-        if t >= warmup:
+        if n >= warmup:
             times.append(dt)
+        n += 1
     per_sample_step = sum(times) / len(times)
     est_full = per_sample_step * c_total / c_sample
     cores = max([d.get("num_threads", 1) for d in threadpool_info()] + [1])
+    names = ", ".join(f"{p.rows}x{p.cols}" for p in sub.params[:6]) + (" ..." if len(sub.params) > 6 else "")
     return {"value": 1.0 / est_full, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{len(idx)} of {len(wl.params)} parameters of {wl.name} (all {wl.num_workers} workers, full "
-                      f"step each), {per_sample_step:.2f} s per sample step; extrapolated to the whole workload by "
-                      f"literal float64 operation count (x{c_total / c_sample:.1f})",
-            "sample_seconds_per_step": per_sample_step}
+            "sample": f"{len(idx)} of {len(wl.params)} parameters of {wl.name} (one per distinct shape: {names}); per "
+                      f"parameter one worker's momentum + PolarNS (float64, short side) + sign + pack and the shared "
+                      f"vote / local polar / update; {per_sample_step:.2f} s per sample step over {len(times)} timed "
+                      f"steps; extrapolated to the whole workload ({wl.num_workers} workers, all parameters) by "
+                      f"float64 operation count (x{c_total / c_sample:.1f})",
+            "sample_seconds_per_step": per_sample_step, "extrapolated": True}
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the ncu
-# captures summarised under profiles/; None for workloads without a capture of the current kernel.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    ("c2_resnet50", "ns_gemm_tc_kernel"): 525.7e6,   # mean of 5 Gram (230.5 MB) and 5 apply (820.8 MB) launches
+# ncu DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the Newton-Schulz launches per unit of work, from
+# the captures summarised in profiles/ (small cases; the traffic of these launches grows in proportion to the entries
+# they process): bytes per (entry, worker) of one Gram launch and of one apply launch.
+NCU_NS_TRAFFIC_PER_ENTRY = {
+    # workload family -> (gram bytes per entry and worker, apply bytes per entry and worker, capture it comes from)
+    "large": (3.61, 12.81, "c5:4096x4096:4 (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
+    "c2_resnet50": (2.26, 8.05, "c2 (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
 }
 
 
@@ -170,9 +218,18 @@ def max_over_ranks(values, dist=None, device="cpu"):
     return [float(v) for v in t]
 
 
-def whole_job_value(ms_step, world):
-    """Replicas only: every rank runs one full step per `ms_step`, so the job does `world` steps in that time."""
-    return world * 1e3 / ms_step
+def whole_job_value(ms_step, world, sharded=False):
+    """Steps per second of the whole job.  Replicas: every rank runs one full step per `ms_step`, so the job does
+    `world` steps in that time.  Sharded workers: all ranks together complete one step per `ms_step`."""
+    return (1 if sharded else world) * 1e3 / ms_step
+
+
+def shard_workers(num_workers, world, rank):
+    """Contiguous, equal shards of the worker axis: (offset, count) of `rank`, or None when M % world != 0."""
+    if world <= 1 or num_workers % world != 0:
+        return None
+    per = num_workers // world
+    return rank * per, per
 
 
 def describe(wl):
@@ -190,10 +247,218 @@ def run_reference(args, wl):
     line = {"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": describe(wl),
-            "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample", "extrapolated")},
             "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ GPU measurement
+def kernel_report(wl, opt, stage_ms, peaks, clocks, timed_region_s, ns_scale="fro", power_iters=2):
+    """Per-kernel-family figures of one workload from its staged timings: algorithmic bytes / flops (the method's
+    own), the implementation's Newton-Schulz HBM bytes, achieved rates and roofline fractions."""
+    M = wl.num_workers
+    mat = [p for p in wl.params if p.kind == "matrix"]
+    plain = [p for p in wl.params if p.kind == "plain"]
+    gb = {"f32": 4, "bf16": 2}
+    K = wl.ns_steps
+    slots = M + (1 if wl.local_polar else 0)
+    ns_flops = opt.ns_flops_per_step
+    ns_exec = opt.ns_executed_flops_per_step
+    mom_bytes = sum(M * p.numel * (gb[p.dtype] + 4 + 4 + 2) for p in mat) + \
+        sum(p.numel * (M * (gb[p.dtype] + 8) + 2 * gb[p.dtype] + M / 8 + 1 / 8) for p in plain)
+    if ns_scale == "spectral":      # the power iteration reads the float32 momentum 2P + 1 more times
+        mom_bytes += sum(M * p.numel * 4 * (2 * power_iters + 1) for p in mat)
+    vote_bytes = sum(p.numel * (M / 8 + 1 / 8 + (2 if wl.local_polar else 2 * gb[p.dtype])) for p in mat)
+    kernels = {}
+    if stage_ms["momentum"] > 0:
+        a = mom_bytes / stage_ms["momentum"] / 1e6
+        kernels["momentum+plain"] = {"ms": stage_ms["momentum"], "bound": "hbm", "algorithmic_bytes": mom_bytes,
+                                     "achieved_gbs": a, "frac_of_measured_copy": a / peaks["hbm_gbs"],
+                                     "frac_of_nominal_8000": a / NOMINAL_HBM_GBS}
+    ns_ms = stage_ms["newton_schulz"] + stage_ms["local_polar"]
+    if ns_ms > 0 and ns_flops > 0:
+        launches = 2 * K * (2 if wl.local_polar else 1)
+        tf = ns_flops / ns_ms / 1e9
+        # The method's own memory traffic of the Newton-Schulz stage: the momentum is read once and one bit per entry
+        # and worker is written (plus, for the local polar step, the +-1 matrix in and the weights in and out).
+        method_bytes = sum(M * p.numel * (4 + 1 / 8) for p in mat) + \
+            (sum(p.numel * (2 + 2 * gb[p.dtype]) for p in mat) if wl.local_polar else 0)
+        # What this implementation moves: per entry, batch slot and iteration the Gram product reads the bf16 iterate
+        # (2 B), the apply product reads it again as an operand (2 B) and moves the hi + lo pair in and out (8 B).
+        impl_bytes = sum(12.0 * p.numel * K * slots for p in mat)
+        kernels["ns_gemm_tc"] = {
+            "ms": ns_ms, "bound": "tensor", "launches": launches, "algorithmic_flops": ns_flops,
+            "executed_flops": ns_exec, "achieved_tflops": tf, "executed_tflops": ns_exec / ns_ms / 1e9,
+            "frac_of_burst_peak": tf / peaks["bf16_tflops"], "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
+            "frac_of_nominal_2250": tf / NOMINAL_BF16_TFLOPS,
+            "method_bytes": method_bytes, "implementation_bytes": impl_bytes,
+            "implementation_gbs": impl_bytes / ns_ms / 1e6,
+            "implementation_gbs_frac_of_measured_copy": impl_bytes / ns_ms / 1e6 / peaks["hbm_gbs"]}
+    if stage_ms["vote_update"] > 0 and vote_bytes > 0:
+        a = vote_bytes / stage_ms["vote_update"] / 1e6
+        kernels["vote_update"] = {"ms": stage_ms["vote_update"], "bound": "hbm", "algorithmic_bytes": vote_bytes,
+                                  "achieved_gbs": a, "frac_of_measured_copy": a / peaks["hbm_gbs"],
+                                  "frac_of_nominal_8000": a / NOMINAL_HBM_GBS}
+    return kernels
+
+
+def roofline_of(wl, kernels, peaks, clocks, timed_ns_seconds):
+    """`roofline` object of the dominant kernel family."""
+    dom = max(kernels, key=lambda k: kernels[k]["ms"])
+    kd = kernels[dom]
+    if kd["bound"] == "tensor":
+        launches = kd["launches"]
+        achieved = kd["achieved_tflops"]
+        # Which measured cuBLAS rate is the fair denominator: the burst figure when the timed Newton-Schulz work is
+        # short or the clock stayed near its maximum, the sustained one when the region is seconds long and the
+        # clock settled under the power cap.
+        sm, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+        near_max = bool(sm and mx and sm >= 0.9 * mx)
+        use_sustained = timed_ns_seconds >= 1.0 and not near_max
+        peak = peaks["bf16_tflops_sustained"] if use_sustained else peaks["bf16_tflops"]
+        fam = "c2_resnet50" if wl.name.startswith("c2") else "large"
+        g_b, a_b, src = NCU_NS_TRAFFIC_PER_ENTRY[fam]
+        units = sum(p.numel for p in wl.params if p.kind == "matrix") * \
+            (wl.num_workers + (1 if wl.local_polar else 0)) / (2.0 if wl.local_polar else 1.0)
+        # mean over a step's Gram and apply launches (a local polar launch processes 1 / M of a workers' launch)
+        traffic = 0.5 * (g_b + a_b) * units
+        return {"kernel": "ns_gemm_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": achieved / peak,
+                "frac_is": ("of measured sustained cuBLAS bf16 (timed Newton-Schulz work %.1f s, median SM clock %s MHz)"
+                            if use_sustained else
+                            "of measured burst cuBLAS bf16 (timed Newton-Schulz work %.1f s, median SM clock %s MHz)")
+                           % (timed_ns_seconds, sm),
+                "frac_of_burst_peak": kd["frac_of_burst_peak"], "frac_of_sustained_peak": kd["frac_of_sustained_peak"],
+                "frac_of_nominal_2250": kd["frac_of_nominal_2250"],
+                "algorithmic_flops_per_launch": kd["algorithmic_flops"] / launches,
+                "executed_flops_per_launch": kd["executed_flops"] / launches,
+                "executed_tflops": kd["executed_tflops"], "ms_per_launch": kd["ms"] / launches,
+                "traffic": traffic, "traffic_source": "ncu capture of " + src + ", scaled by (entries x batch slots)",
+                "peak_source": peaks["source"]}
+    achieved = kd["achieved_gbs"]
+    return {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved / peaks["hbm_gbs"], "traffic": None, "bytes_per_launch": kd["algorithmic_bytes"],
+            "ms_per_launch": kd["ms"], "peak_source": peaks["source"] + " (copy bandwidth)",
+            "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS}
+
+
+def measure(wl, args, dev, dist, rank, world, local_rank, steps, warmup, with_e2e):
+    """Device-timed steps, staged timings and (optionally) the host-buffer leg of one workload."""
+    import torch
+    from paper_2605_16311_b200 import binding as B
+    from paper_2605_16311_b200 import workloads as wlmod
+
+    shard = shard_workers(wl.num_workers, world, rank)
+    sharded = shard is not None
+    kw = {}
+    if sharded:
+        kw = {"worker_offset": shard[0], "local_workers": shard[1]}
+    opt = B.SignMuon(wl.params, wl.num_workers, momentum=wl.momentum, lr=wl.lr, ns_steps=wl.ns_steps,
+                     local_polar=wl.local_polar, device=dev, host_staging=with_e2e, ns_scale=args.ns_scale,
+                     power_iters=args.power_iters, **kw)
+    if args.ns_scale == "spectral":     # seeded start vectors of the power iteration, reused by every step
+        flat = torch.zeros(opt.power_start_size, dtype=torch.float32, device=dev)
+        for p, v in enumerate(wlmod.make_power_start(wl, 0, dev)):
+            if v is not None:
+                off, _ = opt.power_start_segment(p)
+                lo = shard[0] if sharded else 0
+                v = v[lo: lo + opt.local_workers]
+                flat[off: off + v.numel()] = v.reshape(-1)
+        opt.set_power_start(flat)
+    weights = wlmod.make_weights(wl, dev)
+    signal = wlmod.make_signal(wl, dev)
+    n_sets = 2                                           # fresh noise per step, rotating pre-drawn sets
+    grad_sets = []
+    for t in range(n_sets):
+        gs = wlmod.make_grads(wl, signal, t, dev)
+        if sharded:                                      # this rank's workers only
+            gs = [g[shard[0]: shard[0] + shard[1]].contiguous() for g in gs]
+        grad_sets.append(gs)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def full_step(t):
+        if sharded:
+            opt.step_sharded(weights, grad_sets[t % n_sets], wl.lr, dist)
+        else:
+            opt.step(weights, grad_sets[t % n_sets], wl.lr)
+
+    # ---------------------------------------------------------------- device-resident timing
+    for t in range(warmup):
+        full_step(t)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(steps):
+        full_step(t)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    status = opt.status()
+    if status != B.OK:
+        raise RuntimeError(f"device status after the timed region: {status}")
+
+    # ---------------------------------------------------------------- per-stage timing (same steps, events between stages)
+    stages = [("momentum", B.STAGE_MOMENTUM), ("newton_schulz", B.STAGE_NS), ("exchange", None),
+              ("vote_update", B.STAGE_VOTE), ("local_polar", B.STAGE_LOCAL_POLAR)]
+    n_stage_steps = max(3, min(steps, 20))
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(n_stage_steps)]
+    for t in range(n_stage_steps):
+        evs[t][0].record()
+        for i, (_, mask) in enumerate(stages):
+            if mask is None:
+                if sharded:
+                    opt.exchange_payloads(dist)
+            else:
+                opt.step(weights, grad_sets[t % n_sets], wl.lr, stages=mask)
+            evs[t][i + 1].record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    stage_ms = {name: statistics.mean(evs[t][i].elapsed_time(evs[t][i + 1]) for t in range(n_stage_steps))
+                for i, (name, _) in enumerate(stages)}
+
+    # ---------------------------------------------------------------- end to end with host buffers
+    e2e_ms, h2d, d2h = float("nan"), 0, 0
+    if with_e2e:
+        host_w = [w.cpu().pin_memory() for w in weights]
+        host_g = [[g.cpu().pin_memory() for g in gs] for gs in grad_sets]
+        h2d = sum(w.numel() * w.element_size() for w in host_w) + sum(g.numel() * g.element_size() for g in host_g[0])
+        d2h = sum(w.numel() * w.element_size() for w in host_w)
+        e2e_steps = max(3, min(steps, 20))
+
+        def host_step(t):
+            if sharded:
+                opt.step_host_sharded(host_w, host_g[t % n_sets], wl.lr, dist)
+            else:
+                opt.step_host(host_w, host_g[t % n_sets], wl.lr)
+        for t in range(2):
+            host_step(t)
+        barrier()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record()
+        for t in range(e2e_steps):
+            host_step(t)
+        h1.record()
+        barrier()
+        e2e_ms = h0.elapsed_time(h1) / e2e_steps
+        del host_w, host_g
+
+    ms_step, e2e_ms = max_over_ranks([ms_total / steps, e2e_ms], dist, dev)
+    ns_seconds = (stage_ms["newton_schulz"] + stage_ms["local_polar"]) * n_stage_steps / 1e3
+    res = {"ms_per_step": ms_step, "e2e_ms": e2e_ms, "h2d": h2d, "d2h": d2h, "stage_ms": stage_ms, "clocks": clocks,
+           "launches_per_step": opt.launches_per_step, "sharded": sharded, "timed_ns_seconds": ns_seconds,
+           "kernels": kernel_report(wl, opt, stage_ms, load_peaks(), clocks, ns_seconds, args.ns_scale, args.power_iters)}
+    opt.close()
+    del opt, weights, signal, grad_sets
+    torch.cuda.empty_cache()
+    return res
 
 
 def run_ours(args, wl):
@@ -217,156 +482,58 @@ def run_ours(args, wl):
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     B.load_library()
+    peaks = load_peaks()
 
-    opt = B.SignMuon(wl.params, wl.num_workers, momentum=wl.momentum, lr=wl.lr, ns_steps=wl.ns_steps,
-                     local_polar=wl.local_polar, device=dev, host_staging=True, ns_scale=args.ns_scale,
-                     power_iters=args.power_iters)
-    if args.ns_scale == "spectral":     # seeded start vectors of the power iteration, reused by every step
-        flat = torch.zeros(opt.power_start_size, dtype=torch.float32, device=dev)
-        for p, v in enumerate(wlmod.make_power_start(wl, 0, dev)):
-            if v is not None:
-                off, _ = opt.power_start_segment(p)
-                flat[off: off + v.numel()] = v.reshape(-1)
-        opt.set_power_start(flat)
-    weights = wlmod.make_weights(wl, dev)
-    signal = wlmod.make_signal(wl, dev)
-    n_sets = 2                                           # fresh noise per step, rotating pre-drawn sets
-    grad_sets = [wlmod.make_grads(wl, signal, t, dev) for t in range(n_sets)]
-    torch.cuda.synchronize()
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    # ---------------------------------------------------------------- device-resident timing
-    for t in range(args.warmup):
-        opt.step(weights, grad_sets[t % n_sets], wl.lr)
-    barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for t in range(args.steps):
-        opt.step(weights, grad_sets[t % n_sets], wl.lr)
-    e1.record()
-    barrier()
-    ms_total = e0.elapsed_time(e1)
-    status = opt.status()
-    if status != B.OK:
-        raise RuntimeError(f"device status after the timed region: {status}")
-
-    # ---------------------------------------------------------------- per-stage timing (same steps, events between stages)
-    stages = [("momentum", B.STAGE_MOMENTUM), ("newton_schulz", B.STAGE_NS), ("vote_update", B.STAGE_VOTE),
-              ("local_polar", B.STAGE_LOCAL_POLAR)]
-    n_stage_steps = max(3, min(args.steps, 20))
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(n_stage_steps)]
-    for t in range(n_stage_steps):
-        evs[t][0].record()
-        for i, (_, mask) in enumerate(stages):
-            opt.step(weights, grad_sets[t % n_sets], wl.lr, stages=mask)
-            evs[t][i + 1].record()
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    stage_ms = {name: statistics.mean(evs[t][i].elapsed_time(evs[t][i + 1]) for t in range(n_stage_steps))
-                for i, (name, _) in enumerate(stages)}
-
-    # ---------------------------------------------------------------- end to end with host buffers
-    host_w = [w.cpu().pin_memory() for w in weights]
-    host_g = [[g.cpu().pin_memory() for g in gs] for gs in grad_sets]
-    h2d = sum(w.numel() * w.element_size() for w in host_w) + sum(g.numel() * g.element_size() for g in host_g[0])
-    d2h = sum(w.numel() * w.element_size() for w in host_w)
-    e2e_steps = 0 if args.no_e2e else max(3, min(args.steps, 30))
-    for t in range(0 if args.no_e2e else 2):
-        opt.step_host(host_w, host_g[t % n_sets], wl.lr)
-    barrier()
-    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    h0.record()
-    for t in range(e2e_steps):
-        opt.step_host(host_w, host_g[t % n_sets], wl.lr)
-    h1.record()
-    barrier()
-    e2e_ms = h0.elapsed_time(h1) / e2e_steps if e2e_steps else float("nan")
-
-    # ---------------------------------------------------------------- reduce over ranks
-    ms_step, e2e_ms = max_over_ranks([ms_total / args.steps, e2e_ms], dist, dev)
+    main = measure(wl, args, dev, dist, rank, world, local_rank, args.steps, args.warmup, with_e2e=not args.no_e2e)
+    secondary = {}
+    if not args.no_secondary:
+        for name in ("c2", "c3"):
+            wl2 = wlmod.by_name(name)
+            if wl2.name == wl.name:
+                continue
+            r = measure(wl2, args, dev, dist, rank, world, local_rank, max(5, min(args.steps, 20)), 3, with_e2e=False)
+            k = r["kernels"]
+            secondary[wl2.name] = {
+                "config": describe(wl2), "ms_per_step": r["ms_per_step"],
+                "steps_per_sec": whole_job_value(r["ms_per_step"], world, r["sharded"]),
+                "stage_ms": r["stage_ms"], "clocks": r["clocks"],
+                "ns_tflops": k.get("ns_gemm_tc", {}).get("achieved_tflops"),
+                "ns_executed_tflops": k.get("ns_gemm_tc", {}).get("executed_tflops"),
+                "ns_frac_of_burst_peak": k.get("ns_gemm_tc", {}).get("frac_of_burst_peak"),
+                "momentum_gbs": k.get("momentum+plain", {}).get("achieved_gbs"),
+                "vote_update_gbs": k.get("vote_update", {}).get("achieved_gbs"),
+                "kernels": k}
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    peaks = load_peaks()
-    M = wl.num_workers
-    mat = [p for p in wl.params if p.kind == "matrix"]
-    plain = [p for p in wl.params if p.kind == "plain"]
-    gb = {"f32": 4, "bf16": 2}
-    ns_flops = opt.ns_flops_per_step
-    lp_frac = (1.0 / (M + 1)) if wl.local_polar else 0.0
-    mom_bytes = sum(M * p.numel * (gb[p.dtype] + 4 + 4 + 2) for p in mat) + \
-        sum(p.numel * (M * (gb[p.dtype] + 8) + 2 * gb[p.dtype] + M / 8 + 1 / 8) for p in plain)
-    vote_bytes = sum(p.numel * (M / 8 + 1 / 8 + (2 if wl.local_polar else 2 * gb[p.dtype])) for p in mat)
-    n_ns_launches = 2 * wl.ns_steps
-    if args.ns_scale == "spectral":      # the power iteration reads the float32 momentum 2P + 1 more times
-        mom_bytes += sum(M * p.numel * 4 * (2 * args.power_iters + 1) for p in mat)
-    kernels = {}
-    if stage_ms["momentum"] > 0:
-        kernels["momentum+plain"] = {"ms": stage_ms["momentum"], "bound": "hbm", "algorithmic_bytes": mom_bytes,
-                                     "achieved_gbs": mom_bytes / stage_ms["momentum"] / 1e6}
-    ns_ms = stage_ms["newton_schulz"] + stage_ms["local_polar"]
-    if ns_ms > 0 and ns_flops > 0:
-        kernels["ns_gemm_tc"] = {"ms": ns_ms, "bound": "tensor", "algorithmic_flops": ns_flops,
-                                 "launches": n_ns_launches * (2 if wl.local_polar else 1),
-                                 "achieved_tflops": ns_flops / ns_ms / 1e9}
-    if "ns_gemm_tc" in kernels:
-        # the iteration's own memory traffic: per entry, worker and iteration the Gram product reads the bf16 iterate
-        # (2 B), the apply product reads it again as an operand (2 B) and moves hi + lo in and out (8 B)
-        ns_bytes = sum(12.0 * p.numel * wl.ns_steps * (M + (1 if wl.local_polar else 0)) for p in mat)
-        kernels["ns_gemm_tc"].update({"hbm_algorithmic_bytes": ns_bytes, "hbm_achieved_gbs": ns_bytes / ns_ms / 1e6,
-                                      "hbm_frac_of_measured": ns_bytes / ns_ms / 1e6 / peaks["hbm_gbs"]})
-    if stage_ms["vote_update"] > 0 and vote_bytes > 0:
-        kernels["vote_update"] = {"ms": stage_ms["vote_update"], "bound": "hbm", "algorithmic_bytes": vote_bytes,
-                                  "achieved_gbs": vote_bytes / stage_ms["vote_update"] / 1e6}
-    # dominant kernel family of the step
-    dom = max(kernels, key=lambda k: kernels[k]["ms"])
-    kd = kernels[dom]
-    if kd["bound"] == "tensor":
-        launches = kd["launches"]
-        per_launch_ms = kd["ms"] / launches
-        achieved = kd["achieved_tflops"]
-        peak = peaks["bf16_tflops_sustained"]
-        roof = {"kernel": "ns_gemm_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((wl.name, "ns_gemm_tc_kernel")),
-                "flops_per_launch": ns_flops / launches, "ms_per_launch": per_launch_ms,
-                "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
-                "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0}
-    else:
-        achieved = kd["achieved_gbs"]
-        peak = peaks["hbm_gbs"]
-        roof = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "bytes_per_launch": kd["algorithmic_bytes"],
-                "ms_per_launch": kd["ms"], "peak_source": peaks["source"] + " (copy bandwidth)",
-                "frac_of_nominal_8000": achieved / 8000.0}
-
     cpu = None
     if not args.no_cpu_baseline:
-        cpu = time_oracle(wl, 1, 0, args.cpu_baseline_flops)
-        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        cpu = time_oracle(wl, 1, 0, args.oracle_flops, min_seconds=args.cpu_baseline_seconds)
+        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample", "extrapolated")}
 
-    line = {"metric": METRIC, "value": whole_job_value(ms_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+    kernels = main["kernels"]
+    sharded = main["sharded"]
+    line = {"metric": METRIC, "value": whole_job_value(main["ms_per_step"], world, sharded), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": main["ms_per_step"],
+            "higher_is_better": True, "scaling": "strong" if sharded else "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": dict(describe(wl), ns_scale=args.ns_scale,
                            **({"power_iters": args.power_iters} if args.ns_scale == "spectral" else {})),
-            "clocks": clocks,
+            "clocks": main["clocks"],
             "e2e": (None if args.no_e2e else
-                    {"value": whole_job_value(e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms}),
-            "gpu_launches": opt.launches_per_step * args.steps,
-            "roofline": roof, "cpu_baseline": cpu,
-            "stage_ms": stage_ms, "kernels": kernels,
-            "ns_tflops": ns_flops / ns_ms / 1e9 if ns_ms > 0 else None,
-            "multi_gpu": "replicas only" if world > 1 else None}
+                    {"value": whole_job_value(main["e2e_ms"], world, sharded), "unit": UNIT,
+                     "h2d_bytes_per_step": main["h2d"], "d2h_bytes_per_step": main["d2h"],
+                     "ms_per_step": main["e2e_ms"]}),
+            "gpu_launches": main["launches_per_step"] * args.steps,
+            "roofline": roofline_of(wl, kernels, peaks, main["clocks"], main["timed_ns_seconds"]),
+            "cpu_baseline": cpu, "stage_ms": main["stage_ms"], "kernels": kernels,
+            "ns_tflops": kernels.get("ns_gemm_tc", {}).get("achieved_tflops"),
+            "secondary": secondary,
+            "multi_gpu": (None if world == 1 else
+                          ("workers sharded over ranks, packed payload all-gathered (NCCL)" if sharded
+                           else "replicas only (M not divisible by the number of ranks)"))}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -385,8 +552,8 @@ def run_sweep(args):
     build_mod.build()
     B.load_library()
     peaks = load_peaks()
-    sides = [512, 1024, 2048, 4096, 8192]
-    shapes = [(n, n) for n in sides] + [(512, 2048), (2048, 512), (1024, 4096), (4096, 1024), (2048, 8192), (8192, 2048)]
+    shapes = wlmod.sweep_shapes() if not args.sweep_shapes else \
+        [tuple(int(v) for v in s.split("x")) for s in args.sweep_shapes.split(",")]
     workers = [int(x) for x in args.sweep_workers.split(",")]
     for (r, c) in shapes:
         for M in workers:
@@ -418,9 +585,12 @@ def run_sweep(args):
                 vote_bytes = d * (M / 8 + 1 / 8 + 4)
                 line = {"workload": f"c5:{r}x{c}:{M}:{K}", "rows": r, "cols": c, "num_workers": M, "ns_steps": K,
                         "ns_ms": ms[1], "ns_tflops": ns_flops / ms[1] / 1e9,
+                        "ns_executed_tflops": opt.ns_executed_flops_per_step / ms[1] / 1e9,
+                        "ns_frac_of_burst_peak": ns_flops / ms[1] / 1e9 / peaks["bf16_tflops"],
                         "ns_frac_of_sustained_peak": ns_flops / ms[1] / 1e9 / peaks["bf16_tflops_sustained"],
                         "momentum_ms": ms[0], "momentum_gbs": mom_bytes / ms[0] / 1e6,
                         "vote_update_ms": ms[2], "vote_update_gbs": vote_bytes / ms[2] / 1e6,
+                        "vote_update_frac_of_measured_copy": vote_bytes / ms[2] / 1e6 / peaks["hbm_gbs"],
                         "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"]}
                 print(json.dumps(line), flush=True)
                 opt.close()
@@ -431,21 +601,23 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c2", help="c1 | c2 | c3 | c4 | c4_nolp | c5:ROWSxCOLS:M[:K]")
+    ap.add_argument("--workload", default="c4", help="c1 | c2 | c3 | c4 | c4_nolp | c5:ROWSxCOLS:M[:K]")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
-    ap.add_argument("--oracle-flops", type=float, default=1.2e11,
-                    help="float64 operation budget of one oracle sample step")
-    ap.add_argument("--cpu-baseline-flops", type=float, default=2.5e12,
-                    help="float64 operation budget of the oracle sample timed beside the GPU run")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the secondary workloads (c2, c3)")
+    ap.add_argument("--oracle-flops", type=float, default=3.0e12,
+                    help="float64 operation budget of one oracle sample step (reference arm and cpu_baseline leg)")
+    ap.add_argument("--cpu-baseline-seconds", type=float, default=10.0,
+                    help="the cpu_baseline leg repeats its sample step until this much time has passed")
     ap.add_argument("--ns-scale", default="fro", choices=["fro", "spectral"],
                     help="Alg. 4 scale: Frobenius norm (default, the benchmark configuration) or power iteration")
     ap.add_argument("--power-iters", type=int, default=2)
     ap.add_argument("--sweep", action="store_true", help="run the kernel sweep (config 5) and print one line per point")
     ap.add_argument("--sweep-workers", default="1,2,4,8,16,32")
+    ap.add_argument("--sweep-shapes", default="", help="comma-separated ROWSxCOLS list (default: the whole sweep)")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)

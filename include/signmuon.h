@@ -57,7 +57,8 @@ enum {
   SIGNMUON_ERR_TIMEOUT = -6,          /* a bounded device-side wait ran out (see signmuon_status) */
   SIGNMUON_ERR_UNSUPPORTED_ARCH = -7, /* current device is not compute capability 10.x */
   SIGNMUON_ERR_MISALIGNED = -8,       /* a device pointer is not 16-byte aligned */
-  SIGNMUON_ERR_TOO_LARGE = -9         /* problem exceeds a fixed capacity (signmuon_momentum_norm_noalloc) */
+  SIGNMUON_ERR_TOO_LARGE = -9,        /* problem exceeds a fixed capacity (signmuon_momentum_norm_noalloc) */
+  SIGNMUON_ERR_NO_MEMORY = -10        /* a host allocation (context, pinned table mirror) failed */
 };
 
 typedef enum { SIGNMUON_F32 = 0, SIGNMUON_BF16 = 1 } signmuon_dtype;
@@ -126,7 +127,8 @@ enum {
 
 /* Creates a context from a HOST config (Alg. 2 "Input"). Touches no GPU.
  * Errors: INVALID_ARG (null, M outside [1,255], beta outside [0,1), K < 0, lambda < 0,
- * unknown enum), BAD_SHAPE. On error *out is set to NULL. */
+ * unknown enum), BAD_SHAPE (a side < 1 or > 2^24, more than 2^36 entries, a matrix parameter whose longer side
+ * exceeds 128 * 65535), NO_MEMORY. On error *out is set to NULL. */
 int signmuon_create(const signmuon_config* config, signmuon_ctx** out);
 
 /* Bytes the caller must provide: `state` = momenta of all workers (float32 [M][d] per parameter,
@@ -140,7 +142,8 @@ int signmuon_state_bytes(const signmuon_ctx* ctx, size_t* state, size_t* workspa
  * prepares the device-side tables on `cuda_stream` (a cudaStream_t, NULL = legacy default stream).
  * `zero_state` != 0 clears the momenta (Mom_0 = 0); pass 0 when restoring a checkpointed state.
  * `dev_staging` may be NULL when signmuon_step_host is not used.
- * Errors: BUFFER_TOO_SMALL, MISALIGNED, UNSUPPORTED_ARCH, CUDA. */
+ * Also allocates (once per context) a few KB of pinned HOST memory that mirrors the parameter tables.
+ * Errors: BUFFER_TOO_SMALL, MISALIGNED, UNSUPPORTED_ARCH, NO_MEMORY, CUDA. */
 int signmuon_bind(signmuon_ctx* ctx, void* dev_state, size_t state_bytes, void* dev_workspace,
                   size_t workspace_bytes, void* dev_staging, size_t staging_bytes, int zero_state,
                   void* cuda_stream);
@@ -149,6 +152,8 @@ int signmuon_bind(signmuon_ctx* ctx, void* dev_state, size_t state_bytes, void* 
  *   weights: HOST array of num_params DEVICE pointers, W_p [rows][cols] in weight_dtype, updated in place
  *   grads:   HOST array of num_params DEVICE pointers, G_p [M][rows][cols] in grad_dtype (worker-major), read only
  *   lr:      eta_t for this step; a negative value selects config.lr
+ * The device keeps the pointer tables of the last four distinct (weights, grads) pointer sets: a call with a
+ * set seen before uploads nothing; a new set costs one small asynchronous copy from pinned memory.
  * Errors: NOT_BOUND, INVALID_ARG, MISALIGNED, CUDA (sticky launch error). */
 int signmuon_step(signmuon_ctx* ctx, void* const* weights, const void* const* grads, float lr,
                   void* cuda_stream);
@@ -187,8 +192,18 @@ int signmuon_debug_tap(const signmuon_ctx* ctx, int32_t what, int32_t param, int
                        const void** dev_ptr, size_t* bytes, int64_t* ld);
 
 /* Synchronises `cuda_stream`, then reads the device status word: OK, TIMEOUT (a bounded wait in a
- * kernel gave up; results of that step are invalid) or CUDA. */
+ * kernel gave up; results of that step are invalid) or CUDA.  TIMEOUT stays until the next signmuon_bind. */
 int signmuon_status(signmuon_ctx* ctx, void* cuda_stream);
+
+/* Failure detection.  Every wait inside the Newton-Schulz kernels (on a TMA transfer, a tensor-core commit, an
+ * epilogue hand-over) is bounded: after `limit_ns` nanoseconds (0 selects the default of two seconds) the waiting
+ * thread records TIMEOUT in the status word and its CTA drains and exits, so a step can fail but not hang.
+ * signmuon_selftest_wait_timeout enqueues a one-thread kernel that performs exactly that wait on a barrier nothing
+ * ever signals, with the given limit (at most two seconds): afterwards signmuon_status must report TIMEOUT, and
+ * signmuon_bind clears it.  Lets a deployment check the detection path without disturbing a step.
+ * Errors: INVALID_ARG, NOT_BOUND, CUDA. */
+int signmuon_set_wait_limit(signmuon_ctx* ctx, uint64_t limit_ns);
+int signmuon_selftest_wait_timeout(signmuon_ctx* ctx, uint64_t limit_ns, void* cuda_stream);
 
 /* Start vectors of the power iteration (Alg. 5, "Sample v in R^c"), needed when ns_scale is
  * SIGNMUON_SCALE_SPECTRAL: the method draws them at random, so the caller passes them in.
@@ -217,6 +232,12 @@ int signmuon_launches_per_step(const signmuon_ctx* ctx, int32_t* launches);
  * more "worker" for the local polar step), s = min(rows, cols), l = max(rows, cols). */
 int signmuon_ns_flops_per_step(const signmuon_ctx* ctx, double* flops);
 
+/* Flops the tensor cores are actually asked for per step by the tile schedule of the bound context: whole
+ * 256 x 256 x 64 (or 128 x 128 x 64) blocks per scheduled tile, so ragged edges count in full, while the mirror
+ * tiles of the symmetric Gram products (Alg. 4: A = Y Y^T), which are never computed, do not count.  Differs from
+ * signmuon_ns_flops_per_step, the algorithm's own 4 s^2 l K.  Errors: INVALID_ARG, NOT_BOUND. */
+int signmuon_ns_executed_flops_per_step(const signmuon_ctx* ctx, double* flops);
+
 /* Capacity of the built-in scratch of signmuon_momentum_norm_noalloc: one float per 8192 entries per
  * worker, i.e. num_workers * ceil(rows*cols / 8192) must not exceed it (about 5.4e8 entries over all
  * workers; e.g. 4096 x 4096 with 32 workers just fits). */
@@ -232,12 +253,16 @@ int signmuon_ns_flops_per_step(const signmuon_ctx* ctx, double* flops);
  * they can still hand over a workspace; this call needs none.  Its only scratch - the per-block partial
  * sums of the norm reduction - lives in a fixed 256 KB array inside the library image, present on every
  * GPU that loads the library until the process exits.  The call itself allocates nothing and calls
- * nothing that allocates.
+ * nothing that allocates (one caveat: the first call on a device is where the CUDA runtime may load the
+ * library's device code and place that array; warm the entry point up once, outside any stream capture,
+ * before the region that must not allocate).
  *
  *   dev_grads        DEVICE [M][rows*cols] grad_dtype, read only
  *   dev_weights      DEVICE [rows*cols] weight_dtype, read only; may be NULL when weight_decay == 0
  *   dev_momentum     DEVICE [M][rows*cols] float32, updated in place
- *   dev_operand_bf16 DEVICE [M][rows*cols] bf16, written: bf16(momentum), the Newton-Schulz operand
+ *   dev_operand_bf16 DEVICE [M][rows*cols] bf16, written dense (row pitch = cols): bf16(momentum).  This is
+ *                    the layout of signmuon_step's Newton-Schulz operand only when cols is a multiple of 8
+ *                    (the regular path pads rows to a multiple of 8 elements)
  *   dev_scales       DEVICE [M][2] float32, written: 1/max(sigma,eps)^2 and 1/max(sigma,eps)
  * rows*cols must be a multiple of 8 and all array pointers 16-byte aligned.
  *
@@ -246,7 +271,8 @@ int signmuon_ns_flops_per_step(const signmuon_ctx* ctx, double* flops);
  * call overwrites the part it uses before reading it, so no clearing is needed between calls, but calls
  * that may run concurrently on one GPU (different streams without ordering) race - keep them ordered.
  * The first call on each device resolves the array's device address; make that call outside any stream
- * capture.  Other errors: INVALID_ARG, BAD_SHAPE, MISALIGNED, CUDA. */
+ * capture.  Other errors: INVALID_ARG, BAD_SHAPE, MISALIGNED, UNSUPPORTED_ARCH (current device is not
+ * compute capability 10.x), CUDA (one of this call's own two launches was refused). */
 int signmuon_momentum_norm_noalloc(const void* dev_grads, int32_t grad_dtype, const void* dev_weights,
                                    int32_t weight_dtype, float* dev_momentum, void* dev_operand_bf16,
                                    float* dev_scales, int64_t rows, int64_t cols, int32_t num_workers,

@@ -26,13 +26,15 @@ TAP_MOMENTUM, TAP_POLAR, TAP_VOTE_BITS, TAP_WORKER_BITS, TAP_NORM = 0, 1, 2, 3, 
 EXPORTS = [
     "signmuon_create", "signmuon_state_bytes", "signmuon_bind", "signmuon_step", "signmuon_run_stages",
     "signmuon_step_host", "signmuon_packed_payload", "signmuon_payload_segment", "signmuon_debug_tap",
-    "signmuon_status", "signmuon_launches_per_step", "signmuon_ns_flops_per_step",
+    "signmuon_status", "signmuon_launches_per_step", "signmuon_ns_flops_per_step", "signmuon_ns_executed_flops_per_step",
     "signmuon_power_start_size", "signmuon_power_start_segment", "signmuon_set_power_start",
-    "signmuon_sign_agreement",
+    "signmuon_sign_agreement", "signmuon_set_wait_limit", "signmuon_selftest_wait_timeout",
     "signmuon_momentum_norm_noalloc", "signmuon_destroy", "signmuon_error_string",
 ]
 NOALLOC_MAX_PARTIALS = 65536
+ERR_TIMEOUT = -6
 ERR_TOO_LARGE = -9
+ERR_NO_MEMORY = -10
 
 
 class ParamStruct(C.Structure):
@@ -73,10 +75,13 @@ def load_library() -> C.CDLL:
     lib.signmuon_status.argtypes = [vp, vp]
     lib.signmuon_launches_per_step.argtypes = [vp, C.POINTER(i32)]
     lib.signmuon_ns_flops_per_step.argtypes = [vp, C.POINTER(C.c_double)]
+    lib.signmuon_ns_executed_flops_per_step.argtypes = [vp, C.POINTER(C.c_double)]
     lib.signmuon_power_start_size.argtypes = [vp, C.POINTER(sz)]
     lib.signmuon_power_start_segment.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
     lib.signmuon_set_power_start.argtypes = [vp, vp, sz]
     lib.signmuon_sign_agreement.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), vp]
+    lib.signmuon_set_wait_limit.argtypes = [vp, C.c_uint64]
+    lib.signmuon_selftest_wait_timeout.argtypes = [vp, C.c_uint64, vp]
     lib.signmuon_momentum_norm_noalloc.argtypes = [vp, i32, vp, i32, vp, vp, vp, C.c_int64, C.c_int64, i32,
                                                    f32, f32, f32, vp]
     lib.signmuon_destroy.argtypes = [vp]
@@ -197,6 +202,12 @@ def signmuon_ns_flops_per_step(ctx: int) -> float:
     return f.value
 
 
+def signmuon_ns_executed_flops_per_step(ctx: int) -> float:
+    f = C.c_double()
+    _check(load_library().signmuon_ns_executed_flops_per_step(ctx, C.byref(f)), "signmuon_ns_executed_flops_per_step")
+    return f.value
+
+
 def signmuon_power_start_size(ctx: int) -> int:
     n = C.c_size_t()
     _check(load_library().signmuon_power_start_size(ctx, C.byref(n)), "signmuon_power_start_size")
@@ -221,6 +232,15 @@ def signmuon_sign_agreement(ctx: int, num_workers: int, stream: int):
     _check(load_library().signmuon_sign_agreement(ctx, agree, C.byref(entries), stream or None),
            "signmuon_sign_agreement")
     return list(agree), entries.value
+
+
+def signmuon_set_wait_limit(ctx: int, limit_ns: int):
+    _check(load_library().signmuon_set_wait_limit(ctx, limit_ns), "signmuon_set_wait_limit")
+
+
+def signmuon_selftest_wait_timeout(ctx: int, limit_ns: int, stream: int):
+    _check(load_library().signmuon_selftest_wait_timeout(ctx, limit_ns, stream or None),
+           "signmuon_selftest_wait_timeout")
 
 
 def signmuon_momentum_norm_noalloc(grads_ptr: int, grad_dtype: int, weights_ptr: int, weight_dtype: int,
@@ -280,6 +300,20 @@ class SignMuon:
                           self.workspace_bytes, self.staging.data_ptr() if host_staging else 0,
                           self.staging_bytes if host_staging else 0, True, stream)
         self._ptr_cache = None
+
+    def rebind(self, zero_state: bool = True):
+        """Binds the same buffers again (clears the device status word; optionally the momenta)."""
+        with torch.cuda.device(self.device):
+            stream = torch.cuda.current_stream(self.device).cuda_stream
+            signmuon_bind(self.ctx, self.state.data_ptr(), self.state_bytes, self.workspace.data_ptr(),
+                          self.workspace_bytes, self.staging.data_ptr() if self.staging is not None else 0,
+                          self.staging_bytes if self.staging is not None else 0, zero_state, stream)
+
+    def set_wait_limit(self, limit_ns: int):
+        signmuon_set_wait_limit(self.ctx, limit_ns)
+
+    def selftest_wait_timeout(self, limit_ns: int):
+        signmuon_selftest_wait_timeout(self.ctx, limit_ns, torch.cuda.current_stream(self.device).cuda_stream)
 
     def close(self):
         if self.ctx:
@@ -356,3 +390,7 @@ class SignMuon:
     @property
     def ns_flops_per_step(self) -> float:
         return signmuon_ns_flops_per_step(self.ctx)
+
+    @property
+    def ns_executed_flops_per_step(self) -> float:
+        return signmuon_ns_executed_flops_per_step(self.ctx)

@@ -9,7 +9,9 @@ namespace signmuon {
 constexpr int EW_THREADS = 256;
 constexpr int MOM_CHUNK = 8192;        // entries per block of the momentum kernel (256 threads x 8 x 4)
 constexpr int PLAIN_CHUNK = 2048;      // entries per block of the plain-parameter kernel (8 warps x 256)
-constexpr int VOTE_WORDS = 256;        // payload words per block of the vote kernel (8 warps x 32)
+constexpr int VOTE_THREADS = 128;      // vote kernel: 4 warps per block
+constexpr int VOTE_WARP_WORDS = 128;   // payload words per warp (4 consecutive words per lane: 128-bit loads)
+constexpr int VOTE_WORDS = VOTE_WARP_WORDS * VOTE_THREADS / 32;   // payload words per block
 constexpr int PACK_CHUNK = 1024;       // entries per block of the stand-alone pack kernel (small: it only sees small, ragged matrices)
 
 // Finds the list slot whose block range contains `block` (`starts` is ascending, one entry per slot).
@@ -195,7 +197,7 @@ __device__ __forceinline__ void store8(bf16* p, const float (&x)[8]) {
 template <typename GT, typename WT>
 __device__ __forceinline__ void plain_warp_vec(const ParamDev& pd, int64_t base, int M, float beta, float lambda,
                                                float step, uint32_t* __restrict__ bits,
-                                               uint32_t* __restrict__ vote_words, int64_t words_per_worker) {
+                                               uint32_t* __restrict__ vote_words, int64_t bits_pitch) {
   const int lane = threadIdx.x & 31;
   const int64_t d = pd.d;
   const int64_t i0 = base + 8 * lane;
@@ -223,7 +225,7 @@ __device__ __forceinline__ void plain_warp_vec(const ParamDev& pd, int64_t base,
     }
     store8(mom + (int64_t)m * d, mv);
     const uint32_t wordv = __reduce_or_sync(group, byte << shift);
-    if ((lane & 3) == 0) out[(int64_t)m * words_per_worker] = wordv;
+    if ((lane & 3) == 0) out[(int64_t)m * bits_pitch] = wordv;
   };
   int m = 0;
   for (; m + 1 < M; m += 2) {
@@ -256,30 +258,30 @@ __device__ __forceinline__ void plain_warp_vec(const ParamDev& pd, int64_t base,
 template <typename GT, typename WT>
 __device__ __forceinline__ void plain_warp_scalar(const ParamDev& pd, int64_t base, int M, float beta, float lambda,
                                                   float step, uint32_t* __restrict__ bits,
-                                                  uint32_t* __restrict__ vote_words, int64_t words_per_worker);
+                                                  uint32_t* __restrict__ vote_words, int64_t bits_pitch);
 
 template <typename GT, typename WT>
 __device__ __forceinline__ void plain_block(const ParamDev& pd, uint32_t chunk, int M, float beta,
                                             float lambda, float step, uint32_t* __restrict__ bits,
-                                            uint32_t* __restrict__ vote_words, int64_t words_per_worker) {
+                                            uint32_t* __restrict__ vote_words, int64_t bits_pitch) {
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int64_t d = pd.d;
   if ((d & 7) == 0 && (int64_t)chunk * PLAIN_CHUNK + (warp + 1) * 256 <= d) {
     plain_warp_vec<GT, WT>(pd, (int64_t)chunk * PLAIN_CHUNK + warp * 256, M, beta, lambda, step, bits, vote_words,
-                           words_per_worker);
+                           bits_pitch);
     return;
   }
   // ragged tail (or an unaligned parameter): the warp's 256 entries as two scalar passes of 128
   for (int pass = 0; pass < 2; ++pass)
     plain_warp_scalar<GT, WT>(pd, (int64_t)chunk * PLAIN_CHUNK + warp * 256 + pass * 128, M, beta, lambda, step, bits,
-                              vote_words, words_per_worker);
+                              vote_words, bits_pitch);
 }
 
 template <typename GT, typename WT>
 __device__ __forceinline__ void plain_warp_scalar(const ParamDev& pd, int64_t base, int M, float beta,
                                                   float lambda, float step, uint32_t* __restrict__ bits,
-                                                  uint32_t* __restrict__ vote_words, int64_t words_per_worker) {
+                                                  uint32_t* __restrict__ vote_words, int64_t bits_pitch) {
   const int lane = threadIdx.x & 31;
   const int64_t d = pd.d;
   if (base >= d) return;
@@ -319,7 +321,7 @@ __device__ __forceinline__ void plain_warp_scalar(const ParamDev& pd, int64_t ba
       if (lane == k) mine = word;
     }
     if (lane < 4 && word0 + lane < pd.n_words)
-      bits[(int64_t)m * words_per_worker + pd.word_off + word0 + lane] = mine;
+      bits[(int64_t)m * bits_pitch + pd.word_off + word0 + lane] = mine;
   }
   uint32_t vmine = 0;
 #pragma unroll
@@ -343,17 +345,17 @@ __global__ void __launch_bounds__(EW_THREADS) plain_params_kernel(const ParamDev
                                                                   int M, float beta, float lambda, float lr,
                                                                   uint32_t* __restrict__ bits,
                                                                   uint32_t* __restrict__ vote_words,
-                                                                  int64_t words_per_worker) {
+                                                                  int64_t bits_pitch) {
   const int slot = find_slot(starts, n_list, blockIdx.x);
   const ParamDev pd = params[list[slot]];
   const uint32_t chunk = blockIdx.x - starts[slot];
   const float step = lr * pd.upd_scale;
   if (pd.gdtype == 0) {
-    if (pd.wdtype == 0) plain_block<float, float>(pd, chunk, M, beta, lambda, step, bits, vote_words, words_per_worker);
-    else plain_block<float, bf16>(pd, chunk, M, beta, lambda, step, bits, vote_words, words_per_worker);
+    if (pd.wdtype == 0) plain_block<float, float>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch);
+    else plain_block<float, bf16>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch);
   } else {
-    if (pd.wdtype == 0) plain_block<bf16, float>(pd, chunk, M, beta, lambda, step, bits, vote_words, words_per_worker);
-    else plain_block<bf16, bf16>(pd, chunk, M, beta, lambda, step, bits, vote_words, words_per_worker);
+    if (pd.wdtype == 0) plain_block<bf16, float>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch);
+    else plain_block<bf16, bf16>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch);
   }
 }
 
@@ -366,7 +368,7 @@ __global__ void __launch_bounds__(EW_THREADS) pack_kernel(const ParamDev* __rest
                                                           const int32_t* __restrict__ list,
                                                           const uint32_t* __restrict__ starts, int n_list,
                                                           int src_buf, int from_momentum,
-                                                          uint32_t* __restrict__ bits, int64_t words_per_worker) {
+                                                          uint32_t* __restrict__ bits, int64_t bits_pitch) {
   const int slot = find_slot(starts, n_list, blockIdx.x);
   const ParamDev pd = params[list[slot]];
   const uint32_t local = blockIdx.x - starts[slot];
@@ -392,116 +394,177 @@ __global__ void __launch_bounds__(EW_THREADS) pack_kernel(const ParamDev* __rest
     }
     const uint32_t word = __ballot_sync(0xffffffffu, b);
     const int64_t wi = i >> 5;
-    if (lane == 0 && wi < pd.n_words) bits[(int64_t)m * words_per_worker + pd.word_off + wi] = word;
+    if (lane == 0 && wi < pd.n_words) bits[(int64_t)m * bits_pitch + pd.word_off + wi] = word;
   }
 }
 
 // ---------------------------------------------------------------------------------------------
 // Majority vote from the packed words (App. B: c = sum_m b^(m), S = sign(2c - M), ties -> +1) and
 // the weight update W <- W - eta S (Alg. 3), or, for the local polar step, S as a bf16 +-1 matrix.
-// Lane t of a warp loads word (base + t) of every worker (coalesced rows) and keeps the 32
-// per-position counts as bit-sliced counter planes; the comparison c >= ceil(M/2) is the carry
-// out of a bit-sliced addition of 2^PLANES - ceil(M/2).  The vote words are then exchanged by
-// shuffle so that lane l updates entry 32 k + l of word k: coalesced weight traffic.
+//
+// A warp owns an aligned group of 128 words of the payload's word index (the workers' rows are 128-byte
+// aligned in the workspace, so lane l reads words 4l..4l+3 of every worker as one 128-bit load, eight rows in
+// flight).  The 32 per-position counts of each word are kept as bit-sliced counter planes (about three logic
+// operations per worker word instead of 32 unpacks); the comparison c >= ceil(M/2) is the carry out of a
+// bit-sliced addition of 2^PLANES - ceil(M/2).  The 128 vote words then go through shared memory so that the
+// weights (or the +-1 matrix) move as 128-bit vectors too; the first batch of weight vectors is requested
+// before the payload, so both latencies overlap.  Words of the group outside the parameter are masked.
 // ---------------------------------------------------------------------------------------------
 template <int PLANES>
-__device__ __forceinline__ uint32_t vote_word(const uint32_t* __restrict__ bits, int64_t words_per_worker,
-                                              int64_t word_index, int M) {
+struct VoteCounter {
   uint32_t c[PLANES];
+  __device__ __forceinline__ void clear() {
 #pragma unroll
-  for (int b = 0; b < PLANES; ++b) c[b] = 0;
-  auto add_word = [&](uint32_t carry) {
+    for (int b = 0; b < PLANES; ++b) c[b] = 0;
+  }
+  __device__ __forceinline__ void add(uint32_t carry) {
 #pragma unroll
     for (int b = 0; b < PLANES; ++b) {
       const uint32_t t = c[b] & carry;
       c[b] ^= carry;
       carry = t;
     }
-  };
-  const uint32_t* col = bits + word_index;
-  int m = 0;
-  for (; m + 3 < M; m += 4) {          // four workers' words in flight
-    uint32_t w4[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) w4[k] = __ldcs(col + (int64_t)(m + k) * words_per_worker);
-#pragma unroll
-    for (int k = 0; k < 4; ++k) add_word(w4[k]);
   }
-  for (; m < M; ++m) add_word(__ldcs(col + (int64_t)m * words_per_worker));
-  const uint32_t add = (1u << PLANES) - (uint32_t)((M + 1) >> 1);
-  uint32_t carry = 0;
+  // bit set <=> count >= ceil(M/2) <=> 2c - M >= 0
+  __device__ __forceinline__ uint32_t majority(int M) const {
+    const uint32_t add = (1u << PLANES) - (uint32_t)((M + 1) >> 1);
+    uint32_t carry = 0;
 #pragma unroll
-  for (int b = 0; b < PLANES; ++b) {
-    const uint32_t kb = ((add >> b) & 1u) ? 0xffffffffu : 0u;
-    carry = (c[b] & kb) | (carry & (c[b] ^ kb));
+    for (int b = 0; b < PLANES; ++b) {
+      const uint32_t kb = ((add >> b) & 1u) ? 0xffffffffu : 0u;
+      carry = (c[b] & kb) | (carry & (c[b] ^ kb));
+    }
+    return carry;
   }
-  return carry;   // bit set <=> count >= ceil(M/2) <=> 2c - M >= 0
-}
+};
+
+template <typename WT> __host__ __device__ constexpr int write_sbar_vec_entries() { return 16 / (int)sizeof(WT); }
 
 template <int PLANES, typename WT>
-__device__ __forceinline__ void vote_block(const ParamDev& pd, uint32_t chunk, int M, float step, int write_sbar,
-                                           const uint32_t* __restrict__ bits, uint32_t* __restrict__ vote_words,
-                                           int64_t words_per_worker) {
+__device__ __forceinline__ void vote_warp(const ParamDev& pd, int64_t g0, int M, float step, int write_sbar,
+                                          const uint32_t* __restrict__ bits, uint32_t* __restrict__ vote_words,
+                                          int64_t bits_pitch, uint32_t* sv) {
+  constexpr int ROWS = PLANES >= 8 ? 4 : 8;             // worker rows in flight per lane
+  constexpr int EPV = write_sbar_vec_entries<WT>();     // entries per 128-bit weight vector (float: 4, bf16: 8)
   const int lane = threadIdx.x & 31;
-  const int warp = threadIdx.x >> 5;
-  const int64_t wbase = (int64_t)chunk * VOTE_WORDS + warp * 32;
-  if (wbase >= pd.n_words) return;
-  const int64_t my_word = wbase + lane;
-  uint32_t v = 0;
-  if (my_word < pd.n_words) {
-    v = vote_word<PLANES>(bits, words_per_worker, pd.word_off + my_word, M);
-    vote_words[pd.word_off + my_word] = v;
-  }
+  const int64_t lo = pd.word_off, hi = (int64_t)pd.word_off + pd.n_words;
+  if (g0 >= hi || g0 + VOTE_WARP_WORDS <= lo) return;
+  const int64_t g = g0 + 4 * lane;                      // this lane's first word (global word index)
+  const bool lane_full = g >= lo && g + 4 <= hi;
+  const int64_t e0 = (g0 - lo) * 32;                    // entry of the group's first word (negative: group starts before the parameter)
+  const int64_t d = pd.d;
+  // 128-bit path: every vector lies inside one vote word; it needs 16-byte aligned rows of whole vectors
+  const bool vec = write_sbar ? (pd.vec_ok != 0) : ((d & 7) == 0);
   WT* w = reinterpret_cast<WT*>(pd.W);
   bf16* sbar = pd.y0 + (int64_t)M * pd.rows * pd.ldy;   // slot M of operand buffer 0: input of the local polar step
-  const int64_t e0 = wbase * 32;                        // first entry of this warp's 1024
-  if (pd.vec_ok && e0 + 1024 <= pd.d) {
-    // 128-bit path: the warp's 1024 entries are 256 float4 (fp32 weights) or 128 uint4 (bf16 weights or the
-    // +-1 matrix); a lane's vector lies inside one vote word, fetched from its owner lane by shuffle.
-    if (!write_sbar && sizeof(WT) == 4) {
-      float4* w4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(w) + e0);
-      float4 x[8];
+
+  // The group's entries as 128-bit vectors: vector i of the group covers entries e0 + i * epv .. + epv - 1
+  // (epv = 4 float32 or 8 bf16), all inside vote word i / (32 / epv).  Valid when the entry is inside the parameter.
+  const int epv = write_sbar ? 8 : EPV;
+  const int n_batches = (VOTE_WARP_WORDS * 32 / epv) / (8 * 32);      // 8 vectors per lane and batch
+  uint4* vbase = write_sbar ? reinterpret_cast<uint4*>(sbar) : reinterpret_cast<uint4*>(w);
+  auto vec_valid = [&](int i) -> bool {
+    const int64_t e = e0 + (int64_t)i * epv;
+    return e >= 0 && e < d;
+  };
+  auto vec_ptr = [&](int i) -> uint4* {                 // 16-byte units from the start of the parameter
+    return vbase + (e0 / epv + i);
+  };
+  uint4 x[8];                                           // float4 bit patterns or 8 bf16 each
+  const bool rmw = vec && !write_sbar;
+  if (rmw) {                                            // first batch of weight vectors: independent of the vote
 #pragma unroll
-      for (int it = 0; it < 8; ++it) x[it] = __ldcs(w4 + it * 32 + lane);
+    for (int it = 0; it < 8; ++it) {
+      const int i = it * 32 + lane;
+      x[it] = vec_valid(i) ? __ldcs(vec_ptr(i)) : make_uint4(0, 0, 0, 0);
+    }
+  }
+
+  // ---- vote of this lane's four words
+  VoteCounter<PLANES> cnt[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) cnt[j].clear();
+  const uint32_t* col = bits + g;
+  if (lane_full) {
+    int m = 0;
+    for (; m + ROWS <= M; m += ROWS) {
+      uint4 r[ROWS];
+#pragma unroll
+      for (int k = 0; k < ROWS; ++k) r[k] = __ldcs(reinterpret_cast<const uint4*>(col + (int64_t)(m + k) * bits_pitch));
+#pragma unroll
+      for (int k = 0; k < ROWS; ++k) { cnt[0].add(r[k].x); cnt[1].add(r[k].y); cnt[2].add(r[k].z); cnt[3].add(r[k].w); }
+    }
+    for (; m < M; ++m) {
+      const uint4 r = __ldcs(reinterpret_cast<const uint4*>(col + (int64_t)m * bits_pitch));
+      cnt[0].add(r.x); cnt[1].add(r.y); cnt[2].add(r.z); cnt[3].add(r.w);
+    }
+  } else {
+    for (int m = 0; m < M; ++m) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (g + j >= lo && g + j < hi) cnt[j].add(__ldcs(col + (int64_t)m * bits_pitch + j));
+    }
+  }
+  uint32_t v[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) v[j] = cnt[j].majority(M);
+  if (lane_full) {
+    *reinterpret_cast<uint4*>(vote_words + g) = make_uint4(v[0], v[1], v[2], v[3]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (g + j >= lo && g + j < hi) vote_words[g + j] = v[j];
+  }
+  *reinterpret_cast<uint4*>(sv + 4 * lane) = make_uint4(v[0], v[1], v[2], v[3]);
+  __syncwarp();
+
+  if (vec) {
+#pragma unroll 1
+    for (int batch = 0; batch < n_batches; ++batch) {
+      if (batch > 0 && rmw) {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+          const int i = (batch * 8 + it) * 32 + lane;
+          x[it] = vec_valid(i) ? __ldcs(vec_ptr(i)) : make_uint4(0, 0, 0, 0);
+        }
+      }
 #pragma unroll
       for (int it = 0; it < 8; ++it) {
-        const uint32_t bits4 = __shfl_sync(0xffffffffu, v, it * 4 + (lane >> 3)) >> ((lane & 7) * 4);
-        x[it].x -= (bits4 & 1u) ? step : -step;
-        x[it].y -= (bits4 & 2u) ? step : -step;
-        x[it].z -= (bits4 & 4u) ? step : -step;
-        x[it].w -= (bits4 & 8u) ? step : -step;
-        __stcs(w4 + it * 32 + lane, x[it]);
-      }
-    } else {
-      uint4* w8 = write_sbar ? reinterpret_cast<uint4*>(sbar + e0) : reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(w) + e0);
-      uint4 x[4];
+        const int i = (batch * 8 + it) * 32 + lane;
+        if (!vec_valid(i)) continue;
+        uint4 o;
+        if (!write_sbar && sizeof(WT) == 4) {           // 4 float32: a nibble of word i / 8
+          const uint32_t b4 = sv[i >> 3] >> ((i & 7) * 4);
+          o.x = __float_as_uint(__uint_as_float(x[it].x) - ((b4 & 1u) ? step : -step));
+          o.y = __float_as_uint(__uint_as_float(x[it].y) - ((b4 & 2u) ? step : -step));
+          o.z = __float_as_uint(__uint_as_float(x[it].z) - ((b4 & 4u) ? step : -step));
+          o.w = __float_as_uint(__uint_as_float(x[it].w) - ((b4 & 8u) ? step : -step));
+        } else {                                        // 8 bf16: a byte of word i / 4
+          const uint32_t b8 = sv[i >> 2] >> ((i & 3) * 8);
+          const uint32_t in[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
+          uint32_t ov[4];
 #pragma unroll
-      for (int it = 0; it < 4; ++it) x[it] = write_sbar ? make_uint4(0, 0, 0, 0) : __ldcs(w8 + it * 32 + lane);
-#pragma unroll
-      for (int it = 0; it < 4; ++it) {
-        const uint32_t bits8 = __shfl_sync(0xffffffffu, v, it * 8 + (lane >> 2)) >> ((lane & 3) * 8);
-        const uint32_t in[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
-        uint32_t o[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const bool p0 = (bits8 >> (2 * e)) & 1u, p1 = (bits8 >> (2 * e + 1)) & 1u;
-          if (write_sbar) {
-            o[e] = pack_bf16x2(p0 ? 1.f : -1.f, p1 ? 1.f : -1.f);
-          } else {
-            o[e] = pack_bf16x2(__uint_as_float(in[e] << 16) - (p0 ? step : -step),
-                               __uint_as_float(in[e] & 0xffff0000u) - (p1 ? step : -step));
+          for (int e = 0; e < 4; ++e) {
+            const bool p0 = (b8 >> (2 * e)) & 1u, p1 = (b8 >> (2 * e + 1)) & 1u;
+            if (write_sbar) ov[e] = (p0 ? 0x3f80u : 0xbf80u) | ((p1 ? 0x3f80u : 0xbf80u) << 16);      // bf16 +-1
+            else ov[e] = pack_bf16x2(__uint_as_float(in[e] << 16) - (p0 ? step : -step),
+                                     __uint_as_float(in[e] & 0xffff0000u) - (p1 ? step : -step));
           }
+          o = make_uint4(ov[0], ov[1], ov[2], ov[3]);
         }
-        __stcs(w8 + it * 32 + lane, make_uint4(o[0], o[1], o[2], o[3]));
+        __stcs(vec_ptr(i), o);
       }
     }
     return;
   }
-#pragma unroll 4
-  for (int k = 0; k < 32; ++k) {
-    const uint32_t vk = __shfl_sync(0xffffffffu, v, k);
-    const int64_t i = (wbase + k) * 32 + lane;
-    if (i < pd.d) {
+  // scalar path: rows that are padded in the operand buffer (the +-1 matrix of a parameter whose column count is
+  // not a multiple of 8), or d not a multiple of 8
+  for (int k = 0; k < VOTE_WARP_WORDS; ++k) {
+    const int64_t gw = g0 + k;
+    if (gw < lo || gw >= hi) continue;
+    const uint32_t vk = sv[k];
+    const int64_t i = (gw - lo) * 32 + lane;
+    if (i < d) {
       const bool plus = (vk >> lane) & 1u;
       if (write_sbar) {
         int64_t o = i;
@@ -520,19 +583,23 @@ __device__ __forceinline__ void vote_block(const ParamDev& pd, uint32_t chunk, i
 }
 
 template <int PLANES>
-__global__ void __launch_bounds__(EW_THREADS) vote_update_kernel(const ParamDev* __restrict__ params,
-                                                                 const int32_t* __restrict__ list,
-                                                                 const uint32_t* __restrict__ starts, int n_list,
-                                                                 int M, float lr, int write_sbar,
-                                                                 const uint32_t* __restrict__ bits,
-                                                                 uint32_t* __restrict__ vote_words,
-                                                                 int64_t words_per_worker) {
+__global__ void __launch_bounds__(VOTE_THREADS) vote_update_kernel(const ParamDev* __restrict__ params,
+                                                                   const int32_t* __restrict__ list,
+                                                                   const uint32_t* __restrict__ starts, int n_list,
+                                                                   int M, float lr, int write_sbar,
+                                                                   const uint32_t* __restrict__ bits,
+                                                                   uint32_t* __restrict__ vote_words,
+                                                                   int64_t bits_pitch) {
+  __shared__ __align__(16) uint32_t sv_all[VOTE_THREADS / 32][VOTE_WARP_WORDS];
   const int slot = find_slot(starts, n_list, blockIdx.x);
   const ParamDev pd = params[list[slot]];
   const uint32_t chunk = blockIdx.x - starts[slot];
+  const int warp = threadIdx.x >> 5;
+  // first word of this warp's group: groups are aligned in the payload's word index, not in the parameter
+  const int64_t g0 = ((int64_t)(pd.word_off / VOTE_WORDS) + chunk) * VOTE_WORDS + warp * VOTE_WARP_WORDS;
   const float step = lr * pd.upd_scale;
-  if (pd.wdtype == 0) vote_block<PLANES, float>(pd, chunk, M, step, write_sbar, bits, vote_words, words_per_worker);
-  else vote_block<PLANES, bf16>(pd, chunk, M, step, write_sbar, bits, vote_words, words_per_worker);
+  if (pd.wdtype == 0) vote_warp<PLANES, float>(pd, g0, M, step, write_sbar, bits, vote_words, bits_pitch, sv_all[warp]);
+  else vote_warp<PLANES, bf16>(pd, g0, M, step, write_sbar, bits, vote_words, bits_pitch, sv_all[warp]);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -542,10 +609,10 @@ __global__ void __launch_bounds__(EW_THREADS) vote_update_kernel(const ParamDev*
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(EW_THREADS) sign_agreement_kernel(const uint32_t* __restrict__ bits,
                                                                     const uint32_t* __restrict__ vote_words,
-                                                                    int64_t words_per_worker,
+                                                                    int64_t words_per_worker, int64_t bits_pitch,
                                                                     unsigned long long* __restrict__ agree) {
   const int m = blockIdx.y;
-  const uint32_t* mine = bits + (int64_t)m * words_per_worker;
+  const uint32_t* mine = bits + (int64_t)m * bits_pitch;
   unsigned int acc = 0;   // at most 32 bits x (words / threads) per thread: far below 2^32
   for (int64_t i = (int64_t)blockIdx.x * EW_THREADS + threadIdx.x; i < words_per_worker; i += (int64_t)gridDim.x * EW_THREADS)
     acc += __popc(~(__ldg(mine + i) ^ __ldg(vote_words + i)));

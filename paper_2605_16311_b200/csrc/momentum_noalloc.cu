@@ -16,7 +16,10 @@
 //     are read, so nothing has to be cleared between calls, but two calls that overlap on the GPU
 //     (different streams, no ordering between them) race on it.  Keep calls stream-ordered.
 //   * the first call on each device looks up the array's device address (cudaGetSymbolAddress with
-//     that device current).  Make that first call outside any stream capture.
+//     that device current).  Make that first call outside any stream capture.  That first call is also
+//     where the CUDA runtime may load this library's device code onto the GPU and place the array
+//     (lazy module loading): "allocates nothing" describes every call after it, and this one as far as
+//     the library's own code goes.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -147,12 +150,22 @@ __global__ void norm_noalloc_kernel(const float* __restrict__ partials, uint32_t
   }
 }
 
+// Launches return their own status (cudaLaunchKernelEx), so an earlier, unrelated error that is still
+// pending in the runtime is neither reported as this call's nor cleared by it.
+cudaLaunchConfig_t launch_config(unsigned blocks, unsigned threads, cudaStream_t s) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks, 1, 1);
+  cfg.blockDim = dim3(threads, 1, 1);
+  cfg.stream = s;
+  return cfg;
+}
+
 template <typename GT, typename WT>
-void launch_noalloc(const void* g, const void* w, float* mom, void* operand, float* partials, int64_t d,
-                    uint32_t cpw, int M, float beta, float lambda, cudaStream_t s) {
-  momentum_noalloc_kernel<GT, WT><<<(unsigned)(cpw * (uint32_t)M), NA_THREADS, 0, s>>>(
-      static_cast<const GT*>(g), static_cast<const WT*>(w), mom, static_cast<bf16*>(operand), partials, d, cpw, beta,
-      lambda);
+cudaError_t launch_noalloc(const void* g, const void* w, float* mom, void* operand, float* partials, int64_t d,
+                           uint32_t cpw, int M, float beta, float lambda, cudaStream_t s) {
+  const cudaLaunchConfig_t cfg = launch_config(cpw * (uint32_t)M, NA_THREADS, s);
+  return cudaLaunchKernelEx(&cfg, momentum_noalloc_kernel<GT, WT>, static_cast<const GT*>(g),
+                            static_cast<const WT*>(w), mom, static_cast<bf16*>(operand), partials, d, cpw, beta, lambda);
 }
 
 }  // namespace
@@ -177,23 +190,33 @@ extern "C" int signmuon_momentum_norm_noalloc(const void* dev_grads, int32_t gra
   if ((align & 15) || (reinterpret_cast<uintptr_t>(dev_scales) & 3)) return SIGNMUON_ERR_MISALIGNED;
   if (!(eps > 0.f)) eps = 1e-12f;
 
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+    return SIGNMUON_ERR_CUDA;
+  if (major != 10) return SIGNMUON_ERR_UNSUPPORTED_ARCH;   // the library image holds sm_100a code only
+
   float* partials = nullptr;                           // device address of g_noalloc_partials on this device
   const int rc = scratch_for_current_device(&partials);
   if (rc != SIGNMUON_OK) return rc;
 
   cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
   const uint32_t c = (uint32_t)cpw;
+  cudaError_t err;
   if (grad_dtype == SIGNMUON_F32) {
     if (weight_dtype == SIGNMUON_F32)
-      launch_noalloc<float, float>(dev_grads, dev_weights, dev_momentum, dev_operand_bf16, partials, d, c, num_workers, momentum, weight_decay, s);
+      err = launch_noalloc<float, float>(dev_grads, dev_weights, dev_momentum, dev_operand_bf16, partials, d, c, num_workers, momentum, weight_decay, s);
     else
-      launch_noalloc<float, bf16>(dev_grads, dev_weights, dev_momentum, dev_operand_bf16, partials, d, c, num_workers, momentum, weight_decay, s);
+      err = launch_noalloc<float, bf16>(dev_grads, dev_weights, dev_momentum, dev_operand_bf16, partials, d, c, num_workers, momentum, weight_decay, s);
   } else {
     if (weight_dtype == SIGNMUON_F32)
-      launch_noalloc<bf16, float>(dev_grads, dev_weights, dev_momentum, dev_operand_bf16, partials, d, c, num_workers, momentum, weight_decay, s);
+      err = launch_noalloc<bf16, float>(dev_grads, dev_weights, dev_momentum, dev_operand_bf16, partials, d, c, num_workers, momentum, weight_decay, s);
     else
-      launch_noalloc<bf16, bf16>(dev_grads, dev_weights, dev_momentum, dev_operand_bf16, partials, d, c, num_workers, momentum, weight_decay, s);
+      err = launch_noalloc<bf16, bf16>(dev_grads, dev_weights, dev_momentum, dev_operand_bf16, partials, d, c, num_workers, momentum, weight_decay, s);
   }
-  norm_noalloc_kernel<<<(num_workers * 32 + 255) / 256, 256, 0, s>>>(partials, c, num_workers, eps, dev_scales);
-  return cudaGetLastError() == cudaSuccess ? SIGNMUON_OK : SIGNMUON_ERR_CUDA;
+  if (err != cudaSuccess) return SIGNMUON_ERR_CUDA;
+  const cudaLaunchConfig_t ncfg = launch_config((unsigned)(num_workers * 32 + 255) / 256, 256, s);
+  err = cudaLaunchKernelEx(&ncfg, norm_noalloc_kernel, static_cast<const float*>(partials), c, (int)num_workers, eps,
+                           dev_scales);
+  return err == cudaSuccess ? SIGNMUON_OK : SIGNMUON_ERR_CUDA;
 }

@@ -37,8 +37,8 @@
 // Gram products are symmetric: only tiles on or above the diagonal are scheduled and an off-diagonal tile is
 // also stored transposed.  A problem may carry up to three operand pairs ("segments") that are accumulated
 // into the same tile along K: split-precision products (hi hi + lo hi + hi lo) of the spectral scale.
-// Every wait is bounded: after about two seconds a waiting thread records STATUS_TIMEOUT in the
-// status word, raises a CTA-wide abort flag and the CTA drains and exits (TMEM is freed).
+// Every wait is bounded: after the launch's wait limit (two seconds by default) a waiting thread records
+// STATUS_TIMEOUT in the status word, raises a CTA-wide abort flag and the CTA drains and exits (TMEM is freed).
 #pragma once
 
 #include <cuda.h>
@@ -57,7 +57,7 @@ constexpr int EPI_NCOL = 256 / EPI_WARPS;    // columns of a chunk one math thre
 static_assert(EPI_WARPS == 8 || EPI_WARPS == 16, "8 or 16 epilogue math warps");
 constexpr int GEMM_THREADS = 32 * (3 + EPI_WARPS);   // warp 0: operand TMA, warp 1: MMA, then the epilogue math warps,
                                                      // last warp: epilogue TMA (C loads, result stores)
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
+constexpr uint64_t DEFAULT_WAIT_LIMIT_NS = 2000000000ull;   // two seconds unless the caller sets another limit
 
 struct GemmLaunchArgs {
   const CUtensorMap* tmaps;
@@ -67,6 +67,7 @@ struct GemmLaunchArgs {
   const ParamDev* params;
   uint32_t* status;
   float lr;
+  uint64_t wait_limit_ns;           // after this long a waiting thread gives up and the CTA aborts
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -99,7 +100,7 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 }
 // Bounded wait. Returns false when the CTA is aborting (this or another thread ran out of time).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* status) {
+                                          uint32_t* status, uint64_t limit_ns) {
   uint32_t spins = 0;
   uint64_t t0 = 0;
   while (!mbar_try_wait(bar, parity)) {
@@ -108,7 +109,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       const uint64_t now = global_timer_ns();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > WAIT_LIMIT_NS) {
+      } else if (now - t0 > limit_ns) {
         *abort_flag = 1;
         atomicExch(status, (uint32_t)STATUS_TIMEOUT);
         return false;
@@ -391,7 +392,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
           if (seg == 1) { mapA = args.tmaps + pr.tmapA2; mapB = args.tmaps + pr.tmapB2; }
           else if (seg == 2) { mapA = args.tmaps + pr.tmapA3; mapB = args.tmaps + pr.tmapB3; }
           for (int kb = 0; kb < nk; ++kb, ++it) {
-            if (!mbar_wait(smem_u32(&empty_bar[0]) + 8u * s, par, abort_flag, args.status)) { ok = false; break; }
+            if (!mbar_wait(smem_u32(&empty_bar[0]) + 8u * s, par, abort_flag, args.status, args.wait_limit_ns)) { ok = false; break; }
             // the "full" barrier of the pair is CTA 0's: it expects the bytes of both CTAs
             const uint32_t fb = full0 + 8u * s;
             if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[0]) + 8u * s, stage_tx);
@@ -446,11 +447,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         const bool share_ab = KIND == 0 && B_ROWS == GEMM_BM && pr.diag_share != 0 && te.tm == te.tn;
         const uint32_t acc = tcount & 1u;
         const uint32_t acc_round = tcount >> 1;
-        if (!mbar_wait(smem_u32(&tmem_empty_bar[acc]), (acc_round & 1u) ^ 1u, abort_flag, args.status)) { ok = false; break; }
+        if (!mbar_wait(smem_u32(&tmem_empty_bar[acc]), (acc_round & 1u) ^ 1u, abort_flag, args.status, args.wait_limit_ns)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = 0; kb < nk; ++kb) {
-          if (!mbar_wait(smem_u32(&full_bar[0]) + 8u * s, par, abort_flag, args.status)) { ok = false; break; }
+          if (!mbar_wait(smem_u32(&full_bar[0]) + 8u * s, par, abort_flag, args.status, args.wait_limit_ns)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + s * STAGE_BYTES;
           const uint32_t sb = share_ab ? sa : sa + A_BYTES;
@@ -543,7 +544,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
             const uint32_t b = g % EPI_BUFS;
             const uint32_t buf = epi_base + b * BUF_BYTES;
             const int col0 = n0 + ch * 64;
-            if (!mbar_wait(smem_u32(&buf_ready_bar[b]), (g / EPI_BUFS) & 1u, abort_flag, args.status)) { ok = false; break; }
+            if (!mbar_wait(smem_u32(&buf_ready_bar[b]), (g / EPI_BUFS) & 1u, abort_flag, args.status, args.wait_limit_ns)) { ok = false; break; }
             if (store_hi) {
               tma_store_3d(mapO0, col0, row0, batch_o, buf);
               if (store_lo) tma_store_3d(mapO1, col0, row0, batch_o, buf + EPI_HALF_BYTES);
@@ -596,7 +597,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
         const bool mirror = KIND == 0 && pr.sym != 0 && pr.gram_lo == 0 && te.tn != te.tm && rows_live;   // off-diagonal Gram tile
         const uint32_t acc = tcount & 1u;
         const uint32_t acc_round = tcount >> 1;
-        ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_round & 1u, abort_flag, args.status);
+        ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_round & 1u, abort_flag, args.status, args.wait_limit_ns);
         ok = __all_sync(0xffffffffu, ok);        // the whole warp takes the same exit
         if (!ok) break;
         tc_fence_after();
@@ -606,7 +607,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
           const uint32_t b = g % EPI_BUFS;
           const uint32_t buf = epi_base + b * BUF_BYTES;
           const int col0 = n0 + ch * 64 + sub * NC;    // first of this thread's columns
-          ok = mbar_wait(smem_u32(&c_full_bar[b]), (g / EPI_BUFS) & 1u, abort_flag, args.status);
+          ok = mbar_wait(smem_u32(&c_full_bar[b]), (g / EPI_BUFS) & 1u, abort_flag, args.status, args.wait_limit_ns);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           float v[NC];
@@ -640,7 +641,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
               // of this lane quarter still have to read: all of them finish reading before any writes.
               __syncwarp();
               if (lane == 0) mbar_arrive(smem_u32(&row_pair_bar[q]));
-              ok = mbar_wait(smem_u32(&row_pair_bar[q]), f32_chunks & 1u, abort_flag, args.status);
+              ok = mbar_wait(smem_u32(&row_pair_bar[q]), f32_chunks & 1u, abort_flag, args.status, args.wait_limit_ns);
               ++f32_chunks;
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) break;
@@ -722,6 +723,21 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
     __syncthreads();
     if (warp == 1)
       asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// Self-test of the bounded wait: one thread waits, with the same mbar_wait as the product kernel, on an mbarrier
+// that nothing ever arrives at.  The wait runs out after `limit_ns`, the status word receives STATUS_TIMEOUT
+// and the kernel returns normally; the context stays usable.
+__global__ void wait_timeout_probe_kernel(uint32_t* status, uint64_t limit_ns) {
+  __shared__ uint64_t never_bar;
+  __shared__ uint32_t abort_word;
+  if (threadIdx.x == 0) {
+    abort_word = 0;
+    mbar_init(smem_u32(&never_bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    volatile uint32_t* abort_flag = &abort_word;
+    mbar_wait(smem_u32(&never_bar), 0u, abort_flag, status, limit_ns);
   }
 }
 

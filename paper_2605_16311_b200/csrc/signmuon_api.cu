@@ -7,6 +7,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <queue>
 #include <vector>
@@ -74,10 +75,12 @@ struct signmuon_ctx {
   uint32_t mom_blocks = 0, plain_blocks = 0, vote_blocks = 0, packfb_blocks = 0, xv_blocks = 0, xtu_blocks = 0;
   size_t power_start_floats = 0;          // length of the start-vector array (scale = spectral)
   const float* d_power_start = nullptr;   // caller's start vectors (device)
-  uint64_t words_per_worker = 0;
+  uint64_t words_per_worker = 0;          // payload words of one worker (the bytes it would transmit / 4)
+  uint64_t bits_pitch = 0;                // words between two workers' payloads in the workspace (128-byte rows)
   int64_t entries = 0;
   size_t state_bytes = 0, workspace_bytes = 0, staging_bytes = 0;
   // workspace offsets
+  size_t paramdev_stride = 0;             // bytes between two copies of the parameter table
   size_t off_status = 0, off_paramdev = 0, off_lists = 0, off_bits = 0, off_vote = 0, off_tmaps = 0,
          off_problems = 0, off_tables_end = 0;
   size_t off_list_matrix = 0, off_list_plain = 0, off_list_packfb = 0, off_starts_mom = 0, off_starts_plain = 0,
@@ -99,10 +102,24 @@ struct signmuon_ctx {
   cudaEvent_t ev_loaded[2] = {nullptr, nullptr}, ev_consumed[2] = {nullptr, nullptr};
   uint64_t host_steps = 0;
   int num_sms = 0;
-  std::vector<ParamDev> paramdev;         // host copy of the device table
-  bool paramdev_uploaded = false;
+  // Parameter tables.  The device keeps PARAM_TABLES copies of the ParamDev table, one per set of caller
+  // pointers (weights, gradients) seen recently: a caller that alternates between a few sets of buffers (two
+  // gradient buffers, the two staging sets of signmuon_step_host) finds its table already on the device and
+  // the step uploads nothing.  A new set takes the least recently used slot; its image is written into that
+  // slot's pinned host mirror and copied asynchronously (the slot's event guards the mirror's reuse).
+  std::vector<ParamDev> paramdev;         // template: everything except W and G
+  ParamDev* h_tables = nullptr;           // pinned host mirrors, [PARAM_TABLES][num_params]
+  cudaEvent_t ev_table[4] = {nullptr, nullptr, nullptr, nullptr};
+  std::vector<const void*> table_key[4];  // W pointers then G pointers of the set a slot holds (empty: free)
+  uint64_t table_used[4] = {0, 0, 0, 0};
+  uint64_t table_clock = 0;
+  int cur_table = 0;                      // slot of the step being enqueued
+  uint64_t wait_limit_ns = DEFAULT_WAIT_LIMIT_NS;
+  double executed_flops = 0;              // flops the scheduled tiles issue per step (known once the tile tables exist)
   int sticky = SIGNMUON_OK;
 };
+
+namespace { constexpr int PARAM_TABLES = 4; }
 
 namespace {
 
@@ -295,7 +312,7 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
           pr.epi = EPI_APPLY_PACK;
           pr.store_out = keep ? 1 : 0;
           // payload word of this (param, worker): resolved at bind from off_bits
-          pr.bits_out = reinterpret_cast<uint32_t*>((size_t)m * c->words_per_worker * 4 + (size_t)pl.word_off * 4);
+          pr.bits_out = reinterpret_cast<uint32_t*>((size_t)m * c->bits_pitch * 4 + (size_t)pl.word_off * 4);
         } else pr.epi = EPI_APPLY;
       }
       out.push_back(pr);
@@ -332,6 +349,7 @@ int plan_layout(signmuon_ctx* c) {
   }
   if (words >= (1ull << 32)) return SIGNMUON_ERR_BAD_SHAPE;
   c->words_per_worker = words;
+  c->bits_pitch = round_up((size_t)words, 32);
   c->state_bytes = state;
 
   // block ranges of the element-wise kernels
@@ -344,7 +362,14 @@ int plan_layout(signmuon_ctx* c) {
   if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
   c->plain_blocks = (uint32_t)b;
   b = 0;
-  for (int32_t p : c->matrix_list) { c->vote_starts.push_back((uint32_t)b); b += (c->plan[p].n_words + VOTE_WORDS - 1) / VOTE_WORDS; }
+  // vote kernel: blocks own VOTE_WORDS-aligned groups of the payload's word index; a parameter gets every group it
+  // touches (a group shared by two parameters is visited once for each, masked)
+  for (int32_t p : c->matrix_list) {
+    const ParamPlan& pl = c->plan[p];
+    c->vote_starts.push_back((uint32_t)b);
+    b += ((uint64_t)pl.word_off + pl.n_words + VOTE_WORDS - 1) / VOTE_WORDS - pl.word_off / VOTE_WORDS;
+  }
+  if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
   c->vote_blocks = (uint32_t)b;
   b = 0;
   for (int32_t p : c->matrix_list) {
@@ -380,7 +405,8 @@ int plan_layout(signmuon_ctx* c) {
   // workspace layout: small tables first, then the large buffers
   size_t off = 0;
   c->off_status = off; off += ALIGN;
-  c->off_paramdev = off; off += round_up(c->params.size() * sizeof(ParamDev), ALIGN);
+  c->paramdev_stride = round_up(c->params.size() * sizeof(ParamDev), ALIGN);
+  c->off_paramdev = off; off += PARAM_TABLES * c->paramdev_stride;
   auto place = [&](size_t& slot, size_t bytes) { slot = off; off += round_up(std::max<size_t>(bytes, 4), ALIGN); };
   place(c->off_list_matrix, c->matrix_list.size() * 4);
   place(c->off_list_plain, c->plain_list.size() * 4);
@@ -402,8 +428,8 @@ int plan_layout(signmuon_ctx* c) {
       pl.pi_scal_off = off; off += round_up((size_t)M * 8, ALIGN);
     }
   }
-  c->off_bits = off; off += round_up((size_t)M * words * 4, ALIGN);
-  c->off_vote = off; off += round_up((size_t)words * 4, ALIGN);
+  c->off_bits = off; off += round_up((size_t)M * c->bits_pitch * 4, ALIGN);
+  c->off_vote = off; off += round_up((size_t)c->bits_pitch * 4, ALIGN);
   // tensor maps
   c->off_tmaps = off;
   int nt = 0;
@@ -476,14 +502,15 @@ int plan_layout(signmuon_ctx* c) {
 }
 
 PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
+  static std::once_flag once;
   static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
-  if (!fn) {
+  std::call_once(once, [] {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
       fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
-  }
+  });
   return fn;
 }
 
@@ -586,12 +613,17 @@ bool configure_kernels(int* max_pairs) {
   return true;
 }
 
+// Device address of the parameter table of the step being enqueued.
+const ParamDev* cur_paramdev(const signmuon_ctx* c) {
+  return reinterpret_cast<const ParamDev*>(c->d_ws + c->off_paramdev + (size_t)c->cur_table * c->paramdev_stride);
+}
+
 void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s) {
   const TileTable& tt = c->tables[lp.tile_table];
   if (tt.tiles.empty()) return;
   const GemmProblem* probs = reinterpret_cast<const GemmProblem*>(c->d_ws + c->off_problems) + lp.problem_base;
   const TileEntry* tiles = reinterpret_cast<const TileEntry*>(c->d_ws + tt.tiles_off);
-  const ParamDev* pd = reinterpret_cast<const ParamDev*>(c->d_ws + c->off_paramdev);
+  const ParamDev* pd = cur_paramdev(c);
   if (c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) {
     ns_gemm_simt_kernel<<<(unsigned)tt.tiles.size(), 128, 0, s>>>(probs, tiles, tt.bn, pd, lr);
     return;
@@ -604,6 +636,7 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
   a.params = pd;
   a.status = reinterpret_cast<uint32_t*>(c->d_ws + c->off_status);
   a.lr = lr;
+  a.wait_limit_ns = c->wait_limit_ns;
   const bool gram = (lp.tile_table & 1) == 0;
   if (tt.ctas == 2) {
     if (gram) launch_tc<NS_GEMM_PAIR_GRAM>(a, tt.grid, s);
@@ -616,35 +649,70 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
 
 template <int PLANES>
 void launch_vote(signmuon_ctx* c, float lr, int write_sbar, cudaStream_t s) {
-  vote_update_kernel<PLANES><<<c->vote_blocks, EW_THREADS, 0, s>>>(
-      reinterpret_cast<const ParamDev*>(c->d_ws + c->off_paramdev),
+  vote_update_kernel<PLANES><<<c->vote_blocks, VOTE_THREADS, 0, s>>>(
+      cur_paramdev(c),
       reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_matrix),
       reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_vote), (int)c->matrix_list.size(),
       c->cfg.num_workers, lr, write_sbar, reinterpret_cast<const uint32_t*>(c->d_ws + c->off_bits),
-      reinterpret_cast<uint32_t*>(c->d_ws + c->off_vote), (int64_t)c->words_per_worker);
+      reinterpret_cast<uint32_t*>(c->d_ws + c->off_vote), (int64_t)c->bits_pitch);
 }
 
+void invalidate_tables(signmuon_ctx* c) {
+  for (int t = 0; t < PARAM_TABLES; ++t) c->table_key[t].clear();
+}
+
+// Selects (or fills) the device-side parameter table that holds this call's weight and gradient pointers.
 int upload_params(signmuon_ctx* c, void* const* weights, const void* const* grads, cudaStream_t s) {
-  bool changed = !c->paramdev_uploaded;
-  for (size_t p = 0; p < c->params.size(); ++p) {
+  const size_t n = c->params.size();
+  for (size_t p = 0; p < n; ++p) {
     if (!weights[p] || !grads[p]) return SIGNMUON_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(weights[p]) & 15) || (reinterpret_cast<uintptr_t>(grads[p]) & 15))
       return SIGNMUON_ERR_MISALIGNED;
-    if (c->paramdev[p].W != weights[p] || c->paramdev[p].G != grads[p]) {
-      c->paramdev[p].W = weights[p];
-      c->paramdev[p].G = grads[p];
-      changed = true;
+  }
+  ++c->table_clock;
+  for (int t = 0; t < PARAM_TABLES; ++t) {
+    const std::vector<const void*>& key = c->table_key[t];
+    if (key.size() != 2 * n) continue;
+    bool same = true;
+    for (size_t p = 0; p < n && same; ++p) same = key[p] == weights[p] && key[n + p] == grads[p];
+    if (same) {
+      c->cur_table = t;
+      c->table_used[t] = c->table_clock;
+      return SIGNMUON_OK;
     }
   }
-  if (changed) {
-    // pageable source: the runtime stages it before returning, so the host copy may change afterwards
-    if (cudaMemcpyAsync(c->d_ws + c->off_paramdev, c->paramdev.data(), c->paramdev.size() * sizeof(ParamDev),
-                        cudaMemcpyHostToDevice, s) != cudaSuccess) {
-      c->sticky = SIGNMUON_ERR_CUDA;
-      return c->sticky;
-    }
-    c->paramdev_uploaded = true;
+  int victim = -1;
+  for (int t = 0; t < PARAM_TABLES && victim < 0; ++t)
+    if (c->table_key[t].empty()) victim = t;
+  if (victim < 0) {
+    victim = 0;
+    for (int t = 1; t < PARAM_TABLES; ++t)
+      if (c->table_used[t] < c->table_used[victim]) victim = t;
   }
+  // miss: the least recently used slot takes this pointer set.  Its pinned mirror may still be the source of
+  // the copy that filled the slot last time (long finished in practice): wait for that copy only.
+  ParamDev* mirror = c->h_tables + (size_t)victim * n;
+  if (cudaEventSynchronize(c->ev_table[victim]) != cudaSuccess) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+  std::vector<const void*>& key = c->table_key[victim];
+  key.resize(2 * n);
+  for (size_t p = 0; p < n; ++p) {
+    mirror[p] = c->paramdev[p];
+    mirror[p].W = weights[p];
+    mirror[p].G = grads[p];
+    key[p] = weights[p];
+    key[n + p] = grads[p];
+  }
+  // Kernels of earlier steps that read this slot were enqueued on the caller's stream before this copy: a
+  // context is used from one stream at a time, so the copy is ordered behind them.
+  if (cudaMemcpyAsync(c->d_ws + c->off_paramdev + (size_t)victim * c->paramdev_stride, mirror, n * sizeof(ParamDev),
+                      cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaEventRecord(c->ev_table[victim], s) != cudaSuccess) {
+    key.clear();
+    c->sticky = SIGNMUON_ERR_CUDA;
+    return c->sticky;
+  }
+  c->cur_table = victim;
+  c->table_used[victim] = c->table_clock;
   return SIGNMUON_OK;
 }
 
@@ -659,7 +727,7 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
   int rc = upload_params(c, weights, grads, s);
   if (rc != SIGNMUON_OK) return rc;
   const int M = c->cfg.num_workers, K = c->cfg.ns_steps;
-  const ParamDev* pd = reinterpret_cast<const ParamDev*>(c->d_ws + c->off_paramdev);
+  const ParamDev* pd = cur_paramdev(c);
   uint32_t* bits = reinterpret_cast<uint32_t*>(c->d_ws + c->off_bits);
   uint32_t* vote = reinterpret_cast<uint32_t*>(c->d_ws + c->off_vote);
   const int nm = (int)c->matrix_list.size(), np = (int)c->plain_list.size();
@@ -693,7 +761,7 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
       plain_params_kernel<<<c->plain_blocks, EW_THREADS, 0, s>>>(
           pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_plain),
           reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_plain), np, M, c->cfg.momentum,
-          c->cfg.weight_decay, lr, bits, vote, (int64_t)c->words_per_worker);
+          c->cfg.weight_decay, lr, bits, vote, (int64_t)c->bits_pitch);
     }
   }
   if ((mask & SIGNMUON_STAGE_NS) && nm) {
@@ -702,7 +770,7 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
       pack_kernel<<<c->packfb_blocks, EW_THREADS, 0, s>>>(
           pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_packfb),
           reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_packfb), (int)c->packfb_list.size(), K & 1,
-          K == 0 ? 1 : 0, bits, (int64_t)c->words_per_worker);
+          K == 0 ? 1 : 0, bits, (int64_t)c->bits_pitch);
     }
   }
   const bool lp_ns = c->cfg.local_polar && K > 0;
@@ -718,7 +786,8 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
     unsigned long long* agree = reinterpret_cast<unsigned long long*>(c->d_ws + c->off_agree);
     if (cudaMemsetAsync(agree, 0, (size_t)M * 8, s) != cudaSuccess) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
     const unsigned gx = (unsigned)std::min<uint64_t>((c->words_per_worker + EW_THREADS - 1) / EW_THREADS, 1024);
-    sign_agreement_kernel<<<dim3(gx, (unsigned)M), EW_THREADS, 0, s>>>(bits, vote, (int64_t)c->words_per_worker, agree);
+    sign_agreement_kernel<<<dim3(gx, (unsigned)M), EW_THREADS, 0, s>>>(bits, vote, (int64_t)c->words_per_worker,
+                                                                             (int64_t)c->bits_pitch, agree);
   }
   if ((mask & SIGNMUON_STAGE_LOCAL_POLAR) && nm && lp_ns) {
     for (const LaunchPlan& lp : c->lp_launches) launch_gemm(c, lp, lr, s);
@@ -750,10 +819,12 @@ int signmuon_create(const signmuon_config* config, signmuon_ctx** out) {
     if (p.kind != SIGNMUON_PARAM_MATRIX && p.kind != SIGNMUON_PARAM_PLAIN) return SIGNMUON_ERR_INVALID_ARG;
     if (!valid_dtype(p.weight_dtype) || !valid_dtype(p.grad_dtype)) return SIGNMUON_ERR_INVALID_ARG;
     if (p.kind == SIGNMUON_PARAM_MATRIX && std::min(p.rows, p.cols) > 65536 * 2) return SIGNMUON_ERR_BAD_SHAPE;
+    // tile coordinates are 16-bit, in units of at least 128 rows or columns
+    if (p.kind == SIGNMUON_PARAM_MATRIX && (std::max(p.rows, p.cols) + 127) / 128 > 65535) return SIGNMUON_ERR_BAD_SHAPE;
     if (p.rows * p.cols > (1ll << 36)) return SIGNMUON_ERR_BAD_SHAPE;
   }
   signmuon_ctx* c = new (std::nothrow) signmuon_ctx();
-  if (!c) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c) return SIGNMUON_ERR_NO_MEMORY;
   c->cfg = *config;
   if (!(c->cfg.eps > 0.f)) c->cfg.eps = 1e-12f;
   c->params.assign(config->params, config->params + config->num_params);
@@ -800,6 +871,19 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
   }
   c->host_steps = 0;
   const int M = c->cfg.num_workers;
+  if (!c->h_tables) {   // pinned host mirrors of the parameter tables and the events that guard their reuse
+    void* hp = nullptr;
+    if (cudaHostAlloc(&hp, PARAM_TABLES * c->params.size() * sizeof(ParamDev), cudaHostAllocDefault) != cudaSuccess) {
+      cudaGetLastError();
+      return SIGNMUON_ERR_NO_MEMORY;
+    }
+    c->h_tables = static_cast<ParamDev*>(hp);
+    for (int t = 0; t < PARAM_TABLES; ++t)
+      if (cudaEventCreateWithFlags(&c->ev_table[t], cudaEventDisableTiming) != cudaSuccess) {
+        c->sticky = SIGNMUON_ERR_CUDA;
+        return c->sticky;
+      }
+  }
 
   // host image of the table area [0, off_tables_end) minus the big buffers: assemble piecewise
   auto up = [&](size_t off, const void* src, size_t bytes) -> bool {
@@ -808,8 +892,8 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
   };
   bool ok = cudaMemsetAsync(c->d_ws + c->off_status, 0, ALIGN, s) == cudaSuccess;
   if (zero_state) ok = ok && cudaMemsetAsync(c->d_state, 0, c->state_bytes, s) == cudaSuccess;
-  ok = ok && cudaMemsetAsync(c->d_ws + c->off_bits, 0, (size_t)M * c->words_per_worker * 4, s) == cudaSuccess;
-  ok = ok && cudaMemsetAsync(c->d_ws + c->off_vote, 0, (size_t)c->words_per_worker * 4, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->d_ws + c->off_bits, 0, (size_t)M * c->bits_pitch * 4, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->d_ws + c->off_vote, 0, (size_t)c->bits_pitch * 4, s) == cudaSuccess;
 
   // parameter table (W/G filled in at the first step)
   c->paramdev.assign(c->params.size(), ParamDev());
@@ -839,7 +923,7 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     d.upd_scale = eq2 ? (float)(1.0 / std::sqrt((double)pl.rows * (double)pl.cols)) : 1.f;
     d.vec_ok = (pl.d % 8 == 0 && pl.ldy == pl.cols) ? 1 : 0;
   }
-  c->paramdev_uploaded = false;
+  invalidate_tables(c);
   ok = ok && up(c->off_list_matrix, c->matrix_list.data(), c->matrix_list.size() * 4);
   ok = ok && up(c->off_list_plain, c->plain_list.data(), c->plain_list.size() * 4);
   ok = ok && up(c->off_list_packfb, c->packfb_list.data(), c->packfb_list.size() * 4);
@@ -865,6 +949,22 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
                      tt.ctas == 2 ? max_pairs : c->num_sms);
     ok = ok && up(tt.tiles_off, tt.tiles.data(), tt.tiles.size() * sizeof(TileEntry));
     ok = ok && up(tt.cta_off, tt.cta_start.data(), tt.cta_start.size() * 4);
+  }
+  // Flops the tensor cores are asked for per step: every scheduled tile issues whole bm x bn x 64 blocks (ragged
+  // edges are zero-filled, skipped mirror tiles of the symmetric Gram products are not issued at all), once per
+  // operand segment; each tile table is launched K times.
+  c->executed_flops = 0;
+  for (int t = 0; t < 4; ++t) {
+    const TileTable& tt = c->tables[t];
+    const std::vector<LaunchPlan>& ls = (t < 2) ? c->ns_launches : c->lp_launches;
+    if (ls.empty()) continue;
+    double f = 0;
+    for (const TileEntry& te : tt.tiles) {
+      const GemmProblem& pr = c->problems[ls[t & 1].problem_base + te.problem];
+      const double kblocks = (double)((pr.K + GEMM_BK - 1) / GEMM_BK) * (pr.nseg > 1 ? pr.nseg : 1);
+      f += 2.0 * tt.bm * tt.bn * GEMM_BK * kblocks;
+    }
+    c->executed_flops += f * c->cfg.ns_steps;
   }
   // (moved up) kernels configured before the tile tables are split
   std::vector<CUtensorMap> maps((size_t)c->num_tmaps);
@@ -992,7 +1092,7 @@ int signmuon_packed_payload(const signmuon_ctx* c, int32_t worker, const uint32_
   if (entries) *entries = (size_t)c->entries;
   if (dev_ptr) {
     if (!c->bound) { *dev_ptr = nullptr; return SIGNMUON_ERR_NOT_BOUND; }
-    *dev_ptr = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_bits) + (size_t)worker * c->words_per_worker;
+    *dev_ptr = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_bits) + (size_t)worker * c->bits_pitch;
   }
   return SIGNMUON_OK;
 }
@@ -1025,7 +1125,7 @@ int signmuon_debug_tap(const signmuon_ctx* c, int32_t what, int32_t param, int32
     case SIGNMUON_TAP_VOTE_BITS:
       ptr = c->d_ws + c->off_vote + (size_t)pl.word_off * 4; nbytes = (size_t)pl.n_words * 4; break;
     case SIGNMUON_TAP_WORKER_BITS:
-      ptr = c->d_ws + c->off_bits + ((size_t)worker * c->words_per_worker + pl.word_off) * 4;
+      ptr = c->d_ws + c->off_bits + ((size_t)worker * c->bits_pitch + pl.word_off) * 4;
       nbytes = (size_t)pl.n_words * 4; break;
     case SIGNMUON_TAP_NORM:
       if (pl.kind != SIGNMUON_PARAM_MATRIX) return SIGNMUON_ERR_INVALID_ARG;
@@ -1052,6 +1152,21 @@ int signmuon_status(signmuon_ctx* c, void* cuda_stream) {
   return word == STATUS_OK ? SIGNMUON_OK : SIGNMUON_ERR_TIMEOUT;
 }
 
+int signmuon_set_wait_limit(signmuon_ctx* c, uint64_t limit_ns) {
+  if (!c) return SIGNMUON_ERR_INVALID_ARG;
+  c->wait_limit_ns = limit_ns ? limit_ns : DEFAULT_WAIT_LIMIT_NS;
+  return SIGNMUON_OK;
+}
+
+int signmuon_selftest_wait_timeout(signmuon_ctx* c, uint64_t limit_ns, void* cuda_stream) {
+  if (!c || limit_ns == 0 || limit_ns > DEFAULT_WAIT_LIMIT_NS) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  if (c->sticky != SIGNMUON_OK) return c->sticky;
+  wait_timeout_probe_kernel<<<1, 32, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
+      reinterpret_cast<uint32_t*>(c->d_ws + c->off_status), limit_ns);
+  return check_launch(c);
+}
+
 int signmuon_power_start_size(const signmuon_ctx* c, size_t* floats) {
   if (!c || !floats) return SIGNMUON_ERR_INVALID_ARG;
   *floats = c->power_start_floats;
@@ -1076,7 +1191,7 @@ int signmuon_set_power_start(signmuon_ctx* c, const float* dev_vectors, size_t f
   if (c->d_power_start != dev_vectors) {
     c->d_power_start = dev_vectors;
     for (int32_t p : c->matrix_list) c->paramdev[p].pi_start = dev_vectors + c->plan[p].pi_start_off;
-    c->paramdev_uploaded = false;     // the table goes to the device again with the next step
+    invalidate_tables(c);             // every cached table goes to the device again when it is next used
   }
   return SIGNMUON_OK;
 }
@@ -1124,6 +1239,13 @@ int signmuon_ns_flops_per_step(const signmuon_ctx* c, double* flops) {
   return SIGNMUON_OK;
 }
 
+int signmuon_ns_executed_flops_per_step(const signmuon_ctx* c, double* flops) {
+  if (!c || !flops) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  *flops = c->executed_flops;
+  return SIGNMUON_OK;
+}
+
 void signmuon_destroy(signmuon_ctx* c) {
   if (!c) return;
   if (c->copy_stream) {
@@ -1134,6 +1256,9 @@ void signmuon_destroy(signmuon_ctx* c) {
     }
     cudaStreamDestroy(c->copy_stream);
   }
+  for (int t = 0; t < PARAM_TABLES; ++t)
+    if (c->ev_table[t]) { cudaEventSynchronize(c->ev_table[t]); cudaEventDestroy(c->ev_table[t]); }
+  if (c->h_tables) cudaFreeHost(c->h_tables);
   delete c;
 }
 
@@ -1149,6 +1274,7 @@ const char* signmuon_error_string(int code) {
     case SIGNMUON_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
     case SIGNMUON_ERR_MISALIGNED: return "device pointer is not sufficiently aligned";
     case SIGNMUON_ERR_TOO_LARGE: return "problem exceeds the fixed capacity of this entry point";
+    case SIGNMUON_ERR_NO_MEMORY: return "host memory allocation failed";
     default: return "unknown error";
   }
 }

@@ -39,10 +39,13 @@ def _np64(t: torch.Tensor) -> np.ndarray:
 def check_param_step(opt: B.SignMuon, wl, p_idx: int, w_before: torch.Tensor, w_after: torch.Tensor,
                      grads: torch.Tensor, mom_before: Optional[np.ndarray], lr: float, weight_decay: float = 0.0,
                      check_polar: bool = True, report: Optional[dict] = None, power_start=None, power_iters: int = 2,
-                     ns_workers: Optional[Sequence[int]] = None):
+                     ns_workers: Optional[Sequence[int]] = None, have_polar: bool = True):
     """Checks every stage of parameter p_idx for the step just run. Returns the oracle momentum
     (float64, [M, r, c]) evolved from `mom_before` (None = zeros).  `ns_workers` restricts the Newton-Schulz
-    comparison (the costly part of the oracle) to those workers; every other stage covers all workers."""
+    comparison (the costly part of the oracle) to those workers; every other stage covers all workers.
+    `have_polar` = False: the context was created without FLAG_KEEP_POLAR (the configuration a caller and the
+    benchmark run), so Y_K of a parameter whose sign bits are packed in the last epilogue is never stored: its
+    value comparison is skipped, the sign-bit comparison with the oracle stays."""
     p = wl.params[p_idx]
     M, r, c, d = wl.num_workers, p.rows, p.cols, p.rows * p.cols
     K = wl.ns_steps
@@ -87,7 +90,7 @@ def check_param_step(opt: B.SignMuon, wl, p_idx: int, w_before: torch.Tensor, w_
                 continue
             u_or = O.polar_ns_short_side(mom_gpu[m], K, 1e-12, sigma_arg)
             rms = math.sqrt(float(np.mean(u_or ** 2)))
-            if K > 0:
+            if K > 0 and (have_polar or c % 32 != 0):      # rows that do not hold whole words keep Y_K for the pack kernel
                 u_gpu = _np64(opt.tap(B.TAP_POLAR, p_idx, m))
                 rel = np.linalg.norm(u_gpu - u_or) / np.linalg.norm(u_or)
                 rep["polar_relfro"] = max(rep.get("polar_relfro", 0.0), float(rel))
@@ -159,9 +162,10 @@ def check_param_step(opt: B.SignMuon, wl, p_idx: int, w_before: torch.Tensor, w_
 
 def run_and_check(wl, steps: int, flags: int = B.FLAG_KEEP_POLAR, sample: Optional[Sequence[int]] = None,
                   device: str = "cuda:0", check_polar: bool = True, report: Optional[dict] = None,
-                  ns_workers: Optional[Sequence[int]] = None):
+                  ns_workers: Optional[Sequence[int]] = None, capture: Optional[dict] = None):
     """Runs `steps` optimizer steps of workload `wl` on the GPU and checks the sampled parameters
-    (default: all) against the oracle after every step."""
+    (default: all) against the oracle after every step.  `capture` (a dict) receives the payload of every
+    worker after every step and the final weights, for bit-level comparisons between two runs."""
     opt = make_optimizer(wl, flags=flags)
     weights = wlmod.make_weights(wl, device)
     signal = wlmod.make_signal(wl, device)
@@ -191,7 +195,12 @@ def run_and_check(wl, steps: int, flags: int = B.FLAG_KEEP_POLAR, sample: Option
             mom_or[p] = check_param_step(opt, wl, p, before[p], weights[p], grads[p], mom_or[p], wl.lr,
                                          check_polar=check_polar, report=rep,
                                          power_start=None if starts is None else starts[p],
-                                         power_iters=wl.extra.get("power_iters", 2), ns_workers=ns_workers)
+                                         power_iters=wl.extra.get("power_iters", 2), ns_workers=ns_workers,
+                                         have_polar=bool(flags & B.FLAG_KEEP_POLAR))
             mom_or[p] = np.stack([_np64(opt.tap(B.TAP_MOMENTUM, p, m)) for m in range(wl.num_workers)])
+        if capture is not None:
+            capture.setdefault("payloads", []).append([opt.payload(m).clone() for m in range(wl.num_workers)])
+    if capture is not None:
+        capture["weights"] = [w.clone() for w in weights]
     opt.close()
     return rep

@@ -53,10 +53,27 @@ def test_reference_arm_prints_one_json_line():
     import json
     import subprocess
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
-                          "--warmup", "0", "--oracle-flops", "2e9"], check=True, capture_output=True, text=True).stdout
+                          "--warmup", "0", "--workload", "c2", "--oracle-flops", "2e9"], check=True, capture_output=True, text=True).stdout
     lines = [l for l in out.splitlines() if l.strip()]
     assert len(lines) == 1
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["metric"] == "signmuon_optimizer_steps_per_sec" and d["value"] > 0
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["config"]["workload"] == "c2_resnet50"
+    assert d["cpu_baseline"]["extrapolated"] is True
+
+
+def test_reference_arm_and_cpu_baseline_share_one_sample_plan():
+    """Both oracle timings of bench.py draw their sample from the same plan: one parameter per distinct shape
+    inside the operation budget, at least one matrix, so their extrapolations agree by construction."""
+    import bench
+    from paper_2605_16311_b200 import workloads as wlmod
+    c4 = wlmod.config4()
+    idx, c_sample, c_total = bench.oracle_sample_plan(c4, 3.0e12)
+    assert idx == [0]                                           # one 4096 x 4096 matrix
+    assert c_total / c_sample > 30                              # 8 workers x 6 matrices against one worker of one
+    c2 = wlmod.config2()
+    idx2, s2, t2 = bench.oracle_sample_plan(c2, 3.0e12)
+    assert len(idx2) == len({(p.rows, p.cols) for p in c2.params})   # every distinct ResNet-50 shape fits
+    assert bench.shard_workers(8, 4, 3) == (6, 2) and bench.shard_workers(8, 3, 0) is None
+    assert bench.whole_job_value(4.0, 2, sharded=True) == 250.0

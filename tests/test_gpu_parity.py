@@ -178,6 +178,44 @@ def test_llama_layer_without_local_polar_and_sweep_extremes():
     print(rep, rep2, rep3)
 
 
+def _same_bits_and_weights(a: dict, b: dict):
+    for pa, pb in zip(a["payloads"], b["payloads"]):
+        for x, y in zip(pa, pb):
+            assert torch.equal(x, y)
+    for x, y in zip(a["weights"], b["weights"]):
+        assert torch.equal(x, y)
+
+
+def test_default_flags_path_against_oracle():
+    """The configuration a caller (and the benchmark) runs: no FLAG_KEEP_POLAR, so the last apply epilogue
+    writes payload words only and Y_K never reaches memory.  Worker sign bits against the oracle's PolarNS of
+    the GPU's own momentum (>= 99.9 %, mismatches confined to |oracle| < 1e-3 RMS), vote and update from the
+    GPU's own payload, and payload words + weights bit-identical to a run that also stores Y_K."""
+    from parity_utils import run_and_check
+    cases = [(wlmod.config1(), 3, None),
+             (_wl([(200, 328), (328, 200), (64, 147), (130, 64), (96, 96), (1, 160), (300, 1)], 3), 2, None),
+             (_wl([(256, 768), (768, 256), (1, 768)], 4, dtype="bf16", local_polar=True, lr=0.01,
+                  kinds=["matrix", "matrix", "plain"]), 2, None)]
+    c2 = wlmod.config2()
+    names = [p.name for p in c2.params]
+    cases.append((c2, 2, [0, 1, names.index("s0b0.conv3"), names.index("s1b0.conv2"), names.index("s2b0.down"),
+                          names.index("s3b2.conv2"), names.index("fc")]))
+    for wl, steps, sample in cases:
+        plain, kept = {}, {}
+        rep = run_and_check(wl, steps=steps, flags=0, sample=sample, capture=plain)
+        assert rep["sign_match_min"] >= 0.999
+        run_and_check(wl, steps=steps, flags=B.FLAG_KEEP_POLAR, sample=sample, capture=kept, check_polar=False)
+        _same_bits_and_weights(plain, kept)
+
+
+def test_default_flags_path_full_llama_layer_sampled():
+    """Config 4 at full size in the benchmark's launch configuration (flags = 0, local polar on)."""
+    from parity_utils import run_and_check
+    rep = run_and_check(wlmod.config4(), steps=1, flags=0, sample=[0, 4], ns_workers=[5])
+    assert rep["sign_match_min"] >= 0.999
+    print(rep)
+
+
 def test_weight_decay_and_step_lr_override():
     from parity_utils import check_param_step, make_optimizer
     import numpy as np
@@ -216,6 +254,59 @@ def test_stage_calls_equal_one_step_and_determinism():
         for a, b in zip(outs[0][0], other[0]):
             assert torch.equal(a, b)                       # bit-identical weights
         assert torch.equal(outs[0][1], other[1]) and torch.equal(outs[0][2], other[2])
+
+
+def test_bounded_wait_runs_out_and_the_context_recovers():
+    """Failure detection without a fault: a one-thread kernel performs the Newton-Schulz kernels' bounded wait on
+    a barrier that nothing signals, with a 1 ms limit.  The kernel returns, the status word reports the timeout,
+    a new bind clears it, and the context then steps exactly like a fresh one."""
+    wl = _wl([(256, 320), (64, 147)], 3, local_polar=True, lr=0.01)
+    sig = wlmod.make_signal(wl, "cuda:0")
+    g = wlmod.make_grads(wl, sig, 0, "cuda:0")
+    opt = B.SignMuon(wl.params, 3, lr=0.01, local_polar=True)
+    assert opt.status() == B.OK
+    opt.selftest_wait_timeout(1_000_000)
+    assert opt.status() == B.ERR_TIMEOUT
+    assert opt.status() == B.ERR_TIMEOUT          # stays until the next bind
+    with pytest.raises(B.SignMuonError):
+        opt.selftest_wait_timeout(0)              # a limit is mandatory
+    opt.rebind()
+    assert opt.status() == B.OK
+    opt.set_wait_limit(500_000_000)               # a shorter (still generous) limit for the real kernels
+    w = wlmod.make_weights(wl, "cuda:0")
+    opt.step(w, g)
+    assert opt.status() == B.OK
+    fresh = B.SignMuon(wl.params, 3, lr=0.01, local_polar=True)
+    w2 = wlmod.make_weights(wl, "cuda:0")
+    fresh.step(w2, g)
+    assert fresh.status() == B.OK
+    for a, b in zip(w, w2):
+        assert torch.equal(a, b)
+    assert torch.equal(opt.payload(1), fresh.payload(1))
+    opt.close(); fresh.close()
+
+
+def test_pointer_table_cache_with_more_buffer_sets_than_slots():
+    """Six gradient buffer sets used in rotation (the device keeps four pointer tables) against one context
+    that always sees the same buffers: identical weights and payloads after every step."""
+    wl = _wl([(128, 256), (64, 147), (1, 40)], 3, kinds=["matrix", "matrix", "plain"])
+    sig = wlmod.make_signal(wl, "cuda:0")
+    sets = [wlmod.make_grads(wl, sig, t, "cuda:0") for t in range(6)]
+    fixed = [torch.empty_like(x) for x in sets[0]]
+    a, b = B.SignMuon(wl.params, 3), B.SignMuon(wl.params, 3)
+    wa, wb = wlmod.make_weights(wl, "cuda:0"), wlmod.make_weights(wl, "cuda:0")
+    for t in range(14):
+        gs = sets[(t * 5) % 6] if t % 3 else sets[t % 6]
+        a.step(wa, gs)
+        for dst, src in zip(fixed, gs):
+            dst.copy_(src)
+        b.step(wb, fixed)
+        torch.cuda.synchronize()
+        for x, y in zip(wa, wb):
+            assert torch.equal(x, y)
+        assert torch.equal(a.payload(2), b.payload(2))
+    assert a.status() == B.OK and b.status() == B.OK
+    a.close(); b.close()
 
 
 def test_garbage_worker_is_outvoted():

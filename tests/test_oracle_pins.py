@@ -293,6 +293,31 @@ def test_step_update_is_plus_minus_eta_and_plain_kind():
             assert np.array_equal(tr[0].bits, (tr[0].mom.reshape(3, -1) >= 0).astype(np.uint8))
 
 
+def test_step_hands_weight_decay_to_the_momentum():
+    """Alg. 2 "Apply weight decay" at step level: beta = 0 and a constant gradient give Mom = G + lambda W,
+    worked by hand on a 2 x 2 plain parameter (so that no Newton-Schulz intervenes):
+        W = [[1, -2], [4, 0.5]], G = [[0.5, 0.1], [-1.5, -0.1]], lambda = 0.25
+        Mom = [[0.75, -0.4], [-0.5, 0.025]]  -> bits [[1, 0], [0, 1]]  -> W' = W - 0.5 * [[+1, -1], [-1, +1]].
+    Without the decay term the signs of the entries (1,0) and (1,1) would flip."""
+    spec = O.ParamSpec(2, 2, "plain")
+    cfg = O.OracleConfig(num_workers=2, momentum=0.0, lr=0.5, ns_steps=0, weight_decay=0.25)
+    st = O.init_state([spec], cfg)
+    w = np.array([[1.0, -2.0], [4.0, 0.5]])
+    g = np.array([[0.5, 0.1], [-1.5, -0.1]])
+    new_w, tr = O.step([spec], cfg, st, [w], [np.stack([g, g])])
+    assert np.allclose(tr[0].mom[0], np.array([[0.75, -0.4], [-0.5, 0.025]]), rtol=1e-15, atol=1e-17)
+    assert np.array_equal(tr[0].mom[1], tr[0].mom[0]) and np.array_equal(st.mom[0], tr[0].mom)
+    assert tr[0].vote_bits.tolist() == [1, 0, 0, 1]
+    assert np.array_equal(new_w[0], np.array([[0.5, -1.5], [4.5, 0.0]]))
+    # matrix kind, K = 3: the decayed momentum is what enters PolarNS
+    spec_m = O.ParamSpec(2, 2, "matrix")
+    cfg_m = O.OracleConfig(num_workers=1, momentum=0.0, lr=0.5, ns_steps=3, weight_decay=0.25)
+    _, tr_m = O.step([spec_m], cfg_m, O.init_state([spec_m], cfg_m), [w], [g[None]])
+    u, sv, vt = np.linalg.svd(np.array([[0.75, -0.4], [-0.5, 0.025]]))
+    expect = (u * f_scalar(sv / math.sqrt(np.sum(sv ** 2)), 3)) @ vt
+    assert np.allclose(tr_m[0].polar[0], expect, rtol=1e-12, atol=1e-15)
+
+
 def test_step_matrix_sign_is_scale_invariant_and_eq2_scale():
     spec = O.ParamSpec(6, 4, "matrix")
     w = RNG.normal(size=(6, 4))

@@ -6,10 +6,13 @@ allocator lock); it keeps its reduction scratch in a fixed array inside the libr
 that pytest collects it last: a run that stops at the first failure has then already run everything else.
 The test drives two calls in a row through the C ABI - the second one reuses the built-in scratch that the
 first left behind - and compares momentum, bf16 operand and norm factors with what signmuon_run_stages
-produces for the same inputs.
+produces for the same inputs, and with the float64 oracle's momentum recursion and Frobenius norm.
 """
+import numpy as np
 import pytest
 import torch
+
+import oracle as O
 
 from paper_2605_16311_b200 import binding as B
 from paper_2605_16311_b200 import workloads as wlmod
@@ -46,6 +49,8 @@ def test_noalloc_matches_regular_momentum_stage_twice(dtype, rows, cols, M, wd):
     operand = torch.empty(M, d, dtype=torch.bfloat16, device=dev)
     scales = torch.empty(M, 2, dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream().cuda_stream
+    w64 = weights[0].float().cpu().numpy().astype(np.float64)
+    mom_or = np.zeros((M, rows, cols))                                 # the oracle's momentum, evolved alongside
     for step in range(2):                                              # two calls in a row, shared scratch
         grads = wlmod.make_grads(wl, signal, step, dev)
         opt.step(weights, grads, stages=B.STAGE_MOMENTUM)
@@ -62,4 +67,16 @@ def test_noalloc_matches_regular_momentum_stage_twice(dtype, rows, cols, M, wd):
             assert (operand[m].float() - ref_op).abs().max() <= 2e-6 * ref_op.abs().max() + 2 ** -8 * 2e-6
             ref_sc = opt.tap(B.TAP_NORM, 0, m)
             assert torch.allclose(scales[m], ref_sc, rtol=1e-5, atol=0)
+        # against the oracle (Alg. 2 momentum, Alg. 4 sigma = ||Mom||_F): the tolerances of the staged parity tests
+        g64 = grads[0].float().cpu().numpy().astype(np.float64)
+        mom_gpu = mom.cpu().numpy().astype(np.float64).reshape(M, rows, cols)
+        for m in range(M):
+            mom_or[m] = O.momentum_update(mom_or[m], g64[m], w64, 0.9, wd)
+            assert np.max(np.abs(mom_gpu[m] - mom_or[m])) <= 2e-6 * np.max(np.abs(mom_or[m]))
+            sigma = max(O.frobenius_norm(mom_gpu[m]), 1e-12)
+            sc = scales[m].cpu().numpy().astype(np.float64)
+            assert abs(sc[1] * sigma - 1.0) <= 1e-5 and abs(sc[0] * sigma * sigma - 1.0) <= 2e-5
+            assert np.array_equal(operand[m].float().cpu().numpy().reshape(rows, cols),
+                                  O.round_to_bf16(mom_gpu[m]))          # the operand is the rounded momentum
+        mom_or = mom_gpu.copy()                                         # staged: continue from the GPU's state
     opt.close()
