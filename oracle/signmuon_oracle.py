@@ -19,7 +19,8 @@ Pins (tests/test_oracle_pins.py): SVD closed form of the K-step map, the
 polar-factor error bound of the Newton-Schulz theorem, literal-vs-short-side
 equality, brute-force vote counting, int8-sum vs popcount vote, the packed size
 s1 = ceil(d/8) and the 32x ratio, the ResNet-50 worked example of App. B, and
-the closed form of the momentum recursion; for PowerIter: rank-one matrices
+the closed form of the momentum recursion; the Muon comparison step against the SVD form of its
+direction and the exact polar factor in the converged band; for PowerIter: rank-one matrices
 (exact after one round), the diagonal closed form, the sigma_max lower bound and
 its limit against numpy's SVD, P = 0.  The end-to-end multi-step weight
 trajectory has no printed example in the paper: beyond the per-stage pins it is
@@ -40,7 +41,7 @@ __all__ = [
     "pack_bits", "unpack_bits", "bytes_to_words", "words_to_bytes",
     "majority_vote_sum", "majority_vote_popcount", "local_polar",
     "apply_update", "payload_bytes", "round_to_bf16", "init_state", "step",
-    "step_param", "StepTrace",
+    "step_param", "StepTrace", "muon_step_param",
 ]
 
 
@@ -347,6 +348,29 @@ def step_param(spec: ParamSpec, cfg: OracleConfig, mom, weight, grads, lr=None,
     new_weight = apply_update(weight64, direction, lr)
     return StepTrace(mom=new_mom, polar=polar, bits=bits, vote_bits=vote_bits,
                      direction=direction, new_weight=new_weight)
+
+
+def muon_step_param(spec: ParamSpec, cfg: OracleConfig, mom, weight, grads, lr=None, short_side=False):
+    """Full-precision Muon, the comparison optimizer of Sec. 5.1: Alg. 1 without the sign line.
+
+    Data-parallel form with float gradient averaging (the float32 all-reduce that App. B compares against):
+        G = mean_m G^(m);  G~ = G + lambda W;  Mom <- beta Mom + (1 - beta) G~      (one momentum, [r, c])
+        U = PolarNS(Mom; K, eps, fro);  W <- W - eta U
+    Returns (new momentum, U, new weight), all float64.  Plain ("vector-like") parameters have no polar factor:
+    they keep the sign update of step_param and are not handled here.
+    """
+    if spec.kind != "matrix":
+        raise ValueError("muon_step_param handles matrix parameters only")
+    lr = cfg.lr if lr is None else lr
+    r, c = spec.rows, spec.cols
+    weight64 = np.asarray(weight, dtype=np.float64).reshape(r, c)
+    grads = np.asarray(grads, dtype=np.float64).reshape(cfg.num_workers, r, c)
+    g_mean = grads.sum(axis=0) / cfg.num_workers
+    new_mom = momentum_update(np.asarray(mom, dtype=np.float64).reshape(r, c), g_mean, weight64, cfg.momentum,
+                              cfg.weight_decay)
+    ns = polar_ns_short_side if short_side else polar_ns
+    u = ns(new_mom, cfg.ns_steps, cfg.eps)
+    return new_mom, u, apply_update(weight64, u, lr)
 
 
 def step(params: Sequence[ParamSpec], cfg: OracleConfig, state: OracleState, weights, grads,

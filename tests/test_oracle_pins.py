@@ -354,6 +354,42 @@ def test_step_local_polar_direction():
     assert np.allclose(tr2.direction, -expect_d, rtol=1e-10, atol=1e-13)
 
 
+def test_muon_step_direction_is_the_svd_form_of_the_mean_gradient():
+    """Full-precision Muon (Sec. 5.1's comparison optimizer; Alg. 1 without the sign): with beta = 0 the direction is
+    PolarNS of the workers' mean gradient, whose K-step closed form comes from a float64 SVD; with singular values in
+    the band where the iteration has converged it is the polar factor U V^T itself."""
+    rng = np.random.default_rng(7)
+    spec = O.ParamSpec(6, 9, "matrix")
+    cfg = O.OracleConfig(num_workers=3, momentum=0.0, lr=0.25, ns_steps=4)
+    w = rng.normal(size=(6, 9))
+    g = rng.normal(size=(3, 6, 9))
+    mom, u, new_w = O.muon_step_param(spec, cfg, np.zeros((6, 9)), w, g)
+    mean = (g[0] + g[1] + g[2]) / 3.0
+    assert np.allclose(mom, mean, rtol=1e-15, atol=1e-17)
+    uu, sv, vt = np.linalg.svd(mean, full_matrices=False)
+    expect = (uu * f_scalar(sv / math.sqrt(np.sum(sv ** 2)), 4)) @ vt
+    assert np.allclose(u, expect, rtol=1e-10, atol=1e-13)
+    assert np.allclose(new_w, w - 0.25 * expect, rtol=1e-12, atol=1e-15)
+    # momentum carried over: second step from the returned momentum, beta = 0.9, weight decay coupled
+    cfg2 = O.OracleConfig(num_workers=3, momentum=0.9, lr=0.25, ns_steps=0, weight_decay=0.5)
+    mom2, u2, _ = O.muon_step_param(spec, cfg2, mom, w, g)
+    assert np.allclose(mom2, 0.9 * mean + 0.1 * (mean + 0.5 * w), rtol=1e-14)
+    assert np.allclose(u2, mom2 / np.linalg.norm(mom2), rtol=1e-14)          # K = 0: the normalised momentum
+    # converged band: a rank-2 gradient with singular values (0.8, 0.6) of the normalised matrix -> U V^T
+    q1, _ = np.linalg.qr(rng.normal(size=(7, 2)))
+    q2, _ = np.linalg.qr(rng.normal(size=(5, 2)))
+    x = 3.0 * (q1 * np.array([0.8, 0.6])) @ q2.T
+    cfg3 = O.OracleConfig(num_workers=1, momentum=0.0, lr=1.0, ns_steps=8)
+    _, u3, w3 = O.muon_step_param(O.ParamSpec(7, 5, "matrix"), cfg3, np.zeros((7, 5)), np.zeros((7, 5)), x[None])
+    assert np.linalg.norm(u3 - q1 @ q2.T, 2) <= 0.64 ** (2 ** 8) + 1e-12
+    assert np.allclose(w3, -(q1 @ q2.T), atol=1e-10)
+    # short-side route gives the same step; a plain parameter is refused
+    _, u_s, _ = O.muon_step_param(spec, cfg, np.zeros((6, 9)), w, g, short_side=True)
+    assert np.allclose(u_s, u, rtol=1e-10, atol=1e-13)
+    with pytest.raises(ValueError):
+        O.muon_step_param(O.ParamSpec(1, 9, "plain"), cfg, np.zeros((1, 9)), w[:1], g[:, :1])
+
+
 # --------------------------------------------------------------------------- #
 # Alg. 5 (PowerIter) and Alg. 4 with scale = spectral
 # --------------------------------------------------------------------------- #
