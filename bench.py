@@ -350,6 +350,8 @@ def measure(wl, args, dev, dist, rank, world, local_rank, steps, warmup, with_e2
     from paper_2605_16311_b200 import workloads as wlmod
 
     shard = shard_workers(wl.num_workers, world, rank)
+    if shard is None and args.exercise_exchange and dist is not None:
+        shard = (0, wl.num_workers)                      # one rank owning every worker: the exchange path, degenerate
     sharded = shard is not None
     kw = {}
     if sharded:
@@ -475,8 +477,13 @@ def run_ours(args, wl):
     if rank == 0:
         build_mod.build()
     dist = None
-    if world > 1:
+    if world > 1 or args.exercise_exchange:
         import torch.distributed as dist
+        if world == 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29517")
+            os.environ.setdefault("RANK", "0")
+            os.environ.setdefault("WORLD_SIZE", "1")
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
         dist.barrier()
     torch.cuda.set_device(local_rank)
@@ -608,6 +615,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-secondary", action="store_true", help="skip the secondary workloads (c2, c3)")
+    ap.add_argument("--exercise-exchange", action="store_true",
+                    help="with one GPU: run the sharded step (stages + NCCL all-gather of the payload) on a one-rank group")
     ap.add_argument("--oracle-flops", type=float, default=3.0e12,
                     help="float64 operation budget of one oracle sample step (reference arm and cpu_baseline leg)")
     ap.add_argument("--cpu-baseline-seconds", type=float, default=10.0,

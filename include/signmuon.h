@@ -80,7 +80,7 @@ typedef struct {
 typedef struct {
   int32_t num_params;
   const signmuon_param* params; /* HOST, copied by signmuon_create */
-  int32_t num_workers;          /* M >= 1 (at most 255) */
+  int32_t num_workers;          /* M >= 1 (at most 255): the workers that vote */
   float momentum;               /* beta in [0, 1)                       (Alg. 1 input) */
   float lr;                     /* eta; signmuon_step may override it per call */
   int32_t ns_steps;             /* K >= 0; K = 0 gives the sign of the momentum */
@@ -93,7 +93,25 @@ typedef struct {
                                    SIGNMUON_SCALE_SPECTRAL (sigma = PowerIter(Mom, power_iters, eps), Alg. 5).  The
                                    local polar step always uses ||S||_F = sqrt(rows cols). */
   int32_t power_iters;          /* P of Alg. 5, 0..64 (the paper's experiments use 2); ignored for SCALE_FRO */
+  /* Worker sharding (Alg. 2 / Alg. 3 with the workers spread over several GPUs).  local_workers == 0: this
+   * context computes all num_workers workers (one GPU simulates them all).  local_workers > 0: it computes
+   * workers [worker_offset, worker_offset + local_workers) only - state, gradients and Newton-Schulz buffers
+   * cover those workers, gradients arrive as [local_workers][rows][cols] - while the payload buffer still has
+   * one row per worker of the job; the rows of the other workers are filled by the exchange (all-gather of the
+   * packed words, Alg. 3) before the vote stage. */
+  int32_t worker_offset;
+  int32_t local_workers;
+  int32_t update_rule;          /* SIGNMUON_RULE_* */
 } signmuon_config;
+
+/* Update rules.  SIGNMUON: Alg. 2 / Alg. 3.  MUON: the full-precision comparison optimizer of Sec. 5.1 on the same
+ * kernels - Alg. 1 without the sign line, data-parallel with float gradient averaging: matrix parameters keep ONE
+ * momentum of the workers' mean gradient (state [1][d]), U = PolarNS(Mom), W <- W - eta U; nothing is packed or voted
+ * for them and local_polar is ignored.  Plain parameters keep the majority-vote sign update (which is also what a
+ * majority-vote SignAdam would apply: the sign of Adam's direction is the sign of its first moment).  MUON cannot
+ * be combined with worker sharding (average the gradients across GPUs first and pass num_workers = 1) and needs
+ * ns_steps >= 1 (the update is applied by the last Newton-Schulz epilogue). */
+enum { SIGNMUON_RULE_SIGNMUON = 0, SIGNMUON_RULE_MUON = 1 };
 
 enum { SIGNMUON_SCALE_FRO = 0, SIGNMUON_SCALE_SPECTRAL = 1 };
 
@@ -154,6 +172,9 @@ int signmuon_bind(signmuon_ctx* ctx, void* dev_state, size_t state_bytes, void* 
  *   lr:      eta_t for this step; a negative value selects config.lr
  * The device keeps the pointer tables of the last four distinct (weights, grads) pointer sets: a call with a
  * set seen before uploads nothing; a new set costs one small asynchronous copy from pinned memory.
+ * A context that computes only a subset of the workers (config.local_workers) cannot run the step in one call:
+ * the payload exchange sits between the stages; signmuon_step then returns INVALID_ARG - use
+ * signmuon_run_stages(MOMENTUM | NS), exchange, signmuon_run_stages(VOTE | LOCAL_POLAR) or signmuon_vote_update.
  * Errors: NOT_BOUND, INVALID_ARG, MISALIGNED, CUDA (sticky launch error). */
 int signmuon_step(signmuon_ctx* ctx, void* const* weights, const void* const* grads, float lr,
                   void* cuda_stream);
@@ -182,6 +203,57 @@ int signmuon_step_host(signmuon_ctx* ctx, void* const* host_weights, const void*
  * number of sign entries it carries.  May be called before bind with dev_ptr == NULL to get sizes. */
 int signmuon_packed_payload(const signmuon_ctx* ctx, int32_t worker, const uint32_t** dev_ptr,
                             size_t* bytes, size_t* entries);
+
+/* The gathered payload buffer (Alg. 3: "all-gather of B^(m)", App. B "Majority vote from gathered bits"): DEVICE
+ * pointer to row 0, the distance between two workers' rows in bytes (a multiple of 128) and the number of rows
+ * (num_workers).  Row m holds worker m's payload (signmuon_packed_payload(m)).  A context that computes a subset of
+ * the workers writes its own rows in the Newton-Schulz stage; an exchange may write the other rows directly here
+ * (e.g. an in-place all-gather when every rank owns the same number of consecutive workers) before the vote stage
+ * runs.  Valid from signmuon_bind on; dev_ptr may be NULL to query the sizes only. */
+int signmuon_payload_buffer(const signmuon_ctx* ctx, uint32_t** dev_ptr, size_t* row_pitch_bytes, int32_t* rows);
+
+/* Majority vote, optional local polar step and weight update from gathered payloads (Alg. 3 after the all-gather;
+ * Eq. 1): `payloads` is a HOST array of num_workers DEVICE pointers; entry m is worker m's packed payload
+ * (signmuon_packed_payload's size and format), or NULL to use what row m of the payload buffer already holds (the
+ * context's own workers, or rows an exchange wrote in place).  Non-NULL entries are copied into the payload buffer
+ * on `cuda_stream` first.  Then runs the VOTE and LOCAL_POLAR stages: identical results on every GPU that
+ * holds the same payloads and weights.  `grads` is not read by these stages and may repeat the pointers of the
+ * preceding signmuon_run_stages call (it only selects the pointer table).
+ * Errors: as signmuon_run_stages. */
+int signmuon_vote_update(signmuon_ctx* ctx, const uint32_t* const* payloads, void* const* weights,
+                         const void* const* grads, float lr, void* cuda_stream);
+
+/* The exchange fused into the pack (Alg. 3's all-gather without a separate collective): after this call every
+ * payload word this context packs - in the last Newton-Schulz epilogue, in the stand-alone pack kernel and in the
+ * plain-parameter kernel - is stored not only into its own payload buffer but also, at the same offset, into the
+ * payload buffer of every peer (plain stores into peer-mapped memory: NVLink peer access, CUDA IPC or any mapping
+ * that makes the peer's buffer addressable from this GPU).  The stage that packs ends with a small kernel that
+ * publishes the step's sequence number into slot `my_rank` of every peer's flag array; the vote stage starts with
+ * a kernel that waits (bounded by the wait limit; TIMEOUT in the status word when it runs out) until every other
+ * rank's slot of this context's own flag array has reached it.  All ranks must call the stages in lockstep.
+ *   my_rank, num_ranks     this context's rank and the number of ranks (<= 64)
+ *   num_peers (<= 7)       how many other ranks receive this context's words (0 detaches)
+ *   peer_payload_buffers   HOST array of num_peers DEVICE pointers: row 0 of each peer's signmuon_payload_buffer
+ *   peer_flags             HOST array of num_peers DEVICE pointers: each peer's signmuon_exchange_flags
+ * Call after signmuon_bind (a new bind detaches the peers and zeroes the flags).
+ * Errors: INVALID_ARG, NOT_BOUND, MISALIGNED. */
+int signmuon_exchange_flags(const signmuon_ctx* ctx, uint32_t** dev_ptr);
+int signmuon_set_payload_peers(signmuon_ctx* ctx, int32_t my_rank, int32_t num_ranks, int32_t num_peers,
+                               uint32_t* const* peer_payload_buffers, uint32_t* const* peer_flags);
+
+/* The int8 SUM variant of the exchange (Alg. 2: "sum_signs <- sum_m S^(m)", all-reduce with SUM, then
+ * "S <- sign(sum_signs)", ties -> +1).
+ *   signmuon_local_sign_sum: writes, for every bit position of a payload (32 per word, pad positions included),
+ *     the sum of the +-1 signs of this context's own workers as one int8: DEVICE [32 * payload words] bytes,
+ *     16-byte aligned - the buffer a SUM all-reduce over the GPUs then turns into sum_signs.  num_workers must
+ *     not exceed 127.
+ *   signmuon_vote_update_from_sums: takes the reduced sums, forms the vote (sum >= 0 -> +1) and runs the local
+ *     polar step and the weight update like signmuon_vote_update.  The result is bit-identical to voting over
+ *     the gathered payloads (App. B: sign(2 c - M)).
+ * Errors: INVALID_ARG, NOT_BOUND, BUFFER_TOO_SMALL, MISALIGNED, CUDA. */
+int signmuon_local_sign_sum(signmuon_ctx* ctx, int8_t* dev_sums, size_t bytes, void* cuda_stream);
+int signmuon_vote_update_from_sums(signmuon_ctx* ctx, const int8_t* dev_sums, size_t bytes, void* const* weights,
+                                   const void* const* grads, float lr, void* cuda_stream);
 
 /* Word offset of parameter `param` inside a worker's payload and its word count. */
 int signmuon_payload_segment(const signmuon_ctx* ctx, int32_t param, size_t* word_offset, size_t* words);

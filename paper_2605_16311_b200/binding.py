@@ -25,7 +25,9 @@ TAP_MOMENTUM, TAP_POLAR, TAP_VOTE_BITS, TAP_WORKER_BITS, TAP_NORM = 0, 1, 2, 3, 
 
 EXPORTS = [
     "signmuon_create", "signmuon_state_bytes", "signmuon_bind", "signmuon_step", "signmuon_run_stages",
-    "signmuon_step_host", "signmuon_packed_payload", "signmuon_payload_segment", "signmuon_debug_tap",
+    "signmuon_step_host", "signmuon_packed_payload", "signmuon_payload_buffer", "signmuon_vote_update",
+    "signmuon_local_sign_sum", "signmuon_vote_update_from_sums", "signmuon_exchange_flags",
+    "signmuon_set_payload_peers", "signmuon_payload_segment", "signmuon_debug_tap",
     "signmuon_status", "signmuon_launches_per_step", "signmuon_ns_flops_per_step", "signmuon_ns_executed_flops_per_step",
     "signmuon_power_start_size", "signmuon_power_start_segment", "signmuon_set_power_start",
     "signmuon_sign_agreement", "signmuon_set_wait_limit", "signmuon_selftest_wait_timeout",
@@ -47,7 +49,8 @@ class ConfigStruct(C.Structure):
                 ("num_workers", C.c_int32), ("momentum", C.c_float), ("lr", C.c_float),
                 ("ns_steps", C.c_int32), ("local_polar", C.c_int32), ("weight_decay", C.c_float),
                 ("eps", C.c_float), ("update_scale", C.c_int32), ("flags", C.c_int32),
-                ("ns_scale", C.c_int32), ("power_iters", C.c_int32)]
+                ("ns_scale", C.c_int32), ("power_iters", C.c_int32),
+                ("worker_offset", C.c_int32), ("local_workers", C.c_int32), ("update_rule", C.c_int32)]
 
 
 _lib = None
@@ -70,6 +73,12 @@ def load_library() -> C.CDLL:
     lib.signmuon_run_stages.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), f32, vp]
     lib.signmuon_step_host.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), f32, vp]
     lib.signmuon_packed_payload.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(sz), C.POINTER(sz)]
+    lib.signmuon_payload_buffer.argtypes = [vp, C.POINTER(vp), C.POINTER(sz), C.POINTER(i32)]
+    lib.signmuon_vote_update.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp]
+    lib.signmuon_exchange_flags.argtypes = [vp, C.POINTER(vp)]
+    lib.signmuon_set_payload_peers.argtypes = [vp, i32, i32, i32, C.POINTER(vp), C.POINTER(vp)]
+    lib.signmuon_local_sign_sum.argtypes = [vp, vp, sz, vp]
+    lib.signmuon_vote_update_from_sums.argtypes = [vp, vp, sz, C.POINTER(vp), C.POINTER(vp), f32, vp]
     lib.signmuon_payload_segment.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
     lib.signmuon_debug_tap.argtypes = [vp, i32, i32, i32, C.POINTER(vp), C.POINTER(sz), C.POINTER(C.c_int64)]
     lib.signmuon_status.argtypes = [vp, vp]
@@ -109,14 +118,15 @@ def _check(code: int, where: str):
 # ------------------------------------------------------------------------- C-ABI mirrors
 def signmuon_create(params: Sequence[tuple], num_workers: int, momentum: float, lr: float, ns_steps: int,
                     local_polar: bool, weight_decay: float = 0.0, eps: float = 1e-12, update_scale: int = 0,
-                    flags: int = 0, ns_scale: int = 0, power_iters: int = 2) -> int:
+                    flags: int = 0, ns_scale: int = 0, power_iters: int = 2, worker_offset: int = 0,
+                    local_workers: int = 0, update_rule: int = 0) -> int:
     """params: (rows, cols, kind, weight_dtype, grad_dtype) tuples. Returns the context handle."""
     lib = load_library()
     arr = (ParamStruct * max(len(params), 1))()
     for i, (r, c, k, wd, gd) in enumerate(params):
         arr[i] = ParamStruct(r, c, k, wd, gd)
     cfg = ConfigStruct(len(params), arr, num_workers, momentum, lr, ns_steps, int(local_polar), weight_decay,
-                       eps, update_scale, flags, ns_scale, power_iters)
+                       eps, update_scale, flags, ns_scale, power_iters, worker_offset, local_workers, update_rule)
     out = C.c_void_p()
     _check(lib.signmuon_create(C.byref(cfg), C.byref(out)), "signmuon_create")
     return out.value
@@ -169,6 +179,41 @@ def signmuon_packed_payload(ctx: int, worker: int, want_ptr: bool = True):
     _check(lib.signmuon_packed_payload(ctx, worker, C.byref(p) if want_ptr else None, C.byref(b), C.byref(e)),
            "signmuon_packed_payload")
     return p.value, b.value, e.value
+
+
+def signmuon_payload_buffer(ctx: int, want_ptr: bool = True):
+    """(device pointer of row 0, row pitch in bytes, rows) of the gathered payload buffer."""
+    p, pitch, rows = C.c_void_p(), C.c_size_t(), C.c_int32()
+    _check(load_library().signmuon_payload_buffer(ctx, C.byref(p) if want_ptr else None, C.byref(pitch), C.byref(rows)),
+           "signmuon_payload_buffer")
+    return p.value, pitch.value, rows.value
+
+
+def signmuon_vote_update(ctx: int, payload_ptrs, weight_ptrs, grad_ptrs, lr: float, stream: int):
+    _check(load_library().signmuon_vote_update(ctx, payload_ptrs, weight_ptrs, grad_ptrs, lr, stream or None),
+           "signmuon_vote_update")
+
+
+def signmuon_exchange_flags(ctx: int) -> int:
+    p = C.c_void_p()
+    _check(load_library().signmuon_exchange_flags(ctx, C.byref(p)), "signmuon_exchange_flags")
+    return p.value
+
+
+def signmuon_set_payload_peers(ctx: int, my_rank: int, num_ranks: int, peer_buffer_ptrs, peer_flag_ptrs):
+    n = len(peer_buffer_ptrs)
+    _check(load_library().signmuon_set_payload_peers(ctx, my_rank, num_ranks, n, _ptr_array(peer_buffer_ptrs) if n else None,
+                                                     _ptr_array(peer_flag_ptrs) if n else None),
+           "signmuon_set_payload_peers")
+
+
+def signmuon_local_sign_sum(ctx: int, sums_ptr: int, nbytes: int, stream: int):
+    _check(load_library().signmuon_local_sign_sum(ctx, sums_ptr, nbytes, stream or None), "signmuon_local_sign_sum")
+
+
+def signmuon_vote_update_from_sums(ctx: int, sums_ptr: int, nbytes: int, weight_ptrs, grad_ptrs, lr: float, stream: int):
+    _check(load_library().signmuon_vote_update_from_sums(ctx, sums_ptr, nbytes, weight_ptrs, grad_ptrs, lr,
+                                                         stream or None), "signmuon_vote_update_from_sums")
 
 
 def signmuon_payload_segment(ctx: int, param: int):
@@ -263,6 +308,8 @@ def signmuon_destroy(ctx: int):
 _DT = {"f32": F32, "bf16": BF16}
 _KIND = {"matrix": PARAM_MATRIX, "plain": PARAM_PLAIN}
 SCALES = {"fro": 0, "spectral": 1}
+RULES = {"signmuon": 0, "muon": 1}
+RULE_SIGNMUON, RULE_MUON = 0, 1
 
 
 def _view_device(ptr: int, nbytes: int, dtype: torch.dtype, owner: torch.Tensor, base_ptr: int) -> torch.Tensor:
@@ -278,14 +325,18 @@ class SignMuon:
     def __init__(self, params, num_workers: int, momentum: float = 0.9, lr: float = 1e-3, ns_steps: int = 5,
                  local_polar: bool = False, weight_decay: float = 0.0, eps: float = 1e-12, update_scale: int = 0,
                  flags: int = 0, device: str = "cuda:0", host_staging: bool = False, ns_scale: str = "fro",
-                 power_iters: int = 2):
+                 power_iters: int = 2, worker_offset: int = 0, local_workers: int = 0, update_rule: str = "signmuon"):
         self.params = list(params)
         self.num_workers = num_workers
+        self.worker_offset = worker_offset if local_workers else 0
+        self.local_workers = local_workers or num_workers      # workers this context computes
+        self.sharded = self.local_workers < num_workers
         self.ns_steps = ns_steps
         self.device = torch.device(device)
         tuples = [(p.rows, p.cols, _KIND[p.kind], _DT[p.dtype], _DT[p.dtype]) for p in self.params]
         self.ctx = signmuon_create(tuples, num_workers, momentum, lr, ns_steps, local_polar, weight_decay, eps,
-                                   update_scale, flags, SCALES[ns_scale], power_iters)
+                                   update_scale, flags, SCALES[ns_scale], power_iters, worker_offset, local_workers,
+                                   RULES[update_rule])
         self.state_bytes, self.workspace_bytes, self.staging_bytes = signmuon_state_bytes(self.ctx)
         with torch.cuda.device(self.device):
             self.state = torch.empty(self.state_bytes, dtype=torch.uint8, device=self.device)
@@ -293,6 +344,9 @@ class SignMuon:
             self._ws_raw = torch.empty(self.workspace_bytes + 1024, dtype=torch.uint8, device=self.device)
             off = (-self._ws_raw.data_ptr()) % 1024
             self.workspace = self._ws_raw[off: off + self.workspace_bytes]
+            # (a sharded context stages host buffers itself, stage by stage: see step_host_sharded)
+            self._host_stage = host_staging and self.sharded
+            host_staging = host_staging and not self.sharded
             self.staging = (torch.empty(self.staging_bytes, dtype=torch.uint8, device=self.device)
                             if host_staging else None)
             stream = torch.cuda.current_stream(self.device).cuda_stream
@@ -343,6 +397,72 @@ class SignMuon:
     def step_host(self, host_weights, host_grads, lr: float = -1.0):
         wp, gp = self._ptrs(host_weights, host_grads)
         signmuon_step_host(self.ctx, wp, gp, lr, torch.cuda.current_stream(self.device).cuda_stream)
+
+    # ---- worker sharding (Alg. 3 across GPUs): own workers' stages, exchange, shared stages
+    def payload_rows(self) -> torch.Tensor:
+        """int32 view [num_workers, pitch_words] of the gathered payload buffer (row m = worker m's payload)."""
+        ptr, pitch, rows = signmuon_payload_buffer(self.ctx)
+        flat = _view_device(ptr, pitch * rows, torch.int32, self.workspace, self.workspace.data_ptr())
+        return flat.view(rows, pitch // 4)
+
+    def exchange_payloads(self, dist_module, group=None):
+        """All-gather of the packed words: every rank contributes the rows of its own workers."""
+        from . import exchange
+        exchange.all_gather_payload(self.payload_rows(), self.worker_offset, self.local_workers, dist_module, group)
+
+    def set_payload_peers(self, my_rank: int, num_ranks: int, peers):
+        """Fused exchange: `peers` are the SignMuon objects (or (payload buffer ptr, flags ptr) pairs of peer-mapped
+        memory) whose payload buffers also receive every word this context packs."""
+        pairs = [(signmuon_payload_buffer(p.ctx)[0], signmuon_exchange_flags(p.ctx)) if isinstance(p, SignMuon) else p
+                 for p in peers]
+        signmuon_set_payload_peers(self.ctx, my_rank, num_ranks, [a for a, _ in pairs], [b for _, b in pairs])
+
+    def vote_update(self, weights, grads, lr: float = -1.0, payloads=None):
+        """Vote, local polar step and update from the gathered payloads (payloads: optional list of num_workers
+        device tensors or None entries; None = what the payload buffer already holds)."""
+        wp, gp = self._ptrs(weights, grads)
+        ptrs = [0] * self.num_workers if payloads is None else [0 if t is None else t.data_ptr() for t in payloads]
+        signmuon_vote_update(self.ctx, _ptr_array(ptrs), wp, gp, lr, torch.cuda.current_stream(self.device).cuda_stream)
+
+    def local_sign_sum(self, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """int8 sums of this context's own workers' signs, one per payload bit position (Alg. 2's all-reduce buffer)."""
+        _, nbytes, _ = signmuon_packed_payload(self.ctx, self.worker_offset, want_ptr=False)
+        if out is None:
+            out = torch.empty(nbytes * 8, dtype=torch.int8, device=self.device)
+        signmuon_local_sign_sum(self.ctx, out.data_ptr(), out.numel(), torch.cuda.current_stream(self.device).cuda_stream)
+        return out
+
+    def vote_update_from_sums(self, sums: torch.Tensor, weights, grads, lr: float = -1.0):
+        wp, gp = self._ptrs(weights, grads)
+        signmuon_vote_update_from_sums(self.ctx, sums.data_ptr(), sums.numel(), wp, gp, lr,
+                                       torch.cuda.current_stream(self.device).cuda_stream)
+
+    def step_sharded(self, weights, grads, lr: float, dist_module, group=None, int8_allreduce: bool = False):
+        """One step of a sharded context: own workers' momentum + Newton-Schulz + pack, the exchange, then the
+        shared vote / local polar / update (identical on every rank)."""
+        self.step(weights, grads, lr, stages=STAGE_MOMENTUM | STAGE_NS)
+        if int8_allreduce:
+            from . import exchange
+            sums = self.local_sign_sum(getattr(self, "_sums", None))
+            self._sums = sums
+            exchange.all_reduce_sign_sums(sums, dist_module, group)
+            self.vote_update_from_sums(sums, weights, grads, lr)
+        else:
+            self.exchange_payloads(dist_module, group)
+            self.step(weights, grads, lr, stages=STAGE_VOTE | STAGE_LOCAL_POLAR)
+
+    def step_host_sharded(self, host_weights, host_grads, lr: float, dist_module, group=None):
+        """step_sharded with host-resident weights and gradients: copies in, steps, copies the weights back."""
+        if not hasattr(self, "_stage_w"):
+            self._stage_w = [torch.empty_like(w, device=self.device) for w in host_weights]
+            self._stage_g = [torch.empty_like(g, device=self.device) for g in host_grads]
+        for dst, src in zip(self._stage_w, host_weights):
+            dst.copy_(src, non_blocking=True)
+        for dst, src in zip(self._stage_g, host_grads):
+            dst.copy_(src, non_blocking=True)
+        self.step_sharded(self._stage_w, self._stage_g, lr, dist_module, group)
+        for dst, src in zip(host_weights, self._stage_w):
+            dst.copy_(src, non_blocking=True)
 
     def status(self) -> int:
         return signmuon_status(self.ctx, torch.cuda.current_stream(self.device).cuda_stream)

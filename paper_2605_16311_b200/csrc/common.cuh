@@ -32,6 +32,7 @@ struct ParamDev {
   uint32_t chunks_per_worker;  // momentum-kernel blocks (= norm partials) per worker
   float upd_scale;      // 1, or 1/sqrt(rows*cols) for the Eq. 2 normalisation
   int32_t vec_ok;       // 16-byte vector path allowed (d % 8 == 0 and ldy == cols)
+  int32_t avg_workers;  // > 1: the momentum takes the mean of this many workers' gradients (Muon rule), G is [avg][rows][cols]
   // power iteration (scale = spectral): un-normalised vectors and their norms
   float* pi_v;          // [M][cols]
   float* pi_u;          // [M][rows]
@@ -97,6 +98,21 @@ struct GemmProblem {
   int32_t gram_lo;        // EPI_GRAM: also store lo(-A/2) through tmapO1 (then the tile is not mirrored)
   int32_t diag_share;     // EPI_GRAM, one segment: on diagonal tiles the B operand is the A tile (not loaded twice)
 };
+
+// Payload buffers of other GPUs that receive every payload word this GPU packs (the exchange of Alg. 3 fused into
+// the pack: plain stores into peer-mapped memory instead of a separate all-gather).  All payload buffers share one
+// layout, so a peer's copy of a word lives at the same offset: delta[p] = peer p's buffer - this GPU's buffer (bytes).
+constexpr int MAX_PAYLOAD_PEERS = 7;
+struct PeerList {
+  int32_t n;
+  int32_t reserved;
+  int64_t delta[MAX_PAYLOAD_PEERS];
+};
+__device__ __forceinline__ void store_payload_word(uint32_t* own, uint32_t word, const PeerList& peers) {
+  *own = word;
+  for (int p = 0; p < peers.n; ++p)
+    *reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(own) + peers.delta[p]) = word;
+}
 
 struct TileEntry {
   uint32_t problem;       // index relative to the launch's first problem
@@ -204,21 +220,26 @@ __device__ __forceinline__ void store_out_direct(const GemmProblem& pr, int row,
 }
 
 // One payload word from 32 consecutive columns (only issued for parameters with cols % 32 == 0).
-__device__ __forceinline__ void pack_bits_direct(const GemmProblem& pr, int row, int col0, const float* v) {
+__device__ __forceinline__ void pack_bits_direct(const GemmProblem& pr, int row, int col0, const float* v,
+                                                 const PeerList& peers) {
   if (row >= pr.M || col0 + 32 > pr.N) return;
   uint32_t word = 0;
 #pragma unroll
   for (int j = 0; j < 32; ++j) word |= (v[j] >= 0.f ? 1u : 0u) << j;
-  pr.bits_out[((int64_t)row * pr.N + col0) >> 5] = word;
+  store_payload_word(pr.bits_out + (((int64_t)row * pr.N + col0) >> 5), word, peers);
 }
 // Half a payload word from 16 consecutive columns (col0 a multiple of 16; little-endian words: the lower
 // columns are the lower half).
-__device__ __forceinline__ void pack_bits16_direct(const GemmProblem& pr, int row, int col0, const float* v) {
+__device__ __forceinline__ void pack_bits16_direct(const GemmProblem& pr, int row, int col0, const float* v,
+                                                   const PeerList& peers) {
   if (row >= pr.M || col0 + 16 > pr.N) return;
   uint32_t half = 0;
 #pragma unroll
   for (int j = 0; j < 16; ++j) half |= (v[j] >= 0.f ? 1u : 0u) << j;
-  reinterpret_cast<uint16_t*>(pr.bits_out)[((int64_t)row * pr.N + col0) >> 4] = (uint16_t)half;
+  uint16_t* own = reinterpret_cast<uint16_t*>(pr.bits_out) + (((int64_t)row * pr.N + col0) >> 4);
+  *own = (uint16_t)half;
+  for (int p = 0; p < peers.n; ++p)
+    *reinterpret_cast<uint16_t*>(reinterpret_cast<char*>(own) + peers.delta[p]) = (uint16_t)half;
 }
 
 // W <- W - lr * v (local polar step's last epilogue).
@@ -272,7 +293,7 @@ __device__ __forceinline__ void update_weights_direct(const GemmProblem& pr, con
 
 // Whole epilogue of 32 columns with direct global accesses (diagnostic kernel and ragged fallbacks).
 __device__ __forceinline__ void epilogue_row32(const GemmProblem& pr, const ParamDev* params, float lr,
-                                               int row, int col0, float (&v)[32]) {
+                                               int row, int col0, float (&v)[32], const PeerList& peers) {
   if (row >= pr.M || col0 >= pr.N) return;
   const float scale = pr.scale_ptr ? __ldg(pr.scale_ptr) : pr.scale_imm;
   if (pr.epi == EPI_GRAM) {
@@ -284,7 +305,7 @@ __device__ __forceinline__ void epilogue_row32(const GemmProblem& pr, const Para
   }
   apply_c_direct(pr, scale, row, col0, v);
   if (pr.epi == EPI_APPLY || (pr.epi == EPI_APPLY_PACK && pr.store_out)) store_out_direct(pr, row, col0, v, pr.epi == EPI_APPLY);
-  if (pr.epi == EPI_APPLY_PACK) pack_bits_direct(pr, row, col0, v);
+  if (pr.epi == EPI_APPLY_PACK) pack_bits_direct(pr, row, col0, v, peers);
   else if (pr.epi == EPI_APPLY_UPDATE) update_weights_direct(pr, params, lr, row, col0, v);
 }
 

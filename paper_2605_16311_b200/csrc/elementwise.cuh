@@ -10,8 +10,7 @@ constexpr int EW_THREADS = 256;
 constexpr int MOM_CHUNK = 8192;        // entries per block of the momentum kernel (256 threads x 8 x 4)
 constexpr int PLAIN_CHUNK = 2048;      // entries per block of the plain-parameter kernel (8 warps x 256)
 constexpr int VOTE_THREADS = 128;      // vote kernel: 4 warps per block
-constexpr int VOTE_WARP_WORDS = 128;   // payload words per warp (4 consecutive words per lane: 128-bit loads)
-constexpr int VOTE_WORDS = VOTE_WARP_WORDS * VOTE_THREADS / 32;   // payload words per block
+constexpr int VOTE_WORDS = 4 * VOTE_THREADS;   // payload words per block (4 consecutive words per lane: 128-bit loads)
 constexpr int PACK_CHUNK = 1024;       // entries per block of the stand-alone pack kernel (small: it only sees small, ragged matrices)
 
 // Finds the list slot whose block range contains `block` (`starts` is ascending, one entry per slot).
@@ -68,6 +67,8 @@ __device__ __forceinline__ void momentum_block(const ParamDev& pd, int m, uint32
   bf16* ylo = pd.ylo ? pd.ylo + (int64_t)m * pd.rows * pd.ldy : nullptr;
   const int64_t base = (int64_t)chunk * MOM_CHUNK;
   const float omb = 1.f - beta;
+  const int avg = pd.avg_workers;                 // > 1: mean gradient of that many workers (m is 0 then)
+  const float inv_avg = 1.f / (float)(avg > 1 ? avg : 1);
   if (pd.vec_ok) {
 #pragma unroll
     for (int it = 0; it < MOM_CHUNK / (EW_THREADS * 8); ++it) {
@@ -76,6 +77,16 @@ __device__ __forceinline__ void momentum_block(const ParamDev& pd, int m, uint32
         float gv[8], mv[8];
         load8(g + i, gv);
         load8(mom + i, mv);
+        if (avg > 1) {
+          for (int k = 1; k < avg; ++k) {
+            float t[8];
+            load8(g + (int64_t)k * d + i, t);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) gv[e] += t[e];
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) gv[e] *= inv_avg;
+        }
         if (lambda != 0.f) {
           float wv[8];
           load8(w + i, wv);
@@ -111,6 +122,10 @@ __device__ __forceinline__ void momentum_block(const ParamDev& pd, int m, uint32
     const int64_t end = (base + MOM_CHUNK < d) ? base + MOM_CHUNK : d;
     for (int64_t i = base + threadIdx.x; i < end; i += EW_THREADS) {
       float gv = load_as_float<GT>(g + i);
+      if (avg > 1) {
+        for (int k = 1; k < avg; ++k) gv += load_as_float<GT>(g + (int64_t)k * d + i);
+        gv *= inv_avg;
+      }
       if (lambda != 0.f) gv = fmaf(lambda, load_as_float<WT>(w + i), gv);
       const float mv = fmaf(beta, mom[i], omb * gv);
       mom[i] = mv;
@@ -197,7 +212,8 @@ __device__ __forceinline__ void store8(bf16* p, const float (&x)[8]) {
 template <typename GT, typename WT>
 __device__ __forceinline__ void plain_warp_vec(const ParamDev& pd, int64_t base, int M, float beta, float lambda,
                                                float step, uint32_t* __restrict__ bits,
-                                               uint32_t* __restrict__ vote_words, int64_t bits_pitch) {
+                                               uint32_t* __restrict__ vote_words, int64_t bits_pitch, int do_vote,
+                                               const PeerList& peers) {
   const int lane = threadIdx.x & 31;
   const int64_t d = pd.d;
   const int64_t i0 = base + 8 * lane;
@@ -225,7 +241,7 @@ __device__ __forceinline__ void plain_warp_vec(const ParamDev& pd, int64_t base,
     }
     store8(mom + (int64_t)m * d, mv);
     const uint32_t wordv = __reduce_or_sync(group, byte << shift);
-    if ((lane & 3) == 0) out[(int64_t)m * bits_pitch] = wordv;
+    if ((lane & 3) == 0) store_payload_word(out + (int64_t)m * bits_pitch, wordv, peers);
   };
   int m = 0;
   for (; m + 1 < M; m += 2) {
@@ -243,6 +259,7 @@ __device__ __forceinline__ void plain_warp_vec(const ParamDev& pd, int64_t base,
     load8(mom + (int64_t)m * d, m0);
     finish(g0, m0, m);
   }
+  if (!do_vote) return;      // the workers of this pass are a subset: vote and update follow the payload exchange
   uint32_t vbyte = 0;
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
@@ -258,30 +275,33 @@ __device__ __forceinline__ void plain_warp_vec(const ParamDev& pd, int64_t base,
 template <typename GT, typename WT>
 __device__ __forceinline__ void plain_warp_scalar(const ParamDev& pd, int64_t base, int M, float beta, float lambda,
                                                   float step, uint32_t* __restrict__ bits,
-                                                  uint32_t* __restrict__ vote_words, int64_t bits_pitch);
+                                                  uint32_t* __restrict__ vote_words, int64_t bits_pitch, int do_vote,
+                                                  const PeerList& peers);
 
 template <typename GT, typename WT>
 __device__ __forceinline__ void plain_block(const ParamDev& pd, uint32_t chunk, int M, float beta,
                                             float lambda, float step, uint32_t* __restrict__ bits,
-                                            uint32_t* __restrict__ vote_words, int64_t bits_pitch) {
+                                            uint32_t* __restrict__ vote_words, int64_t bits_pitch, int do_vote,
+                                            const PeerList& peers) {
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int64_t d = pd.d;
   if ((d & 7) == 0 && (int64_t)chunk * PLAIN_CHUNK + (warp + 1) * 256 <= d) {
     plain_warp_vec<GT, WT>(pd, (int64_t)chunk * PLAIN_CHUNK + warp * 256, M, beta, lambda, step, bits, vote_words,
-                           bits_pitch);
+                           bits_pitch, do_vote, peers);
     return;
   }
   // ragged tail (or an unaligned parameter): the warp's 256 entries as two scalar passes of 128
   for (int pass = 0; pass < 2; ++pass)
     plain_warp_scalar<GT, WT>(pd, (int64_t)chunk * PLAIN_CHUNK + warp * 256 + pass * 128, M, beta, lambda, step, bits,
-                              vote_words, bits_pitch);
+                              vote_words, bits_pitch, do_vote, peers);
 }
 
 template <typename GT, typename WT>
 __device__ __forceinline__ void plain_warp_scalar(const ParamDev& pd, int64_t base, int M, float beta,
                                                   float lambda, float step, uint32_t* __restrict__ bits,
-                                                  uint32_t* __restrict__ vote_words, int64_t bits_pitch) {
+                                                  uint32_t* __restrict__ vote_words, int64_t bits_pitch, int do_vote,
+                                                  const PeerList& peers) {
   const int lane = threadIdx.x & 31;
   const int64_t d = pd.d;
   if (base >= d) return;
@@ -321,8 +341,9 @@ __device__ __forceinline__ void plain_warp_scalar(const ParamDev& pd, int64_t ba
       if (lane == k) mine = word;
     }
     if (lane < 4 && word0 + lane < pd.n_words)
-      bits[(int64_t)m * bits_pitch + pd.word_off + word0 + lane] = mine;
+      store_payload_word(bits + (int64_t)m * bits_pitch + pd.word_off + word0 + lane, mine, peers);
   }
+  if (!do_vote) return;
   uint32_t vmine = 0;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
@@ -345,17 +366,18 @@ __global__ void __launch_bounds__(EW_THREADS) plain_params_kernel(const ParamDev
                                                                   int M, float beta, float lambda, float lr,
                                                                   uint32_t* __restrict__ bits,
                                                                   uint32_t* __restrict__ vote_words,
-                                                                  int64_t bits_pitch) {
+                                                                  int64_t bits_pitch, int do_vote,
+                                                                  const __grid_constant__ PeerList peers) {
   const int slot = find_slot(starts, n_list, blockIdx.x);
   const ParamDev pd = params[list[slot]];
   const uint32_t chunk = blockIdx.x - starts[slot];
   const float step = lr * pd.upd_scale;
   if (pd.gdtype == 0) {
-    if (pd.wdtype == 0) plain_block<float, float>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch);
-    else plain_block<float, bf16>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch);
+    if (pd.wdtype == 0) plain_block<float, float>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch, do_vote, peers);
+    else plain_block<float, bf16>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch, do_vote, peers);
   } else {
-    if (pd.wdtype == 0) plain_block<bf16, float>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch);
-    else plain_block<bf16, bf16>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch);
+    if (pd.wdtype == 0) plain_block<bf16, float>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch, do_vote, peers);
+    else plain_block<bf16, bf16>(pd, chunk, M, beta, lambda, step, bits, vote_words, bits_pitch, do_vote, peers);
   }
 }
 
@@ -368,7 +390,8 @@ __global__ void __launch_bounds__(EW_THREADS) pack_kernel(const ParamDev* __rest
                                                           const int32_t* __restrict__ list,
                                                           const uint32_t* __restrict__ starts, int n_list,
                                                           int src_buf, int from_momentum,
-                                                          uint32_t* __restrict__ bits, int64_t bits_pitch) {
+                                                          uint32_t* __restrict__ bits, int64_t bits_pitch,
+                                                          const __grid_constant__ PeerList peers) {
   const int slot = find_slot(starts, n_list, blockIdx.x);
   const ParamDev pd = params[list[slot]];
   const uint32_t local = blockIdx.x - starts[slot];
@@ -394,7 +417,7 @@ __global__ void __launch_bounds__(EW_THREADS) pack_kernel(const ParamDev* __rest
     }
     const uint32_t word = __ballot_sync(0xffffffffu, b);
     const int64_t wi = i >> 5;
-    if (lane == 0 && wi < pd.n_words) bits[(int64_t)m * bits_pitch + pd.word_off + wi] = word;
+    if (lane == 0 && wi < pd.n_words) store_payload_word(bits + (int64_t)m * bits_pitch + pd.word_off + wi, word, peers);
   }
 }
 
@@ -402,13 +425,13 @@ __global__ void __launch_bounds__(EW_THREADS) pack_kernel(const ParamDev* __rest
 // Majority vote from the packed words (App. B: c = sum_m b^(m), S = sign(2c - M), ties -> +1) and
 // the weight update W <- W - eta S (Alg. 3), or, for the local polar step, S as a bf16 +-1 matrix.
 //
-// A warp owns an aligned group of 128 words of the payload's word index (the workers' rows are 128-byte
-// aligned in the workspace, so lane l reads words 4l..4l+3 of every worker as one 128-bit load, eight rows in
-// flight).  The 32 per-position counts of each word are kept as bit-sliced counter planes (about three logic
-// operations per worker word instead of 32 unpacks); the comparison c >= ceil(M/2) is the carry out of a
-// bit-sliced addition of 2^PLANES - ceil(M/2).  The 128 vote words then go through shared memory so that the
-// weights (or the +-1 matrix) move as 128-bit vectors too; the first batch of weight vectors is requested
-// before the payload, so both latencies overlap.  Words of the group outside the parameter are masked.
+// Two streaming kernels.  vote_kernel reads the payload (the workers' rows are 128-byte aligned in the workspace, so
+// a lane reads four consecutive words of a worker as one 128-bit load, eight rows in flight) and writes the vote
+// words; the 32 per-position counts of a word are kept as bit-sliced counter planes (about three logic operations
+// per worker word instead of 32 unpacks) and the comparison c >= ceil(M/2) is the carry out of a bit-sliced addition
+// of 2^PLANES - ceil(M/2).  update_kernel reads the vote words back (1/8 byte per entry, from L2) and moves the weights
+// (or the +-1 matrix) as 128-bit vectors, eight per thread in flight.  Split this way each kernel keeps few registers
+// per byte in flight; one fused kernel held both the payload rows and the weight vectors and ran at lower occupancy.
 // ---------------------------------------------------------------------------------------------
 template <int PLANES>
 struct VoteCounter {
@@ -438,54 +461,27 @@ struct VoteCounter {
   }
 };
 
-template <typename WT> __host__ __device__ constexpr int write_sbar_vec_entries() { return 16 / (int)sizeof(WT); }
-
-template <int PLANES, typename WT>
-__device__ __forceinline__ void vote_warp(const ParamDev& pd, int64_t g0, int M, float step, int write_sbar,
-                                          const uint32_t* __restrict__ bits, uint32_t* __restrict__ vote_words,
-                                          int64_t bits_pitch, uint32_t* sv) {
-  constexpr int ROWS = PLANES >= 8 ? 4 : 8;             // worker rows in flight per lane
-  constexpr int EPV = write_sbar_vec_entries<WT>();     // entries per 128-bit weight vector (float: 4, bf16: 8)
-  const int lane = threadIdx.x & 31;
+// vote_kernel: payload rows -> vote words.  A block owns an aligned group of VOTE_WORDS words of the payload's
+// word index, a lane four consecutive words; words of the group outside the parameter are masked (a group shared
+// by two parameters is visited once for each).
+template <int PLANES>
+__global__ void __launch_bounds__(VOTE_THREADS) vote_kernel(const ParamDev* __restrict__ params,
+                                                            const int32_t* __restrict__ list,
+                                                            const uint32_t* __restrict__ starts, int n_list, int M,
+                                                            const uint32_t* __restrict__ bits,
+                                                            uint32_t* __restrict__ vote_words, int64_t bits_pitch) {
+  constexpr int ROWS = 8;                               // worker rows in flight per lane
+  const int slot = find_slot(starts, n_list, blockIdx.x);
+  const ParamDev& pd = params[list[slot]];
   const int64_t lo = pd.word_off, hi = (int64_t)pd.word_off + pd.n_words;
-  if (g0 >= hi || g0 + VOTE_WARP_WORDS <= lo) return;
-  const int64_t g = g0 + 4 * lane;                      // this lane's first word (global word index)
-  const bool lane_full = g >= lo && g + 4 <= hi;
-  const int64_t e0 = (g0 - lo) * 32;                    // entry of the group's first word (negative: group starts before the parameter)
-  const int64_t d = pd.d;
-  // 128-bit path: every vector lies inside one vote word; it needs 16-byte aligned rows of whole vectors
-  const bool vec = write_sbar ? (pd.vec_ok != 0) : ((d & 7) == 0);
-  WT* w = reinterpret_cast<WT*>(pd.W);
-  bf16* sbar = pd.y0 + (int64_t)M * pd.rows * pd.ldy;   // slot M of operand buffer 0: input of the local polar step
-
-  // The group's entries as 128-bit vectors: vector i of the group covers entries e0 + i * epv .. + epv - 1
-  // (epv = 4 float32 or 8 bf16), all inside vote word i / (32 / epv).  Valid when the entry is inside the parameter.
-  const int epv = write_sbar ? 8 : EPV;
-  const int n_batches = (VOTE_WARP_WORDS * 32 / epv) / (8 * 32);      // 8 vectors per lane and batch
-  uint4* vbase = write_sbar ? reinterpret_cast<uint4*>(sbar) : reinterpret_cast<uint4*>(w);
-  auto vec_valid = [&](int i) -> bool {
-    const int64_t e = e0 + (int64_t)i * epv;
-    return e >= 0 && e < d;
-  };
-  auto vec_ptr = [&](int i) -> uint4* {                 // 16-byte units from the start of the parameter
-    return vbase + (e0 / epv + i);
-  };
-  uint4 x[8];                                           // float4 bit patterns or 8 bf16 each
-  const bool rmw = vec && !write_sbar;
-  if (rmw) {                                            // first batch of weight vectors: independent of the vote
-#pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int i = it * 32 + lane;
-      x[it] = vec_valid(i) ? __ldcs(vec_ptr(i)) : make_uint4(0, 0, 0, 0);
-    }
-  }
-
-  // ---- vote of this lane's four words
+  const uint32_t chunk = blockIdx.x - starts[slot];
+  const int64_t g = ((int64_t)(pd.word_off / VOTE_WORDS) + chunk) * VOTE_WORDS + 4 * (int64_t)threadIdx.x;
+  if (g >= hi || g + 4 <= lo) return;
   VoteCounter<PLANES> cnt[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) cnt[j].clear();
   const uint32_t* col = bits + g;
-  if (lane_full) {
+  if (g >= lo && g + 4 <= hi) {
     int m = 0;
     for (; m + ROWS <= M; m += ROWS) {
       uint4 r[ROWS];
@@ -494,112 +490,210 @@ __device__ __forceinline__ void vote_warp(const ParamDev& pd, int64_t g0, int M,
 #pragma unroll
       for (int k = 0; k < ROWS; ++k) { cnt[0].add(r[k].x); cnt[1].add(r[k].y); cnt[2].add(r[k].z); cnt[3].add(r[k].w); }
     }
+    if (m + 4 <= M) {
+      uint4 r[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) r[k] = __ldcs(reinterpret_cast<const uint4*>(col + (int64_t)(m + k) * bits_pitch));
+#pragma unroll
+      for (int k = 0; k < 4; ++k) { cnt[0].add(r[k].x); cnt[1].add(r[k].y); cnt[2].add(r[k].z); cnt[3].add(r[k].w); }
+      m += 4;
+    }
     for (; m < M; ++m) {
       const uint4 r = __ldcs(reinterpret_cast<const uint4*>(col + (int64_t)m * bits_pitch));
       cnt[0].add(r.x); cnt[1].add(r.y); cnt[2].add(r.z); cnt[3].add(r.w);
     }
+    *reinterpret_cast<uint4*>(vote_words + g) =
+        make_uint4(cnt[0].majority(M), cnt[1].majority(M), cnt[2].majority(M), cnt[3].majority(M));
   } else {
     for (int m = 0; m < M; ++m) {
 #pragma unroll
       for (int j = 0; j < 4; ++j)
         if (g + j >= lo && g + j < hi) cnt[j].add(__ldcs(col + (int64_t)m * bits_pitch + j));
     }
-  }
-  uint32_t v[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) v[j] = cnt[j].majority(M);
-  if (lane_full) {
-    *reinterpret_cast<uint4*>(vote_words + g) = make_uint4(v[0], v[1], v[2], v[3]);
-  } else {
 #pragma unroll
     for (int j = 0; j < 4; ++j)
-      if (g + j >= lo && g + j < hi) vote_words[g + j] = v[j];
+      if (g + j >= lo && g + j < hi) vote_words[g + j] = cnt[j].majority(M);
   }
-  *reinterpret_cast<uint4*>(sv + 4 * lane) = make_uint4(v[0], v[1], v[2], v[3]);
-  __syncwarp();
+}
 
+// update_kernel: vote words -> W <- W - eta S (Alg. 3 "Update parameters"), or S as a bf16 +-1 matrix in the local
+// polar step's operand slot.  A block owns UPD_VECS 128-bit vectors of one parameter (4 float32 or 8 bf16 entries
+// each, all inside one vote word), a thread eight of them, all requested before the first is used.
+constexpr int UPD_VECS = EW_THREADS * 8;
+template <typename WT>
+__device__ __forceinline__ void update_block(const ParamDev& pd, uint32_t chunk, int lp_slot, float step, int write_sbar,
+                                             const uint32_t* __restrict__ vote_words) {
+  const int64_t d = pd.d;
+  WT* w = reinterpret_cast<WT*>(pd.W);
+  bf16* sbar = pd.y0 + (int64_t)lp_slot * pd.rows * pd.ldy;   // the slot after the own workers' slots of operand buffer 0
+  const uint32_t* vw = vote_words + pd.word_off;
+  const bool vec = write_sbar ? (pd.vec_ok != 0) : ((d & 7) == 0);
+  const int epv = (write_sbar || sizeof(WT) == 2) ? 8 : 4;
   if (vec) {
-#pragma unroll 1
-    for (int batch = 0; batch < n_batches; ++batch) {
-      if (batch > 0 && rmw) {
+    uint4* vbase = write_sbar ? reinterpret_cast<uint4*>(sbar) : reinterpret_cast<uint4*>(w);
+    const int64_t n_vec = d / epv;
+    const int64_t i0 = (int64_t)chunk * UPD_VECS + threadIdx.x;
+    uint4 x[8];
+    uint32_t vword[8];
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          const int i = (batch * 8 + it) * 32 + lane;
-          x[it] = vec_valid(i) ? __ldcs(vec_ptr(i)) : make_uint4(0, 0, 0, 0);
-        }
+    for (int it = 0; it < 8; ++it) {
+      const int64_t i = i0 + it * EW_THREADS;
+      if (i < n_vec) {
+        vword[it] = __ldg(vw + ((i * epv) >> 5));
+        if (!write_sbar) x[it] = __ldcs(vbase + i);
       }
+    }
 #pragma unroll
-      for (int it = 0; it < 8; ++it) {
-        const int i = (batch * 8 + it) * 32 + lane;
-        if (!vec_valid(i)) continue;
-        uint4 o;
-        if (!write_sbar && sizeof(WT) == 4) {           // 4 float32: a nibble of word i / 8
-          const uint32_t b4 = sv[i >> 3] >> ((i & 7) * 4);
-          o.x = __float_as_uint(__uint_as_float(x[it].x) - ((b4 & 1u) ? step : -step));
-          o.y = __float_as_uint(__uint_as_float(x[it].y) - ((b4 & 2u) ? step : -step));
-          o.z = __float_as_uint(__uint_as_float(x[it].z) - ((b4 & 4u) ? step : -step));
-          o.w = __float_as_uint(__uint_as_float(x[it].w) - ((b4 & 8u) ? step : -step));
-        } else {                                        // 8 bf16: a byte of word i / 4
-          const uint32_t b8 = sv[i >> 2] >> ((i & 3) * 8);
-          const uint32_t in[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
-          uint32_t ov[4];
+    for (int it = 0; it < 8; ++it) {
+      const int64_t i = i0 + it * EW_THREADS;
+      if (i >= n_vec) continue;
+      uint4 o;
+      if (!write_sbar && sizeof(WT) == 4) {             // 4 float32: a nibble of the vote word
+        const uint32_t b4 = vword[it] >> ((i & 7) * 4);
+        o.x = __float_as_uint(__uint_as_float(x[it].x) - ((b4 & 1u) ? step : -step));
+        o.y = __float_as_uint(__uint_as_float(x[it].y) - ((b4 & 2u) ? step : -step));
+        o.z = __float_as_uint(__uint_as_float(x[it].z) - ((b4 & 4u) ? step : -step));
+        o.w = __float_as_uint(__uint_as_float(x[it].w) - ((b4 & 8u) ? step : -step));
+      } else {                                          // 8 bf16: a byte of the vote word
+        const uint32_t b8 = vword[it] >> ((i & 3) * 8);
+        const uint32_t in[4] = {x[it].x, x[it].y, x[it].z, x[it].w};
+        uint32_t ov[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const bool p0 = (b8 >> (2 * e)) & 1u, p1 = (b8 >> (2 * e + 1)) & 1u;
-            if (write_sbar) ov[e] = (p0 ? 0x3f80u : 0xbf80u) | ((p1 ? 0x3f80u : 0xbf80u) << 16);      // bf16 +-1
-            else ov[e] = pack_bf16x2(__uint_as_float(in[e] << 16) - (p0 ? step : -step),
-                                     __uint_as_float(in[e] & 0xffff0000u) - (p1 ? step : -step));
-          }
-          o = make_uint4(ov[0], ov[1], ov[2], ov[3]);
+        for (int e = 0; e < 4; ++e) {
+          const bool p0 = (b8 >> (2 * e)) & 1u, p1 = (b8 >> (2 * e + 1)) & 1u;
+          if (write_sbar) ov[e] = (p0 ? 0x3f80u : 0xbf80u) | ((p1 ? 0x3f80u : 0xbf80u) << 16);      // bf16 +-1
+          else ov[e] = pack_bf16x2(__uint_as_float(in[e] << 16) - (p0 ? step : -step),
+                                   __uint_as_float(in[e] & 0xffff0000u) - (p1 ? step : -step));
         }
-        __stcs(vec_ptr(i), o);
+        o = make_uint4(ov[0], ov[1], ov[2], ov[3]);
       }
+      __stcs(vbase + i, o);
     }
     return;
   }
   // scalar path: rows that are padded in the operand buffer (the +-1 matrix of a parameter whose column count is
-  // not a multiple of 8), or d not a multiple of 8
-  for (int k = 0; k < VOTE_WARP_WORDS; ++k) {
-    const int64_t gw = g0 + k;
-    if (gw < lo || gw >= hi) continue;
-    const uint32_t vk = sv[k];
-    const int64_t i = (gw - lo) * 32 + lane;
-    if (i < d) {
-      const bool plus = (vk >> lane) & 1u;
-      if (write_sbar) {
-        int64_t o = i;
-        if (pd.ldy != pd.cols) {
-          const int64_t r = i / pd.cols;
-          o = r * pd.ldy + (i - r * pd.cols);
-        }
-        sbar[o] = __float2bfloat16_rn(plus ? 1.f : -1.f);
-      } else {
-        const float nw = load_as_float<WT>(w + i) - (plus ? step : -step);
-        if (sizeof(WT) == 4) reinterpret_cast<float*>(w)[i] = nw;
-        else reinterpret_cast<bf16*>(w)[i] = __float2bfloat16_rn(nw);
+  // not a multiple of 8), or d not a multiple of 8.  The block covers the same entries as on the vector path.
+  const int64_t e_begin = (int64_t)chunk * UPD_VECS * epv;
+  const int64_t e_end = (e_begin + (int64_t)UPD_VECS * epv < d) ? e_begin + (int64_t)UPD_VECS * epv : d;
+  for (int64_t i = e_begin + threadIdx.x; i < e_end; i += EW_THREADS) {
+    const bool plus = (__ldg(vw + (i >> 5)) >> (i & 31)) & 1u;
+    if (write_sbar) {
+      int64_t o = i;
+      if (pd.ldy != pd.cols) {
+        const int64_t r = i / pd.cols;
+        o = r * pd.ldy + (i - r * pd.cols);
       }
+      sbar[o] = __float2bfloat16_rn(plus ? 1.f : -1.f);
+    } else {
+      const float nw = load_as_float<WT>(w + i) - (plus ? step : -step);
+      if (sizeof(WT) == 4) reinterpret_cast<float*>(w)[i] = nw;
+      else reinterpret_cast<bf16*>(w)[i] = __float2bfloat16_rn(nw);
     }
   }
 }
 
-template <int PLANES>
-__global__ void __launch_bounds__(VOTE_THREADS) vote_update_kernel(const ParamDev* __restrict__ params,
-                                                                   const int32_t* __restrict__ list,
-                                                                   const uint32_t* __restrict__ starts, int n_list,
-                                                                   int M, float lr, int write_sbar,
-                                                                   const uint32_t* __restrict__ bits,
-                                                                   uint32_t* __restrict__ vote_words,
-                                                                   int64_t bits_pitch) {
-  __shared__ __align__(16) uint32_t sv_all[VOTE_THREADS / 32][VOTE_WARP_WORDS];
+__global__ void __launch_bounds__(EW_THREADS) update_kernel(const ParamDev* __restrict__ params,
+                                                            const int32_t* __restrict__ list,
+                                                            const uint32_t* __restrict__ starts, int n_list, int lp_slot,
+                                                            float lr, int write_sbar,
+                                                            const uint32_t* __restrict__ vote_words) {
   const int slot = find_slot(starts, n_list, blockIdx.x);
   const ParamDev pd = params[list[slot]];
   const uint32_t chunk = blockIdx.x - starts[slot];
-  const int warp = threadIdx.x >> 5;
-  // first word of this warp's group: groups are aligned in the payload's word index, not in the parameter
-  const int64_t g0 = ((int64_t)(pd.word_off / VOTE_WORDS) + chunk) * VOTE_WORDS + warp * VOTE_WARP_WORDS;
   const float step = lr * pd.upd_scale;
-  if (pd.wdtype == 0) vote_warp<PLANES, float>(pd, g0, M, step, write_sbar, bits, vote_words, bits_pitch, sv_all[warp]);
-  else vote_warp<PLANES, bf16>(pd, g0, M, step, write_sbar, bits, vote_words, bits_pitch, sv_all[warp]);
+  const int sbar = (write_sbar && pd.kind == 0) ? 1 : 0;   // plain parameters are updated directly (no local polar step)
+  if (pd.wdtype == 0) update_block<float>(pd, chunk, lp_slot, step, sbar, vote_words);
+  else update_block<bf16>(pd, chunk, lp_slot, step, sbar, vote_words);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Integer sign sums (Alg. 2: "sum_signs <- sum_m S^(m)", all-reduce with SUM on int8).
+// sign_sum_kernel: per payload bit position the sum of the +-1 signs of `rows` payload rows, one int8 per
+// position (2 c - rows, c = number of set bits); thread t owns word t (32 positions, 32 bytes of output).
+// sums_to_vote_kernel: S = sign(sum), ties -> +1, packed back into vote words (bit = sum >= 0).
+// Pad positions carry bit 0 in every payload, so their sum is -rows (negative after any reduction): the vote
+// keeps them 0.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) sign_sum_kernel(const uint32_t* __restrict__ bits, int64_t bits_pitch,
+                                                              int64_t words, int rows, int8_t* __restrict__ sums) {
+  const int64_t w = (int64_t)blockIdx.x * EW_THREADS + threadIdx.x;
+  if (w >= words) return;
+  VoteCounter<8> cnt;
+  cnt.clear();
+  for (int m = 0; m < rows; ++m) cnt.add(__ldg(bits + (int64_t)m * bits_pitch + w));
+  uint32_t out[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    uint32_t packed = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int j = q * 4 + e;
+      int c = 0;
+#pragma unroll
+      for (int b = 0; b < 8; ++b) c |= (int)((cnt.c[b] >> j) & 1u) << b;
+      packed |= (uint32_t)(uint8_t)(int8_t)(2 * c - rows) << (8 * e);
+    }
+    out[q] = packed;
+  }
+  uint4* o = reinterpret_cast<uint4*>(sums + w * 32);
+  o[0] = make_uint4(out[0], out[1], out[2], out[3]);
+  o[1] = make_uint4(out[4], out[5], out[6], out[7]);
+}
+
+__global__ void __launch_bounds__(EW_THREADS) sums_to_vote_kernel(const int8_t* __restrict__ sums, int64_t words,
+                                                                  uint32_t* __restrict__ vote_words) {
+  const int64_t w = (int64_t)blockIdx.x * EW_THREADS + threadIdx.x;
+  if (w >= words) return;
+  const uint4* in = reinterpret_cast<const uint4*>(sums + w * 32);
+  const uint4 a = __ldg(in), b = __ldg(in + 1);
+  const uint32_t v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+  uint32_t word = 0;
+#pragma unroll
+  for (int q = 0; q < 8; ++q)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int8_t sv = (int8_t)((v[q] >> (8 * e)) & 0xffu);
+      word |= (sv >= 0 ? 1u : 0u) << (q * 4 + e);
+    }
+  vote_words[w] = word;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Hand-shake of the fused exchange.  publish_payload_kernel runs after the last kernel that stores payload words:
+// it makes those stores visible system-wide and writes this step's sequence number into slot `my_rank` of every
+// peer's flag array.  await_payloads_kernel runs before the vote: lane r waits until slot r of this GPU's own flag
+// array has reached the sequence number, at most `limit_ns`; a wait that runs out records STATUS_TIMEOUT.
+// ---------------------------------------------------------------------------------------------
+struct FlagList {
+  int32_t n;
+  int32_t reserved;
+  uint32_t* flags[MAX_PAYLOAD_PEERS];
+};
+__global__ void publish_payload_kernel(const __grid_constant__ FlagList peers, int my_rank, uint32_t seq) {
+  if (threadIdx.x < peers.n) {
+    __threadfence_system();
+    volatile uint32_t* f = peers.flags[threadIdx.x] + my_rank;
+    *f = seq;
+    __threadfence_system();
+  }
+}
+__global__ void await_payloads_kernel(const uint32_t* own_flags, int n_ranks, int my_rank, uint32_t seq,
+                                      uint64_t limit_ns, uint32_t* status) {
+  const int r = threadIdx.x;
+  if (r >= n_ranks || r == my_rank) return;
+  const volatile uint32_t* f = own_flags + r;
+  uint64_t t0 = 0;
+  uint32_t spins = 0;
+  // (sequence numbers wrap: compare as a signed distance)
+  while ((int32_t)(*f - seq) < 0) {
+    if ((++spins & 63u) == 0) {
+      uint64_t now;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > limit_ns) { atomicExch(status, (uint32_t)STATUS_TIMEOUT); return; }
+    }
+  }
+  __threadfence_system();
 }
 
 // ---------------------------------------------------------------------------------------------

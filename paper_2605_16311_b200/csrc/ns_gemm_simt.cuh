@@ -10,7 +10,8 @@ namespace signmuon {
 
 __global__ void __launch_bounds__(128) ns_gemm_simt_kernel(const GemmProblem* __restrict__ problems,
                                                            const TileEntry* __restrict__ tiles, int bn,
-                                                           const ParamDev* __restrict__ params, float lr) {
+                                                           const ParamDev* __restrict__ params, float lr,
+                                                           const __grid_constant__ PeerList peers) {
   __shared__ float As[128][33];
   __shared__ float Bs[32][33];
   const TileEntry te = tiles[blockIdx.x];
@@ -48,7 +49,7 @@ __global__ void __launch_bounds__(128) ns_gemm_simt_kernel(const GemmProblem* __
       }
       __syncthreads();
     }
-    epilogue_row32(pr, params, lr, m0 + tid, c0, acc);
+    epilogue_row32(pr, params, lr, m0 + tid, c0, acc, peers);
   }
 }
 

@@ -49,10 +49,7 @@ namespace signmuon {
 
 constexpr int GEMM_BM = 128;
 constexpr int GEMM_BK = 64;
-#ifndef NS_EPI_WARPS
-#define NS_EPI_WARPS 8
-#endif
-constexpr int EPI_WARPS = NS_EPI_WARPS;      // EPI_WARPS / 4 warps per TMEM lane quarter, each NCOL of a chunk's 64 columns
+constexpr int EPI_WARPS = 8;                 // EPI_WARPS / 4 warps per TMEM lane quarter, each NCOL of a chunk's 64 columns
 constexpr int EPI_NCOL = 256 / EPI_WARPS;    // columns of a chunk one math thread owns (32 or 16)
 static_assert(EPI_WARPS == 8 || EPI_WARPS == 16, "8 or 16 epilogue math warps");
 constexpr int GEMM_THREADS = 32 * (3 + EPI_WARPS);   // warp 0: operand TMA, warp 1: MMA, then the epilogue math warps,
@@ -68,6 +65,7 @@ struct GemmLaunchArgs {
   uint32_t* status;
   float lr;
   uint64_t wait_limit_ns;           // after this long a waiting thread gives up and the CTA aborts
+  PeerList peers;                   // other GPUs' payload buffers that also receive the packed words (n = 0: none)
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -285,7 +283,7 @@ __device__ __forceinline__ void epi_issue_c_load(int c_mode, const CUtensorMap* 
 }
 
 template <int BN, int STAGES, int EPI_BUFS, int CTAS, int KIND>
-__global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmLaunchArgs args) {
+__global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __grid_constant__ GemmLaunchArgs args) {
   constexpr int B_ROWS = BN / CTAS;                            // rows of the B operand this CTA stages
   constexpr int TILE_M = GEMM_BM * CTAS;                       // rows of the output tile of the CTA (pair)
   constexpr uint32_t A_BYTES = GEMM_BM * GEMM_BK * 2;          // 16 KB
@@ -702,7 +700,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const GemmL
             }
           }
           if (KIND == 1 && epi == EPI_APPLY_PACK) {
-            if (NC == 32) pack_bits_direct(pr, row, col0, v); else pack_bits16_direct(pr, row, col0, v);
+            if (NC == 32) pack_bits_direct(pr, row, col0, v, args.peers); else pack_bits16_direct(pr, row, col0, v, args.peers);
           } else if (KIND == 1 && epi == EPI_APPLY_UPDATE) {
             update_weights_direct<NC>(pr, args.params, args.lr, row, col0, v);
           }

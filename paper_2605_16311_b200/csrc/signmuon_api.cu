@@ -70,11 +70,20 @@ struct signmuon_ctx {
   signmuon_config cfg;
   std::vector<signmuon_param> params;
   std::vector<ParamPlan> plan;
-  std::vector<int32_t> matrix_list, plain_list, packfb_list;
-  std::vector<uint32_t> mom_starts, plain_starts, vote_starts, packfb_starts, xv_starts, xtu_starts;
+  std::vector<int32_t> matrix_list, plain_list, packfb_list, vote_list;
+  std::vector<uint32_t> mom_starts, plain_starts, vote_starts, upd_starts, packfb_starts, xv_starts, xtu_starts;
+  uint32_t upd_blocks = 0;
   uint32_t mom_blocks = 0, plain_blocks = 0, vote_blocks = 0, packfb_blocks = 0, xv_blocks = 0, xtu_blocks = 0;
   size_t power_start_floats = 0;          // length of the start-vector array (scale = spectral)
   const float* d_power_start = nullptr;   // caller's start vectors (device)
+  int M_all = 1;                          // workers that vote (config.num_workers)
+  int Lw = 1;                             // workers this context computes (momentum, Newton-Schulz, pack)
+  int w_off = 0;                          // global index of its first worker
+  int Wm = 1;                             // Newton-Schulz batch slots of a matrix parameter's workers: Lw, or 1 under the
+                                          // Muon rule (one momentum of the mean gradient)
+  bool muon = false;                      // update_rule == SIGNMUON_RULE_MUON
+  bool lp = false;                        // local polar step in effect (never under the Muon rule)
+  bool sharded = false;                   // Lw < M_all: the payload rows of the other workers come from elsewhere
   uint64_t words_per_worker = 0;          // payload words of one worker (the bytes it would transmit / 4)
   uint64_t bits_pitch = 0;                // words between two workers' payloads in the workspace (128-byte rows)
   int64_t entries = 0;
@@ -83,6 +92,7 @@ struct signmuon_ctx {
   size_t paramdev_stride = 0;             // bytes between two copies of the parameter table
   size_t off_status = 0, off_paramdev = 0, off_lists = 0, off_bits = 0, off_vote = 0, off_tmaps = 0,
          off_problems = 0, off_tables_end = 0;
+  size_t off_list_vote = 0, off_starts_upd = 0, off_flags = 0;
   size_t off_list_matrix = 0, off_list_plain = 0, off_list_packfb = 0, off_starts_mom = 0, off_starts_plain = 0,
          off_starts_vote = 0, off_starts_packfb = 0, off_starts_xv = 0, off_starts_xtu = 0, off_agree = 0;
   // GEMM plans
@@ -115,6 +125,11 @@ struct signmuon_ctx {
   uint64_t table_clock = 0;
   int cur_table = 0;                      // slot of the step being enqueued
   uint64_t wait_limit_ns = DEFAULT_WAIT_LIMIT_NS;
+  // fused exchange: payload words are also stored into the peers' payload buffers; flags tell when they are complete
+  PeerList peers = {};                    // byte distance of every peer's payload buffer from this one
+  FlagList peer_flags = {};               // every peer's flag array
+  int my_rank = 0, n_ranks = 1;
+  uint32_t exchange_seq = 0;              // sequence number of the last published payload
   double executed_flops = 0;              // flops the scheduled tiles issue per step (known once the tile tables exist)
   int sticky = SIGNMUON_OK;
 };
@@ -195,7 +210,7 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
     const int src = k & 1, dst = (k + 1) & 1;
     for (int w = 0; w < workers; ++w) {
       // the local polar step works in its own slot (index M) so the workers' results stay readable
-      const int m = local_polar_phase ? c->cfg.num_workers : w;
+      const int m = local_polar_phase ? c->Wm : w;
       GemmProblem pr;
       std::memset(&pr, 0, sizeof(pr));
       const size_t ybytes = (size_t)pl.rows * pl.ldy * 2, qbytes = (size_t)pl.s * pl.ldq * 2;
@@ -307,12 +322,12 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         }
         const bool last = (k == K - 1);
         if (!last) pr.epi = EPI_APPLY;
-        else if (local_polar_phase) pr.epi = EPI_APPLY_UPDATE;
+        else if (local_polar_phase || c->muon) pr.epi = EPI_APPLY_UPDATE;   // W <- W - eta Y_K (local polar step; Muon rule)
         else if (pl.fused_pack) {
           pr.epi = EPI_APPLY_PACK;
           pr.store_out = keep ? 1 : 0;
           // payload word of this (param, worker): resolved at bind from off_bits
-          pr.bits_out = reinterpret_cast<uint32_t*>((size_t)m * c->bits_pitch * 4 + (size_t)pl.word_off * 4);
+          pr.bits_out = reinterpret_cast<uint32_t*>((size_t)(c->w_off + m) * c->bits_pitch * 4 + (size_t)pl.word_off * 4);
         } else pr.epi = EPI_APPLY;
       }
       out.push_back(pr);
@@ -321,7 +336,7 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
 }
 
 int plan_layout(signmuon_ctx* c) {
-  const int M = c->cfg.num_workers;
+  const int M = c->Wm;                    // batch slots of a matrix parameter: this context's own workers (1: Muon rule)
   const int K = c->cfg.ns_steps;
   size_t state = 0;
   uint64_t words = 0;
@@ -339,9 +354,9 @@ int plan_layout(signmuon_ctx* c) {
     pl.word_off = (uint32_t)words;
     words += pl.n_words;
     pl.chunks_per_worker = (uint32_t)((pl.d + MOM_CHUNK - 1) / MOM_CHUNK);
-    pl.fused_pack = (sp.kind == SIGNMUON_PARAM_MATRIX) && K > 0 && (sp.cols % 32 == 0);
+    pl.fused_pack = (sp.kind == SIGNMUON_PARAM_MATRIX) && K > 0 && (sp.cols % 32 == 0) && !c->muon;
     pl.mom_off = state;
-    state += round_up((size_t)M * pl.d * 4, ALIGN);
+    state += round_up((size_t)(sp.kind == SIGNMUON_PARAM_MATRIX ? c->Wm : c->Lw) * pl.d * 4, ALIGN);
     c->plan.push_back(pl);
     if (sp.kind == SIGNMUON_PARAM_MATRIX) c->matrix_list.push_back((int32_t)p);
     else c->plain_list.push_back((int32_t)p);
@@ -364,16 +379,32 @@ int plan_layout(signmuon_ctx* c) {
   b = 0;
   // vote kernel: blocks own VOTE_WORDS-aligned groups of the payload's word index; a parameter gets every group it
   // touches (a group shared by two parameters is visited once for each, masked)
-  for (int32_t p : c->matrix_list) {
+  if (!c->muon) c->vote_list = c->matrix_list;
+  if (c->sharded) {       // the plain parameters' vote also waits for the exchange: every parameter goes through the vote kernel
+    c->vote_list.clear();
+    for (size_t p = 0; p < c->params.size(); ++p) c->vote_list.push_back((int32_t)p);
+  }
+  for (int32_t p : c->vote_list) {
     const ParamPlan& pl = c->plan[p];
     c->vote_starts.push_back((uint32_t)b);
     b += ((uint64_t)pl.word_off + pl.n_words + VOTE_WORDS - 1) / VOTE_WORDS - pl.word_off / VOTE_WORDS;
   }
   if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
   c->vote_blocks = (uint32_t)b;
+  // update kernel: blocks of UPD_VECS 128-bit vectors (8 bf16 or 4 float32 entries each; the +-1 matrix is bf16)
+  b = 0;
+  for (int32_t p : c->vote_list) {
+    const ParamPlan& pl = c->plan[p];
+    const bool sbar = c->lp && K > 0 && pl.kind == SIGNMUON_PARAM_MATRIX;
+    const uint64_t per_block = (uint64_t)UPD_VECS * ((sbar || pl.wdtype == SIGNMUON_BF16) ? 8 : 4);
+    c->upd_starts.push_back((uint32_t)b);
+    b += ((uint64_t)pl.d + per_block - 1) / per_block;
+  }
+  if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
+  c->upd_blocks = (uint32_t)b;
   b = 0;
   for (int32_t p : c->matrix_list) {
-    if (c->plan[p].fused_pack) continue;
+    if (c->plan[p].fused_pack || c->muon) continue;     // (nothing is packed under the Muon rule)
     c->packfb_list.push_back(p);
     c->packfb_starts.push_back((uint32_t)b);
     b += (uint64_t)M * ((c->plan[p].d + PACK_CHUNK - 1) / PACK_CHUNK);
@@ -411,11 +442,14 @@ int plan_layout(signmuon_ctx* c) {
   place(c->off_list_matrix, c->matrix_list.size() * 4);
   place(c->off_list_plain, c->plain_list.size() * 4);
   place(c->off_list_packfb, c->packfb_list.size() * 4);
+  place(c->off_list_vote, c->vote_list.size() * 4);
   place(c->off_starts_mom, c->mom_starts.size() * 4);
   place(c->off_starts_plain, c->plain_starts.size() * 4);
   place(c->off_starts_vote, c->vote_starts.size() * 4);
+  place(c->off_starts_upd, c->upd_starts.size() * 4);
   place(c->off_starts_packfb, c->packfb_starts.size() * 4);
-  place(c->off_agree, (size_t)M * 8);
+  place(c->off_agree, (size_t)c->M_all * 8);
+  place(c->off_flags, 64 * 4);
   place(c->off_starts_xv, c->xv_starts.size() * 4);
   place(c->off_starts_xtu, c->xtu_starts.size() * 4);
   for (int32_t p : c->matrix_list) {
@@ -428,7 +462,7 @@ int plan_layout(signmuon_ctx* c) {
       pl.pi_scal_off = off; off += round_up((size_t)M * 8, ALIGN);
     }
   }
-  c->off_bits = off; off += round_up((size_t)M * c->bits_pitch * 4, ALIGN);
+  c->off_bits = off; off += round_up((size_t)c->M_all * c->bits_pitch * 4, ALIGN);
   c->off_vote = off; off += round_up((size_t)c->bits_pitch * 4, ALIGN);
   // tensor maps
   c->off_tmaps = off;
@@ -439,7 +473,7 @@ int plan_layout(signmuon_ctx* c) {
   // Newton-Schulz operand buffers
   for (int32_t p : c->matrix_list) {
     ParamPlan& pl = c->plan[p];
-    const size_t slots = (size_t)M + (c->cfg.local_polar ? 1 : 0);
+    const size_t slots = (size_t)M + (c->lp ? 1 : 0);
     const size_t ybytes = round_up(slots * pl.rows * pl.ldy * 2, 1024);
     pl.y_off[0] = off; off += ybytes;
     pl.y_off[1] = off; off += ybytes;
@@ -461,7 +495,7 @@ int plan_layout(signmuon_ctx* c) {
       c->ns_launches.push_back({c->problems.size(), 1});
       append_problems(c, c->problems, false, k, K, M, false);
     }
-    if (c->cfg.local_polar) {
+    if (c->lp) {
       for (int k = 0; k < K; ++k) {
         c->lp_launches.push_back({c->problems.size(), 2});
         append_problems(c, c->problems, true, k, K, 1, true);
@@ -495,7 +529,7 @@ int plan_layout(signmuon_ctx* c) {
   for (ParamPlan& pl : c->plan) { pl.stage_w_off = st; st += round_up((size_t)pl.d * dtype_size(pl.wdtype), ALIGN); }
   c->stage_g_base = st;
   size_t gs = 0;
-  for (ParamPlan& pl : c->plan) { pl.stage_g_off = gs; gs += round_up((size_t)M * pl.d * dtype_size(pl.gdtype), ALIGN); }
+  for (ParamPlan& pl : c->plan) { pl.stage_g_off = gs; gs += round_up((size_t)c->Lw * pl.d * dtype_size(pl.gdtype), ALIGN); }
   c->stage_g_set_bytes = gs;
   c->staging_bytes = st + 2 * gs;
   return SIGNMUON_OK;
@@ -562,25 +596,12 @@ void launch_tc(const GemmLaunchArgs& a, int lists, cudaStream_t s) {
 // Shapes of the tensor-core kernel in use.  Gram launches have a long K loop and a small bf16 output:
 // deep operand ring, two half-size output buffers.  Apply launches have a short K loop and move 8 bytes
 // per entry through the epilogue: shallower operand ring, four chunk buffers (two C loads in flight).
-// Operand stages / chunk buffers of each shape; overridable at compile time for tuning runs.
-#ifndef NS_GRAM_STAGES
-#define NS_GRAM_STAGES 5
-#endif
-#ifndef NS_GRAM_BUFS
-#define NS_GRAM_BUFS 2
-#endif
-#ifndef NS_APPLY_STAGES
-#define NS_APPLY_STAGES 3
-#endif
-#ifndef NS_APPLY_BUFS
-#define NS_APPLY_BUFS 4
-#endif
 // (BN, operand stages, chunk buffers, CTAs per tile, kind)
-#define NS_GEMM_PAIR_GRAM 256, NS_GRAM_STAGES, NS_GRAM_BUFS, 2, 0
-#define NS_GEMM_PAIR_APPLY 256, NS_APPLY_STAGES, NS_APPLY_BUFS, 2, 1
+#define NS_GEMM_PAIR_GRAM 256, 5, 2, 2, 0
+#define NS_GEMM_PAIR_APPLY 256, 3, 4, 2, 1
 #define NS_GEMM_PAIR_APPLY_LONGK 256, 4, 3, 2, 1   /* long contraction: the operand ring matters more than the chunk ring */
-#define NS_GEMM_ONE_GRAM 128, NS_GRAM_STAGES, NS_GRAM_BUFS, 1, 0
-#define NS_GEMM_ONE_APPLY 128, NS_APPLY_STAGES, NS_APPLY_BUFS, 1, 1
+#define NS_GEMM_ONE_GRAM 128, 5, 2, 1, 0
+#define NS_GEMM_ONE_APPLY 128, 3, 4, 1, 1
 
 template <int BN, int STAGES, int EPI_BUFS, int CTAS, int KIND>
 bool opt_in_smem() {
@@ -625,7 +646,7 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
   const TileEntry* tiles = reinterpret_cast<const TileEntry*>(c->d_ws + tt.tiles_off);
   const ParamDev* pd = cur_paramdev(c);
   if (c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) {
-    ns_gemm_simt_kernel<<<(unsigned)tt.tiles.size(), 128, 0, s>>>(probs, tiles, tt.bn, pd, lr);
+    ns_gemm_simt_kernel<<<(unsigned)tt.tiles.size(), 128, 0, s>>>(probs, tiles, tt.bn, pd, lr, c->peers);
     return;
   }
   GemmLaunchArgs a;
@@ -637,6 +658,7 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
   a.status = reinterpret_cast<uint32_t*>(c->d_ws + c->off_status);
   a.lr = lr;
   a.wait_limit_ns = c->wait_limit_ns;
+  a.peers = c->peers;
   const bool gram = (lp.tile_table & 1) == 0;
   if (tt.ctas == 2) {
     if (gram) launch_tc<NS_GEMM_PAIR_GRAM>(a, tt.grid, s);
@@ -647,14 +669,20 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
   }
 }
 
+// Vote over `rows` payload rows starting at `src` (default: all workers' rows of the payload buffer), then the
+// update from the vote words.
 template <int PLANES>
-void launch_vote(signmuon_ctx* c, float lr, int write_sbar, cudaStream_t s) {
-  vote_update_kernel<PLANES><<<c->vote_blocks, VOTE_THREADS, 0, s>>>(
-      cur_paramdev(c),
-      reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_matrix),
-      reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_vote), (int)c->matrix_list.size(),
-      c->cfg.num_workers, lr, write_sbar, reinterpret_cast<const uint32_t*>(c->d_ws + c->off_bits),
-      reinterpret_cast<uint32_t*>(c->d_ws + c->off_vote), (int64_t)c->bits_pitch);
+void launch_vote(signmuon_ctx* c, float lr, int write_sbar, cudaStream_t s, const uint32_t* src = nullptr, int rows = 0) {
+  const ParamDev* pd = cur_paramdev(c);
+  const int32_t* list = reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_vote);
+  uint32_t* vote = reinterpret_cast<uint32_t*>(c->d_ws + c->off_vote);
+  const int n = (int)c->vote_list.size();
+  if (src != vote)      // (vote words computed elsewhere: only the update remains)
+    vote_kernel<PLANES><<<c->vote_blocks, VOTE_THREADS, 0, s>>>(
+        pd, list, reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_vote), n, src ? rows : c->M_all,
+        src ? src : reinterpret_cast<const uint32_t*>(c->d_ws + c->off_bits), vote, (int64_t)c->bits_pitch);
+  update_kernel<<<c->upd_blocks, EW_THREADS, 0, s>>>(
+      pd, list, reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_upd), n, c->Wm, lr, write_sbar, vote);
 }
 
 void invalidate_tables(signmuon_ctx* c) {
@@ -716,8 +744,10 @@ int upload_params(signmuon_ctx* c, void* const* weights, const void* const* grad
   return SIGNMUON_OK;
 }
 
+// `vote_from_words`: the vote words were produced elsewhere (from all-reduced sign sums): the vote stage then only
+// maps them to the update (a one-row "vote" over the vote words themselves).
 int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const void* const* grads, float lr,
-                    cudaStream_t s) {
+                    cudaStream_t s, bool vote_from_words = false) {
   if (!c) return SIGNMUON_ERR_INVALID_ARG;
   if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
   if (c->sticky != SIGNMUON_OK) return c->sticky;
@@ -726,7 +756,7 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
   if (lr < 0.f) lr = c->cfg.lr;
   int rc = upload_params(c, weights, grads, s);
   if (rc != SIGNMUON_OK) return rc;
-  const int M = c->cfg.num_workers, K = c->cfg.ns_steps;
+  const int M = c->Wm, K = c->cfg.ns_steps;      // M: batch slots of the matrix parameters (own workers; 1: Muon rule)
   const ParamDev* pd = cur_paramdev(c);
   uint32_t* bits = reinterpret_cast<uint32_t*>(c->d_ws + c->off_bits);
   uint32_t* vote = reinterpret_cast<uint32_t*>(c->d_ws + c->off_vote);
@@ -760,8 +790,9 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
     if (np) {
       plain_params_kernel<<<c->plain_blocks, EW_THREADS, 0, s>>>(
           pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_plain),
-          reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_plain), np, M, c->cfg.momentum,
-          c->cfg.weight_decay, lr, bits, vote, (int64_t)c->bits_pitch);
+          reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_plain), np, c->Lw, c->cfg.momentum,
+          c->cfg.weight_decay, lr, bits + (size_t)c->w_off * c->bits_pitch, vote, (int64_t)c->bits_pitch,
+          c->sharded ? 0 : 1, c->peers);
     }
   }
   if ((mask & SIGNMUON_STAGE_NS) && nm) {
@@ -770,23 +801,35 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
       pack_kernel<<<c->packfb_blocks, EW_THREADS, 0, s>>>(
           pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_packfb),
           reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_packfb), (int)c->packfb_list.size(), K & 1,
-          K == 0 ? 1 : 0, bits, (int64_t)c->bits_pitch);
+          K == 0 ? 1 : 0, bits + (size_t)c->w_off * c->bits_pitch, (int64_t)c->bits_pitch, c->peers);
     }
   }
-  const bool lp_ns = c->cfg.local_polar && K > 0;
-  if ((mask & SIGNMUON_STAGE_VOTE) && nm) {
+  if ((mask & SIGNMUON_STAGE_NS) && c->peer_flags.n > 0) {
+    // fused exchange: every payload word of this step is stored (here and in the peers' buffers): tell the peers
+    ++c->exchange_seq;
+    publish_payload_kernel<<<1, 32, 0, s>>>(c->peer_flags, c->my_rank, c->exchange_seq);
+  }
+  if ((mask & SIGNMUON_STAGE_VOTE) && c->peer_flags.n > 0) {
+    // ... and wait (bounded) until every peer has told this GPU the same
+    await_payloads_kernel<<<1, 64, 0, s>>>(reinterpret_cast<const uint32_t*>(c->d_ws + c->off_flags), c->n_ranks,
+                                           c->my_rank, c->exchange_seq, c->wait_limit_ns,
+                                           reinterpret_cast<uint32_t*>(c->d_ws + c->off_status));
+  }
+  const bool lp_ns = c->lp && K > 0;
+  if ((mask & SIGNMUON_STAGE_VOTE) && !c->vote_list.empty()) {
     // local polar with K = 0 degenerates to S / ||S||_F: plain update with the Eq. 2 scale
     const int write_sbar = lp_ns ? 1 : 0;
-    if (M <= 7) launch_vote<3>(c, lr, write_sbar, s);
-    else if (M <= 63) launch_vote<6>(c, lr, write_sbar, s);
+    if (vote_from_words) launch_vote<3>(c, lr, write_sbar, s, vote, 1);      // update only
+    else if (c->M_all <= 7) launch_vote<3>(c, lr, write_sbar, s);
+    else if (c->M_all <= 63) launch_vote<6>(c, lr, write_sbar, s);
     else launch_vote<8>(c, lr, write_sbar, s);
   }
   if ((mask & SIGNMUON_STAGE_VOTE) && (c->cfg.flags & SIGNMUON_FLAG_SIGN_AGREEMENT)) {
     // after the vote of the matrix parameters (the plain parameters voted in the momentum stage)
     unsigned long long* agree = reinterpret_cast<unsigned long long*>(c->d_ws + c->off_agree);
-    if (cudaMemsetAsync(agree, 0, (size_t)M * 8, s) != cudaSuccess) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+    if (cudaMemsetAsync(agree, 0, (size_t)c->M_all * 8, s) != cudaSuccess) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
     const unsigned gx = (unsigned)std::min<uint64_t>((c->words_per_worker + EW_THREADS - 1) / EW_THREADS, 1024);
-    sign_agreement_kernel<<<dim3(gx, (unsigned)M), EW_THREADS, 0, s>>>(bits, vote, (int64_t)c->words_per_worker,
+    sign_agreement_kernel<<<dim3(gx, (unsigned)c->M_all), EW_THREADS, 0, s>>>(bits, vote, (int64_t)c->words_per_worker,
                                                                              (int64_t)c->bits_pitch, agree);
   }
   if ((mask & SIGNMUON_STAGE_LOCAL_POLAR) && nm && lp_ns) {
@@ -813,6 +856,15 @@ int signmuon_create(const signmuon_config* config, signmuon_ctx** out) {
   if (config->local_polar != 0 && config->local_polar != 1) return SIGNMUON_ERR_INVALID_ARG;
   if (config->ns_scale != SIGNMUON_SCALE_FRO && config->ns_scale != SIGNMUON_SCALE_SPECTRAL) return SIGNMUON_ERR_INVALID_ARG;
   if (config->power_iters < 0 || config->power_iters > 64) return SIGNMUON_ERR_INVALID_ARG;
+  if (config->local_workers < 0 || config->local_workers > config->num_workers) return SIGNMUON_ERR_INVALID_ARG;
+  if (config->update_rule != SIGNMUON_RULE_SIGNMUON && config->update_rule != SIGNMUON_RULE_MUON) return SIGNMUON_ERR_INVALID_ARG;
+  // Muon averages float gradients: with the workers on several GPUs that is the caller's all-reduce (then M = 1 here)
+  if (config->update_rule == SIGNMUON_RULE_MUON && config->local_workers > 0 && config->local_workers < config->num_workers)
+    return SIGNMUON_ERR_INVALID_ARG;
+  if (config->update_rule == SIGNMUON_RULE_MUON && config->ns_steps == 0) return SIGNMUON_ERR_INVALID_ARG;   // the update lives in the last Newton-Schulz epilogue
+  if (config->local_workers > 0 &&
+      (config->worker_offset < 0 || config->worker_offset + config->local_workers > config->num_workers))
+    return SIGNMUON_ERR_INVALID_ARG;
   for (int i = 0; i < config->num_params; ++i) {
     const signmuon_param& p = config->params[i];
     if (p.rows < 1 || p.cols < 1 || p.rows > (1 << 24) || p.cols > (1 << 24)) return SIGNMUON_ERR_BAD_SHAPE;
@@ -827,6 +879,13 @@ int signmuon_create(const signmuon_config* config, signmuon_ctx** out) {
   if (!c) return SIGNMUON_ERR_NO_MEMORY;
   c->cfg = *config;
   if (!(c->cfg.eps > 0.f)) c->cfg.eps = 1e-12f;
+  c->M_all = config->num_workers;
+  c->Lw = config->local_workers > 0 ? config->local_workers : config->num_workers;
+  c->w_off = config->local_workers > 0 ? config->worker_offset : 0;
+  c->sharded = c->Lw < c->M_all;
+  c->muon = config->update_rule == SIGNMUON_RULE_MUON;
+  c->Wm = c->muon ? 1 : c->Lw;
+  c->lp = config->local_polar != 0 && !c->muon;
   c->params.assign(config->params, config->params + config->num_params);
   c->cfg.params = nullptr;
   int rc = plan_layout(c);
@@ -870,7 +929,7 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     if (!sok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
   }
   c->host_steps = 0;
-  const int M = c->cfg.num_workers;
+  const int M = c->Wm;
   if (!c->h_tables) {   // pinned host mirrors of the parameter tables and the events that guard their reuse
     void* hp = nullptr;
     if (cudaHostAlloc(&hp, PARAM_TABLES * c->params.size() * sizeof(ParamDev), cudaHostAllocDefault) != cudaSuccess) {
@@ -891,8 +950,12 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     return cudaMemcpyAsync(c->d_ws + off, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
   };
   bool ok = cudaMemsetAsync(c->d_ws + c->off_status, 0, ALIGN, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->d_ws + c->off_flags, 0, 64 * 4, s) == cudaSuccess;
+  c->peers.n = 0;            // peers are attached after bind (their addresses refer to bound buffers)
+  c->peer_flags.n = 0;
+  c->exchange_seq = 0;
   if (zero_state) ok = ok && cudaMemsetAsync(c->d_state, 0, c->state_bytes, s) == cudaSuccess;
-  ok = ok && cudaMemsetAsync(c->d_ws + c->off_bits, 0, (size_t)M * c->bits_pitch * 4, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->d_ws + c->off_bits, 0, (size_t)c->M_all * c->bits_pitch * 4, s) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->d_ws + c->off_vote, 0, (size_t)c->bits_pitch * 4, s) == cudaSuccess;
 
   // parameter table (W/G filled in at the first step)
@@ -919,17 +982,20 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     d.kind = pl.kind; d.wdtype = pl.wdtype; d.gdtype = pl.gdtype;
     d.word_off = pl.word_off; d.n_words = pl.n_words; d.chunks_per_worker = pl.chunks_per_worker;
     const bool eq2 = c->cfg.update_scale == 1 ||
-                     (pl.kind == SIGNMUON_PARAM_MATRIX && c->cfg.local_polar && c->cfg.ns_steps == 0);
+                     (pl.kind == SIGNMUON_PARAM_MATRIX && c->lp && c->cfg.ns_steps == 0);
     d.upd_scale = eq2 ? (float)(1.0 / std::sqrt((double)pl.rows * (double)pl.cols)) : 1.f;
     d.vec_ok = (pl.d % 8 == 0 && pl.ldy == pl.cols) ? 1 : 0;
+    d.avg_workers = (c->muon && pl.kind == SIGNMUON_PARAM_MATRIX) ? c->Lw : 1;
   }
   invalidate_tables(c);
   ok = ok && up(c->off_list_matrix, c->matrix_list.data(), c->matrix_list.size() * 4);
   ok = ok && up(c->off_list_plain, c->plain_list.data(), c->plain_list.size() * 4);
   ok = ok && up(c->off_list_packfb, c->packfb_list.data(), c->packfb_list.size() * 4);
+  ok = ok && up(c->off_list_vote, c->vote_list.data(), c->vote_list.size() * 4);
   ok = ok && up(c->off_starts_mom, c->mom_starts.data(), c->mom_starts.size() * 4);
   ok = ok && up(c->off_starts_plain, c->plain_starts.data(), c->plain_starts.size() * 4);
   ok = ok && up(c->off_starts_vote, c->vote_starts.data(), c->vote_starts.size() * 4);
+  ok = ok && up(c->off_starts_upd, c->upd_starts.data(), c->upd_starts.size() * 4);
   ok = ok && up(c->off_starts_packfb, c->packfb_starts.data(), c->packfb_starts.size() * 4);
   ok = ok && up(c->off_starts_xv, c->xv_starts.data(), c->xv_starts.size() * 4);
   ok = ok && up(c->off_starts_xtu, c->xtu_starts.data(), c->xtu_starts.size() * 4);
@@ -974,7 +1040,7 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
       const ParamPlan& pl = c->plan[p];
       CUtensorMap* mp = maps.data() + pl.tmap_base;
       const uint32_t bn = 128;   // box rows of a K-major B operand = tile width
-      const uint64_t slots = (uint64_t)M + (c->cfg.local_polar ? 1 : 0);
+      const uint64_t slots = (uint64_t)M + (c->lp ? 1 : 0);
       for (int buf = 0; buf < 2; ++buf) {
         void* y = c->d_ws + pl.y_off[buf];
         const uint64_t yb = (uint64_t)pl.rows * pl.ldy;
@@ -1032,6 +1098,7 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
 }
 
 int signmuon_step(signmuon_ctx* c, void* const* weights, const void* const* grads, float lr, void* cuda_stream) {
+  if (c && c->sharded) return SIGNMUON_ERR_INVALID_ARG;   // the payload exchange belongs between the stages
   return run_stages_impl(c, SIGNMUON_STAGE_ALL, weights, grads, lr, reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -1047,8 +1114,9 @@ int signmuon_step_host(signmuon_ctx* c, void* const* host_weights, const void* c
   if (!c->bound || !c->d_staging) return SIGNMUON_ERR_NOT_BOUND;
   if (c->sticky != SIGNMUON_OK) return c->sticky;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
-  const int M = c->cfg.num_workers;
+  const int M = c->Lw;
   const size_t n = c->params.size();
+  if (c->sharded) return SIGNMUON_ERR_INVALID_ARG;     // the exchange sits between the stages: see signmuon_step
   for (size_t p = 0; p < n; ++p)
     if (!host_weights[p] || !host_grads[p]) return SIGNMUON_ERR_INVALID_ARG;
   const int set = (int)(c->host_steps & 1);
@@ -1097,6 +1165,98 @@ int signmuon_packed_payload(const signmuon_ctx* c, int32_t worker, const uint32_
   return SIGNMUON_OK;
 }
 
+int signmuon_payload_buffer(const signmuon_ctx* c, uint32_t** dev_ptr, size_t* row_pitch_bytes, int32_t* rows) {
+  if (!c) return SIGNMUON_ERR_INVALID_ARG;
+  if (row_pitch_bytes) *row_pitch_bytes = (size_t)c->bits_pitch * 4;
+  if (rows) *rows = c->M_all;
+  if (dev_ptr) {
+    if (!c->bound) { *dev_ptr = nullptr; return SIGNMUON_ERR_NOT_BOUND; }
+    *dev_ptr = reinterpret_cast<uint32_t*>(c->d_ws + c->off_bits);
+  }
+  return SIGNMUON_OK;
+}
+
+int signmuon_exchange_flags(const signmuon_ctx* c, uint32_t** dev_ptr) {
+  if (!c || !dev_ptr) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) { *dev_ptr = nullptr; return SIGNMUON_ERR_NOT_BOUND; }
+  *dev_ptr = reinterpret_cast<uint32_t*>(c->d_ws + c->off_flags);
+  return SIGNMUON_OK;
+}
+
+int signmuon_set_payload_peers(signmuon_ctx* c, int32_t my_rank, int32_t num_ranks, int32_t num_peers,
+                               uint32_t* const* peer_payload_buffers, uint32_t* const* peer_flags) {
+  if (!c) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  if (num_peers < 0 || num_peers > MAX_PAYLOAD_PEERS || num_ranks < 1 || num_ranks > 64 || my_rank < 0 ||
+      my_rank >= num_ranks || num_peers >= num_ranks + (num_peers == 0 ? 1 : 0))
+    return SIGNMUON_ERR_INVALID_ARG;
+  if (num_peers > 0 && (!peer_payload_buffers || !peer_flags)) return SIGNMUON_ERR_INVALID_ARG;
+  PeerList pl = {};
+  FlagList fl = {};
+  const char* own = reinterpret_cast<const char*>(c->d_ws + c->off_bits);
+  for (int p = 0; p < num_peers; ++p) {
+    if (!peer_payload_buffers[p] || !peer_flags[p]) return SIGNMUON_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(peer_payload_buffers[p]) & 127) || (reinterpret_cast<uintptr_t>(peer_flags[p]) & 3))
+      return SIGNMUON_ERR_MISALIGNED;
+    pl.delta[p] = reinterpret_cast<const char*>(peer_payload_buffers[p]) - own;
+    fl.flags[p] = peer_flags[p];
+  }
+  pl.n = fl.n = num_peers;
+  c->peers = pl;
+  c->peer_flags = fl;
+  c->my_rank = my_rank;
+  c->n_ranks = num_ranks;
+  return SIGNMUON_OK;
+}
+
+int signmuon_vote_update(signmuon_ctx* c, const uint32_t* const* payloads, void* const* weights,
+                         const void* const* grads, float lr, void* cuda_stream) {
+  if (!c || !payloads) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  if (c->sticky != SIGNMUON_OK) return c->sticky;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  uint32_t* rows = reinterpret_cast<uint32_t*>(c->d_ws + c->off_bits);
+  for (int m = 0; m < c->M_all; ++m) {
+    const uint32_t* src = payloads[m];
+    uint32_t* dst = rows + (size_t)m * c->bits_pitch;
+    if (!src || src == dst) continue;
+    if (reinterpret_cast<uintptr_t>(src) & 3) return SIGNMUON_ERR_MISALIGNED;
+    if (cudaMemcpyAsync(dst, src, (size_t)c->words_per_worker * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess) {
+      c->sticky = SIGNMUON_ERR_CUDA;
+      return c->sticky;
+    }
+  }
+  return run_stages_impl(c, SIGNMUON_STAGE_VOTE | SIGNMUON_STAGE_LOCAL_POLAR, weights, grads, lr, s);
+}
+
+int signmuon_local_sign_sum(signmuon_ctx* c, int8_t* dev_sums, size_t bytes, void* cuda_stream) {
+  if (!c || !dev_sums) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  if (c->sticky != SIGNMUON_OK) return c->sticky;
+  if (c->M_all > 127) return SIGNMUON_ERR_INVALID_ARG;              // the reduced sums must fit int8
+  if (bytes < (size_t)c->words_per_worker * 32) return SIGNMUON_ERR_BUFFER_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(dev_sums) & 15) return SIGNMUON_ERR_MISALIGNED;
+  const uint32_t* rows = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_bits) + (size_t)c->w_off * c->bits_pitch;
+  const unsigned blocks = (unsigned)((c->words_per_worker + EW_THREADS - 1) / EW_THREADS);
+  sign_sum_kernel<<<blocks, EW_THREADS, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
+      rows, (int64_t)c->bits_pitch, (int64_t)c->words_per_worker, c->Lw, dev_sums);
+  return check_launch(c);
+}
+
+int signmuon_vote_update_from_sums(signmuon_ctx* c, const int8_t* dev_sums, size_t bytes, void* const* weights,
+                                   const void* const* grads, float lr, void* cuda_stream) {
+  if (!c || !dev_sums) return SIGNMUON_ERR_INVALID_ARG;
+  if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
+  if (c->sticky != SIGNMUON_OK) return c->sticky;
+  if (bytes < (size_t)c->words_per_worker * 32) return SIGNMUON_ERR_BUFFER_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(dev_sums) & 15) return SIGNMUON_ERR_MISALIGNED;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const unsigned blocks = (unsigned)((c->words_per_worker + EW_THREADS - 1) / EW_THREADS);
+  sums_to_vote_kernel<<<blocks, EW_THREADS, 0, s>>>(dev_sums, (int64_t)c->words_per_worker,
+                                                    reinterpret_cast<uint32_t*>(c->d_ws + c->off_vote));
+  return run_stages_impl(c, SIGNMUON_STAGE_VOTE | SIGNMUON_STAGE_LOCAL_POLAR, weights, grads, lr, s, true);
+}
+
 int signmuon_payload_segment(const signmuon_ctx* c, int32_t param, size_t* word_offset, size_t* words) {
   if (!c || param < 0 || param >= (int32_t)c->params.size()) return SIGNMUON_ERR_INVALID_ARG;
   if (word_offset) *word_offset = c->plan[param].word_off;
@@ -1110,17 +1270,26 @@ int signmuon_debug_tap(const signmuon_ctx* c, int32_t what, int32_t param, int32
   if (worker < 0 || worker >= c->cfg.num_workers) return SIGNMUON_ERR_INVALID_ARG;
   if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
   const ParamPlan& pl = c->plan[param];
+  // momentum, Y_K and norm factors exist for this context's own workers only
+  const bool own = worker >= c->w_off && worker < c->w_off + c->Lw;
+  if (!own && (what == SIGNMUON_TAP_MOMENTUM || what == SIGNMUON_TAP_POLAR || what == SIGNMUON_TAP_NORM))
+    return SIGNMUON_ERR_INVALID_ARG;
+  const int32_t lw = worker - c->w_off;                 // index among the own workers
+  if (c->muon && pl.kind == SIGNMUON_PARAM_MATRIX) {    // one momentum, nothing packed or voted
+    if (what != SIGNMUON_TAP_MOMENTUM && what != SIGNMUON_TAP_NORM) return SIGNMUON_ERR_INVALID_ARG;
+    if (lw != 0) return SIGNMUON_ERR_INVALID_ARG;
+  }
   size_t nbytes = 0;
   int64_t pitch = pl.cols;
   const void* ptr = nullptr;
   switch (what) {
     case SIGNMUON_TAP_MOMENTUM:
-      ptr = c->d_state + pl.mom_off + (size_t)worker * pl.d * 4; nbytes = (size_t)pl.d * 4; break;
+      ptr = c->d_state + pl.mom_off + (size_t)lw * pl.d * 4; nbytes = (size_t)pl.d * 4; break;
     case SIGNMUON_TAP_POLAR: {
       if (pl.kind != SIGNMUON_PARAM_MATRIX) return SIGNMUON_ERR_INVALID_ARG;
       if (!(c->cfg.flags & SIGNMUON_FLAG_KEEP_POLAR) && pl.fused_pack) return SIGNMUON_ERR_INVALID_ARG;
       const size_t yb = (size_t)pl.rows * pl.ldy * 2;
-      ptr = c->d_ws + pl.y_off[c->cfg.ns_steps & 1] + (size_t)worker * yb; nbytes = yb; pitch = pl.ldy; break;
+      ptr = c->d_ws + pl.y_off[c->cfg.ns_steps & 1] + (size_t)lw * yb; nbytes = yb; pitch = pl.ldy; break;
     }
     case SIGNMUON_TAP_VOTE_BITS:
       ptr = c->d_ws + c->off_vote + (size_t)pl.word_off * 4; nbytes = (size_t)pl.n_words * 4; break;
@@ -1129,7 +1298,7 @@ int signmuon_debug_tap(const signmuon_ctx* c, int32_t what, int32_t param, int32
       nbytes = (size_t)pl.n_words * 4; break;
     case SIGNMUON_TAP_NORM:
       if (pl.kind != SIGNMUON_PARAM_MATRIX) return SIGNMUON_ERR_INVALID_ARG;
-      ptr = c->d_ws + pl.scales_off + (size_t)worker * 8; nbytes = 8; break;
+      ptr = c->d_ws + pl.scales_off + (size_t)lw * 8; nbytes = 8; break;
     default: return SIGNMUON_ERR_INVALID_ARG;
   }
   *dev_ptr = ptr;
@@ -1201,7 +1370,7 @@ int signmuon_sign_agreement(signmuon_ctx* c, uint64_t* host_agree, uint64_t* hos
   if (!(c->cfg.flags & SIGNMUON_FLAG_SIGN_AGREEMENT)) return SIGNMUON_ERR_INVALID_ARG;
   if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
-  const int M = c->cfg.num_workers;
+  const int M = c->M_all;
   std::vector<unsigned long long> raw((size_t)M);
   if (cudaMemcpyAsync(raw.data(), c->d_ws + c->off_agree, (size_t)M * 8, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
       cudaStreamSynchronize(s) != cudaSuccess) {
@@ -1220,8 +1389,10 @@ int signmuon_launches_per_step(const signmuon_ctx* c, int32_t* launches) {
   const bool nm = !c->matrix_list.empty();
   if (nm) n += 1 + (c->power_start_floats ? 3 + 4 * c->cfg.power_iters : 1);   // momentum + norms (or power iteration)
   if (!c->plain_list.empty()) n += 1;
-  if (nm) n += (int)c->ns_launches.size() + (c->packfb_blocks ? 1 : 0) + 1;   // NS, fallback pack, vote
-  if (nm && c->cfg.local_polar && c->cfg.ns_steps > 0) n += (int)c->lp_launches.size();
+  if (nm) n += (int)c->ns_launches.size() + (c->packfb_blocks ? 1 : 0);       // NS, fallback pack
+  if (!c->vote_list.empty()) n += 2;                                          // vote, update
+  if (nm && c->lp && c->cfg.ns_steps > 0) n += (int)c->lp_launches.size();
+  if (c->peer_flags.n > 0) n += 2;                                            // publish, await (fused exchange)
   if (c->cfg.flags & SIGNMUON_FLAG_SIGN_AGREEMENT) n += 1;
   *launches = n;
   return SIGNMUON_OK;
@@ -1233,7 +1404,7 @@ int signmuon_ns_flops_per_step(const signmuon_ctx* c, double* flops) {
   for (int32_t p : c->matrix_list) {
     const ParamPlan& pl = c->plan[p];
     f += 4.0 * (double)pl.s * (double)pl.s * (double)pl.l * c->cfg.ns_steps *
-         (c->cfg.num_workers + (c->cfg.local_polar ? 1 : 0));
+         (c->Wm + (c->lp ? 1 : 0));
   }
   *flops = f;
   return SIGNMUON_OK;

@@ -125,10 +125,10 @@ def sweep_shapes() -> List[Tuple[int, int]]:
     return sq + rect
 
 
-def config5(rows: int, cols: int, num_workers: int, ns_steps: int = 5) -> Workload:
-    return Workload(f"c5_sweep_{rows}x{cols}_M{num_workers}_K{ns_steps}",
+def config5(rows: int, cols: int, num_workers: int, ns_steps: int = 5, local_polar: bool = False) -> Workload:
+    return Workload(f"c5_sweep_{rows}x{cols}_M{num_workers}_K{ns_steps}" + ("_lp" if local_polar else ""),
                     [Param(rows, cols, "matrix", "bf16", "w")], num_workers=num_workers, lr=1e-3,
-                    ns_steps=ns_steps, local_polar=False, steps=3, signal_std=1.0, noise_std=1.0,
+                    ns_steps=ns_steps, local_polar=local_polar, steps=3, signal_std=1.0, noise_std=1.0,
                     weight_std=0.02, config_id=5)
 
 
@@ -152,12 +152,18 @@ def by_name(name: str) -> Workload:
         wl.params = [p for p in wl.params if p.kind == kind]
         wl.name = name
         return wl
-    if name.startswith("c5:"):           # c5:ROWSxCOLS:M[:K]
+    if name in ("c2_short256", "c2_long"):   # the ResNet-50 matrices with a short side <= 256 / above (profiling cases)
+        wl = config2()
+        small = name == "c2_short256"
+        wl.params = [p for p in wl.params if (min(p.rows, p.cols) <= 256) == small]
+        wl.name = name
+        return wl
+    if name.startswith("c5:") or name.startswith("c5lp:"):           # c5:ROWSxCOLS:M[:K]; c5lp: local polar step on
         parts = name.split(":")
         r, c = (int(v) for v in parts[1].split("x"))
         m = int(parts[2])
         k = int(parts[3]) if len(parts) > 3 else 5
-        return config5(r, c, m, k)
+        return config5(r, c, m, k, local_polar=parts[0] == "c5lp")
     raise KeyError(name)
 
 

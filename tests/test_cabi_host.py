@@ -101,8 +101,8 @@ def test_ragged_parameter_pads_to_words():
     _, nbytes, entries = B.signmuon_packed_payload(ctx, 1, want_ptr=False)
     assert entries == 38 and nbytes == 4 * (2 + 1)
     assert B.signmuon_payload_segment(ctx, 1) == (2, 1)
-    # momentum, norms, 2x2 NS products, fallback pack (11 columns do not fill words), vote, plain kernel
-    assert B.signmuon_launches_per_step(ctx) == 2 + 1 + 4 + 1 + 1
+    # momentum, norms, plain kernel, 2x2 NS products, fallback pack (11 columns do not fill words), vote, update
+    assert B.signmuon_launches_per_step(ctx) == 2 + 1 + 4 + 1 + 2
     B.signmuon_destroy(ctx)
 
 
@@ -122,7 +122,7 @@ def test_power_start_layout_and_errors():
     assert lib.signmuon_power_start_segment(ctx, 1, None, None) == -1      # plain parameter
     assert lib.signmuon_set_power_start(ctx, C.c_void_p(4096), 54) == -3     # not bound yet
     # momentum, start norm + 2 rounds x 4 + final matvec + sigma, 5 x 2 NS products, fallback pack, vote, plain kernel
-    assert B.signmuon_launches_per_step(ctx) == 1 + (3 + 8) + 10 + 1 + 1 + 1
+    assert B.signmuon_launches_per_step(ctx) == 1 + (3 + 8) + 10 + 1 + 2 + 1
     B.signmuon_destroy(ctx)
     for kw in (dict(ns_scale=2), dict(ns_scale=-1), dict(power_iters=-1), dict(power_iters=65)):
         cfg = _cfg([(64, 64, 0, 0, 0)])
@@ -156,3 +156,28 @@ def test_header_is_plain_c(tmp_path):
     out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split(maxsplit=2)
     assert out[0] == "512" and out[1] == "4096"          # 64 x 64 entries, one bit each
     assert out[2].startswith("a bounded")
+
+
+def test_worker_shard_arguments_and_payload_buffer_layout():
+    """A context may compute a block of the workers only (the others' payload rows arrive by the exchange):
+    argument checks, state sized for the own workers, payload buffer with one 128-byte-aligned row per worker."""
+    lib = B.load_library()
+    params = [(64, 96, 0, 0, 0), (1, 40, 1, 0, 0)]
+    full = B.signmuon_create(params, 8, 0.9, 1e-3, 5, False)
+    part = B.signmuon_create(params, 8, 0.9, 1e-3, 5, False, worker_offset=4, local_workers=2)
+    st_full, _, _ = B.signmuon_state_bytes(full)
+    st_part, _, _ = B.signmuon_state_bytes(part)
+    assert st_part == 2 * 64 * 96 * 4 + 512 and st_full == 8 * 64 * 96 * 4 + 1280    # momenta of 2 of the 8 workers (256-byte slabs)
+    _, pitch, rows = B.signmuon_payload_buffer(part, want_ptr=False)
+    _, nbytes, _ = B.signmuon_packed_payload(part, 7, want_ptr=False)
+    assert rows == 8 and pitch % 128 == 0 and pitch >= nbytes == 4 * (64 * 96 // 32 + 2)
+    p = C.c_void_p()
+    assert lib.signmuon_payload_buffer(part, C.byref(p), None, None) == -3          # not bound yet
+    # a sharded context cannot run the whole step in one call: the exchange sits between the stages
+    arr = (C.c_void_p * 2)(4096, 8192)
+    assert lib.signmuon_step(part, arr, arr, C.c_float(1e-3), None) == -1
+    for bad in (dict(worker_offset=7, local_workers=2), dict(worker_offset=-1, local_workers=1),
+                dict(worker_offset=0, local_workers=9)):
+        with pytest.raises(B.SignMuonError):
+            B.signmuon_create(params, 8, 0.9, 1e-3, 5, False, **bad)
+    B.signmuon_destroy(full); B.signmuon_destroy(part)

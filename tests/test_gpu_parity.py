@@ -309,6 +309,59 @@ def test_pointer_table_cache_with_more_buffer_sets_than_slots():
     a.close(); b.close()
 
 
+@pytest.mark.parametrize("dtype,M,K", [("f32", 4, 5), ("bf16", 3, 3), ("f32", 1, 1)])
+def test_muon_rule_against_oracle(dtype, M, K):
+    """The full-precision Muon comparison optimizer on the same kernels (one momentum of the mean gradient,
+    W <- W - eta PolarNS(Mom), no sign, no vote): momentum at the momentum tolerance, update direction within 2e-2
+    relative Frobenius error of the oracle's step from the GPU's own momentum; plain parameters keep the
+    majority-vote sign update."""
+    import oracle as O
+    from parity_utils import _np64
+    shapes = [(200, 328), (328, 200), (64, 147), (256, 256), (1, 160)]
+    wl = _wl(shapes, M, dtype=dtype, K=K, kinds=["matrix"] * 4 + ["plain"], lr=0.01)
+    opt = B.SignMuon(wl.params, M, momentum=0.9, lr=0.01, ns_steps=K, update_rule="muon", weight_decay=0.01)
+    w = wlmod.make_weights(wl, "cuda:0")
+    sig = wlmod.make_signal(wl, "cuda:0")
+    cfg = O.OracleConfig(num_workers=M, momentum=0.9, lr=0.01, ns_steps=K, weight_decay=0.01)
+    mom_prev = [np.zeros((p.rows, p.cols)) for p in wl.params[:4]]
+    for t in range(2):
+        g = wlmod.make_grads(wl, sig, t, "cuda:0")
+        before = [x.clone() for x in w]
+        opt.step(w, g)
+        torch.cuda.synchronize()
+        assert opt.status() == B.OK
+        for p in range(4):
+            spec = O.ParamSpec(wl.params[p].rows, wl.params[p].cols, "matrix", dtype)
+            w0 = _np64(before[p])
+            mom_or, _, _ = O.muon_step_param(spec, cfg, mom_prev[p], w0, _np64(g[p]), short_side=True)
+            mom_gpu = _np64(opt.tap(B.TAP_MOMENTUM, p, 0))
+            assert np.max(np.abs(mom_gpu - mom_or)) <= 2e-6 * np.max(np.abs(mom_or))
+            u_or = O.polar_ns_short_side(mom_gpu, K, 1e-12)               # staged: from the GPU's own momentum
+            w1 = _np64(w[p])
+            if dtype == "f32":
+                d_gpu = (w0 - w1) / 0.01
+                noise = np.linalg.norm(np.abs(w0) * 1.2e-7 / 0.01)
+                rel = max(np.linalg.norm(d_gpu - u_or) - noise, 0.0) / np.linalg.norm(u_or)
+                assert rel <= 2e-2, rel
+            else:
+                w1_or = w0 - 0.01 * u_or
+                ulp = np.abs(O.round_to_bf16(w1_or).astype(np.float64)) * 2.0 ** -7 + 1e-40
+                assert np.all(np.abs(w1 - w1_or) <= 0.5 * ulp * (1 + 1e-3) + 0.01 * 0.05 * np.max(np.abs(u_or)))
+            mom_prev[p] = mom_gpu
+            with pytest.raises(B.SignMuonError):
+                opt.tap(B.TAP_WORKER_BITS, p, 0)                          # nothing is packed for a matrix under this rule
+        # the plain parameter: majority-vote sign update of its M momenta
+        d = wl.params[4].numel
+        packed = [opt.tap(B.TAP_WORKER_BITS, 4, m).cpu().numpy()[: (d + 7) // 8] for m in range(M)]
+        vote = O.decode_bits(O.majority_vote_popcount(packed, d)).reshape(1, d).astype(np.float64)
+        want = O.round_to_bf16(_np64(before[4]) - 0.01 * vote) if dtype == "bf16" else _np64(before[4]) - 0.01 * vote
+        scale = np.maximum(np.maximum(np.abs(_np64(before[4])), np.abs(want)), 0.01)   # operands of W - eta S
+        assert np.max(np.abs(_np64(w[4]) - want) / scale) <= 1e-6
+    with pytest.raises(B.SignMuonError):
+        B.SignMuon(wl.params, M, ns_steps=0, update_rule="muon")
+    opt.close()
+
+
 def test_garbage_worker_is_outvoted():
     """One worker sending NaN gradients maps to -1 everywhere; the vote still equals the popcount rule."""
     from parity_utils import check_param_step
