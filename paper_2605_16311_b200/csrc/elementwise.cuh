@@ -9,8 +9,7 @@ namespace signmuon {
 constexpr int EW_THREADS = 256;
 constexpr int MOM_CHUNK = 8192;        // entries per block of the momentum kernel (256 threads x 8 x 4)
 constexpr int PLAIN_CHUNK = 2048;      // entries per block of the plain-parameter kernel (8 warps x 256)
-constexpr int VOTE_THREADS = 128;      // vote kernel: 4 warps per block
-constexpr int VOTE_WORDS = 4 * VOTE_THREADS;   // payload words per block (4 consecutive words per lane: 128-bit loads)
+constexpr int VOTE_THREADS = 128;      // vote kernel: 4 warps per block, 4 consecutive payload words per thread (128-bit loads)
 constexpr int PACK_CHUNK = 1024;       // entries per block of the stand-alone pack kernel (small: it only sees small, ragged matrices)
 
 // Finds the list slot whose block range contains `block` (`starts` is ascending, one entry per slot).
@@ -461,59 +460,58 @@ struct VoteCounter {
   }
 };
 
-// vote_kernel: payload rows -> vote words.  A block owns an aligned group of VOTE_WORDS words of the payload's
-// word index, a lane four consecutive words; words of the group outside the parameter are masked (a group shared
-// by two parameters is visited once for each).
+// vote_kernel: payload rows -> vote words, over a few contiguous word ranges of the payload (the matrix parameters'
+// words; everything when the plain parameters are voted here too).  The vote of a bit position does not depend on
+// the parameter it belongs to, so the kernel needs no parameter table: a thread owns four consecutive words of the
+// concatenated ranges.  Range bounds are multiples of four words (rounded outwards by the host: a few neighbouring
+// words of a plain parameter or pad words may be voted again, with the same result).
+constexpr int MAX_VOTE_RANGES = 8;
+struct VoteRanges {
+  int32_t n;
+  int32_t reserved;
+  int64_t begin[MAX_VOTE_RANGES];     // first word of the range
+  int64_t quads_before[MAX_VOTE_RANGES + 1];   // four-word groups in the ranges before this one; [n] = total
+};
 template <int PLANES>
-__global__ void __launch_bounds__(VOTE_THREADS) vote_kernel(const ParamDev* __restrict__ params,
-                                                            const int32_t* __restrict__ list,
-                                                            const uint32_t* __restrict__ starts, int n_list, int M,
+__global__ void __launch_bounds__(VOTE_THREADS) vote_kernel(const __grid_constant__ VoteRanges ranges, int M,
                                                             const uint32_t* __restrict__ bits,
                                                             uint32_t* __restrict__ vote_words, int64_t bits_pitch) {
   constexpr int ROWS = 8;                               // worker rows in flight per lane
-  const int slot = find_slot(starts, n_list, blockIdx.x);
-  const ParamDev& pd = params[list[slot]];
-  const int64_t lo = pd.word_off, hi = (int64_t)pd.word_off + pd.n_words;
-  const uint32_t chunk = blockIdx.x - starts[slot];
-  const int64_t g = ((int64_t)(pd.word_off / VOTE_WORDS) + chunk) * VOTE_WORDS + 4 * (int64_t)threadIdx.x;
-  if (g >= hi || g + 4 <= lo) return;
+  // the update kernel that follows may start its prologue (and request its weights) while this grid still runs
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int64_t q = (int64_t)blockIdx.x * VOTE_THREADS + threadIdx.x;
+  if (q >= ranges.quads_before[ranges.n]) return;
+  int r = 0;
+#pragma unroll
+  for (int i = 1; i < MAX_VOTE_RANGES; ++i)
+    if (i < ranges.n && q >= ranges.quads_before[i]) r = i;
+  const int64_t g = ranges.begin[r] + 4 * (q - ranges.quads_before[r]);
   VoteCounter<PLANES> cnt[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) cnt[j].clear();
   const uint32_t* col = bits + g;
-  if (g >= lo && g + 4 <= hi) {
-    int m = 0;
-    for (; m + ROWS <= M; m += ROWS) {
-      uint4 r[ROWS];
+  int m = 0;
+  for (; m + ROWS <= M; m += ROWS) {
+    uint4 v[ROWS];
 #pragma unroll
-      for (int k = 0; k < ROWS; ++k) r[k] = __ldcs(reinterpret_cast<const uint4*>(col + (int64_t)(m + k) * bits_pitch));
+    for (int k = 0; k < ROWS; ++k) v[k] = __ldcs(reinterpret_cast<const uint4*>(col + (int64_t)(m + k) * bits_pitch));
 #pragma unroll
-      for (int k = 0; k < ROWS; ++k) { cnt[0].add(r[k].x); cnt[1].add(r[k].y); cnt[2].add(r[k].z); cnt[3].add(r[k].w); }
-    }
-    if (m + 4 <= M) {
-      uint4 r[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) r[k] = __ldcs(reinterpret_cast<const uint4*>(col + (int64_t)(m + k) * bits_pitch));
-#pragma unroll
-      for (int k = 0; k < 4; ++k) { cnt[0].add(r[k].x); cnt[1].add(r[k].y); cnt[2].add(r[k].z); cnt[3].add(r[k].w); }
-      m += 4;
-    }
-    for (; m < M; ++m) {
-      const uint4 r = __ldcs(reinterpret_cast<const uint4*>(col + (int64_t)m * bits_pitch));
-      cnt[0].add(r.x); cnt[1].add(r.y); cnt[2].add(r.z); cnt[3].add(r.w);
-    }
-    *reinterpret_cast<uint4*>(vote_words + g) =
-        make_uint4(cnt[0].majority(M), cnt[1].majority(M), cnt[2].majority(M), cnt[3].majority(M));
-  } else {
-    for (int m = 0; m < M; ++m) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-        if (g + j >= lo && g + j < hi) cnt[j].add(__ldcs(col + (int64_t)m * bits_pitch + j));
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (g + j >= lo && g + j < hi) vote_words[g + j] = cnt[j].majority(M);
+    for (int k = 0; k < ROWS; ++k) { cnt[0].add(v[k].x); cnt[1].add(v[k].y); cnt[2].add(v[k].z); cnt[3].add(v[k].w); }
   }
+  if (m + 4 <= M) {
+    uint4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) v[k] = __ldcs(reinterpret_cast<const uint4*>(col + (int64_t)(m + k) * bits_pitch));
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { cnt[0].add(v[k].x); cnt[1].add(v[k].y); cnt[2].add(v[k].z); cnt[3].add(v[k].w); }
+    m += 4;
+  }
+  for (; m < M; ++m) {
+    const uint4 v = __ldcs(reinterpret_cast<const uint4*>(col + (int64_t)m * bits_pitch));
+    cnt[0].add(v.x); cnt[1].add(v.y); cnt[2].add(v.z); cnt[3].add(v.w);
+  }
+  *reinterpret_cast<uint4*>(vote_words + g) =
+      make_uint4(cnt[0].majority(M), cnt[1].majority(M), cnt[2].majority(M), cnt[3].majority(M));
 }
 
 // update_kernel: vote words -> W <- W - eta S (Alg. 3 "Update parameters"), or S as a bf16 +-1 matrix in the local
@@ -535,13 +533,19 @@ __device__ __forceinline__ void update_block(const ParamDev& pd, uint32_t chunk,
     const int64_t i0 = (int64_t)chunk * UPD_VECS + threadIdx.x;
     uint4 x[8];
     uint32_t vword[8];
+    if (!write_sbar) {
+#pragma unroll
+      for (int it = 0; it < 8; ++it) {
+        const int64_t i = i0 + it * EW_THREADS;
+        if (i < n_vec) x[it] = __ldcs(vbase + i);
+      }
+    }
+    // the vote words come from the grid launched just before this one, which may still be running
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 #pragma unroll
     for (int it = 0; it < 8; ++it) {
       const int64_t i = i0 + it * EW_THREADS;
-      if (i < n_vec) {
-        vword[it] = __ldg(vw + ((i * epv) >> 5));
-        if (!write_sbar) x[it] = __ldcs(vbase + i);
-      }
+      if (i < n_vec) vword[it] = __ldcg(vw + ((i * epv) >> 5));
     }
 #pragma unroll
     for (int it = 0; it < 8; ++it) {
@@ -573,10 +577,11 @@ __device__ __forceinline__ void update_block(const ParamDev& pd, uint32_t chunk,
   }
   // scalar path: rows that are padded in the operand buffer (the +-1 matrix of a parameter whose column count is
   // not a multiple of 8), or d not a multiple of 8.  The block covers the same entries as on the vector path.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int64_t e_begin = (int64_t)chunk * UPD_VECS * epv;
   const int64_t e_end = (e_begin + (int64_t)UPD_VECS * epv < d) ? e_begin + (int64_t)UPD_VECS * epv : d;
   for (int64_t i = e_begin + threadIdx.x; i < e_end; i += EW_THREADS) {
-    const bool plus = (__ldg(vw + (i >> 5)) >> (i & 31)) & 1u;
+    const bool plus = (__ldcg(vw + (i >> 5)) >> (i & 31)) & 1u;
     if (write_sbar) {
       int64_t o = i;
       if (pd.ldy != pd.cols) {

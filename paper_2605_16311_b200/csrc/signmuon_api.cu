@@ -71,7 +71,7 @@ struct signmuon_ctx {
   std::vector<signmuon_param> params;
   std::vector<ParamPlan> plan;
   std::vector<int32_t> matrix_list, plain_list, packfb_list, vote_list;
-  std::vector<uint32_t> mom_starts, plain_starts, vote_starts, upd_starts, packfb_starts, xv_starts, xtu_starts;
+  std::vector<uint32_t> mom_starts, plain_starts, upd_starts, packfb_starts, xv_starts, xtu_starts;
   uint32_t upd_blocks = 0;
   uint32_t mom_blocks = 0, plain_blocks = 0, vote_blocks = 0, packfb_blocks = 0, xv_blocks = 0, xtu_blocks = 0;
   size_t power_start_floats = 0;          // length of the start-vector array (scale = spectral)
@@ -94,7 +94,7 @@ struct signmuon_ctx {
          off_problems = 0, off_tables_end = 0;
   size_t off_list_vote = 0, off_starts_upd = 0, off_flags = 0;
   size_t off_list_matrix = 0, off_list_plain = 0, off_list_packfb = 0, off_starts_mom = 0, off_starts_plain = 0,
-         off_starts_vote = 0, off_starts_packfb = 0, off_starts_xv = 0, off_starts_xtu = 0, off_agree = 0;
+         off_starts_packfb = 0, off_starts_xv = 0, off_starts_xtu = 0, off_agree = 0;
   // GEMM plans
   std::vector<GemmProblem> problems;      // pointers filled at bind
   std::vector<LaunchPlan> ns_launches, lp_launches;
@@ -130,6 +130,7 @@ struct signmuon_ctx {
   FlagList peer_flags = {};               // every peer's flag array
   int my_rank = 0, n_ranks = 1;
   uint32_t exchange_seq = 0;              // sequence number of the last published payload
+  VoteRanges vote_ranges = {};            // word ranges of the payload the vote kernel covers
   double executed_flops = 0;              // flops the scheduled tiles issue per step (known once the tile tables exist)
   int sticky = SIGNMUON_OK;
 };
@@ -377,20 +378,34 @@ int plan_layout(signmuon_ctx* c) {
   if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
   c->plain_blocks = (uint32_t)b;
   b = 0;
-  // vote kernel: blocks own VOTE_WORDS-aligned groups of the payload's word index; a parameter gets every group it
-  // touches (a group shared by two parameters is visited once for each, masked)
   if (!c->muon) c->vote_list = c->matrix_list;
   if (c->sharded) {       // the plain parameters' vote also waits for the exchange: every parameter goes through the vote kernel
     c->vote_list.clear();
     for (size_t p = 0; p < c->params.size(); ++p) c->vote_list.push_back((int32_t)p);
   }
-  for (int32_t p : c->vote_list) {
-    const ParamPlan& pl = c->plan[p];
-    c->vote_starts.push_back((uint32_t)b);
-    b += ((uint64_t)pl.word_off + pl.n_words + VOTE_WORDS - 1) / VOTE_WORDS - pl.word_off / VOTE_WORDS;
+  // vote kernel: the payload words of these parameters as a few contiguous ranges with bounds rounded outwards to
+  // four words (parameters follow one another in the payload, so neighbours merge); too many ranges: everything
+  {
+    VoteRanges vr = {};
+    std::vector<std::pair<int64_t, int64_t>> rg;
+    for (int32_t p : c->vote_list) {
+      const ParamPlan& pl = c->plan[p];
+      const int64_t lo = (int64_t)pl.word_off / 4 * 4, hi = ((int64_t)pl.word_off + pl.n_words + 3) / 4 * 4;
+      if (!rg.empty() && lo <= rg.back().second) rg.back().second = std::max(rg.back().second, hi);
+      else rg.push_back({lo, hi});
+    }
+    if ((int)rg.size() > MAX_VOTE_RANGES) rg.assign(1, {0, ((int64_t)words + 3) / 4 * 4});
+    vr.n = (int32_t)rg.size();
+    int64_t quads = 0;
+    for (int i = 0; i < vr.n; ++i) {
+      vr.begin[i] = rg[i].first;
+      vr.quads_before[i] = quads;
+      quads += (rg[i].second - rg[i].first) / 4;
+    }
+    vr.quads_before[vr.n] = quads;
+    c->vote_ranges = vr;
+    c->vote_blocks = (uint32_t)((quads + VOTE_THREADS - 1) / VOTE_THREADS);
   }
-  if (b >= (1ull << 31)) return SIGNMUON_ERR_BAD_SHAPE;
-  c->vote_blocks = (uint32_t)b;
   // update kernel: blocks of UPD_VECS 128-bit vectors (8 bf16 or 4 float32 entries each; the +-1 matrix is bf16)
   b = 0;
   for (int32_t p : c->vote_list) {
@@ -445,7 +460,6 @@ int plan_layout(signmuon_ctx* c) {
   place(c->off_list_vote, c->vote_list.size() * 4);
   place(c->off_starts_mom, c->mom_starts.size() * 4);
   place(c->off_starts_plain, c->plain_starts.size() * 4);
-  place(c->off_starts_vote, c->vote_starts.size() * 4);
   place(c->off_starts_upd, c->upd_starts.size() * 4);
   place(c->off_starts_packfb, c->packfb_starts.size() * 4);
   place(c->off_agree, (size_t)c->M_all * 8);
@@ -679,10 +693,22 @@ void launch_vote(signmuon_ctx* c, float lr, int write_sbar, cudaStream_t s, cons
   const int n = (int)c->vote_list.size();
   if (src != vote)      // (vote words computed elsewhere: only the update remains)
     vote_kernel<PLANES><<<c->vote_blocks, VOTE_THREADS, 0, s>>>(
-        pd, list, reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_vote), n, src ? rows : c->M_all,
-        src ? src : reinterpret_cast<const uint32_t*>(c->d_ws + c->off_bits), vote, (int64_t)c->bits_pitch);
-  update_kernel<<<c->upd_blocks, EW_THREADS, 0, s>>>(
-      pd, list, reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_upd), n, c->Wm, lr, write_sbar, vote);
+        c->vote_ranges, src ? rows : c->M_all, src ? src : reinterpret_cast<const uint32_t*>(c->d_ws + c->off_bits),
+        vote, (int64_t)c->bits_pitch);
+  // Programmatic dependent launch: the update grid may begin (and request its weight vectors) while the vote grid
+  // drains; it waits for the vote grid's completion before it reads a vote word.
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(c->upd_blocks, 1, 1);
+  cfg.blockDim = dim3(EW_THREADS, 1, 1);
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, update_kernel, pd, list, reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_upd), n,
+                     c->Wm, lr, write_sbar, static_cast<const uint32_t*>(vote));
 }
 
 void invalidate_tables(signmuon_ctx* c) {
@@ -994,7 +1020,6 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
   ok = ok && up(c->off_list_vote, c->vote_list.data(), c->vote_list.size() * 4);
   ok = ok && up(c->off_starts_mom, c->mom_starts.data(), c->mom_starts.size() * 4);
   ok = ok && up(c->off_starts_plain, c->plain_starts.data(), c->plain_starts.size() * 4);
-  ok = ok && up(c->off_starts_vote, c->vote_starts.data(), c->vote_starts.size() * 4);
   ok = ok && up(c->off_starts_upd, c->upd_starts.data(), c->upd_starts.size() * 4);
   ok = ok && up(c->off_starts_packfb, c->packfb_starts.data(), c->packfb_starts.size() * 4);
   ok = ok && up(c->off_starts_xv, c->xv_starts.data(), c->xv_starts.size() * 4);
