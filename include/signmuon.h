@@ -121,6 +121,8 @@ enum {
                                      kernel instead of the tensor-core kernel (slow; for fault isolation) */
   SIGNMUON_FLAG_GEMM_1CTA = 4,    /* run the tensor-core kernel with one CTA per 128 x 128 tile instead of
                                      CTA pairs on 256 x 256 tiles (same results; for comparison) */
+  SIGNMUON_FLAG_LP_GRAM_BF16 = 32, /* run the first Gram product of the local polar step on the bf16 copy of the vote
+                                     matrix instead of its FP8 (E4M3) copy (same result bit for bit; for comparison) */
   SIGNMUON_FLAG_SIGN_AGREEMENT = 16 /* count, every step, how many of each worker's sign bits equal the vote
                                      (one more small kernel; read with signmuon_sign_agreement) */
 };

@@ -32,6 +32,9 @@ struct ParamDev {
   uint32_t chunks_per_worker;  // momentum-kernel blocks (= norm partials) per worker
   float upd_scale;      // 1, or 1/sqrt(rows*cols) for the Eq. 2 normalisation
   int32_t vec_ok;       // 16-byte vector path allowed (d % 8 == 0 and ldy == cols)
+  uint8_t* sbar8;       // matrix params with the local polar step: the vote matrix once more as FP8 (E4M3) +-1 bytes,
+                        // [rows][ld8]: operand of the step's first Gram product (null: not kept)
+  int32_t ld8;          // row pitch of sbar8 in bytes (cols rounded up to 16)
   int32_t avg_workers;  // > 1: the momentum takes the mean of this many workers' gradients (Muon rule), G is [avg][rows][cols]
   // power iteration (scale = spectral): un-normalised vectors and their norms
   float* pi_v;          // [M][cols]
@@ -95,6 +98,8 @@ struct GemmProblem {
   // tile, every segment contracting over the same K.
   int32_t nseg;           // 0 or 1: one pair
   int32_t tmapA2, tmapB2, tmapA3, tmapB3;
+  int32_t fp8;            // operands are FP8 (E4M3) bytes: 128 elements per 128-byte row, tensor-core kind f8f6f4.  Used for
+                          // the first Gram product of the local polar step, whose operand is the exact +-1 vote matrix
   int32_t gram_lo;        // EPI_GRAM: also store lo(-A/2) through tmapO1 (then the tile is not mirrored)
   int32_t diag_share;     // EPI_GRAM, one segment: on diagonal tiles the B operand is the A tile (not loaded twice)
 };

@@ -570,6 +570,20 @@ __device__ __forceinline__ void update_block(const ParamDev& pd, uint32_t chunk,
                                    __uint_as_float(in[e] & 0xffff0000u) - (p1 ? step : -step));
         }
         o = make_uint4(ov[0], ov[1], ov[2], ov[3]);
+        if (write_sbar && pd.sbar8) {                   // the same eight signs as E4M3 bytes (+1 = 0x38, -1 = 0xb8)
+          uint32_t lo4 = 0, hi4 = 0;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            lo4 |= (((b8 >> e) & 1u) ? 0x38u : 0xb8u) << (8 * e);
+            hi4 |= (((b8 >> (4 + e)) & 1u) ? 0x38u : 0xb8u) << (8 * e);
+          }
+          int64_t off = i * 8;                          // dense when the byte pitch equals the column count
+          if (pd.ld8 != pd.cols) {
+            const int64_t r = off / pd.cols;
+            off = r * pd.ld8 + (off - r * pd.cols);
+          }
+          __stcs(reinterpret_cast<uint2*>(pd.sbar8 + off), make_uint2(lo4, hi4));
+        }
       }
       __stcs(vbase + i, o);
     }
@@ -589,6 +603,10 @@ __device__ __forceinline__ void update_block(const ParamDev& pd, uint32_t chunk,
         o = r * pd.ldy + (i - r * pd.cols);
       }
       sbar[o] = __float2bfloat16_rn(plus ? 1.f : -1.f);
+      if (pd.sbar8) {
+        const int64_t r = i / pd.cols;
+        pd.sbar8[r * pd.ld8 + (i - r * pd.cols)] = plus ? (uint8_t)0x38 : (uint8_t)0xb8;
+      }
     } else {
       const float nw = load_as_float<WT>(w + i) - (plus ? step : -step);
       if (sizeof(WT) == 4) reinterpret_cast<float*>(w)[i] = nw;

@@ -165,6 +165,25 @@ __device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// FP8 (E4M3 x E4M3 -> fp32) forms of the same instructions: K = 32 elements (32 bytes) per instruction.
+__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_f8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -245,14 +264,16 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   return d;
 }
 
-// Instruction descriptor, kind::f16: D fp32 (bits [4,6) = 1), A/B bf16 (bits [7,10) = [10,13) = 1),
-// bit 15 / 16: A / B contiguous along M / N, bits [17,23) N >> 3, bits [24,29) M >> 4
+// Instruction descriptor: D fp32 (bits [4,6) = 1), A/B format in bits [7,10) and [10,13) (kind::f16: 1 = bf16;
+// kind::f8f6f4: 0 = E4M3), bit 15 / 16: A / B contiguous along M / N, bits [17,23) N >> 3, bits [24,29) M >> 4
 // (M = 128 for one CTA, 256 for a CTA pair).
-__device__ __forceinline__ uint32_t instr_desc(int m, int n, int a_mn, int b_mn) {
+__device__ __forceinline__ uint32_t instr_desc(int m, int n, int a_mn, int b_mn, int fp8 = 0) {
   uint32_t d = 0;
   d |= 1u << 4;
-  d |= 1u << 7;
-  d |= 1u << 10;
+  if (!fp8) {
+    d |= 1u << 7;
+    d |= 1u << 10;
+  }
   d |= (uint32_t)(a_mn & 1) << 15;
   d |= (uint32_t)(b_mn & 1) << 16;
   d |= (uint32_t)(n >> 3) << 17;
@@ -380,7 +401,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
         const int n0 = te.tn * BN + (int)cta_rank * B_ROWS;            // this CTA's rows of B
         const int batch = pr.batch;
         const int a_mn = pr.a_mn, b_mn = pr.b_mn;
-        const int nk = (pr.K + GEMM_BK - 1) / GEMM_BK;
+        // FP8 operands (Gram launches only): a stage still holds 128 bytes along K, i.e. 128 elements instead of 64,
+        // and an MN-major tile is one 128-wide chunk of 128 k-rows instead of two 64-wide chunks of 64
+        const bool fp8 = KIND == 0 && pr.fp8 != 0;
+        const int kelem = fp8 ? 2 * GEMM_BK : GEMM_BK;
+        const int nk = (pr.K + kelem - 1) / kelem;
         const int nseg = pr.nseg > 1 ? pr.nseg : 1;           // split-precision products: segments along K
         // Diagonal tile of a one-segment Gram product: this CTA's B rows are its A rows, so B is not loaded
         // and the MMA reads the A tile for both operands (B_ROWS == GEMM_BM and equal box shapes).
@@ -396,9 +421,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
             if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[0]) + 8u * s, stage_tx);
             const uint32_t sa = smem_base + s * STAGE_BYTES;
             const uint32_t sb = sa + A_BYTES;
-            const int k0 = kb * GEMM_BK;
+            const int k0 = kb * kelem;
             if (!a_mn) {
               load_operand(sa, mapA, k0, m0, batch, fb);
+            } else if (fp8) {
+              load_operand(sa, mapA, m0, k0, batch, fb);
             } else {
 #pragma unroll
               for (int c = 0; c < GEMM_BM / 64; ++c) load_operand(sa + c * 8192, mapA, m0 + 64 * c, k0, batch, fb);
@@ -406,6 +433,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
             if (share_ab) {
             } else if (!b_mn) {
               load_operand(sb, mapB, k0, n0, batch, fb);
+            } else if (fp8) {
+              load_operand(sb, mapB, n0, k0, batch, fb);
             } else {
 #pragma unroll
               for (int c = 0; c < B_ROWS / 64; ++c) load_operand(sb + c * 8192, mapB, n0 + 64 * c, k0, batch, fb);
@@ -440,8 +469,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
         const TileEntry te = args.tiles[t];
         const GemmProblem& pr = args.problems[te.problem];
         const int a_mn = pr.a_mn, b_mn = pr.b_mn;
-        const int nk = ((pr.K + GEMM_BK - 1) / GEMM_BK) * (pr.nseg > 1 ? pr.nseg : 1);
-        const uint32_t idesc = instr_desc(TILE_M, BN, a_mn, b_mn);
+        const bool fp8 = KIND == 0 && pr.fp8 != 0;
+        const int kelem = fp8 ? 2 * GEMM_BK : GEMM_BK;
+        const int nk = ((pr.K + kelem - 1) / kelem) * (pr.nseg > 1 ? pr.nseg : 1);
+        const uint32_t idesc = instr_desc(TILE_M, BN, a_mn, b_mn, fp8 ? 1 : 0);
+        // MN-major operands: bytes between the 16 (bf16) or 32 (FP8) k-rows of consecutive instructions, and between
+        // 128-byte-wide chunks along M/N (a 128-row FP8 tile is a single chunk)
+        const uint32_t mn_step = fp8 ? 4096u : 2048u, mn_lbo = fp8 ? 16384u : 8192u;
         const bool share_ab = KIND == 0 && B_ROWS == GEMM_BM && pr.diag_share != 0 && te.tm == te.tn;
         const uint32_t acc = tcount & 1u;
         const uint32_t acc_round = tcount >> 1;
@@ -455,10 +489,14 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
           const uint32_t sb = share_ab ? sa : sa + A_BYTES;
 #pragma unroll
           for (int kk = 0; kk < GEMM_BK / 16; ++kk) {
-            const uint64_t adesc = a_mn ? smem_desc(sa + kk * 2048, 8192, 1024) : smem_desc(sa + kk * 32, 16, 1024);
-            const uint64_t bdesc = b_mn ? smem_desc(sb + kk * 2048, 8192, 1024) : smem_desc(sb + kk * 32, 16, 1024);
-            if (CTAS == 2) tc_mma_f16_pair(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
-            else tc_mma_f16(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
+            const uint64_t adesc = a_mn ? smem_desc(sa + kk * mn_step, mn_lbo, 1024) : smem_desc(sa + kk * 32, 16, 1024);
+            const uint64_t bdesc = b_mn ? smem_desc(sb + kk * mn_step, mn_lbo, 1024) : smem_desc(sb + kk * 32, 16, 1024);
+            const uint32_t accum = (kb | kk) != 0 ? 1u : 0u;
+            if (fp8) {
+              if (CTAS == 2) tc_mma_f8_pair(d_tmem, adesc, bdesc, idesc, accum); else tc_mma_f8(d_tmem, adesc, bdesc, idesc, accum);
+            } else {
+              if (CTAS == 2) tc_mma_f16_pair(d_tmem, adesc, bdesc, idesc, accum); else tc_mma_f16(d_tmem, adesc, bdesc, idesc, accum);
+            }
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
           if (CTAS == 2) tc_commit_pair(smem_u32(&empty_bar[0]) + 8u * s); else tc_commit(smem_u32(&empty_bar[0]) + 8u * s);

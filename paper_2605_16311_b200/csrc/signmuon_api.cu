@@ -43,11 +43,14 @@ struct ParamPlan {
   size_t stage_w_off, stage_g_off;                    // bytes into the host-staging buffer
   size_t pi_v_off, pi_u_off, pi_scal_off;             // power iteration (scale = spectral), bytes into the workspace
   size_t pi_start_off;                                // floats into the caller's start-vector array
+  size_t s8_off;                                      // FP8 copy of the vote matrix (local polar step), bytes into the workspace
+  int32_t ld8;                                        // its row pitch in bytes (cols rounded up to 16)
+  bool lp_fp8;                                        // the local polar step's first Gram product runs on FP8 operands
 };
 
 // indices of a parameter's tensor maps relative to tmap_base
 enum { TM_Y0_K128 = 0, TM_Y0_KBN, TM_Y0_MN, TM_Y1_K128, TM_Y1_KBN, TM_Y1_MN, TM_Q_K128, TM_Q_KBN, TM_LO0_K128, TM_MOM_F32,
-       TM_Q_BOX64, TM_LO1_K128, TM_LO0_MN, TM_LO1_MN, TM_QLO_K128, TM_QLO_KBN, TM_PER_PARAM };
+       TM_Q_BOX64, TM_LO1_K128, TM_LO0_MN, TM_LO1_MN, TM_QLO_K128, TM_QLO_KBN, TM_S8, TM_PER_PARAM };
 
 struct LaunchPlan {        // one grouped GEMM launch
   size_t problem_base;     // index of its first problem in the problem array
@@ -157,7 +160,8 @@ void build_tile_table(TileTable& tt, const std::vector<GemmProblem>& probs, size
     // consecutive tiles overlap, so a tile costs the longer of the two; a 64-column chunk of an apply epilogue
     // (C in, combine, hi/lo out) takes about five such units, a chunk of a Gram epilogue about one (measured
     // per-chunk cycle counts).
-    const int nk = ((pr.K + GEMM_BK - 1) / GEMM_BK) * (pr.nseg > 1 ? pr.nseg : 1);
+    const int kelem = pr.fp8 ? 2 * GEMM_BK : GEMM_BK;        // elements of K per 128-byte stage row
+    const int nk = ((pr.K + kelem - 1) / kelem) * (pr.nseg > 1 ? pr.nseg : 1);
     const int per_chunk = (pr.epi == EPI_GRAM) ? 1 : 5;
     for (int a = 0; a < tm; ++a)
       for (int b = (pr.sym ? a : 0); b < tn; ++b) {   // symmetric results: tiles on or above the diagonal
@@ -255,6 +259,14 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
             pr.tmapA2 = pr.tmapA;             pr.tmapB2 = pl.tmap_base + lmn;
             pr.tmapA3 = pl.tmap_base + lmn;   pr.tmapB3 = pr.tmapB;
           }
+        }
+        if (k == 0 && local_polar_phase && pl.lp_fp8) {
+          // S S^T of the exact +-1 vote matrix: E4M3 operands (one byte per entry, twice the tensor-core rate);
+          // products are +-1 and their fp32 sums are exact integers, so the result equals the bf16 product's bit for bit
+          pr.fp8 = 1;
+          pr.A = pr.B = reinterpret_cast<const bf16*>(pl.s8_off);
+          pr.tmapA = pr.tmapB = pl.tmap_base + TM_S8;
+          pr.batch = 0;                              // the FP8 copy has a single slot
         }
         if (k == 0) {
           if (local_polar_phase) pr.scale_imm = (float)(1.0 / ((double)pl.rows * (double)pl.cols));
@@ -356,6 +368,9 @@ int plan_layout(signmuon_ctx* c) {
     words += pl.n_words;
     pl.chunks_per_worker = (uint32_t)((pl.d + MOM_CHUNK - 1) / MOM_CHUNK);
     pl.fused_pack = (sp.kind == SIGNMUON_PARAM_MATRIX) && K > 0 && (sp.cols % 32 == 0) && !c->muon;
+    pl.ld8 = (int32_t)round_up((size_t)sp.cols, 16);
+    pl.lp_fp8 = sp.kind == SIGNMUON_PARAM_MATRIX && c->lp && K > 0 &&
+                !(c->cfg.flags & (SIGNMUON_FLAG_SIMT_GEMM | SIGNMUON_FLAG_LP_GRAM_BF16));
     pl.mom_off = state;
     state += round_up((size_t)(sp.kind == SIGNMUON_PARAM_MATRIX ? c->Wm : c->Lw) * pl.d * 4, ALIGN);
     c->plan.push_back(pl);
@@ -497,6 +512,7 @@ int plan_layout(signmuon_ctx* c) {
       pl.lo_off[1] = off; off += ybytes;
       pl.qlo_off = off; off += round_up(slots * pl.s * pl.ldq * 2, 1024);
     }
+    if (pl.lp_fp8) { pl.s8_off = off; off += round_up((size_t)pl.rows * pl.ld8, 1024); }
   }
   // GEMM problems: K x (gram, apply) for the workers, and again for the local polar step
   c->problems.clear();
@@ -574,6 +590,19 @@ bool encode_map(CUtensorMap* map, void* base, uint64_t inner, uint64_t rows, uin
   cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, gdim, gstr, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 3-D byte tensor {cols, rows, 1} with a {128, 128, 1} box and 128-byte swizzle (FP8 operands).
+bool encode_map_u8(CUtensorMap* map, void* base, uint64_t cols, uint64_t rows, uint64_t pitch_bytes) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[3] = {cols, rows, 1};
+  cuuint64_t gstr[2] = {pitch_bytes, pitch_bytes * rows};
+  cuuint32_t box[3] = {128u, 128u, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, base, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -1012,6 +1041,8 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     d.upd_scale = eq2 ? (float)(1.0 / std::sqrt((double)pl.rows * (double)pl.cols)) : 1.f;
     d.vec_ok = (pl.d % 8 == 0 && pl.ldy == pl.cols) ? 1 : 0;
     d.avg_workers = (c->muon && pl.kind == SIGNMUON_PARAM_MATRIX) ? c->Lw : 1;
+    d.sbar8 = pl.lp_fp8 ? c->d_ws + pl.s8_off : nullptr;
+    d.ld8 = pl.ld8;
   }
   invalidate_tables(c);
   ok = ok && up(c->off_list_matrix, c->matrix_list.data(), c->matrix_list.size() * 4);
@@ -1052,9 +1083,12 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     double f = 0;
     for (const TileEntry& te : tt.tiles) {
       const GemmProblem& pr = c->problems[ls[t & 1].problem_base + te.problem];
-      const double kblocks = (double)((pr.K + GEMM_BK - 1) / GEMM_BK) * (pr.nseg > 1 ? pr.nseg : 1);
-      f += 2.0 * tt.bm * tt.bn * GEMM_BK * kblocks;
+      const int kelem = pr.fp8 ? 2 * GEMM_BK : GEMM_BK;
+      const double kblocks = (double)((pr.K + kelem - 1) / kelem) * (pr.nseg > 1 ? pr.nseg : 1);
+      f += 2.0 * tt.bm * tt.bn * kelem * kblocks;
     }
+    // (a tile table serves the K launches of its kind; the FP8 first Gram of the local polar step has the same
+    // tiles and, per tile, the same flops as the bf16 Gram launches that follow it)
     c->executed_flops += f * c->cfg.ns_steps;
   }
   // (moved up) kernels configured before the tile tables are split
@@ -1088,6 +1122,8 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
         ok = ok && encode_map(mp + TM_QLO_K128, c->d_ws + pl.qlo_off, pl.s, pl.s, slots, pl.ldq, qb, 128);
         ok = ok && encode_map(mp + TM_QLO_KBN, c->d_ws + pl.qlo_off, pl.s, pl.s, slots, pl.ldq, qb, bn);
       }
+      if (pl.lp_fp8)          // FP8 copy of the vote matrix: {128 bytes x 128 rows} boxes serve K-major and MN-major tiles
+        ok = ok && encode_map_u8(mp + TM_S8, c->d_ws + pl.s8_off, pl.cols, pl.rows, pl.ld8);
       if (pl.cols % 4 == 0)   // float32 momentum as the first iteration's C operand
         ok = ok && encode_map(mp + TM_MOM_F32, c->d_state + pl.mom_off, pl.cols, pl.rows, M, pl.cols, (uint64_t)pl.d, 128,
                               true);

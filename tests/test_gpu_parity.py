@@ -362,6 +362,29 @@ def test_muon_rule_against_oracle(dtype, M, K):
     opt.close()
 
 
+@pytest.mark.parametrize("flags", [0, B.FLAG_GEMM_1CTA])
+def test_local_polar_first_gram_in_fp8_equals_bf16_bit_for_bit(flags):
+    """The local polar step's first Gram product reads the vote matrix as E4M3 bytes (+-1 are exact, the fp32
+    sums of +-1 products are exact integers): the weights after the step equal, bit for bit, those of a run
+    whose first Gram product uses the bf16 copy.  Wide, tall, square and ragged shapes; K-major and MN-major tiles."""
+    shapes = [(200, 328), (328, 200), (64, 147), (256, 256), (512, 1152), (1152, 512), (130, 48)]
+    for dtype, M in (("f32", 3), ("bf16", 4)):
+        wl = _wl(shapes, M, dtype=dtype, local_polar=True, lr=0.01)
+        sig = wlmod.make_signal(wl, "cuda:0")
+        outs = []
+        for extra in (0, B.FLAG_LP_GRAM_BF16):
+            opt = B.SignMuon(wl.params, M, lr=0.01, local_polar=True, flags=flags | extra)
+            w = wlmod.make_weights(wl, "cuda:0")
+            for t in range(2):
+                opt.step(w, wlmod.make_grads(wl, sig, t, "cuda:0"))
+            torch.cuda.synchronize()
+            assert opt.status() == B.OK
+            outs.append(w)
+            opt.close()
+        for a, b in zip(*outs):
+            assert torch.equal(a, b)
+
+
 def test_garbage_worker_is_outvoted():
     """One worker sending NaN gradients maps to -1 everywhere; the vote still equals the popcount rule."""
     from parity_utils import check_param_step
