@@ -123,6 +123,9 @@ enum {
                                      CTA pairs on 256 x 256 tiles (same results; for comparison) */
   SIGNMUON_FLAG_LP_GRAM_BF16 = 32, /* run the first Gram product of the local polar step on the bf16 copy of the vote
                                      matrix instead of its FP8 (E4M3) copy (same result bit for bit; for comparison) */
+  SIGNMUON_FLAG_NO_GRAM_SPACE = 64, /* run every Newton-Schulz iteration on the full matrix, also for parameters with a
+                                     short side of at most 256 (whose iteration otherwise runs in Gram space on chip;
+                                     same map, two passes over the matrix instead of 2 K; for comparison) */
   SIGNMUON_FLAG_SIGN_AGREEMENT = 16 /* count, every step, how many of each worker's sign bits equal the vote
                                      (one more small kernel; read with signmuon_sign_agreement) */
 };

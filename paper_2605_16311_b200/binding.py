@@ -20,6 +20,7 @@ OK = 0
 F32, BF16 = 0, 1
 PARAM_MATRIX, PARAM_PLAIN = 0, 1
 FLAG_KEEP_POLAR, FLAG_SIMT_GEMM, FLAG_GEMM_1CTA, FLAG_SIGN_AGREEMENT, FLAG_LP_GRAM_BF16 = 1, 2, 4, 16, 32
+FLAG_NO_GRAM_SPACE = 64
 STAGE_MOMENTUM, STAGE_NS, STAGE_VOTE, STAGE_LOCAL_POLAR, STAGE_ALL = 1, 2, 4, 8, 15
 TAP_MOMENTUM, TAP_POLAR, TAP_VOTE_BITS, TAP_WORKER_BITS, TAP_NORM = 0, 1, 2, 3, 4
 

@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsignmuon.so")
 SOURCES = ["signmuon_api.cu", "momentum_noalloc.cu"]
-HEADERS = ["common.cuh", "elementwise.cuh", "ns_gemm_simt.cuh", "ns_gemm_sm100.cuh",
+HEADERS = ["common.cuh", "elementwise.cuh", "ns_gemm_simt.cuh", "ns_gemm_sm100.cuh", "ns_chain_sm100.cuh",
            os.path.join("..", "..", "include", "signmuon.h")]
 
 

@@ -35,6 +35,7 @@ struct ParamDev {
   uint8_t* sbar8;       // matrix params with the local polar step: the vote matrix once more as FP8 (E4M3) +-1 bytes,
                         // [rows][ld8]: operand of the step's first Gram product (null: not kept)
   int32_t ld8;          // row pitch of sbar8 in bytes (cols rounded up to 16)
+  int32_t yk_buf;       // matrix params: which operand buffer (0: y0, 1: y1) holds Y_K after the last apply product
   int32_t avg_workers;  // > 1: the momentum takes the mean of this many workers' gradients (Muon rule), G is [avg][rows][cols]
   // power iteration (scale = spectral): un-normalised vectors and their norms
   float* pi_v;          // [M][cols]
@@ -52,7 +53,7 @@ struct ParamDev {
 // decide such signs with a 2^-9 relative error of a term that is not small.
 enum : int32_t {
   EPI_GRAM = 0,          // out = bf16(-0.5 * scale * acc)                      (the "-A/2" of 3I/2 - A/2)
-  EPI_APPLY = 1,         // y = scale * (acc + 1.5 * C); out = hi(y), out_lo = lo(y)   (Y_{k+1})
+  EPI_APPLY = 1,         // y = scale * (acc + own * C), own = 1.5; out = hi(y), out_lo = lo(y)   (Y_{k+1})
   EPI_APPLY_PACK = 2,    // sign bits of y -> payload words (hi(y) optionally stored)
   EPI_APPLY_UPDATE = 3   // W -= lr * y                                          (local polar step)
 };
@@ -98,6 +99,9 @@ struct GemmProblem {
   // tile, every segment contracting over the same K.
   int32_t nseg;           // 0 or 1: one pair
   int32_t tmapA2, tmapB2, tmapA3, tmapB3;
+  float own_coef;         // APPLY*: coefficient of the own term, y = scale * (acc + own_coef * C): 1.5 for one Newton-Schulz
+                          // step; 1.5^K when the product applies K steps at once (iteration carried out in Gram space)
+  int32_t hi_only;        // EPI_APPLY: store hi(y) only (the lo buffer is still being read as an operand)
   int32_t fp8;            // operands are FP8 (E4M3) bytes: 128 elements per 128-byte row, tensor-core kind f8f6f4.  Used for
                           // the first Gram product of the local polar step, whose operand is the exact +-1 vote matrix
   int32_t gram_lo;        // EPI_GRAM: also store lo(-A/2) through tmapO1 (then the tile is not mirrored)
@@ -160,12 +164,13 @@ __device__ __forceinline__ void store_hi_lo(bf16* o, bf16* olo, const float (&v)
 // ---- epilogue building blocks, each over 32 consecutive columns [col0, col0+32) of output row `row`;
 // rows/columns outside the problem are skipped.
 
-// v <- scale * (v + 1.5 * C) with C read directly from global memory.
+// v <- scale * (v + own * C) with C read directly from global memory (own = 1.5 for a Newton-Schulz step).
 template <int NC = 32>
 __device__ __forceinline__ void apply_c_direct(const GemmProblem& pr, float scale, int row, int col0, float* v) {
   if (row >= pr.M || col0 >= pr.N) return;
   const bool full = (col0 + NC <= pr.N);
   const int n_valid = full ? NC : pr.N - col0;
+  const float own = pr.own_coef;
   if (pr.c_mode == C_F32) {
     const float* c = reinterpret_cast<const float*>(pr.C) + (int64_t)row * pr.ldc + col0;
     if (full && ((pr.ldc & 3) == 0)) {
@@ -173,14 +178,14 @@ __device__ __forceinline__ void apply_c_direct(const GemmProblem& pr, float scal
 #pragma unroll
       for (int q = 0; q < NC / 4; ++q) {
         const float4 t = __ldg(c4 + q);
-        v[4 * q] = scale * fmaf(1.5f, t.x, v[4 * q]);
-        v[4 * q + 1] = scale * fmaf(1.5f, t.y, v[4 * q + 1]);
-        v[4 * q + 2] = scale * fmaf(1.5f, t.z, v[4 * q + 2]);
-        v[4 * q + 3] = scale * fmaf(1.5f, t.w, v[4 * q + 3]);
+        v[4 * q] = scale * fmaf(own, t.x, v[4 * q]);
+        v[4 * q + 1] = scale * fmaf(own, t.y, v[4 * q + 1]);
+        v[4 * q + 2] = scale * fmaf(own, t.z, v[4 * q + 2]);
+        v[4 * q + 3] = scale * fmaf(own, t.w, v[4 * q + 3]);
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < NC; ++j) v[j] = (j < n_valid) ? scale * fmaf(1.5f, __ldg(c + j), v[j]) : 0.f;
+      for (int j = 0; j < NC; ++j) v[j] = (j < n_valid) ? scale * fmaf(own, __ldg(c + j), v[j]) : 0.f;
     }
   } else {
     const bf16* c = reinterpret_cast<const bf16*>(pr.C) + (int64_t)row * pr.ldc + col0;
@@ -197,8 +202,8 @@ __device__ __forceinline__ void apply_c_direct(const GemmProblem& pr, float scal
         for (int e = 0; e < 4; ++e) {
           const float c0 = __uint_as_float(w[e] << 16) + __uint_as_float(wl[e] << 16);
           const float c1 = __uint_as_float(w[e] & 0xffff0000u) + __uint_as_float(wl[e] & 0xffff0000u);
-          v[q * 8 + 2 * e] = scale * fmaf(1.5f, c0, v[q * 8 + 2 * e]);
-          v[q * 8 + 2 * e + 1] = scale * fmaf(1.5f, c1, v[q * 8 + 2 * e + 1]);
+          v[q * 8 + 2 * e] = scale * fmaf(own, c0, v[q * 8 + 2 * e]);
+          v[q * 8 + 2 * e + 1] = scale * fmaf(own, c1, v[q * 8 + 2 * e + 1]);
         }
       }
     } else {
@@ -206,7 +211,7 @@ __device__ __forceinline__ void apply_c_direct(const GemmProblem& pr, float scal
       for (int j = 0; j < NC; ++j) {
         float cv = 0.f;
         if (j < n_valid) cv = __bfloat162float(c[j]) + (cl ? __bfloat162float(cl[j]) : 0.f);
-        v[j] = (j < n_valid) ? scale * fmaf(1.5f, cv, v[j]) : 0.f;
+        v[j] = (j < n_valid) ? scale * fmaf(own, cv, v[j]) : 0.f;
       }
     }
   }
@@ -309,7 +314,8 @@ __device__ __forceinline__ void epilogue_row32(const GemmProblem& pr, const Para
     return;
   }
   apply_c_direct(pr, scale, row, col0, v);
-  if (pr.epi == EPI_APPLY || (pr.epi == EPI_APPLY_PACK && pr.store_out)) store_out_direct(pr, row, col0, v, pr.epi == EPI_APPLY);
+  if (pr.epi == EPI_APPLY || (pr.epi == EPI_APPLY_PACK && pr.store_out))
+    store_out_direct(pr, row, col0, v, pr.epi == EPI_APPLY && pr.hi_only == 0);
   if (pr.epi == EPI_APPLY_PACK) pack_bits_direct(pr, row, col0, v, peers);
   else if (pr.epi == EPI_APPLY_UPDATE) update_weights_direct(pr, params, lr, row, col0, v);
 }

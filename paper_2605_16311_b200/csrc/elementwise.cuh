@@ -382,13 +382,13 @@ __global__ void __launch_bounds__(EW_THREADS) plain_params_kernel(const ParamDev
 
 // ---------------------------------------------------------------------------------------------
 // Stand-alone sign + pack (Alg. 3 "PackBits") for matrix parameters whose rows do not hold whole
-// payload words (cols % 32 != 0), and for K = 0.  Source: bf16 Y_K [M][rows][ldy], or for K = 0
-// the float32 momentum itself.
+// payload words (cols % 32 != 0), and for K = 0.  Source: bf16 Y_K [M][rows][ldy] in the operand buffer the
+// parameter's last apply product wrote, or for K = 0 the float32 momentum itself.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(EW_THREADS) pack_kernel(const ParamDev* __restrict__ params,
                                                           const int32_t* __restrict__ list,
                                                           const uint32_t* __restrict__ starts, int n_list,
-                                                          int src_buf, int from_momentum,
+                                                          int from_momentum,
                                                           uint32_t* __restrict__ bits, int64_t bits_pitch,
                                                           const __grid_constant__ PeerList peers) {
   const int slot = find_slot(starts, n_list, blockIdx.x);
@@ -398,7 +398,7 @@ __global__ void __launch_bounds__(EW_THREADS) pack_kernel(const ParamDev* __rest
   const int m = local / cpw;
   const uint32_t chunk = local - m * cpw;
   const int lane = threadIdx.x & 31;
-  const bf16* y = (src_buf ? pd.y1 : pd.y0) + (int64_t)m * pd.rows * pd.ldy;
+  const bf16* y = (pd.yk_buf ? pd.y1 : pd.y0) + (int64_t)m * pd.rows * pd.ldy;   // where this parameter's Y_K was left
   const float* mom = pd.mom + (int64_t)m * pd.d;
   const int64_t base = (int64_t)chunk * PACK_CHUNK;
 #pragma unroll 4

@@ -570,7 +570,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
           const int epi = (KIND == 0) ? (int)EPI_GRAM : pr.epi;
           const bool store_hi = (KIND == 0 || epi == EPI_APPLY || (epi == EPI_APPLY_PACK && pr.store_out)) &&
                                 pr.tma_out != 0 && rows_live;
-          const bool store_lo = (KIND == 1 && epi == EPI_APPLY) || (KIND == 0 && pr.gram_lo != 0);
+          const bool store_lo = (KIND == 1 && epi == EPI_APPLY && pr.hi_only == 0) || (KIND == 0 && pr.gram_lo != 0);
           const bool mirror = KIND == 0 && pr.sym != 0 && pr.gram_lo == 0 && te.tn != te.tm && rows_live;
           const CUtensorMap* mapO0 = args.tmaps + pr.tmapO0;
           const CUtensorMap* mapO1 = args.tmaps + pr.tmapO1;
@@ -625,11 +625,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
         int n_chunks = (prN - n0 + 63) / 64;
         if (n_chunks > BN / 64) n_chunks = BN / 64;
         const float scale = pr.scale_ptr ? __ldg(pr.scale_ptr) : pr.scale_imm;
+        const float own = pr.own_coef;           // coefficient of the own term (1.5 for one Newton-Schulz step)
         // a CTA whose 128 rows lie wholly below the matrix moves nothing through TMA (it still drains TMEM)
         const bool rows_live = row0 < prM;
         const bool tma_c = KIND == 1 && pr.tma_c != 0 && rows_live, tma_out = pr.tma_out != 0;
         const bool store_hi = KIND == 0 || epi == EPI_APPLY || (epi == EPI_APPLY_PACK && pr.store_out);
-        const bool store_lo = (KIND == 1 && epi == EPI_APPLY) || (KIND == 0 && pr.gram_lo != 0);
+        const bool store_lo = (KIND == 1 && epi == EPI_APPLY && pr.hi_only == 0) || (KIND == 0 && pr.gram_lo != 0);
         const bool mirror = KIND == 0 && pr.sym != 0 && pr.gram_lo == 0 && te.tn != te.tm && rows_live;   // off-diagonal Gram tile
         const uint32_t acc = tcount & 1u;
         const uint32_t acc_round = tcount >> 1;
@@ -668,10 +669,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
                 const uint32_t c16 = funit0 + (uint32_t)cc;
                 const uint4 u = lds128(buf + fhalf * EPI_HALF_BYTES + row_off + ((c16 ^ sw) << 4));
                 float* o = v + cc * 4;
-                o[0] = scale * fmaf(1.5f, __uint_as_float(u.x), o[0]);
-                o[1] = scale * fmaf(1.5f, __uint_as_float(u.y), o[1]);
-                o[2] = scale * fmaf(1.5f, __uint_as_float(u.z), o[2]);
-                o[3] = scale * fmaf(1.5f, __uint_as_float(u.w), o[3]);
+                o[0] = scale * fmaf(own, __uint_as_float(u.x), o[0]);
+                o[1] = scale * fmaf(own, __uint_as_float(u.y), o[1]);
+                o[2] = scale * fmaf(own, __uint_as_float(u.z), o[2]);
+                o[3] = scale * fmaf(own, __uint_as_float(u.w), o[3]);
               }
               // The bf16 results go to this thread's units of BOTH halves, i.e. into fp32 columns that other warps
               // of this lane quarter still have to read: all of them finish reading before any writes.
@@ -696,8 +697,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
                 for (int e = 0; e < 4; ++e) {
                   const float c0 = __uint_as_float(wh[e] << 16) + __uint_as_float(wl[e] << 16);
                   const float c1 = __uint_as_float(wh[e] & 0xffff0000u) + __uint_as_float(wl[e] & 0xffff0000u);
-                  o[2 * e] = scale * fmaf(1.5f, c0, o[2 * e]);
-                  o[2 * e + 1] = scale * fmaf(1.5f, c1, o[2 * e + 1]);
+                  o[2 * e] = scale * fmaf(own, c0, o[2 * e]);
+                  o[2 * e + 1] = scale * fmaf(own, c1, o[2 * e + 1]);
                 }
               }
             }

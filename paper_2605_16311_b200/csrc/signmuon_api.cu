@@ -18,6 +18,7 @@
 #include "ns_gemm_simt.cuh"
 #include "power_iter.cuh"
 #include "ns_gemm_sm100.cuh"
+#include "ns_chain_sm100.cuh"
 
 using namespace signmuon;
 
@@ -35,6 +36,7 @@ struct ParamPlan {
   int32_t ldy, ldq;
   uint32_t n_words, word_off;
   uint32_t chunks_per_worker;
+  bool gs;               // the workers' Newton-Schulz iteration runs in Gram space (on-chip chain; short side <= 256)
   bool fused_pack;       // sign+pack happens in the last apply epilogue
   size_t mom_off;        // bytes into the state buffer
   size_t y_off[2], lo_off[2], q_off, qlo_off, scales_off, partials_off;   // bytes into the workspace (matrix params)
@@ -54,8 +56,14 @@ enum { TM_Y0_K128 = 0, TM_Y0_KBN, TM_Y0_MN, TM_Y1_K128, TM_Y1_KBN, TM_Y1_MN, TM_
 
 struct LaunchPlan {        // one grouped GEMM launch
   size_t problem_base;     // index of its first problem in the problem array
-  int tile_table;          // which tile table (0 gram, 1 apply, 2 gram local-polar, 3 apply local-polar)
+  size_t problem_count;
+  int tile_table;          // which tile table (TT_*): launches with the same problem structure share one
+  bool gram;               // Gram launch (else apply launch)
 };
+
+// Tile tables.  The workers' first Gram launch and last apply launch also carry the parameters whose iteration runs in
+// Gram space (they take part in no other launch), so those two launches have tables of their own.
+enum { TT_GRAM_FIRST = 0, TT_APPLY_LAST, TT_GRAM, TT_APPLY, TT_LP_GRAM, TT_LP_APPLY, TT_COUNT };
 
 struct TileTable {
   std::vector<TileEntry> tiles;         // ordered by CTA
@@ -65,6 +73,9 @@ struct TileTable {
   int ctas = 1;            // CTAs that share a tile
   bool long_k = false;     // tile-weighted mean contraction length >= 1536 (chooses the apply kernel's rings)
   size_t tiles_off = 0, cta_off = 0;    // bytes into the workspace
+  size_t problem_base = 0, problem_count = 0;   // the launch that defines the table (others using it have the same structure)
+  bool used = false;
+  double flops = 0;                     // flops its tiles issue per launch
 };
 
 }  // namespace
@@ -101,7 +112,12 @@ struct signmuon_ctx {
   // GEMM plans
   std::vector<GemmProblem> problems;      // pointers filled at bind
   std::vector<LaunchPlan> ns_launches, lp_launches;
-  TileTable tables[4];
+  TileTable tables[TT_COUNT];
+  // Newton-Schulz in Gram space (short side <= 256): one chain launch between the first Gram and the last apply launch
+  std::vector<ChainProblem> chain_problems;   // pointers as workspace offsets until bind
+  std::vector<uint32_t> chain_order, chain_pair_start;
+  size_t off_chain_problems = 0, off_chain_order = 0, off_chain_start = 0;
+  int chain_pairs = 0;
   int num_tmaps = 0;
   // binding
   bool split = false;      // Newton-Schulz products of the workers in split precision (scale = spectral)
@@ -207,12 +223,18 @@ size_t count_tiles(const std::vector<GemmProblem>& probs, size_t pbase, size_t p
 // Builds the problem list of the Gram (`gram` = true) or apply product of Newton-Schulz
 // iteration k for `workers` batch slots.  Device pointers are left as byte offsets into the
 // workspace (resolved at bind) in the pointer fields.
+// A parameter whose iteration runs in Gram space takes part in the first Gram launch only (A_0 = Y_0 Y_0^T, stored as
+// the hi/lo pair of -A_0/2 for the chain kernel) and in the last apply launch only (Y_K = T_K Y_0 with
+// T_K = (3/2)^K I + F_K: product F_K Y_0 in split precision, own term (3/2)^K Mom from the float32 momentum).
 void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, int k, int K, int workers,
                      bool local_polar_phase) {
   const bool keep = (c->cfg.flags & SIGNMUON_FLAG_KEEP_POLAR) != 0;
   for (int32_t p : c->matrix_list) {
     const ParamPlan& pl = c->plan[p];
-    const int src = k & 1, dst = (k + 1) & 1;
+    const bool gs = pl.gs && !local_polar_phase;
+    if (gs && (gram ? k != 0 : k != K - 1)) continue;
+    const bool first = gs || k == 0;                 // reads the momentum (scale from memory, float32 own term)
+    const int src = gs ? 0 : (k & 1), dst = gs ? 1 : ((k + 1) & 1);
     for (int w = 0; w < workers; ++w) {
       // the local polar step works in its own slot (index M) so the workers' results stay readable
       const int m = local_polar_phase ? c->Wm : w;
@@ -242,7 +264,7 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         pr.sym = (c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) ? 0 : 1;   // square tiles only (bm == bn in every shape)
         pr.tmapOT = pl.tmap_base + TM_Q_BOX64;
         pr.diag_share = 1;                          // A and B are the same rows of the same matrix on diagonal tiles
-        if (c->split && !local_polar_phase) {       // -A/2 as a hi/lo pair, both triangles computed
+        if ((c->split && !local_polar_phase) || gs) {   // -A/2 as a hi/lo pair, both triangles computed
           pr.gram_lo = 1;
           pr.sym = 0;
           pr.diag_share = 0;                        // the segments pair different operands
@@ -268,7 +290,7 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
           pr.tmapA = pr.tmapB = pl.tmap_base + TM_S8;
           pr.batch = 0;                              // the FP8 copy has a single slot
         }
-        if (k == 0) {
+        if (first) {
           if (local_polar_phase) pr.scale_imm = (float)(1.0 / ((double)pl.rows * (double)pl.cols));
           else pr.scale_ptr = reinterpret_cast<const float*>(pl.scales_off + (size_t)m * 8);
         } else {
@@ -289,7 +311,8 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         const size_t lo = pl.lo_off[split ? src : 0] + m * ybytes;       // lo part of Y_k
         const size_t lo_dst = pl.lo_off[split ? dst : 0] + m * ybytes;   // lo part of Y_{k+1}
         const int tlo = split && src ? TM_LO1_K128 : TM_LO0_K128, tlo_dst = split && dst ? TM_LO1_K128 : TM_LO0_K128;
-        if (split) {      // Q Y ~ Qhi Yhi + Qlo Yhi + Qhi Ylo (three operand segments along K)
+        pr.own_coef = gs ? (float)std::pow(1.5, (double)K) : 1.5f;
+        if (split || gs) {      // Q Y ~ Qhi Yhi + Qlo Yhi + Qhi Ylo (three operand segments along K)
           pr.nseg = 3;
           const int tlo_mn = src ? TM_LO1_MN : TM_LO0_MN;
           if (pl.wide) {
@@ -300,14 +323,14 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
             pr.tmapA3 = pl.tmap_base + tlo;         pr.tmapB3 = pr.tmapB;
           }
         }
-        if (k == 0 && !local_polar_phase) {          // own term from the float32 momentum itself
+        if (first && !local_polar_phase) {           // own term from the float32 momentum itself
           pr.c_mode = C_F32;
           pr.C = reinterpret_cast<const void*>(pl.mom_off + (size_t)m * pl.d * 4);   // offset into the state buffer
           pr.ldc = pl.cols;
         } else {
-          pr.c_mode = (k == 0) ? C_BF16 : C_HILO;    // the +-1 vote matrix is exact in bf16
+          pr.c_mode = first ? C_BF16 : C_HILO;       // the +-1 vote matrix is exact in bf16
           pr.C = reinterpret_cast<const void*>(ysrc);
-          pr.C_lo = (k == 0) ? nullptr : reinterpret_cast<const bf16*>(lo);
+          pr.C_lo = first ? nullptr : reinterpret_cast<const bf16*>(lo);
           pr.ldc = pl.ldy;
         }
         pr.out = reinterpret_cast<void*>(ydst);
@@ -327,13 +350,14 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
           pr.tmapC0 = pl.tmap_base + ty;
           pr.tmapC1 = pl.tmap_base + tlo;
         }
-        if (k == 0) {
+        if (first) {
           if (local_polar_phase) pr.scale_imm = (float)(1.0 / std::sqrt((double)pl.rows * (double)pl.cols));
           else pr.scale_ptr = reinterpret_cast<const float*>(pl.scales_off + (size_t)m * 8 + 4);
         } else {
           pr.scale_imm = 1.f;
         }
         const bool last = (k == K - 1);
+        if (gs && !last) continue;                   // (unreachable: filtered above)
         if (!last) pr.epi = EPI_APPLY;
         else if (local_polar_phase || c->muon) pr.epi = EPI_APPLY_UPDATE;   // W <- W - eta Y_K (local polar step; Muon rule)
         else if (pl.fused_pack) {
@@ -342,6 +366,9 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
           // payload word of this (param, worker): resolved at bind from off_bits
           pr.bits_out = reinterpret_cast<uint32_t*>((size_t)(c->w_off + m) * c->bits_pitch * 4 + (size_t)pl.word_off * 4);
         } else pr.epi = EPI_APPLY;
+        // (the lo part of the source is an operand of this product's other tiles: it must not be overwritten; nothing
+        // reads the lo part of Y_K)
+        if (gs) pr.hi_only = 1;
       }
       out.push_back(pr);
     }
@@ -368,6 +395,11 @@ int plan_layout(signmuon_ctx* c) {
     words += pl.n_words;
     pl.chunks_per_worker = (uint32_t)((pl.d + MOM_CHUNK - 1) / MOM_CHUNK);
     pl.fused_pack = (sp.kind == SIGNMUON_PARAM_MATRIX) && K > 0 && (sp.cols % 32 == 0) && !c->muon;
+    // Gram-space iteration for short sides up to 256: needs at least two iterations to pay, the tensor-core kernels,
+    // and the Frobenius scale (with the spectral scale the products already run in split precision the regular way)
+    pl.gs = sp.kind == SIGNMUON_PARAM_MATRIX && K >= 2 && pl.s <= 256 &&
+            !(c->cfg.flags & (SIGNMUON_FLAG_SIMT_GEMM | SIGNMUON_FLAG_NO_GRAM_SPACE)) &&
+            c->cfg.ns_scale == SIGNMUON_SCALE_FRO;
     pl.ld8 = (int32_t)round_up((size_t)sp.cols, 16);
     pl.lp_fp8 = sp.kind == SIGNMUON_PARAM_MATRIX && c->lp && K > 0 &&
                 !(c->cfg.flags & (SIGNMUON_FLAG_SIMT_GEMM | SIGNMUON_FLAG_LP_GRAM_BF16));
@@ -508,48 +540,70 @@ int plan_layout(signmuon_ctx* c) {
     pl.y_off[1] = off; off += ybytes;
     pl.lo_off[0] = pl.lo_off[1] = off; off += ybytes;
     pl.q_off = off; off += round_up(slots * pl.s * pl.ldq * 2, 1024);
-    if (c->split) {
-      pl.lo_off[1] = off; off += ybytes;
-      pl.qlo_off = off; off += round_up(slots * pl.s * pl.ldq * 2, 1024);
-    }
+    if (c->split) { pl.lo_off[1] = off; off += ybytes; }
+    if (c->split || pl.gs) { pl.qlo_off = off; off += round_up(slots * pl.s * pl.ldq * 2, 1024); }
     if (pl.lp_fp8) { pl.s8_off = off; off += round_up((size_t)pl.rows * pl.ld8, 1024); }
   }
   // GEMM problems: K x (gram, apply) for the workers, and again for the local polar step
   c->problems.clear();
   c->ns_launches.clear();
   c->lp_launches.clear();
+  for (int t = 0; t < TT_COUNT; ++t) c->tables[t] = TileTable();
+  auto add_launch = [&](std::vector<LaunchPlan>& ls, bool gram, int k, int workers, bool lp_phase, int table) {
+    LaunchPlan lp;
+    lp.problem_base = c->problems.size();
+    append_problems(c, c->problems, gram, k, K, workers, lp_phase);
+    lp.problem_count = c->problems.size() - lp.problem_base;
+    lp.tile_table = table;
+    lp.gram = gram;
+    if (lp.problem_count == 0) return;                 // (every parameter of this launch iterates in Gram space)
+    TileTable& tt = c->tables[table];
+    if (!tt.used) { tt.used = true; tt.problem_base = lp.problem_base; tt.problem_count = lp.problem_count; }
+    ls.push_back(lp);
+  };
   if (!c->matrix_list.empty()) {
     for (int k = 0; k < K; ++k) {
-      c->ns_launches.push_back({c->problems.size(), 0});
-      append_problems(c, c->problems, true, k, K, M, false);
-      c->ns_launches.push_back({c->problems.size(), 1});
-      append_problems(c, c->problems, false, k, K, M, false);
+      add_launch(c->ns_launches, true, k, M, false, k == 0 ? TT_GRAM_FIRST : TT_GRAM);
+      add_launch(c->ns_launches, false, k, M, false, k == K - 1 ? TT_APPLY_LAST : TT_APPLY);
     }
     if (c->lp) {
       for (int k = 0; k < K; ++k) {
-        c->lp_launches.push_back({c->problems.size(), 2});
-        append_problems(c, c->problems, true, k, K, 1, true);
-        c->lp_launches.push_back({c->problems.size(), 3});
-        append_problems(c, c->problems, false, k, K, 1, true);
+        add_launch(c->lp_launches, true, k, 1, true, TT_LP_GRAM);
+        add_launch(c->lp_launches, false, k, 1, true, TT_LP_APPLY);
       }
     }
   }
   c->off_problems = off; off += round_up(c->problems.size() * sizeof(GemmProblem), ALIGN);
   // tile tables (sizes do not depend on the SM count; the CTA split is made at bind)
-  const size_t nm = c->matrix_list.size();
-  for (int t = 0; t < 4; ++t) {
+  for (int t = 0; t < TT_COUNT; ++t) {
     TileTable& tt = c->tables[t];
     const bool pair = !(c->cfg.flags & (SIGNMUON_FLAG_GEMM_1CTA | SIGNMUON_FLAG_SIMT_GEMM));
     tt.ctas = pair ? 2 : 1;
     tt.bm = pair ? 256 : 128;
     tt.bn = pair ? 256 : 128;
     size_t ntiles = 0;
-    const std::vector<LaunchPlan>& ls = (t < 2) ? c->ns_launches : c->lp_launches;
-    const size_t per = (t < 2) ? nm * M : nm;
-    if (!ls.empty()) ntiles = count_tiles(c->problems, ls[t & 1].problem_base, per, tt.bm, tt.bn);
+    if (tt.used) ntiles = count_tiles(c->problems, tt.problem_base, tt.problem_count, tt.bm, tt.bn);
     tt.tiles_off = off; off += round_up(std::max<size_t>(ntiles, 1) * sizeof(TileEntry), ALIGN);
     tt.cta_off = off; off += round_up((MAX_CTAS + 1) * 4, ALIGN);
   }
+  // chain problems: one per (Gram-space parameter, worker); -A_0/2 in, F_K out (the hi/lo Gram buffers)
+  c->chain_problems.clear();
+  for (int32_t p : c->matrix_list) {
+    const ParamPlan& pl = c->plan[p];
+    if (!pl.gs) continue;
+    const size_t qbytes = (size_t)pl.s * pl.ldq * 2;
+    for (int m = 0; m < M; ++m) {
+      ChainProblem cp;
+      cp.q_hi = reinterpret_cast<bf16*>(pl.q_off + m * qbytes);
+      cp.q_lo = reinterpret_cast<bf16*>(pl.qlo_off + m * qbytes);
+      cp.s = (int32_t)pl.s;
+      cp.ldq = pl.ldq;
+      c->chain_problems.push_back(cp);
+    }
+  }
+  c->off_chain_problems = off; off += round_up(std::max<size_t>(c->chain_problems.size(), 1) * sizeof(ChainProblem), ALIGN);
+  c->off_chain_order = off; off += round_up(std::max<size_t>(c->chain_problems.size(), 1) * 4, ALIGN);
+  c->off_chain_start = off; off += round_up((MAX_CTAS + 1) * 4, ALIGN);
   c->off_tables_end = off;
   c->workspace_bytes = off;
 
@@ -657,7 +711,9 @@ bool opt_in_smem() {
 // many CTA pairs the device can hold at once.
 bool configure_kernels(int* max_pairs) {
   bool ok = opt_in_smem<NS_GEMM_PAIR_GRAM>() && opt_in_smem<NS_GEMM_PAIR_APPLY>() && opt_in_smem<NS_GEMM_ONE_GRAM>() &&
-            opt_in_smem<NS_GEMM_ONE_APPLY>() && opt_in_smem<NS_GEMM_PAIR_APPLY_LONGK>();
+            opt_in_smem<NS_GEMM_ONE_APPLY>() && opt_in_smem<NS_GEMM_PAIR_APPLY_LONGK>() &&
+            cudaFuncSetAttribute(ns_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)CHAIN_SMEM_BYTES) == cudaSuccess;
   if (!ok) return false;
   cudaLaunchConfig_t cfg;
   std::memset(&cfg, 0, sizeof(cfg));
@@ -702,7 +758,7 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
   a.lr = lr;
   a.wait_limit_ns = c->wait_limit_ns;
   a.peers = c->peers;
-  const bool gram = (lp.tile_table & 1) == 0;
+  const bool gram = lp.gram;
   if (tt.ctas == 2) {
     if (gram) launch_tc<NS_GEMM_PAIR_GRAM>(a, tt.grid, s);
     else if (tt.long_k) launch_tc<NS_GEMM_PAIR_APPLY_LONGK>(a, tt.grid, s);
@@ -714,6 +770,31 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
 
 // Vote over `rows` payload rows starting at `src` (default: all workers' rows of the payload buffer), then the
 // update from the vote words.
+// Gram-space chain of the parameters with a short side up to 256: one CTA pair per (parameter, worker) problem list.
+void launch_chain(signmuon_ctx* c, cudaStream_t s) {
+  ChainLaunchArgs a;
+  a.problems = reinterpret_cast<const ChainProblem*>(c->d_ws + c->off_chain_problems);
+  a.order = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_chain_order);
+  a.pair_start = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_chain_start);
+  a.status = reinterpret_cast<uint32_t*>(c->d_ws + c->off_status);
+  a.wait_limit_ns = c->wait_limit_ns;
+  a.K = c->cfg.ns_steps;
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)c->chain_pairs * 2, 1, 1);
+  cfg.blockDim = dim3(CHAIN_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = CHAIN_SMEM_BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, ns_chain_kernel, a);
+}
+
 template <int PLANES>
 void launch_vote(signmuon_ctx* c, float lr, int write_sbar, cudaStream_t s, const uint32_t* src = nullptr, int rows = 0) {
   const ParamDev* pd = cur_paramdev(c);
@@ -851,11 +932,15 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
     }
   }
   if ((mask & SIGNMUON_STAGE_NS) && nm) {
-    for (const LaunchPlan& lp : c->ns_launches) launch_gemm(c, lp, lr, s);
+    bool chain_done = c->chain_problems.empty();
+    for (const LaunchPlan& lp : c->ns_launches) {
+      if (!chain_done && lp.tile_table != TT_GRAM_FIRST) { launch_chain(c, s); chain_done = true; }
+      launch_gemm(c, lp, lr, s);
+    }
     if (c->packfb_blocks) {
       pack_kernel<<<c->packfb_blocks, EW_THREADS, 0, s>>>(
           pd, reinterpret_cast<const int32_t*>(c->d_ws + c->off_list_packfb),
-          reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_packfb), (int)c->packfb_list.size(), K & 1,
+          reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_packfb), (int)c->packfb_list.size(),
           K == 0 ? 1 : 0, bits + (size_t)c->w_off * c->bits_pitch, (int64_t)c->bits_pitch, c->peers);
     }
   }
@@ -1023,7 +1108,8 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     if (pl.kind == SIGNMUON_PARAM_MATRIX) {
       d.y0 = reinterpret_cast<bf16*>(c->d_ws + pl.y_off[0]);
       d.y1 = reinterpret_cast<bf16*>(c->d_ws + pl.y_off[1]);
-      d.ylo = c->split ? reinterpret_cast<bf16*>(c->d_ws + pl.lo_off[0]) : nullptr;
+      d.ylo = (c->split || pl.gs) ? reinterpret_cast<bf16*>(c->d_ws + pl.lo_off[0]) : nullptr;
+      d.yk_buf = pl.gs ? 1 : (c->cfg.ns_steps & 1);
       d.scales = reinterpret_cast<float*>(c->d_ws + pl.scales_off);
       d.partials = reinterpret_cast<float*>(c->d_ws + pl.partials_off);
       if (c->power_start_floats) {
@@ -1062,34 +1148,63 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
   int max_pairs = 1;
   if (!configure_kernels(&max_pairs)) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
   max_pairs = std::min(max_pairs, MAX_CTAS);
-  for (int t = 0; t < 4; ++t) {
+  for (int t = 0; t < TT_COUNT; ++t) {
     TileTable& tt = c->tables[t];
-    const std::vector<LaunchPlan>& ls = (t < 2) ? c->ns_launches : c->lp_launches;
     tt.tiles.clear();
-    if (ls.empty()) continue;
-    build_tile_table(tt, c->problems, ls[t & 1].problem_base, (t < 2) ? nm * M : nm,
-                     tt.ctas == 2 ? max_pairs : c->num_sms);
+    tt.flops = 0;
+    if (!tt.used) continue;
+    build_tile_table(tt, c->problems, tt.problem_base, tt.problem_count, tt.ctas == 2 ? max_pairs : c->num_sms);
     ok = ok && up(tt.tiles_off, tt.tiles.data(), tt.tiles.size() * sizeof(TileEntry));
     ok = ok && up(tt.cta_off, tt.cta_start.data(), tt.cta_start.size() * 4);
-  }
-  // Flops the tensor cores are asked for per step: every scheduled tile issues whole bm x bn x 64 blocks (ragged
-  // edges are zero-filled, skipped mirror tiles of the symmetric Gram products are not issued at all), once per
-  // operand segment; each tile table is launched K times.
-  c->executed_flops = 0;
-  for (int t = 0; t < 4; ++t) {
-    const TileTable& tt = c->tables[t];
-    const std::vector<LaunchPlan>& ls = (t < 2) ? c->ns_launches : c->lp_launches;
-    if (ls.empty()) continue;
-    double f = 0;
+    // Flops the tensor cores are asked for by one launch of this table: every scheduled tile issues whole
+    // bm x bn x (128 bytes of K) blocks (ragged edges are zero-filled, skipped mirror tiles of the symmetric Gram
+    // products are not issued at all), once per operand segment.
     for (const TileEntry& te : tt.tiles) {
-      const GemmProblem& pr = c->problems[ls[t & 1].problem_base + te.problem];
+      const GemmProblem& pr = c->problems[tt.problem_base + te.problem];
       const int kelem = pr.fp8 ? 2 * GEMM_BK : GEMM_BK;
       const double kblocks = (double)((pr.K + kelem - 1) / kelem) * (pr.nseg > 1 ? pr.nseg : 1);
-      f += 2.0 * tt.bm * tt.bn * kelem * kblocks;
+      tt.flops += 2.0 * tt.bm * tt.bn * kelem * kblocks;
     }
-    // (a tile table serves the K launches of its kind; the FP8 first Gram of the local polar step has the same
-    // tiles and, per tile, the same flops as the bf16 Gram launches that follow it)
-    c->executed_flops += f * c->cfg.ns_steps;
+  }
+  c->executed_flops = 0;
+  for (const LaunchPlan& lp : c->ns_launches) c->executed_flops += c->tables[lp.tile_table].flops;
+  for (const LaunchPlan& lp : c->lp_launches) c->executed_flops += c->tables[lp.tile_table].flops;
+  // chain launch: problems to CTA pairs, longest first (cost ~ s^2: contraction steps x columns walked)
+  c->chain_pairs = 0;
+  if (!c->chain_problems.empty()) {
+    const int K = c->cfg.ns_steps;
+    std::vector<ChainProblem> cps = c->chain_problems;
+    std::vector<uint32_t> idx(cps.size());
+    for (size_t i = 0; i < cps.size(); ++i) {
+      idx[i] = (uint32_t)i;
+      cps[i].q_hi = reinterpret_cast<bf16*>(c->d_ws + reinterpret_cast<size_t>(cps[i].q_hi));
+      cps[i].q_lo = reinterpret_cast<bf16*>(c->d_ws + reinterpret_cast<size_t>(cps[i].q_lo));
+      // products of the chain: A A and A (A A) in every iteration but the last, A F in every iteration but the first
+      c->executed_flops += 3.0 * (K - 1) * 2.0 * 256.0 * 256.0 * (double)(((cps[i].s + 15) / 16) * 16);
+    }
+    std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) { return cps[a].s > cps[b].s; });
+    c->chain_pairs = (int)std::min<size_t>((size_t)max_pairs, cps.size());
+    std::vector<std::vector<uint32_t>> per((size_t)c->chain_pairs);
+    typedef std::pair<long long, int> Load;
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int i = 0; i < c->chain_pairs; ++i) heap.push({0, i});
+    for (uint32_t i : idx) {
+      Load top = heap.top();
+      heap.pop();
+      per[top.second].push_back(i);
+      heap.push({top.first + (long long)cps[i].s * cps[i].s + 4096, top.second});
+    }
+    c->chain_order.clear();
+    c->chain_pair_start.assign((size_t)c->chain_pairs + 1, 0);
+    for (int i = 0; i < c->chain_pairs; ++i) {
+      c->chain_pair_start[i] = (uint32_t)c->chain_order.size();
+      c->chain_order.insert(c->chain_order.end(), per[i].begin(), per[i].end());
+    }
+    c->chain_pair_start[c->chain_pairs] = (uint32_t)c->chain_order.size();
+    ok = ok && up(c->off_chain_problems, cps.data(), cps.size() * sizeof(ChainProblem));
+    ok = ok && up(c->off_chain_order, c->chain_order.data(), c->chain_order.size() * 4);
+    ok = ok && up(c->off_chain_start, c->chain_pair_start.data(), c->chain_pair_start.size() * 4);
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;      // (cps dies with this scope)
   }
   // (moved up) kernels configured before the tile tables are split
   std::vector<CUtensorMap> maps((size_t)c->num_tmaps);
@@ -1118,7 +1233,7 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
         ok = ok && encode_map(mp + (b2 ? TM_LO1_MN : TM_LO0_MN), c->d_ws + pl.lo_off[b2], pl.cols, pl.rows, slots,
                               pl.ldy, (uint64_t)pl.rows * pl.ldy, 64);
       }
-      if (c->split) {
+      if (c->split || pl.gs) {
         ok = ok && encode_map(mp + TM_QLO_K128, c->d_ws + pl.qlo_off, pl.s, pl.s, slots, pl.ldq, qb, 128);
         ok = ok && encode_map(mp + TM_QLO_KBN, c->d_ws + pl.qlo_off, pl.s, pl.s, slots, pl.ldq, qb, bn);
       }
@@ -1350,7 +1465,7 @@ int signmuon_debug_tap(const signmuon_ctx* c, int32_t what, int32_t param, int32
       if (pl.kind != SIGNMUON_PARAM_MATRIX) return SIGNMUON_ERR_INVALID_ARG;
       if (!(c->cfg.flags & SIGNMUON_FLAG_KEEP_POLAR) && pl.fused_pack) return SIGNMUON_ERR_INVALID_ARG;
       const size_t yb = (size_t)pl.rows * pl.ldy * 2;
-      ptr = c->d_ws + pl.y_off[c->cfg.ns_steps & 1] + (size_t)lw * yb; nbytes = yb; pitch = pl.ldy; break;
+      ptr = c->d_ws + pl.y_off[pl.gs ? 1 : (c->cfg.ns_steps & 1)] + (size_t)lw * yb; nbytes = yb; pitch = pl.ldy; break;
     }
     case SIGNMUON_TAP_VOTE_BITS:
       ptr = c->d_ws + c->off_vote + (size_t)pl.word_off * 4; nbytes = (size_t)pl.n_words * 4; break;
@@ -1451,6 +1566,7 @@ int signmuon_launches_per_step(const signmuon_ctx* c, int32_t* launches) {
   if (nm) n += 1 + (c->power_start_floats ? 3 + 4 * c->cfg.power_iters : 1);   // momentum + norms (or power iteration)
   if (!c->plain_list.empty()) n += 1;
   if (nm) n += (int)c->ns_launches.size() + (c->packfb_blocks ? 1 : 0);       // NS, fallback pack
+  if (!c->chain_problems.empty()) n += 1;                                     // Gram-space chain
   if (!c->vote_list.empty()) n += 2;                                          // vote, update
   if (nm && c->lp && c->cfg.ns_steps > 0) n += (int)c->lp_launches.size();
   if (c->peer_flags.n > 0) n += 2;                                            // publish, await (fused exchange)

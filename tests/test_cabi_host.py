@@ -101,8 +101,12 @@ def test_ragged_parameter_pads_to_words():
     _, nbytes, entries = B.signmuon_packed_payload(ctx, 1, want_ptr=False)
     assert entries == 38 and nbytes == 4 * (2 + 1)
     assert B.signmuon_payload_segment(ctx, 1) == (2, 1)
-    # momentum, norms, plain kernel, 2x2 NS products, fallback pack (11 columns do not fill words), vote, update
-    assert B.signmuon_launches_per_step(ctx) == 2 + 1 + 4 + 1 + 2
+    # momentum, norms, plain kernel; the 3 x 11 matrix iterates in Gram space (first Gram product, on-chip chain, last
+    # apply product); fallback pack (11 columns do not fill words), vote, update
+    assert B.signmuon_launches_per_step(ctx) == 2 + 1 + 3 + 1 + 2
+    full = B.signmuon_create([(3, 11, 0, 0, 0), (1, 5, 1, 0, 0)], 3, 0.9, 1e-3, 2, False, flags=B.FLAG_NO_GRAM_SPACE)
+    assert B.signmuon_launches_per_step(full) == 2 + 1 + 4 + 1 + 2          # 2 x 2 products on the full matrix
+    B.signmuon_destroy(full)
     B.signmuon_destroy(ctx)
 
 

@@ -208,6 +208,30 @@ def test_default_flags_path_against_oracle():
         _same_bits_and_weights(plain, kept)
 
 
+@pytest.mark.parametrize("K", [2, 5])
+def test_gram_space_iteration_against_oracle_and_full_matrix_iteration(K):
+    """Short sides up to 256 iterate in Gram space (one Gram launch, the on-chip chain, one apply launch).  Both that
+    path and the per-iteration path (FLAG_NO_GRAM_SPACE) are held to the oracle's Alg. 4 at the same tolerances; their
+    sign bits agree with each other wherever the oracle's value is not next to zero (both are confined to 1e-3 RMS)."""
+    import numpy as np
+    from parity_utils import run_and_check
+    shapes = [(64, 576), (576, 64), (100, 328), (129, 520), (200, 200), (256, 1024), (1024, 256), (256, 256),
+              (64, 147), (8, 64), (320, 512)]
+    wl = _wl(shapes, 3, K=K)
+    rep_gs, rep_full, cap_gs, cap_full = {}, {}, {}, {}
+    run_and_check(wl, steps=2, report=rep_gs, capture=cap_gs)
+    run_and_check(wl, steps=2, flags=B.FLAG_KEEP_POLAR | B.FLAG_NO_GRAM_SPACE, report=rep_full, capture=cap_full)
+    print("gram space:", rep_gs, "\nper iteration:", rep_full)
+    assert rep_gs["polar_relfro"] <= 2e-2 and rep_full["polar_relfro"] <= 2e-2
+    for m in range(wl.num_workers):
+        a = cap_gs["payloads"][0][m].cpu().numpy().view(np.uint8)
+        b = cap_full["payloads"][0][m].cpu().numpy().view(np.uint8)
+        differing = int(np.unpackbits(a ^ b).sum())
+        assert differing <= 2e-3 * wl.numel
+    # default flags (no stored Y_K) on the same set
+    run_and_check(wl, steps=1, flags=0)
+
+
 def test_default_flags_path_full_llama_layer_sampled():
     """Config 4 at full size in the benchmark's launch configuration (flags = 0, local polar on)."""
     from parity_utils import run_and_check
