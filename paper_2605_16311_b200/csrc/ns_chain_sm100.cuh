@@ -14,8 +14,10 @@
 //
 // Per CTA (rank r of the pair): rows [128 r, 128 r + 128) of every matrix.  A symmetric matrix serves as the A operand
 // (its rows) and as the B operand (b(j,k) = X[j][k], rows again), so each CTA only ever needs its own rows: what its
-// threads compute (thread = row = TMEM lane) is what its next MMA reads.  Shared memory: A_hi, A_lo and X (S_hi or
-// F_hi), 64 KB each, K-major with 128-byte swizzle in four 64-column blocks.  Tensor memory: D0 (A-chain), D1 (Z).
+// threads compute is what its next MMA reads.  Thread = row = TMEM lane; the four warps that share a tensor-memory lane
+// quarter split the 32-column chunks between them (a thread always meets the same (row, chunk) cells, so the
+// combination phases need no barrier of their own).  Shared memory: A_hi, A_lo and X (S_hi or F_hi), 64 KB each,
+// K-major with 128-byte swizzle in four 64-column blocks.  Tensor memory: D0 (A-chain), D1 (Z).
 //
 //   input : Q_hi, Q_lo = hi/lo pair of -A_0 / 2 (what the Gram launch stores), [s][ldq] bf16
 //   output: F_K as a hi/lo pair, written over the input; the apply launch then forms
@@ -42,7 +44,8 @@ struct ChainLaunchArgs {
   int32_t K;                    // Newton-Schulz iterations (>= 2)
 };
 
-constexpr int CHAIN_THREADS = 128;
+constexpr int CHAIN_COLGROUPS = 4;                           // warps that share a lane quarter, each walking every 4th chunk
+constexpr int CHAIN_THREADS = 128 * CHAIN_COLGROUPS;
 constexpr uint32_t CHAIN_BUF_BYTES = 128 * 256 * 2;            // 128 rows x 256 columns of bf16
 constexpr size_t CHAIN_SMEM_BYTES = 3 * CHAIN_BUF_BYTES + 1024;
 
@@ -105,7 +108,9 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) ns_chain_kernel(const __grid
   const uint32_t smem_base = (smem_u32(chain_smem_raw) + 1023u) & ~1023u;
   const uint32_t buf_ahi = smem_base, buf_alo = smem_base + CHAIN_BUF_BYTES, buf_x = smem_base + 2 * CHAIN_BUF_BYTES;
   const int warp = threadIdx.x >> 5;
-  const int row = threadIdx.x;                          // row of this CTA's 128 = TMEM lane
+  const int quarter = warp & 3;                         // tensor-memory lane quarter this warp may access
+  const int cg = warp >> 2;                             // which of the 32-column chunks this warp walks: cg, cg + 4, ...
+  const int row = quarter * 32 + (threadIdx.x & 31);    // row of this CTA's 128 = TMEM lane
   const uint32_t rank = cluster_cta_rank();             // rank 0 issues the pair's MMAs
   const uint32_t pair = blockIdx.x >> 1;
   volatile uint32_t* abort_flag = &abort_word;
@@ -124,7 +129,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) ns_chain_kernel(const __grid
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = tmem_slot;
-  const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);     // this warp's lane quarter
+  const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);  // this warp's lane quarter
   const uint32_t d0 = t_lane, d1 = t_lane + 256u;                        // A-chain accumulator, Z = -2 F
   const uint32_t d0_mma = tmem_base, d1_mma = tmem_base + 256u;
 
@@ -167,7 +172,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) ns_chain_kernel(const __grid
     const bool live = grow < s;
 
     // ---- load -A_0/2 (hi/lo), form A_0 = -2 (hi + lo): A buffers <- split(A_0), D1 <- Z_1 = A_0 (F_1 = -A_0 / 2)
-    for (int ch = 0; ch < chunks; ++ch) {
+    for (int ch = cg; ch < chunks; ch += CHAIN_COLGROUPS) {
       float a[32];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
@@ -195,7 +200,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) ns_chain_kernel(const __grid
       const bool last = (k == args.K - 1);
       if (k > 0) {
         // X <- hi(F_k), F_k = -Z_k / 2;  D1 <- 3/2 Z_k + t_k A_k  (the MMA then adds A_k F_k: Z_{k+1})
-        for (int ch = 0; ch < chunks; ++ch) {
+        for (int ch = cg; ch < chunks; ch += CHAIN_COLGROUPS) {
           float z[32], a[32];
           tc_ld32(d1 + ch * 32, z);
           chain_load_row32(buf_ahi, buf_alo, row, ch, a);
@@ -220,7 +225,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) ns_chain_kernel(const __grid
       await_mma();
       if (!last) {
         // X <- hi(S);  D0 <- 9 A_k - 6 S  (the MMA then adds A_k S: 4 A_{k+1})
-        for (int ch = 0; ch < chunks; ++ch) {
+        for (int ch = cg; ch < chunks; ch += CHAIN_COLGROUPS) {
           float sv[32], a[32];
           tc_ld32(d0 + ch * 32, sv);
           chain_load_row32(buf_ahi, buf_alo, row, ch, a);
@@ -240,7 +245,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) ns_chain_kernel(const __grid
         }
         await_mma();
         // A buffers <- split(A_{k+1})
-        for (int ch = 0; ch < chunks; ++ch) {
+        for (int ch = cg; ch < chunks; ch += CHAIN_COLGROUPS) {
           float v[32];
           tc_ld32(d0 + ch * 32, v);
 #pragma unroll
@@ -252,7 +257,7 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) ns_chain_kernel(const __grid
     }
 
     // ---- F_K = -Z_K / 2 as a hi/lo pair, over the input (tensor-memory reads are warp-wide: every lane takes them)
-    for (int ch = 0; ch < chunks; ++ch) {
+    for (int ch = cg; ch < chunks; ch += CHAIN_COLGROUPS) {
       float z[32];
       tc_ld32(d1 + ch * 32, z);
       if (!(live && ok)) continue;
