@@ -139,10 +139,12 @@ __global__ void __launch_bounds__(CHAIN_THREADS, 1) ns_chain_kernel(const __grid
   // One product D (+)= X Y^T-form with both operands K-major in shared memory (rows = this CTA's 128 rows of X as
   // A operand and of Y as B operand), contraction over the first k16 blocks of 16 columns.
   auto issue_product = [&](uint32_t d_tmem, uint32_t buf_a, uint32_t buf_b, uint32_t idesc, int k16, bool accumulate) {
+    // descriptor low words: start address (16-byte units) | leading byte offset 16; K-major, stride byte offset 1024
+    const uint32_t a_lo = ((buf_a >> 4) & 0x3fffu) | (1u << 16), b_lo = ((buf_b >> 4) & 0x3fffu) | (1u << 16);
     for (int ks = 0; ks < k16; ++ks) {
-      const uint32_t off = (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32u;
-      tc_mma_f16_pair(d_tmem, smem_desc(buf_a + off, 16, 1024), smem_desc(buf_b + off, 16, 1024), idesc,
-                      (accumulate || ks > 0) ? 1u : 0u);
+      const uint32_t off16 = (uint32_t)(ks >> 2) * (16384u >> 4) + (uint32_t)(ks & 3) * 2u;
+      tc_mma_words<true, false>(d_tmem, a_lo + off16, b_lo + off16, SMEM_DESC_HI_SBO1024, idesc,
+                                (accumulate || ks > 0) ? 1u : 0u);
     }
   };
   // Everything the threads of both CTAs wrote (shared memory, tensor memory) becomes visible to the MMAs issued next.

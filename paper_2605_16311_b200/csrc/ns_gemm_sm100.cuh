@@ -41,6 +41,8 @@
 // STATUS_TIMEOUT in the status word, raises a CTA-wide abort flag and the CTA drains and exits (TMEM is freed).
 #pragma once
 
+#include <type_traits>
+
 #include <cuda.h>
 
 #include "common.cuh"
@@ -156,47 +158,10 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                           uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// FP8 (E4M3 x E4M3 -> fp32) forms of the same instructions: K = 32 elements (32 bytes) per instruction.
-__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void tc_mma_f8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                               uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// CTA-pair forms: the MMA spans both CTAs; the commit arrives on the barrier at the same offset in both.
-__device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                                uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
+// CTA-pair form: the MMA spans both CTAs; the commit arrives on the barrier at the same offset in both.
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
   const uint16_t mask = 3;
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -262,6 +227,32 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   d |= (uint64_t)1 << 46;
   d |= (uint64_t)2 << 61;
   return d;
+}
+
+// High word of such a descriptor with a stride byte offset of 1024 (every operand tile here), and the MMA issued from
+// the two descriptor words of each operand (A and B share the high word).  kind::f16 takes bf16 x bf16 -> fp32 with
+// K = 16 per instruction, kind::f8f6f4 E4M3 x E4M3 -> fp32 with K = 32 (32 bytes either way).
+constexpr uint32_t SMEM_DESC_HI_SBO1024 = ((1024u >> 4) & 0x3fffu) | (1u << 14) | (2u << 29);
+template <bool PAIR, bool FP8>
+__device__ __forceinline__ void tc_mma_words(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                             uint32_t accumulate) {
+  if (PAIR && FP8) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+  } else if (PAIR) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+  } else if (FP8) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+  } else {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+  }
 }
 
 // Instruction descriptor: D fp32 (bits [4,6) = 1), A/B format in bits [7,10) and [10,13) (kind::f16: 1 = bf16;
@@ -482,26 +473,29 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
         if (!mbar_wait(smem_u32(&tmem_empty_bar[acc]), (acc_round & 1u) ^ 1u, abort_flag, args.status, args.wait_limit_ns)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb = 0; kb < nk; ++kb) {
-          if (!mbar_wait(smem_u32(&full_bar[0]) + 8u * s, par, abort_flag, args.status, args.wait_limit_ns)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t sa = smem_base + s * STAGE_BYTES;
-          const uint32_t sb = share_ab ? sa : sa + A_BYTES;
+        // The descriptors of a tile differ only in their start-address field: the low word is the stage's address
+        // field plus a per-tile constant (leading byte offset), advanced by a per-tile step for each of the four
+        // instructions of a K block; the high word (stride byte offset 1024, version, 128-byte swizzle) never changes.
+        const uint32_t a_lo_const = ((a_mn ? mn_lbo : 16u) >> 4) << 16, b_lo_const = ((b_mn ? mn_lbo : 16u) >> 4) << 16;
+        const uint32_t a_step = (a_mn ? mn_step : 32u) >> 4, b_step = (b_mn ? mn_step : 32u) >> 4;
+        const uint32_t b_off = share_ab ? 0u : A_BYTES;
+        auto run_tile = [&](auto fp8_tag) {
+          constexpr bool FP8 = decltype(fp8_tag)::value;
+          for (int kb = 0; kb < nk; ++kb) {
+            if (!mbar_wait(smem_u32(&full_bar[0]) + 8u * s, par, abort_flag, args.status, args.wait_limit_ns)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = smem_base + s * STAGE_BYTES;
+            const uint32_t a_lo = ((sa >> 4) & 0x3fffu) | a_lo_const, b_lo = (((sa + b_off) >> 4) & 0x3fffu) | b_lo_const;
 #pragma unroll
-          for (int kk = 0; kk < GEMM_BK / 16; ++kk) {
-            const uint64_t adesc = a_mn ? smem_desc(sa + kk * mn_step, mn_lbo, 1024) : smem_desc(sa + kk * 32, 16, 1024);
-            const uint64_t bdesc = b_mn ? smem_desc(sb + kk * mn_step, mn_lbo, 1024) : smem_desc(sb + kk * 32, 16, 1024);
-            const uint32_t accum = (kb | kk) != 0 ? 1u : 0u;
-            if (fp8) {
-              if (CTAS == 2) tc_mma_f8_pair(d_tmem, adesc, bdesc, idesc, accum); else tc_mma_f8(d_tmem, adesc, bdesc, idesc, accum);
-            } else {
-              if (CTAS == 2) tc_mma_f16_pair(d_tmem, adesc, bdesc, idesc, accum); else tc_mma_f16(d_tmem, adesc, bdesc, idesc, accum);
-            }
+            for (int kk = 0; kk < GEMM_BK / 16; ++kk)
+              tc_mma_words<CTAS == 2, FP8>(d_tmem, a_lo + kk * a_step, b_lo + kk * b_step, SMEM_DESC_HI_SBO1024, idesc,
+                                           (kb | kk) != 0 ? 1u : 0u);
+            // frees the stage (in both CTAs of a pair) once these MMAs have read it
+            if (CTAS == 2) tc_commit_pair(smem_u32(&empty_bar[0]) + 8u * s); else tc_commit(smem_u32(&empty_bar[0]) + 8u * s);
+            if (++s == STAGES) { s = 0; par ^= 1u; }
           }
-          // frees the stage (in both CTAs of a pair) once these MMAs have read it
-          if (CTAS == 2) tc_commit_pair(smem_u32(&empty_bar[0]) + 8u * s); else tc_commit(smem_u32(&empty_bar[0]) + 8u * s);
-          if (++s == STAGES) { s = 0; par ^= 1u; }
-        }
+        };
+        if (fp8) run_tile(std::integral_constant<bool, true>{}); else run_tile(std::integral_constant<bool, false>{});
         if (ok) {                                    // accumulator complete
           if (CTAS == 2) tc_commit_pair(smem_u32(&tmem_full_bar[acc])); else tc_commit(smem_u32(&tmem_full_bar[acc]));
         }
