@@ -262,7 +262,6 @@ def kernel_report(wl, opt, stage_ms, peaks, clocks, timed_region_s, ns_scale="fr
     plain = [p for p in wl.params if p.kind == "plain"]
     gb = {"f32": 4, "bf16": 2}
     K = wl.ns_steps
-    slots = M + (1 if wl.local_polar else 0)
     ns_flops = opt.ns_flops_per_step
     ns_exec = opt.ns_executed_flops_per_step
     mom_bytes = sum(M * p.numel * (gb[p.dtype] + 4 + 4 + 2) for p in mat) + \
@@ -285,8 +284,14 @@ def kernel_report(wl, opt, stage_ms, peaks, clocks, timed_region_s, ns_scale="fr
         method_bytes = sum(M * p.numel * (4 + 1 / 8) for p in mat) + \
             (sum(p.numel * (2 + 2 * gb[p.dtype]) for p in mat) if wl.local_polar else 0)
         # What this implementation moves: per entry, batch slot and iteration the Gram product reads the bf16 iterate
-        # (2 B), the apply product reads it again as an operand (2 B) and moves the hi + lo pair in and out (8 B).
-        impl_bytes = sum(12.0 * p.numel * K * slots for p in mat)
+        # (2 B), the apply product reads it again as an operand (2 B) and moves the hi + lo pair in and out (8 B).  A
+        # matrix whose workers iterate in Gram space (short side <= 256, K >= 2, Frobenius scale) crosses HBM twice per
+        # step instead: hi + lo operands of the one Gram product (4 B), hi + lo operands of the one apply product (4 B)
+        # and the float32 momentum as its own term (4 B); the local polar step always iterates on the full matrix.
+        def gram_space(p):
+            return min(p.rows, p.cols) <= 256 and K >= 2 and ns_scale == "fro"
+        impl_bytes = sum(12.0 * p.numel * (M if gram_space(p) else K * M) + (12.0 * p.numel * K if wl.local_polar else 0.0)
+                         for p in mat)
         kernels["ns_gemm_tc"] = {
             "ms": ns_ms, "bound": "tensor", "launches": launches, "algorithmic_flops": ns_flops,
             "executed_flops": ns_exec, "achieved_tflops": tf, "executed_tflops": ns_exec / ns_ms / 1e9,

@@ -37,6 +37,10 @@
 // Gram products are symmetric: only tiles on or above the diagonal are scheduled and an off-diagonal tile is
 // also stored transposed.  A problem may carry up to three operand pairs ("segments") that are accumulated
 // into the same tile along K: split-precision products (hi hi + lo hi + hi lo) of the spectral scale.
+// Warps (384 threads): 0 = TMA of the A operand, 1 = MMA issue, 2..9 = epilogue math, 10 = epilogue TMA, 11 = TMA of the
+// B operand.  The single threads of warps 0, 1 and 11 sit on the critical path of every K block (512 tensor-core cycles
+// on a CTA pair): the MMA thread forms its descriptors by adding a step to precomputed words, and the copies of a
+// stage are split over two threads.
 // Every wait is bounded: after the launch's wait limit (two seconds by default) a waiting thread records
 // STATUS_TIMEOUT in the status word, raises a CTA-wide abort flag and the CTA drains and exits (TMEM is freed).
 #pragma once
@@ -54,8 +58,9 @@ constexpr int GEMM_BK = 64;
 constexpr int EPI_WARPS = 8;                 // EPI_WARPS / 4 warps per TMEM lane quarter, each NCOL of a chunk's 64 columns
 constexpr int EPI_NCOL = 256 / EPI_WARPS;    // columns of a chunk one math thread owns (32 or 16)
 static_assert(EPI_WARPS == 8 || EPI_WARPS == 16, "8 or 16 epilogue math warps");
-constexpr int GEMM_THREADS = 32 * (3 + EPI_WARPS);   // warp 0: operand TMA, warp 1: MMA, then the epilogue math warps,
-                                                     // last warp: epilogue TMA (C loads, result stores)
+constexpr int GEMM_THREADS = 32 * (4 + EPI_WARPS);   // warp 0: TMA of the A operand, warp 1: MMA, then the epilogue math warps,
+                                                     // then the epilogue TMA warp (C loads, result stores), last warp: TMA
+                                                     // of the B operand
 constexpr uint64_t DEFAULT_WAIT_LIMIT_NS = 2000000000ull;   // two seconds unless the caller sets another limit
 
 struct GemmLaunchArgs {
@@ -376,9 +381,15 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
   };
   const int row_shift = (int)cta_rank * GEMM_BM;   // this CTA's rows inside the tile of the pair
 
-  if (warp == 0) {
-    // ===================================================================== TMA producer
+  if (warp == 0 || warp == 3 + EPI_WARPS) {
+    // ===================================================================== TMA producers
+    // Two threads feed the operand ring: one loads the A tiles (and, in CTA 0, posts the bytes a stage expects), the
+    // other the B tiles.  Both wait on the same "stage empty" barriers.  A B copy may complete before the A thread has
+    // posted the expected bytes of its stage: the barrier's transaction count is signed, and its phase cannot end
+    // before that post, which is also the phase's only pending arrival.  (One thread issuing all copies of a stage
+    // - four when both operands are MN-major - was the bound of those launches.)
     if (lane == 0) {
+      const bool do_a = (warp == 0);
       uint32_t it = 0;   // running k-block counter across tiles
       uint32_t s = 0, par = 1;   // ring position and the parity to wait for on its "empty" barrier
       const uint32_t full0 = (CTAS == 2) ? map_to_cta(smem_u32(&full_bar[0]), 0) : smem_u32(&full_bar[0]);
@@ -386,12 +397,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
       for (uint32_t t = tile_begin; t < tile_end && ok; ++t) {
         const TileEntry te = args.tiles[t];
         const GemmProblem& pr = args.problems[te.problem];
-        const CUtensorMap* mapA = args.tmaps + pr.tmapA;
-        const CUtensorMap* mapB = args.tmaps + pr.tmapB;
-        const int m0 = te.tm * TILE_M + (int)cta_rank * GEMM_BM;       // this CTA's rows of A
-        const int n0 = te.tn * BN + (int)cta_rank * B_ROWS;            // this CTA's rows of B
+        const CUtensorMap* map = args.tmaps + (do_a ? pr.tmapA : pr.tmapB);
+        // this CTA's rows of its operand
+        const int r0 = do_a ? te.tm * TILE_M + (int)cta_rank * GEMM_BM : te.tn * BN + (int)cta_rank * B_ROWS;
         const int batch = pr.batch;
-        const int a_mn = pr.a_mn, b_mn = pr.b_mn;
+        const int mn = do_a ? pr.a_mn : pr.b_mn;
         // FP8 operands (Gram launches only): a stage still holds 128 bytes along K, i.e. 128 elements instead of 64,
         // and an MN-major tile is one 128-wide chunk of 128 k-rows instead of two 64-wide chunks of 64
         const bool fp8 = KIND == 0 && pr.fp8 != 0;
@@ -402,33 +412,25 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
         // and the MMA reads the A tile for both operands (B_ROWS == GEMM_BM and equal box shapes).
         const bool share_ab = KIND == 0 && B_ROWS == GEMM_BM && pr.diag_share != 0 && te.tm == te.tn;
         const uint32_t stage_tx = share_ab ? CTAS * A_BYTES : CTAS * STAGE_BYTES;
+        const bool skip = !do_a && share_ab;
+        const int chunks = (do_a ? GEMM_BM : B_ROWS) / 64;
         for (int seg = 0; seg < nseg && ok; ++seg) {
-          if (seg == 1) { mapA = args.tmaps + pr.tmapA2; mapB = args.tmaps + pr.tmapB2; }
-          else if (seg == 2) { mapA = args.tmaps + pr.tmapA3; mapB = args.tmaps + pr.tmapB3; }
+          if (seg == 1) map = args.tmaps + (do_a ? pr.tmapA2 : pr.tmapB2);
+          else if (seg == 2) map = args.tmaps + (do_a ? pr.tmapA3 : pr.tmapB3);
           for (int kb = 0; kb < nk; ++kb, ++it) {
             if (!mbar_wait(smem_u32(&empty_bar[0]) + 8u * s, par, abort_flag, args.status, args.wait_limit_ns)) { ok = false; break; }
             // the "full" barrier of the pair is CTA 0's: it expects the bytes of both CTAs
             const uint32_t fb = full0 + 8u * s;
-            if (cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[0]) + 8u * s, stage_tx);
-            const uint32_t sa = smem_base + s * STAGE_BYTES;
-            const uint32_t sb = sa + A_BYTES;
+            if (do_a && cta_rank == 0) mbar_expect_tx(smem_u32(&full_bar[0]) + 8u * s, stage_tx);
+            const uint32_t dst = smem_base + s * STAGE_BYTES + (do_a ? 0u : A_BYTES);
             const int k0 = kb * kelem;
-            if (!a_mn) {
-              load_operand(sa, mapA, k0, m0, batch, fb);
+            if (skip) {
+            } else if (!mn) {
+              load_operand(dst, map, k0, r0, batch, fb);
             } else if (fp8) {
-              load_operand(sa, mapA, m0, k0, batch, fb);
+              load_operand(dst, map, r0, k0, batch, fb);
             } else {
-#pragma unroll
-              for (int c = 0; c < GEMM_BM / 64; ++c) load_operand(sa + c * 8192, mapA, m0 + 64 * c, k0, batch, fb);
-            }
-            if (share_ab) {
-            } else if (!b_mn) {
-              load_operand(sb, mapB, k0, n0, batch, fb);
-            } else if (fp8) {
-              load_operand(sb, mapB, n0, k0, batch, fb);
-            } else {
-#pragma unroll
-              for (int c = 0; c < B_ROWS / 64; ++c) load_operand(sb + c * 8192, mapB, n0 + 64 * c, k0, batch, fb);
+              for (int c = 0; c < chunks; ++c) load_operand(dst + c * 8192, map, r0 + 64 * c, k0, batch, fb);
             }
             if (++s == STAGES) { s = 0; par ^= 1u; }
           }
@@ -436,7 +438,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
       }
       if (!ok) {
         // Abort path: let the copies already issued land before the CTA's shared memory goes away.
-        if (cta_rank == 0) {
+        if (cta_rank == 0 && do_a) {
           const uint32_t pending = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
           for (uint32_t j = 0; j < pending; ++j) {
             const uint32_t i2 = it - 1 - j;
@@ -444,7 +446,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
             while (!mbar_try_wait(smem_u32(&full_bar[i2 % STAGES]), (i2 / STAGES) & 1u) && ++spins < (1u << 22)) {}
           }
         } else {
-          // the peer's barrier cannot be polled from here: give the copies a fixed 100 us
+          // the barrier that counts these copies is not this thread's to poll: give them a fixed 100 us
           const uint64_t t0 = global_timer_ns();
           while (global_timer_ns() - t0 < 100000ull) {}
         }
@@ -504,7 +506,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
   } else {
     // ===================================================================== epilogue
     // Chunks (64 output columns of this CTA's 128 rows) are numbered g = 0, 1, ... across the CTA's tiles;
-    // chunk g lives in ring buffer g % EPI_BUFS.  For every chunk the TMA thread (warp 10) first makes the
+    // chunk g lives in ring buffer g % EPI_BUFS.  For every chunk the TMA thread (warp 2 + EPI_WARPS) first makes the
     // buffer available - it waits until the store that last used the buffer has left shared memory, then
     // either starts the C loads on c_full_bar (bytes expected) or just arrives on it - and it does so
     // PREFETCH chunks ahead of the chunk whose results it sends off.  A math warp waits on c_full_bar,
