@@ -202,8 +202,8 @@ def time_oracle(wl, steps, warmup, budget_flops, min_seconds=0.0):
 # they process): bytes per (entry, worker) of one Gram launch and of one apply launch.
 NCU_NS_TRAFFIC_PER_ENTRY = {
     # workload family -> (gram bytes per entry and worker, apply bytes per entry and worker, capture it comes from)
-    "large": (3.61, 12.81, "c5:4096x4096:4 (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
-    "c2_resnet50": (2.26, 8.05, "c2 (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
+    "large": (3.65, 12.79, "c5:4096x4096:4 (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
+    "c2_resnet50": (2.19, 7.81, "c2, matrices with a short side of 512 and more (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
 }
 
 
@@ -324,7 +324,9 @@ def roofline_of(wl, kernels, peaks, clocks, timed_ns_seconds):
         peak = peaks["bf16_tflops_sustained"] if use_sustained else peaks["bf16_tflops"]
         fam = "c2_resnet50" if wl.name.startswith("c2") else "large"
         g_b, a_b, src = NCU_NS_TRAFFIC_PER_ENTRY[fam]
-        units = sum(p.numel for p in wl.params if p.kind == "matrix") * \
+        # entries of the matrices that take part in every launch (those with a short side up to 256 iterate in Gram
+        # space and appear in the first Gram and the last apply launch only)
+        units = sum(p.numel for p in wl.params if p.kind == "matrix" and (min(p.rows, p.cols) > 256 or wl.ns_steps < 2)) * \
             (wl.num_workers + (1 if wl.local_polar else 0)) / (2.0 if wl.local_polar else 1.0)
         # mean over a step's Gram and apply launches (a local polar launch processes 1 / M of a workers' launch)
         traffic = 0.5 * (g_b + a_b) * units

@@ -518,9 +518,11 @@ __global__ void __launch_bounds__(VOTE_THREADS) vote_kernel(const __grid_constan
 // polar step's operand slot.  A block owns UPD_VECS 128-bit vectors of one parameter (4 float32 or 8 bf16 entries
 // each, all inside one vote word), a thread eight of them, all requested before the first is used.
 constexpr int UPD_VECS = EW_THREADS * 8;
-template <typename WT>
-__device__ __forceinline__ void update_block(const ParamDev& pd, uint32_t chunk, int lp_slot, float step, int write_sbar,
+// (SBAR is a template parameter so that the plain weight update does not carry the registers of the +-1 matrix stores.)
+template <typename WT, bool SBAR>
+__device__ __forceinline__ void update_block(const ParamDev& pd, uint32_t chunk, int lp_slot, float step,
                                              const uint32_t* __restrict__ vote_words) {
+  constexpr bool write_sbar = SBAR;
   const int64_t d = pd.d;
   WT* w = reinterpret_cast<WT*>(pd.W);
   bf16* sbar = pd.y0 + (int64_t)lp_slot * pd.rows * pd.ldy;   // the slot after the own workers' slots of operand buffer 0
@@ -615,18 +617,24 @@ __device__ __forceinline__ void update_block(const ParamDev& pd, uint32_t chunk,
   }
 }
 
-__global__ void __launch_bounds__(EW_THREADS) update_kernel(const ParamDev* __restrict__ params,
+// LP = the local polar step follows: matrix parameters then receive the +-1 matrix instead of a weight update.  Two
+// kernels, so that the plain weight update (LP = false) is compiled without the registers of the other path.
+template <bool LP>
+__global__ void __launch_bounds__(EW_THREADS, 4) update_kernel(const ParamDev* __restrict__ params,
                                                             const int32_t* __restrict__ list,
                                                             const uint32_t* __restrict__ starts, int n_list, int lp_slot,
-                                                            float lr, int write_sbar,
-                                                            const uint32_t* __restrict__ vote_words) {
+                                                            float lr, const uint32_t* __restrict__ vote_words) {
   const int slot = find_slot(starts, n_list, blockIdx.x);
   const ParamDev pd = params[list[slot]];
   const uint32_t chunk = blockIdx.x - starts[slot];
   const float step = lr * pd.upd_scale;
-  const int sbar = (write_sbar && pd.kind == 0) ? 1 : 0;   // plain parameters are updated directly (no local polar step)
-  if (pd.wdtype == 0) update_block<float>(pd, chunk, lp_slot, step, sbar, vote_words);
-  else update_block<bf16>(pd, chunk, lp_slot, step, sbar, vote_words);
+  if (LP && pd.kind == 0) {                  // plain parameters are updated directly (no local polar step)
+    if (pd.wdtype == 0) update_block<float, true>(pd, chunk, lp_slot, step, vote_words);
+    else update_block<bf16, true>(pd, chunk, lp_slot, step, vote_words);
+  } else {
+    if (pd.wdtype == 0) update_block<float, false>(pd, chunk, lp_slot, step, vote_words);
+    else update_block<bf16, false>(pd, chunk, lp_slot, step, vote_words);
+  }
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -817,8 +817,11 @@ void launch_vote(signmuon_ctx* c, float lr, int write_sbar, cudaStream_t s, cons
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  cudaLaunchKernelEx(&cfg, update_kernel, pd, list, reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_upd), n,
-                     c->Wm, lr, write_sbar, static_cast<const uint32_t*>(vote));
+  const uint32_t* starts = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_starts_upd);
+  if (write_sbar)
+    cudaLaunchKernelEx(&cfg, update_kernel<true>, pd, list, starts, n, c->Wm, lr, static_cast<const uint32_t*>(vote));
+  else
+    cudaLaunchKernelEx(&cfg, update_kernel<false>, pd, list, starts, n, c->Wm, lr, static_cast<const uint32_t*>(vote));
 }
 
 void invalidate_tables(signmuon_ctx* c) {
