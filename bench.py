@@ -340,7 +340,9 @@ def roofline_of(wl, kernels, peaks, clocks, timed_ns_seconds):
                 "frac_of_nominal_2250": kd["frac_of_nominal_2250"],
                 "algorithmic_flops_per_launch": kd["algorithmic_flops"] / launches,
                 "executed_flops_per_launch": kd["executed_flops"] / launches,
-                "executed_tflops": kd["executed_tflops"], "ms_per_launch": kd["ms"] / launches,
+                "executed_tflops": kd["executed_tflops"], "frac_executed": kd["executed_tflops"] / peak,
+                "frac_executed_of_nominal_2250": kd["executed_tflops"] / NOMINAL_BF16_TFLOPS,
+                "ms_per_launch": kd["ms"] / launches,
                 "traffic": traffic, "traffic_source": "ncu capture of " + src + ", scaled by (entries x batch slots)",
                 "peak_source": peaks["source"]}
     achieved = kd["achieved_gbs"]
