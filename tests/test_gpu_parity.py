@@ -432,6 +432,35 @@ def test_garbage_worker_is_outvoted():
     opt.close()
 
 
+def test_degenerate_cases_tiny_matrices_zero_gradient_and_255_workers():
+    """The degenerate ends of the method: matrices of one row, one column or a few entries as MATRIX parameters (the
+    Gram matrix is then 1 x 1 or 2 x 2 and PolarNS keeps the signs), an all-zero gradient (sigma = 0 -> Y = 0 -> every
+    sign bit 1, Alg. 3's note, pad bits 0, W <- W - eta), and the largest worker count the vote supports."""
+    from parity_utils import run_and_check, make_optimizer
+    run_and_check(_wl([(1, 96), (96, 1), (2, 2), (8, 8), (3, 5), (1, 1)], 3), steps=2)
+    run_and_check(_wl([(1, 96), (8, 8), (5, 3)], 2, local_polar=True, lr=0.01), steps=1)
+    run_and_check(_wl([(16, 32), (24, 8), (1, 40)], 255, K=2, kinds=["matrix", "matrix", "plain"]), steps=1,
+                  ns_workers=[0, 254])
+    # all-zero gradients
+    wl = _wl([(64, 96), (40, 7), (1, 33)], 4, kinds=["matrix", "matrix", "plain"])
+    opt = make_optimizer(wl)
+    w = wlmod.make_weights(wl, "cuda:0")
+    before = [x.clone() for x in w]
+    g = [torch.zeros_like(x) for x in wlmod.make_grads(wl, wlmod.make_signal(wl, "cuda:0"), 0, "cuda:0")]
+    opt.step(w, g, wl.lr)
+    torch.cuda.synchronize()
+    assert opt.status() == B.OK
+    import oracle as O
+    for p_idx, p in enumerate(wl.params):
+        d = p.rows * p.cols
+        for m in range(wl.num_workers):
+            bits = O.unpack_bits(opt.tap(B.TAP_WORKER_BITS, p_idx, m).cpu().numpy(), d)
+            assert bits.all()
+        assert O.unpack_bits(opt.tap(B.TAP_VOTE_BITS, p_idx, 0).cpu().numpy(), d).all()
+        assert torch.allclose(w[p_idx], before[p_idx] - wl.lr, rtol=0, atol=1e-9)
+    opt.close()
+
+
 def test_sign_agreement_counts_match_the_payload():
     """Per worker, the number of sign bits equal to the vote, against plain counting on the GPU's own bits
     (ragged parameters: pad bits must not be counted)."""
