@@ -37,10 +37,11 @@
 // Gram products are symmetric: only tiles on or above the diagonal are scheduled and an off-diagonal tile is
 // also stored transposed.  A problem may carry up to three operand pairs ("segments") that are accumulated
 // into the same tile along K: split-precision products (hi hi + lo hi + hi lo) of the spectral scale.
-// Warps (384 threads): 0 = TMA of the A operand, 1 = MMA issue, 2..9 = epilogue math, 10 = epilogue TMA, 11 = TMA of the
-// B operand.  The single threads of warps 0, 1 and 11 sit on the critical path of every K block (512 tensor-core cycles
-// on a CTA pair): the MMA thread forms its descriptors by adding a step to precomputed words, and the copies of a
-// stage are split over two threads.
+// Warps (416 threads): 0 = TMA of the A operand, 1 and 12 = MMA issue (alternate K blocks), 2..9 = epilogue math,
+// 10 = epilogue TMA, 11 = TMA of the B operand.  The single threads of warps 0, 1, 11 and 12 sit on the critical path of
+// every K block (512 tensor-core cycles on a CTA pair): the MMA threads form their descriptors by adding a step to
+// precomputed words and take turns, so that one prepares while the other's instructions run, and the copies of a stage
+// are split over two threads.
 // Every wait is bounded: after the launch's wait limit (two seconds by default) a waiting thread records
 // STATUS_TIMEOUT in the status word, raises a CTA-wide abort flag and the CTA drains and exits (TMEM is freed).
 #pragma once
@@ -58,9 +59,9 @@ constexpr int GEMM_BK = 64;
 constexpr int EPI_WARPS = 8;                 // EPI_WARPS / 4 warps per TMEM lane quarter, each NCOL of a chunk's 64 columns
 constexpr int EPI_NCOL = 256 / EPI_WARPS;    // columns of a chunk one math thread owns (32 or 16)
 static_assert(EPI_WARPS == 8 || EPI_WARPS == 16, "8 or 16 epilogue math warps");
-constexpr int GEMM_THREADS = 32 * (4 + EPI_WARPS);   // warp 0: TMA of the A operand, warp 1: MMA, then the epilogue math warps,
-                                                     // then the epilogue TMA warp (C loads, result stores), last warp: TMA
-                                                     // of the B operand
+constexpr int GEMM_THREADS = 32 * (7 + EPI_WARPS);   // warp 0: TMA of the A operand, warp 1: MMA issue (even K blocks), then the
+                                                     // epilogue math warps, the epilogue TMA warp (C loads, result stores), the
+                                                     // TMA warp of the B operand, last warp: MMA issue (odd K blocks)
 constexpr uint64_t DEFAULT_WAIT_LIMIT_NS = 2000000000ull;   // two seconds unless the caller sets another limit
 
 struct GemmLaunchArgs {
@@ -327,6 +328,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
   __shared__ uint64_t row_pair_bar[4];           // the math warps of a lane quarter (fp32 C chunks only)
   __shared__ uint32_t tmem_slot;
   __shared__ uint32_t abort_word;
+  __shared__ uint32_t issue_turn;               // index of the next K block whose MMAs may be issued (two issuing threads)
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;
@@ -338,12 +340,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
 
   if (threadIdx.x == 0) {
     abort_word = 0;
+    issue_turn = 0;
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
     for (int a = 0; a < 2; ++a) {
-      mbar_init(smem_u32(&tmem_full_bar[a]), 1);
+      mbar_init(smem_u32(&tmem_full_bar[a]), 2);          // one commit of each MMA-issuing thread
       mbar_init(smem_u32(&tmem_empty_bar[a]), EPI_WARPS * CTAS);
     }
     for (int b = 0; b < EPI_BUFS; ++b) {
@@ -381,17 +384,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
   };
   const int row_shift = (int)cta_rank * GEMM_BM;   // this CTA's rows inside the tile of the pair
 
-  if (warp == 0 || warp == 3 + EPI_WARPS) {
+  if (warp == 0 || warp == 3 + EPI_WARPS || warp >= 5 + EPI_WARPS) {
     // ===================================================================== TMA producers
-    // Two threads feed the operand ring: one loads the A tiles (and, in CTA 0, posts the bytes a stage expects), the
-    // other the B tiles.  Both wait on the same "stage empty" barriers.  A B copy may complete before the A thread has
+    // Four threads feed the operand ring, two for the even and two for the odd K blocks: one of each pair loads the A
+    // tiles (and, in CTA 0, posts the bytes a stage expects), the other the B tiles.  Both wait on the same "stage empty" barriers.  A B copy may complete before the A thread has
     // posted the expected bytes of its stage: the barrier's transaction count is signed, and its phase cannot end
     // before that post, which is also the phase's only pending arrival.  (One thread issuing all copies of a stage
     // - four when both operands are MN-major - was the bound of those launches.)
     if (lane == 0) {
-      const bool do_a = (warp == 0);
+      const bool do_a = (warp == 0 || warp == 5 + EPI_WARPS);
+      const uint32_t my_parity = (warp >= 5 + EPI_WARPS) ? 1u : 0u;   // this thread serves the even or the odd K blocks
       uint32_t it = 0;   // running k-block counter across tiles
-      uint32_t s = 0, par = 1;   // ring position and the parity to wait for on its "empty" barrier
       const uint32_t full0 = (CTAS == 2) ? map_to_cta(smem_u32(&full_bar[0]), 0) : smem_u32(&full_bar[0]);
       bool ok = true;
       for (uint32_t t = tile_begin; t < tile_end && ok; ++t) {
@@ -418,6 +421,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
           if (seg == 1) map = args.tmaps + (do_a ? pr.tmapA2 : pr.tmapB2);
           else if (seg == 2) map = args.tmaps + (do_a ? pr.tmapA3 : pr.tmapB3);
           for (int kb = 0; kb < nk; ++kb, ++it) {
+            if ((it & 1u) != my_parity) continue;
+            const uint32_t s = it % (uint32_t)STAGES, par = ((it / (uint32_t)STAGES) & 1u) ^ 1u;   // ring position, parity of its "empty" barrier
             if (!mbar_wait(smem_u32(&empty_bar[0]) + 8u * s, par, abort_flag, args.status, args.wait_limit_ns)) { ok = false; break; }
             // the "full" barrier of the pair is CTA 0's: it expects the bytes of both CTAs
             const uint32_t fb = full0 + 8u * s;
@@ -432,13 +437,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
             } else {
               for (int c = 0; c < chunks; ++c) load_operand(dst + c * 8192, map, r0 + 64 * c, k0, batch, fb);
             }
-            if (++s == STAGES) { s = 0; par ^= 1u; }
           }
         }
       }
       if (!ok) {
         // Abort path: let the copies already issued land before the CTA's shared memory goes away.
-        if (cta_rank == 0 && do_a) {
+        if (cta_rank == 0 && do_a && my_parity == 0) {
           const uint32_t pending = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
           for (uint32_t j = 0; j < pending; ++j) {
             const uint32_t i2 = it - 1 - j;
@@ -452,11 +456,22 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
         }
       }
     }
-  } else if (warp == 1) {
-    // ===================================================================== MMA issuer (CTA 0 of a pair)
+  } else if (warp == 1 || warp == 4 + EPI_WARPS) {
+    // ===================================================================== MMA issuers (CTA 0 of a pair)
+    // A tcgen05.mma occupies its issuing thread for as long as the tensor core takes to accept it, and whatever
+    // else that thread does between two instructions (barrier waits, descriptor arithmetic, the commit) is time in
+    // which the tensor pipe has nothing to do: measured, every cycle of such work lengthens a K block by a cycle.
+    // So two threads issue alternate K blocks.  Each prepares its K block (waits for the stage, forms the
+    // descriptors) while the other one's instructions run, then waits for its turn, issues its four instructions
+    // and passes the turn on.  The turn (a K-block counter in shared memory, handed over between
+    // tcgen05.fence::before_thread_sync and ::after_thread_sync) keeps the instructions of a tile in K order, so the
+    // accumulation order - and with it every result bit - does not depend on timing.  A commit covers the MMAs of its
+    // own thread only: each thread frees the stages it consumed, and both commit to the accumulator's barrier.
     if (lane == 0 && cta_rank == 0) {
+      const uint32_t me = (warp == 1) ? 0u : 1u;
+      const uint32_t turn_addr = smem_u32(&issue_turn);
       uint32_t tcount = 0;
-      uint32_t s = 0, par = 0;   // ring position and the parity to wait for on its "full" barrier
+      uint32_t it0 = 0;                            // index of the tile's first K block in the CTA's K-block sequence
       bool ok = true;
       for (uint32_t t = tile_begin; t < tile_end && ok; ++t, ++tcount) {
         const TileEntry te = args.tiles[t];
@@ -464,7 +479,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
         const int a_mn = pr.a_mn, b_mn = pr.b_mn;
         const bool fp8 = KIND == 0 && pr.fp8 != 0;
         const int kelem = fp8 ? 2 * GEMM_BK : GEMM_BK;
-        const int nk = ((pr.K + kelem - 1) / kelem) * (pr.nseg > 1 ? pr.nseg : 1);
+        const uint32_t nk = (uint32_t)(((pr.K + kelem - 1) / kelem) * (pr.nseg > 1 ? pr.nseg : 1));
         const uint32_t idesc = instr_desc(TILE_M, BN, a_mn, b_mn, fp8 ? 1 : 0);
         // MN-major operands: bytes between the 16 (bf16) or 32 (FP8) k-rows of consecutive instructions, and between
         // 128-byte-wide chunks along M/N (a 128-row FP8 tile is a single chunk)
@@ -483,24 +498,50 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
         const uint32_t b_off = share_ab ? 0u : A_BYTES;
         auto run_tile = [&](auto fp8_tag) {
           constexpr bool FP8 = decltype(fp8_tag)::value;
-          for (int kb = 0; kb < nk; ++kb) {
+          // this thread's K blocks of the tile: those whose index in the CTA's sequence has its parity
+          for (uint32_t kb = (it0 + me) & 1u; kb < nk; kb += 2) {
+            const uint32_t it = it0 + kb;
+            const uint32_t s = it % (uint32_t)STAGES, par = (it / (uint32_t)STAGES) & 1u;
             if (!mbar_wait(smem_u32(&full_bar[0]) + 8u * s, par, abort_flag, args.status, args.wait_limit_ns)) { ok = false; break; }
-            tc_fence_after();
             const uint32_t sa = smem_base + s * STAGE_BYTES;
             const uint32_t a_lo = ((sa >> 4) & 0x3fffu) | a_lo_const, b_lo = (((sa + b_off) >> 4) & 0x3fffu) | b_lo_const;
+            // wait for the turn (bounded like every other wait)
+            {
+              uint32_t v, spins = 0;
+              uint64_t t_first = 0;
+              for (;;) {
+                asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(turn_addr) : "memory");
+                if (v == it) break;
+                if ((++spins & 1023u) == 0) {
+                  if (*abort_flag) { ok = false; break; }
+                  const uint64_t now = global_timer_ns();
+                  if (t_first == 0) t_first = now;
+                  else if (now - t_first > args.wait_limit_ns) {
+                    *abort_flag = 1;
+                    atomicExch(args.status, (uint32_t)STATUS_TIMEOUT);
+                    ok = false;
+                    break;
+                  }
+                }
+              }
+              if (!ok) break;
+            }
+            tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < GEMM_BK / 16; ++kk)
               tc_mma_words<CTAS == 2, FP8>(d_tmem, a_lo + kk * a_step, b_lo + kk * b_step, SMEM_DESC_HI_SBO1024, idesc,
-                                           (kb | kk) != 0 ? 1u : 0u);
+                                           (kb | (uint32_t)kk) != 0 ? 1u : 0u);
+            tc_fence_before();
+            asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(turn_addr), "r"(it + 1u) : "memory");
             // frees the stage (in both CTAs of a pair) once these MMAs have read it
             if (CTAS == 2) tc_commit_pair(smem_u32(&empty_bar[0]) + 8u * s); else tc_commit(smem_u32(&empty_bar[0]) + 8u * s);
-            if (++s == STAGES) { s = 0; par ^= 1u; }
           }
         };
         if (fp8) run_tile(std::integral_constant<bool, true>{}); else run_tile(std::integral_constant<bool, false>{});
-        if (ok) {                                    // accumulator complete
+        if (ok) {                                    // this thread's share of the accumulator is complete
           if (CTAS == 2) tc_commit_pair(smem_u32(&tmem_full_bar[acc])); else tc_commit(smem_u32(&tmem_full_bar[acc]));
         }
+        it0 += nk;
       }
     }
   } else {

@@ -695,8 +695,8 @@ void launch_tc(const GemmLaunchArgs& a, int lists, cudaStream_t s) {
 // per entry through the epilogue: shallower operand ring, four chunk buffers (two C loads in flight).
 // (BN, operand stages, chunk buffers, CTAs per tile, kind)
 #define NS_GEMM_PAIR_GRAM 256, 5, 2, 2, 0
-#define NS_GEMM_PAIR_APPLY 256, 3, 4, 2, 1
-#define NS_GEMM_PAIR_APPLY_LONGK 256, 4, 3, 2, 1   /* long contraction: the operand ring matters more than the chunk ring */
+#define NS_GEMM_PAIR_APPLY 256, 4, 3, 2, 1
+#define NS_GEMM_PAIR_APPLY_LONGK 256, 5, 2, 2, 1   /* long contraction: the operand ring matters more than the chunk ring */
 #define NS_GEMM_ONE_GRAM 128, 5, 2, 1, 0
 #define NS_GEMM_ONE_APPLY 128, 3, 4, 1, 1
 
