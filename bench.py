@@ -202,8 +202,8 @@ def time_oracle(wl, steps, warmup, budget_flops, min_seconds=0.0):
 # they process): bytes per (entry, worker) of one Gram launch and of one apply launch.
 NCU_NS_TRAFFIC_PER_ENTRY = {
     # workload family -> (gram bytes per entry and worker, apply bytes per entry and worker, capture it comes from)
-    "large": (3.65, 12.79, "c5:4096x4096:4 (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
-    "c2_resnet50": (2.19, 7.81, "c2, matrices with a short side of 512 and more (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
+    "large": (3.62, 12.04, "c5:4096x4096:4 (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
+    "c2_resnet50": (2.19, 7.87, "c2, matrices with a short side of 512 and more (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
 }
 
 
