@@ -63,6 +63,34 @@ def test_polar_ns_literal_equals_short_side_larger():
     assert np.max(np.abs(a - b)) <= 1e-13 * np.max(np.abs(a))
 
 
+@pytest.mark.parametrize("shape,K", [((6, 40), 5), ((40, 6), 3), ((9, 9), 2), ((3, 17), 7)])
+def test_gram_space_evaluation_is_the_same_map_as_alg4(shape, K):
+    """The reading the CUDA path relies on for short sides: with A_k = Y_k Y_k^T and P_k = 3/2 I - A_k / 2, Alg. 4's
+    step gives A_{k+1} = P_k A_k P_k = 9/4 A_k - 3/2 A_k^2 + 1/4 A_k^3 and Y_K = (P_{K-1} ... P_0) Y_0; with
+    T_k = (3/2)^k I + F_k the product obeys F_{k+1} = 3/2 F_k - (3/2)^k / 2 A_k - 1/2 A_k F_k, F_0 = 0.  Written out here in
+    numpy (not in the oracle) and compared with the oracle's literal iteration."""
+    x = RNG.normal(size=shape)
+    wide = shape[0] <= shape[1]
+    y0 = x / np.linalg.norm(x)
+    a = y0 @ y0.T if wide else y0.T @ y0
+    f = np.zeros_like(a)
+    t = 1.0
+    for _ in range(K):
+        f, a = 1.5 * f - 0.5 * t * a - 0.5 * a @ f, 2.25 * a - 1.5 * a @ a + 0.25 * a @ a @ a
+        t *= 1.5
+    tk = t * np.eye(a.shape[0]) + f
+    y_gram_space = tk @ y0 if wide else y0 @ tk
+    y_literal = O.polar_ns(x, K)
+    assert np.max(np.abs(y_gram_space - y_literal)) <= 1e-12 * np.max(np.abs(y_literal))
+    # and the s x s matrix the chain carries is the Gram matrix of the literal iterate
+    yk_minus_1 = O.polar_ns(x, K - 1)
+    a_lit = yk_minus_1 @ yk_minus_1.T if wide else yk_minus_1.T @ yk_minus_1
+    a_chain = y0 @ y0.T if wide else y0.T @ y0
+    for _ in range(K - 1):
+        a_chain = 2.25 * a_chain - 1.5 * a_chain @ a_chain + 0.25 * a_chain @ a_chain @ a_chain
+    assert np.max(np.abs(a_chain - a_lit)) <= 1e-12
+
+
 @pytest.mark.parametrize("K", [1, 2, 3, 4, 5])
 def test_newton_schulz_polar_error_bound(K):
     # tall 9 x 2 with singular values 0.8, 0.6: ||X||_F = 1, rho = ||I - X^T X||_op = 0.64
