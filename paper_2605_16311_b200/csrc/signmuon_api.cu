@@ -129,6 +129,7 @@ struct signmuon_ctx {
   // signmuon_step_host: gradients are copied on an internal stream, one step ahead of the compute
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_loaded[2] = {nullptr, nullptr}, ev_consumed[2] = {nullptr, nullptr};
+  cudaEvent_t ev_weights_up = nullptr;       // the last call's weight upload has left the host-to-device copy engine
   uint64_t host_steps = 0;
   int num_sms = 0;
   // Parameter tables.  The device keeps PARAM_TABLES copies of the ParamDev table, one per set of caller
@@ -1069,6 +1070,7 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
       sok = cudaEventCreateWithFlags(&c->ev_loaded[i], cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreateWithFlags(&c->ev_consumed[i], cudaEventDisableTiming) == cudaSuccess;
     }
+    sok = sok && cudaEventCreateWithFlags(&c->ev_weights_up, cudaEventDisableTiming) == cudaSuccess;
     if (!sok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
   }
   c->host_steps = 0;
@@ -1305,6 +1307,10 @@ int signmuon_step_host(signmuon_ctx* c, void* const* host_weights, const void* c
   bool ok = true;
   // gradients: internal stream, as soon as the step that last used this set (two calls ago) has finished
   if (c->host_steps >= 2) ok = cudaStreamWaitEvent(c->copy_stream, c->ev_consumed[set], 0) == cudaSuccess;
+  // ... and behind the previous call's weight upload: that (small) copy becomes ready at the same moment as this
+  // (large) one - when the step before it ends - and must not queue behind it in the host-to-device copy engine, or the
+  // previous call's step would wait for this call's gradients
+  if (c->host_steps >= 1) ok = ok && cudaStreamWaitEvent(c->copy_stream, c->ev_weights_up, 0) == cudaSuccess;
   for (size_t p = 0; p < n && ok; ++p) {
     const ParamPlan& pl = c->plan[p];
     g[p] = gbase + pl.stage_g_off;
@@ -1318,6 +1324,7 @@ int signmuon_step_host(signmuon_ctx* c, void* const* host_weights, const void* c
     w[p] = c->d_staging + pl.stage_w_off;
     ok = cudaMemcpyAsync(w[p], host_weights[p], (size_t)pl.d * dtype_size(pl.wdtype), cudaMemcpyHostToDevice, s) == cudaSuccess;
   }
+  ok = ok && cudaEventRecord(c->ev_weights_up, s) == cudaSuccess;
   ok = ok && cudaStreamWaitEvent(s, c->ev_loaded[set], 0) == cudaSuccess;
   if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
   int rc = run_stages_impl(c, SIGNMUON_STAGE_ALL, w.data(), g.data(), lr, s);
@@ -1605,6 +1612,7 @@ void signmuon_destroy(signmuon_ctx* c) {
       if (c->ev_loaded[i]) cudaEventDestroy(c->ev_loaded[i]);
       if (c->ev_consumed[i]) cudaEventDestroy(c->ev_consumed[i]);
     }
+    if (c->ev_weights_up) cudaEventDestroy(c->ev_weights_up);
     cudaStreamDestroy(c->copy_stream);
   }
   for (int t = 0; t < PARAM_TABLES; ++t)
