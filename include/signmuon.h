@@ -193,12 +193,15 @@ int signmuon_run_stages(signmuon_ctx* ctx, int32_t stage_mask, void* const* weig
 /* Same step with HOST-resident weights and gradients (same layouts as signmuon_step, but HOST
  * pointers inside the HOST arrays; pinned memory recommended): copies them to the staging buffer
  * bound by signmuon_bind, runs the step, copies the weights back, without synchronising the host.
- * The weights travel on `cuda_stream`; the gradients travel on a stream of the library's own into one of
- * two staging sets, so that, when calls follow one another without a synchronisation in between, the
- * gradient copy of a call overlaps the compute and the weight copy-back of the call before it.  As with
- * any asynchronous copy, the host arrays of a call must stay unchanged until that call's work has run
- * (synchronise `cuda_stream`, whose work waits for the gradient copy).  signmuon_bind creates that stream
- * and four events when a staging buffer is given; signmuon_destroy releases them.
+ * The gradients travel on a stream of the library's own into one of two staging sets, so that, when calls follow
+ * one another without a synchronisation in between, the gradient copy of a call overlaps the compute and the weight
+ * copy-back of the call before it.  The weights are copied back on `cuda_stream` at the end of the step.  Their
+ * upload goes first on `cuda_stream` when something before the vote stage needs them (plain parameters, coupled
+ * weight decay, the Muon rule); otherwise it follows the gradients on the library's stream, ordered behind the
+ * previous call's copy-back to the same host arrays, and only the vote stage waits for it.  As with any
+ * asynchronous copy, the host arrays of a call must stay unchanged until that call's work has run: synchronise
+ * `cuda_stream` (its work waits for both uploads) before changing them.  signmuon_bind creates that stream and
+ * five events when a staging buffer is given; signmuon_destroy releases them.
  * Errors as signmuon_step, plus NOT_BOUND when no staging was bound. */
 int signmuon_step_host(signmuon_ctx* ctx, void* const* host_weights, const void* const* host_grads,
                        float lr, void* cuda_stream);

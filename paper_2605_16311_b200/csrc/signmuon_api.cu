@@ -1318,16 +1318,30 @@ int signmuon_step_host(signmuon_ctx* c, void* const* host_weights, const void* c
                          cudaMemcpyHostToDevice, c->copy_stream) == cudaSuccess;
   }
   ok = ok && cudaEventRecord(c->ev_loaded[set], c->copy_stream) == cudaSuccess;
-  // weights: the caller's stream, behind the previous call's copy back to the same host arrays
+  // Weights.  Nothing before the vote stage touches them unless there are plain parameters (updated in the momentum
+  // stage), coupled weight decay (read there) or the Muon rule (updated by the last Newton-Schulz epilogue): then they
+  // too travel on the library's stream, behind the gradients and behind the previous call's copy back to the same
+  // host arrays, and only the vote stage waits for them.  Otherwise they go first, on the caller's stream.
+  const bool late_weights = c->plain_list.empty() && c->cfg.weight_decay == 0.f && !c->muon;
+  cudaStream_t ws = late_weights ? c->copy_stream : s;
+  if (late_weights && c->host_steps >= 1) ok = ok && cudaStreamWaitEvent(ws, c->ev_consumed[set ^ 1], 0) == cudaSuccess;
   for (size_t p = 0; p < n && ok; ++p) {
     const ParamPlan& pl = c->plan[p];
     w[p] = c->d_staging + pl.stage_w_off;
-    ok = cudaMemcpyAsync(w[p], host_weights[p], (size_t)pl.d * dtype_size(pl.wdtype), cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = cudaMemcpyAsync(w[p], host_weights[p], (size_t)pl.d * dtype_size(pl.wdtype), cudaMemcpyHostToDevice, ws) == cudaSuccess;
   }
-  ok = ok && cudaEventRecord(c->ev_weights_up, s) == cudaSuccess;
+  ok = ok && cudaEventRecord(c->ev_weights_up, ws) == cudaSuccess;
   ok = ok && cudaStreamWaitEvent(s, c->ev_loaded[set], 0) == cudaSuccess;
   if (!ok) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
-  int rc = run_stages_impl(c, SIGNMUON_STAGE_ALL, w.data(), g.data(), lr, s);
+  int rc;
+  if (late_weights) {
+    rc = run_stages_impl(c, SIGNMUON_STAGE_MOMENTUM | SIGNMUON_STAGE_NS, w.data(), g.data(), lr, s);
+    if (rc != SIGNMUON_OK) return rc;
+    if (cudaStreamWaitEvent(s, c->ev_weights_up, 0) != cudaSuccess) { c->sticky = SIGNMUON_ERR_CUDA; return c->sticky; }
+    rc = run_stages_impl(c, SIGNMUON_STAGE_VOTE | SIGNMUON_STAGE_LOCAL_POLAR, w.data(), g.data(), lr, s);
+  } else {
+    rc = run_stages_impl(c, SIGNMUON_STAGE_ALL, w.data(), g.data(), lr, s);
+  }
   if (rc != SIGNMUON_OK) return rc;
   for (size_t p = 0; p < n && ok; ++p) {
     const ParamPlan& pl = c->plan[p];

@@ -280,6 +280,31 @@ def test_stage_calls_equal_one_step_and_determinism():
         assert torch.equal(outs[0][1], other[1]) and torch.equal(outs[0][2], other[2])
 
 
+def test_long_contractions_are_bit_reproducible_run_to_run():
+    """Two threads issue the tensor-core instructions of a tile, alternating K blocks; a token keeps them in K order,
+    so the fp32 accumulation order - and every payload and weight bit - must not depend on timing.  Long contractions
+    (many K blocks per tile, both operand majors, the split-precision products of a short-side matrix) over three
+    fresh contexts."""
+    wl = _wl([(1024, 4096), (4096, 1024), (256, 2048), (768, 768)], 3, dtype="bf16", local_polar=True, lr=0.01)
+    sig = wlmod.make_signal(wl, "cuda:0")
+    g = wlmod.make_grads(wl, sig, 0, "cuda:0")
+    outs = []
+    for _ in range(3):
+        opt = B.SignMuon(wl.params, 3, lr=0.01, local_polar=True)
+        w = wlmod.make_weights(wl, "cuda:0")
+        for _step in range(2):
+            opt.step(w, g)
+        torch.cuda.synchronize()
+        assert opt.status() == B.OK
+        outs.append(([x.clone() for x in w], [opt.payload(m).clone() for m in range(3)]))
+        opt.close()
+    for other in outs[1:]:
+        for a, b in zip(outs[0][0], other[0]):
+            assert torch.equal(a, b)
+        for a, b in zip(outs[0][1], other[1]):
+            assert torch.equal(a, b)
+
+
 def test_bounded_wait_runs_out_and_the_context_recovers():
     """Failure detection without a fault: a one-thread kernel performs the Newton-Schulz kernels' bounded wait on
     a barrier that nothing signals, with a 1 ms limit.  The kernel returns, the status word reports the timeout,
@@ -488,23 +513,34 @@ def test_sign_agreement_counts_match_the_payload():
     plain.close()
 
 
-def test_host_resident_step_matches_device_step():
-    """Four host-buffer steps issued back to back (the gradient copies run one step ahead on the library's
-    own stream) against four device-buffer steps on the same inputs: bit-identical weights."""
-    wl = _wl([(128, 256), (64, 147), (1, 40)], 3, kinds=["matrix", "matrix", "plain"])
+@pytest.mark.parametrize("case", ["plain_params", "matrices_only", "matrices_local_polar", "weight_decay"])
+def test_host_resident_step_matches_device_step(case):
+    """Six host-buffer steps issued back to back (the gradient copies run one step ahead on the library's own stream;
+    without plain parameters and weight decay the weights travel there too and only the vote stage waits for them)
+    against six device-buffer steps on the same inputs: bit-identical weights, also when the caller changes the host
+    weights between two calls."""
+    kinds = ["matrix", "matrix", "plain"] if case == "plain_params" else ["matrix", "matrix", "matrix"]
+    shapes = [(128, 256), (64, 147), (1, 40)] if case == "plain_params" else [(128, 256), (64, 147), (320, 512)]
+    lp = case == "matrices_local_polar"
+    wd = 0.01 if case == "weight_decay" else 0.0
+    wl = _wl(shapes, 3, kinds=kinds, local_polar=lp, lr=0.01 if lp else 1e-3)
     sig = wlmod.make_signal(wl, "cuda:0")
-    gs = [wlmod.make_grads(wl, sig, t, "cuda:0") for t in range(4)]
+    gs = [wlmod.make_grads(wl, sig, t, "cuda:0") for t in range(6)]
     w_dev = wlmod.make_weights(wl, "cuda:0")
     w_host = [x.cpu().pin_memory() for x in w_dev]
     g_host = [[x.cpu().pin_memory() for x in g] for g in gs]
-    a = B.SignMuon(wl.params, 3)
-    for g in gs:
+    a = B.SignMuon(wl.params, 3, local_polar=lp, lr=wl.lr, weight_decay=wd)
+    b = B.SignMuon(wl.params, 3, local_polar=lp, lr=wl.lr, weight_decay=wd, host_staging=True)
+    for t, g in enumerate(gs):
+        if t == 3:      # the caller edits the weights between two steps (after synchronising, as the contract asks)
+            torch.cuda.synchronize()
+            for x, y in zip(w_dev, w_host):
+                x.mul_(0.5)
+                y.mul_(0.5)
         a.step(w_dev, g)
-    b = B.SignMuon(wl.params, 3, host_staging=True)
-    for g in g_host:
-        b.step_host(w_host, g)
+        b.step_host(w_host, g_host[t])
     torch.cuda.synchronize()
-    assert b.status() == B.OK
+    assert a.status() == B.OK and b.status() == B.OK
     for x, y in zip(w_dev, w_host):
         assert torch.equal(x.cpu(), y)
     a.close(); b.close()
