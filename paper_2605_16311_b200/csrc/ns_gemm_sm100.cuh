@@ -387,10 +387,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
   if (warp == 0 || warp == 3 + EPI_WARPS || warp >= 5 + EPI_WARPS) {
     // ===================================================================== TMA producers
     // Four threads feed the operand ring, two for the even and two for the odd K blocks: one of each pair loads the A
-    // tiles (and, in CTA 0, posts the bytes a stage expects), the other the B tiles.  Both wait on the same "stage empty" barriers.  A B copy may complete before the A thread has
-    // posted the expected bytes of its stage: the barrier's transaction count is signed, and its phase cannot end
-    // before that post, which is also the phase's only pending arrival.  (One thread issuing all copies of a stage
-    // - four when both operands are MN-major - was the bound of those launches.)
+    // tiles (and, in CTA 0, posts the bytes a stage expects), the other the B tiles.  The two threads of a K block wait
+    // on the same "stage empty" barrier.  A B copy may complete before the A thread has posted the expected bytes of
+    // its stage: the barrier's transaction count is signed, and its phase cannot end before that post, which is also
+    // the phase's only pending arrival.  (One thread issuing all copies of a stage - four when both operands are
+    // MN-major - was the bound of those launches.)
     if (lane == 0) {
       const bool do_a = (warp == 0 || warp == 5 + EPI_WARPS);
       const uint32_t my_parity = (warp >= 5 + EPI_WARPS) ? 1u : 0u;   // this thread serves the even or the odd K blocks
