@@ -305,6 +305,42 @@ def test_long_contractions_are_bit_reproducible_run_to_run():
             assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("local_polar", [False, True])
+def test_step_captured_in_a_cuda_graph_replays_bit_identically(local_polar):
+    """signmuon_step only enqueues work (no allocation, no synchronisation, no upload once the pointer set is known):
+    a step recorded into a CUDA graph - cluster launches, the programmatic dependent launch of the update kernel and the
+    Gram-space chain included - replays to the same bits as the same steps enqueued directly."""
+    wl = _wl([(256, 512), (512, 1024), (64, 147), (1, 96)], 3, local_polar=local_polar, lr=0.01,
+             kinds=["matrix", "matrix", "matrix", "plain"])
+    sig = wlmod.make_signal(wl, "cuda:0")
+    g = wlmod.make_grads(wl, sig, 0, "cuda:0")
+    eager = B.SignMuon(wl.params, 3, lr=0.01, local_polar=local_polar)
+    graphed = B.SignMuon(wl.params, 3, lr=0.01, local_polar=local_polar)
+    w_e = wlmod.make_weights(wl, "cuda:0")
+    w_g = [x.clone() for x in w_e]
+    eager.step(w_e, g)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graphed.step(w_g, g)                       # warm-up on the capture stream: the pointer table is uploaded here
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        graphed.step(w_g, g)
+    # the capture itself runs nothing: three replays against three more eager steps
+    for _ in range(3):
+        graph.replay()
+        eager.step(w_e, g)
+    torch.cuda.synchronize()
+    assert eager.status() == B.OK and graphed.status() == B.OK
+    for a, b in zip(w_e, w_g):
+        assert torch.equal(a, b)
+    for m in range(3):
+        assert torch.equal(eager.payload(m), graphed.payload(m))
+    eager.close(); graphed.close()
+
+
 def test_bounded_wait_runs_out_and_the_context_recovers():
     """Failure detection without a fault: a one-thread kernel performs the Newton-Schulz kernels' bounded wait on
     a barrier that nothing signals, with a 1 ms limit.  The kernel returns, the status word reports the timeout,
