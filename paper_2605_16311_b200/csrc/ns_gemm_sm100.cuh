@@ -511,7 +511,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
               uint32_t v, spins = 0;
               uint64_t t_first = 0;
               for (;;) {
-                asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(turn_addr) : "memory");
+                asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(turn_addr) : "memory");
                 if (v == it) break;
                 if ((++spins & 1023u) == 0) {
                   if (*abort_flag) { ok = false; break; }
@@ -533,7 +533,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
               tc_mma_words<CTAS == 2, FP8>(d_tmem, a_lo + kk * a_step, b_lo + kk * b_step, SMEM_DESC_HI_SBO1024, idesc,
                                            (kb | (uint32_t)kk) != 0 ? 1u : 0u);
             tc_fence_before();
-            asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(turn_addr), "r"(it + 1u) : "memory");
+            asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(turn_addr), "r"(it + 1u) : "memory");
             // frees the stage (in both CTAs of a pair) once these MMAs have read it
             if (CTAS == 2) tc_commit_pair(smem_u32(&empty_bar[0]) + 8u * s); else tc_commit(smem_u32(&empty_bar[0]) + 8u * s);
           }
