@@ -472,6 +472,48 @@ def measure(wl, args, dev, dist, rank, world, local_rank, steps, warmup, with_e2
     return res
 
 
+def live_reference(dev, seconds=1.5):
+    """The box's own library rates, measured in this run for context (boxes of one pool differ by more than 10 % under
+    the power cap): torch.matmul bf16 8192^3 back to back for `seconds` and a 1 Gi-element bf16 copy.  Not on the
+    optimizer's path; `roofline.peak` stays the recorded measurement."""
+    import torch
+    n = 8192
+    a = torch.randn(n, n, device=dev, dtype=torch.bfloat16)
+    b = torch.randn(n, n, device=dev, dtype=torch.bfloat16)
+    c = torch.empty(n, n, device=dev, dtype=torch.bfloat16)
+    for _ in range(3):
+        torch.matmul(a, b, out=c)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(torch.device(dev).index or 0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 0
+    t0 = time.perf_counter()
+    e0.record()
+    while time.perf_counter() - t0 < seconds:
+        for _ in range(20):
+            torch.matmul(a, b, out=c)
+        reps += 20
+        torch.cuda.synchronize()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    tf = 2.0 * n ** 3 * reps / e0.elapsed_time(e1) / 1e9
+    del a, b, c
+    x = torch.empty(1 << 30, device=dev, dtype=torch.bfloat16)
+    y = torch.empty_like(x)
+    for _ in range(2):
+        y.copy_(x)
+    best = 0.0
+    for _ in range(5):
+        e0.record(); y.copy_(x); e1.record(); torch.cuda.synchronize()
+        best = max(best, 2.0 * x.numel() * 2 / e0.elapsed_time(e1) / 1e6)
+    del x, y
+    torch.cuda.empty_cache()
+    return {"cublas_bf16_tflops_sustained": tf, "copy_gbs": best, "sm_mhz": clocks.get("sm_mhz"),
+            "reasons": clocks.get("reasons"), "how": "torch.matmul bf16 8192^3 for %.1f s; b.copy_(a) 1 Gi bf16 elements, best of 5" % seconds}
+
+
 def run_ours(args, wl):
     import torch
     from paper_2605_16311_b200 import binding as B
@@ -524,6 +566,9 @@ def run_ours(args, wl):
             dist.destroy_process_group()
         return
 
+    live = None
+    if world == 1 and not args.no_live_reference and not args.no_e2e:     # (profiling runs pass --no-e2e)
+        live = live_reference(dev)
     cpu = None
     if not args.no_cpu_baseline:
         cpu = time_oracle(wl, 1, 0, args.oracle_flops, min_seconds=args.cpu_baseline_seconds)
@@ -546,6 +591,7 @@ def run_ours(args, wl):
             "roofline": roofline_of(wl, kernels, peaks, main["clocks"], main["timed_ns_seconds"]),
             "cpu_baseline": cpu, "stage_ms": main["stage_ms"], "kernels": kernels,
             "ns_tflops": kernels.get("ns_gemm_tc", {}).get("achieved_tflops"),
+            "live_reference": live,
             "secondary": secondary,
             "multi_gpu": (None if world == 1 else
                           ("workers sharded over ranks, packed payload all-gathered (NCCL)" if sharded
@@ -624,6 +670,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-secondary", action="store_true", help="skip the secondary workloads (c2, c3)")
+    ap.add_argument("--no-live-reference", action="store_true",
+                    help="skip the box's own cuBLAS / copy rates measured beside the result (context only)")
     ap.add_argument("--exercise-exchange", action="store_true",
                     help="with one GPU: run the sharded step (stages + NCCL all-gather of the payload) on a one-rank group")
     ap.add_argument("--oracle-flops", type=float, default=3.0e12,
