@@ -282,7 +282,6 @@ __device__ __forceinline__ void plain_block(const ParamDev& pd, uint32_t chunk, 
                                             float lambda, float step, uint32_t* __restrict__ bits,
                                             uint32_t* __restrict__ vote_words, int64_t bits_pitch, int do_vote,
                                             const PeerList& peers) {
-  const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int64_t d = pd.d;
   if ((d & 7) == 0 && (int64_t)chunk * PLAIN_CHUNK + (warp + 1) * 256 <= d) {

@@ -1211,7 +1211,6 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     ok = ok && up(c->off_chain_start, c->chain_pair_start.data(), c->chain_pair_start.size() * 4);
     ok = ok && cudaStreamSynchronize(s) == cudaSuccess;      // (cps dies with this scope)
   }
-  // (moved up) kernels configured before the tile tables are split
   std::vector<CUtensorMap> maps((size_t)c->num_tmaps);
   const bool need_maps = !(c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) && c->cfg.ns_steps > 0;
   if (need_maps) {
