@@ -592,6 +592,18 @@ def run_ours(args, wl):
             "cpu_baseline": cpu, "stage_ms": main["stage_ms"], "kernels": kernels,
             "ns_tflops": kernels.get("ns_gemm_tc", {}).get("achieved_tflops"),
             "live_reference": live,
+            # the two stated targets, evaluated on this run: Newton-Schulz >= 60 % of the dense bf16 peak (2250 TF nominal),
+            # memory-bound kernels >= 70 % of ~8 TB/s
+            "targets": {
+                "ns_fraction_of_nominal_2250": {
+                    "algorithmic_flops": kernels.get("ns_gemm_tc", {}).get("frac_of_nominal_2250"),
+                    "executed_flops": (kernels["ns_gemm_tc"]["executed_tflops"] / NOMINAL_BF16_TFLOPS
+                                       if "ns_gemm_tc" in kernels else None),
+                    "target": 0.60},
+                "hbm_fraction_of_nominal_8000": {
+                    "momentum": kernels.get("momentum+plain", {}).get("frac_of_nominal_8000"),
+                    "vote_update": kernels.get("vote_update", {}).get("frac_of_nominal_8000"),
+                    "target": 0.70}},
             "secondary": secondary,
             "multi_gpu": (None if world == 1 else
                           ("workers sharded over ranks, packed payload all-gathered (NCCL)" if sharded
