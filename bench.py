@@ -268,7 +268,9 @@ def kernel_report(wl, opt, stage_ms, peaks, clocks, timed_region_s, ns_scale="fr
         sum(p.numel * (M * (gb[p.dtype] + 8) + 2 * gb[p.dtype] + M / 8 + 1 / 8) for p in plain)
     if ns_scale == "spectral":      # the power iteration reads the float32 momentum 2P + 1 more times
         mom_bytes += sum(M * p.numel * 4 * (2 * power_iters + 1) for p in mat)
-    vote_bytes = sum(p.numel * (M / 8 + 1 / 8 + (2 if wl.local_polar else 2 * gb[p.dtype])) for p in mat)
+    # payload rows in, vote words out and in again; then either the weights in and out, or (local polar step next) the
+    # +-1 matrix out as bf16 and as FP8 bytes
+    vote_bytes = sum(p.numel * (M / 8 + 1 / 8 + (3 if wl.local_polar else 2 * gb[p.dtype])) for p in mat)
     kernels = {}
     if stage_ms["momentum"] > 0:
         a = mom_bytes / stage_ms["momentum"] / 1e6
