@@ -146,15 +146,18 @@ def test_full_resnet50_config_sampled():
     print(rep)
 
 
-def test_full_gpt2_config_sampled():
+@pytest.mark.parametrize("flags", [B.FLAG_KEEP_POLAR, 0])
+def test_full_gpt2_config_sampled(flags):
     """Config 3 at full size (12 layers, embeddings and norm gains as plain parameters, M = 16, Student-t noise,
-    local polar on): sampled parameters, Newton-Schulz compared for two of the sixteen workers."""
+    local polar on): sampled parameters, Newton-Schulz compared for two of the sixteen workers; once with Y_K kept
+    for the value comparison, once in the configuration the benchmark times (flags = 0)."""
     from parity_utils import run_and_check
     wl = wlmod.config3()
     names = [p.name for p in wl.params]
     sample = [names.index("h0.qkv"), names.index("h5.attn_proj"), names.index("h11.mlp_proj"), names.index("wpe"),
               names.index("ln7")]
-    rep = run_and_check(wl, steps=1, sample=sample, ns_workers=[0, 15])
+    rep = run_and_check(wl, steps=1, sample=sample, ns_workers=[0, 15], flags=flags)
+    assert rep["sign_match_min"] >= 0.999
     print(rep)
 
 
