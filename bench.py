@@ -551,7 +551,11 @@ def run_ours(args, wl):
             wl2 = wlmod.by_name(name)
             if wl2.name == wl.name:
                 continue
-            r = measure(wl2, args, dev, dist, rank, world, local_rank, max(5, min(args.steps, 20)), 3, with_e2e=False)
+            try:
+                r = measure(wl2, args, dev, dist, rank, world, local_rank, max(5, min(args.steps, 20)), 3, with_e2e=False)
+            except Exception as exc:        # a secondary block must not cost the headline its line
+                secondary[wl2.name] = {"config": describe(wl2), "error": repr(exc)}
+                continue
             k = r["kernels"]
             secondary[wl2.name] = {
                 "config": describe(wl2), "ms_per_step": r["ms_per_step"],
