@@ -63,7 +63,7 @@ struct LaunchPlan {        // one grouped GEMM launch
 
 // Tile tables.  The workers' first Gram launch and last apply launch also carry the parameters whose iteration runs in
 // Gram space (they take part in no other launch), so those two launches have tables of their own.
-enum { TT_GRAM_FIRST = 0, TT_APPLY_LAST, TT_GRAM, TT_APPLY, TT_LP_GRAM, TT_LP_APPLY, TT_COUNT };
+enum { TT_GRAM_FIRST = 0, TT_APPLY_LAST, TT_GRAM, TT_APPLY, TT_LP_GRAM_FIRST, TT_LP_APPLY_LAST, TT_LP_GRAM, TT_LP_APPLY, TT_COUNT };
 
 struct TileTable {
   std::vector<TileEntry> tiles;         // ordered by CTA
@@ -114,10 +114,12 @@ struct signmuon_ctx {
   std::vector<LaunchPlan> ns_launches, lp_launches;
   TileTable tables[TT_COUNT];
   // Newton-Schulz in Gram space (short side <= 256): one chain launch between the first Gram and the last apply launch
-  std::vector<ChainProblem> chain_problems;   // pointers as workspace offsets until bind
-  std::vector<uint32_t> chain_order, chain_pair_start;
-  size_t off_chain_problems = 0, off_chain_order = 0, off_chain_start = 0;
-  int chain_pairs = 0;
+  // Gram-space chain launches: [0] the workers' iterations, [1] the local polar step's (one problem per parameter)
+  struct ChainSet {
+    std::vector<ChainProblem> problems;       // pointers as workspace offsets until bind
+    size_t off_problems = 0, off_order = 0, off_start = 0;
+    int pairs = 0;
+  } chain[2];
   int num_tmaps = 0;
   // binding
   bool split = false;      // Newton-Schulz products of the workers in split precision (scale = spectral)
@@ -232,7 +234,7 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
   const bool keep = (c->cfg.flags & SIGNMUON_FLAG_KEEP_POLAR) != 0;
   for (int32_t p : c->matrix_list) {
     const ParamPlan& pl = c->plan[p];
-    const bool gs = pl.gs && !local_polar_phase;
+    const bool gs = pl.gs;
     if (gs && (gram ? k != 0 : k != K - 1)) continue;
     const bool first = gs || k == 0;                 // reads the momentum (scale from memory, float32 own term)
     const int src = gs ? 0 : (k & 1), dst = gs ? 1 : ((k + 1) & 1);
@@ -265,7 +267,12 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         pr.sym = (c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) ? 0 : 1;   // square tiles only (bm == bn in every shape)
         pr.tmapOT = pl.tmap_base + TM_Q_BOX64;
         pr.diag_share = 1;                          // A and B are the same rows of the same matrix on diagonal tiles
-        if ((c->split && !local_polar_phase) || gs) {   // -A/2 as a hi/lo pair, both triangles computed
+        if (local_polar_phase && gs) {              // -A/2 as a hi/lo pair for the chain; the +-1 operands are exact
+          pr.gram_lo = 1;
+          pr.sym = 0;
+          pr.out_lo = reinterpret_cast<bf16*>(pl.qlo_off + m * qbytes);
+          pr.tmapO1 = pl.tmap_base + TM_QLO_K128;
+        } else if ((c->split && !local_polar_phase) || gs) {   // -A/2 as a hi/lo pair, both triangles computed
           pr.gram_lo = 1;
           pr.sym = 0;
           pr.diag_share = 0;                        // the segments pair different operands
@@ -314,7 +321,7 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         const int tlo = split && src ? TM_LO1_K128 : TM_LO0_K128, tlo_dst = split && dst ? TM_LO1_K128 : TM_LO0_K128;
         pr.own_coef = gs ? (float)std::pow(1.5, (double)K) : 1.5f;
         if (split || gs) {      // Q Y ~ Qhi Yhi + Qlo Yhi + Qhi Ylo (three operand segments along K)
-          pr.nseg = 3;
+          pr.nseg = local_polar_phase ? 2 : 3;        // (the +-1 vote matrix has no lo part)
           const int tlo_mn = src ? TM_LO1_MN : TM_LO0_MN;
           if (pl.wide) {
             pr.tmapA2 = pl.tmap_base + TM_QLO_K128; pr.tmapB2 = pr.tmapB;
@@ -569,8 +576,8 @@ int plan_layout(signmuon_ctx* c) {
     }
     if (c->lp) {
       for (int k = 0; k < K; ++k) {
-        add_launch(c->lp_launches, true, k, 1, true, TT_LP_GRAM);
-        add_launch(c->lp_launches, false, k, 1, true, TT_LP_APPLY);
+        add_launch(c->lp_launches, true, k, 1, true, k == 0 ? TT_LP_GRAM_FIRST : TT_LP_GRAM);
+        add_launch(c->lp_launches, false, k, 1, true, k == K - 1 ? TT_LP_APPLY_LAST : TT_LP_APPLY);
       }
     }
   }
@@ -587,24 +594,28 @@ int plan_layout(signmuon_ctx* c) {
     tt.tiles_off = off; off += round_up(std::max<size_t>(ntiles, 1) * sizeof(TileEntry), ALIGN);
     tt.cta_off = off; off += round_up((MAX_CTAS + 1) * 4, ALIGN);
   }
-  // chain problems: one per (Gram-space parameter, worker); -A_0/2 in, F_K out (the hi/lo Gram buffers)
-  c->chain_problems.clear();
-  for (int32_t p : c->matrix_list) {
-    const ParamPlan& pl = c->plan[p];
-    if (!pl.gs) continue;
-    const size_t qbytes = (size_t)pl.s * pl.ldq * 2;
-    for (int m = 0; m < M; ++m) {
-      ChainProblem cp;
-      cp.q_hi = reinterpret_cast<bf16*>(pl.q_off + m * qbytes);
-      cp.q_lo = reinterpret_cast<bf16*>(pl.qlo_off + m * qbytes);
-      cp.s = (int32_t)pl.s;
-      cp.ldq = pl.ldq;
-      c->chain_problems.push_back(cp);
+  // chain problems: one per (Gram-space parameter, worker), and one per parameter in the local polar step's slot;
+  // -A_0/2 in, F_K out (the hi/lo Gram buffers)
+  for (int set = 0; set < 2; ++set) {
+    signmuon_ctx::ChainSet& cs = c->chain[set];
+    cs.problems.clear();
+    for (int32_t p : c->matrix_list) {
+      const ParamPlan& pl = c->plan[p];
+      if (!pl.gs || (set == 1 && !c->lp)) continue;
+      const size_t qbytes = (size_t)pl.s * pl.ldq * 2;
+      for (int m = (set ? M : 0); m < (set ? M + 1 : M); ++m) {
+        ChainProblem cp;
+        cp.q_hi = reinterpret_cast<bf16*>(pl.q_off + m * qbytes);
+        cp.q_lo = reinterpret_cast<bf16*>(pl.qlo_off + m * qbytes);
+        cp.s = (int32_t)pl.s;
+        cp.ldq = pl.ldq;
+        cs.problems.push_back(cp);
+      }
     }
+    cs.off_problems = off; off += round_up(std::max<size_t>(cs.problems.size(), 1) * sizeof(ChainProblem), ALIGN);
+    cs.off_order = off; off += round_up(std::max<size_t>(cs.problems.size(), 1) * 4, ALIGN);
+    cs.off_start = off; off += round_up((MAX_CTAS + 1) * 4, ALIGN);
   }
-  c->off_chain_problems = off; off += round_up(std::max<size_t>(c->chain_problems.size(), 1) * sizeof(ChainProblem), ALIGN);
-  c->off_chain_order = off; off += round_up(std::max<size_t>(c->chain_problems.size(), 1) * 4, ALIGN);
-  c->off_chain_start = off; off += round_up((MAX_CTAS + 1) * 4, ALIGN);
   c->off_tables_end = off;
   c->workspace_bytes = off;
 
@@ -772,17 +783,18 @@ void launch_gemm(signmuon_ctx* c, const LaunchPlan& lp, float lr, cudaStream_t s
 // Vote over `rows` payload rows starting at `src` (default: all workers' rows of the payload buffer), then the
 // update from the vote words.
 // Gram-space chain of the parameters with a short side up to 256: one CTA pair per (parameter, worker) problem list.
-void launch_chain(signmuon_ctx* c, cudaStream_t s) {
+void launch_chain(signmuon_ctx* c, int set, cudaStream_t s) {
+  const signmuon_ctx::ChainSet& cs = c->chain[set];
   ChainLaunchArgs a;
-  a.problems = reinterpret_cast<const ChainProblem*>(c->d_ws + c->off_chain_problems);
-  a.order = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_chain_order);
-  a.pair_start = reinterpret_cast<const uint32_t*>(c->d_ws + c->off_chain_start);
+  a.problems = reinterpret_cast<const ChainProblem*>(c->d_ws + cs.off_problems);
+  a.order = reinterpret_cast<const uint32_t*>(c->d_ws + cs.off_order);
+  a.pair_start = reinterpret_cast<const uint32_t*>(c->d_ws + cs.off_start);
   a.status = reinterpret_cast<uint32_t*>(c->d_ws + c->off_status);
   a.wait_limit_ns = c->wait_limit_ns;
   a.K = c->cfg.ns_steps;
   cudaLaunchConfig_t cfg;
   std::memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3((unsigned)c->chain_pairs * 2, 1, 1);
+  cfg.gridDim = dim3((unsigned)cs.pairs * 2, 1, 1);
   cfg.blockDim = dim3(CHAIN_THREADS, 1, 1);
   cfg.dynamicSmemBytes = CHAIN_SMEM_BYTES;
   cfg.stream = s;
@@ -936,9 +948,9 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
     }
   }
   if ((mask & SIGNMUON_STAGE_NS) && nm) {
-    bool chain_done = c->chain_problems.empty();
+    bool chain_done = c->chain[0].problems.empty();
     for (const LaunchPlan& lp : c->ns_launches) {
-      if (!chain_done && lp.tile_table != TT_GRAM_FIRST) { launch_chain(c, s); chain_done = true; }
+      if (!chain_done && lp.tile_table != TT_GRAM_FIRST) { launch_chain(c, 0, s); chain_done = true; }
       launch_gemm(c, lp, lr, s);
     }
     if (c->packfb_blocks) {
@@ -977,7 +989,11 @@ int run_stages_impl(signmuon_ctx* c, int32_t mask, void* const* weights, const v
                                                                              (int64_t)c->bits_pitch, agree);
   }
   if ((mask & SIGNMUON_STAGE_LOCAL_POLAR) && nm && lp_ns) {
-    for (const LaunchPlan& lp : c->lp_launches) launch_gemm(c, lp, lr, s);
+    bool chain_done = c->chain[1].problems.empty();
+    for (const LaunchPlan& lp : c->lp_launches) {
+      if (!chain_done && lp.tile_table != TT_LP_GRAM_FIRST) { launch_chain(c, 1, s); chain_done = true; }
+      launch_gemm(c, lp, lr, s);
+    }
   }
   return check_launch(c);
 }
@@ -1174,11 +1190,13 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
   c->executed_flops = 0;
   for (const LaunchPlan& lp : c->ns_launches) c->executed_flops += c->tables[lp.tile_table].flops;
   for (const LaunchPlan& lp : c->lp_launches) c->executed_flops += c->tables[lp.tile_table].flops;
-  // chain launch: problems to CTA pairs, longest first (cost ~ s^2: contraction steps x columns walked)
-  c->chain_pairs = 0;
-  if (!c->chain_problems.empty()) {
+  // chain launches: problems to CTA pairs, longest first (cost ~ s^2: contraction steps x columns walked)
+  for (int set = 0; set < 2; ++set) {
+    signmuon_ctx::ChainSet& cs = c->chain[set];
+    cs.pairs = 0;
+    if (cs.problems.empty()) continue;
     const int K = c->cfg.ns_steps;
-    std::vector<ChainProblem> cps = c->chain_problems;
+    std::vector<ChainProblem> cps = cs.problems;
     std::vector<uint32_t> idx(cps.size());
     for (size_t i = 0; i < cps.size(); ++i) {
       idx[i] = (uint32_t)i;
@@ -1188,28 +1206,27 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
       c->executed_flops += 3.0 * (K - 1) * 2.0 * 256.0 * 256.0 * (double)(((cps[i].s + 15) / 16) * 16);
     }
     std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) { return cps[a].s > cps[b].s; });
-    c->chain_pairs = (int)std::min<size_t>((size_t)max_pairs, cps.size());
-    std::vector<std::vector<uint32_t>> per((size_t)c->chain_pairs);
+    cs.pairs = (int)std::min<size_t>((size_t)max_pairs, cps.size());
+    std::vector<std::vector<uint32_t>> per((size_t)cs.pairs);
     typedef std::pair<long long, int> Load;
     std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
-    for (int i = 0; i < c->chain_pairs; ++i) heap.push({0, i});
+    for (int i = 0; i < cs.pairs; ++i) heap.push({0, i});
     for (uint32_t i : idx) {
       Load top = heap.top();
       heap.pop();
       per[top.second].push_back(i);
       heap.push({top.first + (long long)cps[i].s * cps[i].s + 4096, top.second});
     }
-    c->chain_order.clear();
-    c->chain_pair_start.assign((size_t)c->chain_pairs + 1, 0);
-    for (int i = 0; i < c->chain_pairs; ++i) {
-      c->chain_pair_start[i] = (uint32_t)c->chain_order.size();
-      c->chain_order.insert(c->chain_order.end(), per[i].begin(), per[i].end());
+    std::vector<uint32_t> order, pair_start((size_t)cs.pairs + 1, 0);
+    for (int i = 0; i < cs.pairs; ++i) {
+      pair_start[i] = (uint32_t)order.size();
+      order.insert(order.end(), per[i].begin(), per[i].end());
     }
-    c->chain_pair_start[c->chain_pairs] = (uint32_t)c->chain_order.size();
-    ok = ok && up(c->off_chain_problems, cps.data(), cps.size() * sizeof(ChainProblem));
-    ok = ok && up(c->off_chain_order, c->chain_order.data(), c->chain_order.size() * 4);
-    ok = ok && up(c->off_chain_start, c->chain_pair_start.data(), c->chain_pair_start.size() * 4);
-    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;      // (cps dies with this scope)
+    pair_start[cs.pairs] = (uint32_t)order.size();
+    ok = ok && up(cs.off_problems, cps.data(), cps.size() * sizeof(ChainProblem));
+    ok = ok && up(cs.off_order, order.data(), order.size() * 4);
+    ok = ok && up(cs.off_start, pair_start.data(), pair_start.size() * 4);
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;      // (the host vectors die with this scope)
   }
   std::vector<CUtensorMap> maps((size_t)c->num_tmaps);
   const bool need_maps = !(c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) && c->cfg.ns_steps > 0;
@@ -1589,9 +1606,9 @@ int signmuon_launches_per_step(const signmuon_ctx* c, int32_t* launches) {
   if (nm) n += 1 + (c->power_start_floats ? 3 + 4 * c->cfg.power_iters : 1);   // momentum + norms (or power iteration)
   if (!c->plain_list.empty()) n += 1;
   if (nm) n += (int)c->ns_launches.size() + (c->packfb_blocks ? 1 : 0);       // NS, fallback pack
-  if (!c->chain_problems.empty()) n += 1;                                     // Gram-space chain
+  if (!c->chain[0].problems.empty()) n += 1;                                  // Gram-space chain
   if (!c->vote_list.empty()) n += 2;                                          // vote, update
-  if (nm && c->lp && c->cfg.ns_steps > 0) n += (int)c->lp_launches.size();
+  if (nm && c->lp && c->cfg.ns_steps > 0) n += (int)c->lp_launches.size() + (c->chain[1].problems.empty() ? 0 : 1);
   if (c->peer_flags.n > 0) n += 2;                                            // publish, await (fused exchange)
   if (c->cfg.flags & SIGNMUON_FLAG_SIGN_AGREEMENT) n += 1;
   *launches = n;

@@ -235,6 +235,21 @@ def test_gram_space_iteration_against_oracle_and_full_matrix_iteration(K):
     run_and_check(wl, steps=1, flags=0)
 
 
+def test_local_polar_step_in_gram_space_against_oracle_and_full_matrix_iteration():
+    """The local polar step of matrices with a short side up to 256 also iterates in Gram space (FP8 Gram of the
+    vote matrix, the on-chip chain, one apply launch that updates the weights).  Both that path and the per-iteration
+    one are held to the oracle's Alg. 4 on the vote matrix; the Gram-space path, whose product with the exact +-1 matrix
+    carries only the rounding of F_K, is the more accurate of the two."""
+    from parity_utils import run_and_check
+    shapes = [(64, 576), (576, 64), (100, 328), (200, 200), (256, 1024), (1024, 256), (64, 147), (16, 2048), (320, 512)]
+    wl = _wl(shapes, 4, local_polar=True, lr=0.01)
+    rep_gs = run_and_check(wl, steps=2)
+    rep_full = run_and_check(wl, steps=2, flags=B.FLAG_KEEP_POLAR | B.FLAG_NO_GRAM_SPACE)
+    print("gram space:", rep_gs, "\nper iteration:", rep_full)
+    assert rep_gs["local_polar_relfro"] <= 2e-3
+    assert rep_full["local_polar_relfro"] <= 2e-2
+
+
 def test_default_flags_path_full_llama_layer_sampled():
     """Config 4 at full size in the benchmark's launch configuration (flags = 0, local polar on)."""
     from parity_utils import run_and_check
