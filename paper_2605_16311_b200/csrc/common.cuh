@@ -106,6 +106,12 @@ struct GemmProblem {
                           // the first Gram product of the local polar step, whose operand is the exact +-1 vote matrix
   int32_t gram_lo;        // EPI_GRAM: also store lo(-A/2) through tmapO1 (then the tile is not mirrored)
   int32_t diag_share;     // EPI_GRAM, one segment: on diagonal tiles the B operand is the A tile (not loaded twice)
+  // Products of the Gram-space chain through memory (s x s, symmetric operands and results)
+  int32_t mirror_hi;      // sym != 0: every off-diagonal tile also stores hi(result) transposed with plain stores (used
+                          // where the transposed copy through tmapOT is not available: hi/lo outputs)
+  const bf16* C2;         // EPI_APPLY: second linear term (hi part), same shape and pitch as the output, read with plain
+  const bf16* C2_lo;      //            loads; y = scale * (acc + own_coef * C + c2_coef * (C2 + C2_lo))
+  float c2_coef;
 };
 
 // Payload buffers of other GPUs that receive every payload word this GPU packs (the exchange of Alg. 3 fused into

@@ -670,6 +670,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
         const bool store_hi = KIND == 0 || epi == EPI_APPLY || (epi == EPI_APPLY_PACK && pr.store_out);
         const bool store_lo = (KIND == 1 && epi == EPI_APPLY && pr.hi_only == 0) || (KIND == 0 && pr.gram_lo != 0);
         const bool mirror = KIND == 0 && pr.sym != 0 && pr.gram_lo == 0 && te.tn != te.tm && rows_live;   // off-diagonal Gram tile
+        // symmetric result with hi/lo outputs: the hi part of an off-diagonal tile also goes to the transposed place
+        const bool mirror_hi = pr.sym != 0 && pr.mirror_hi != 0 && te.tn != te.tm && row < prM;
+        bf16* const out_t = reinterpret_cast<bf16*>(pr.out) + row;
+        const int64_t ld_out = pr.ld_out;
+        const bf16* c2_hi = nullptr;
+        const bf16* c2_lo = nullptr;
+        if (KIND == 1 && pr.C2 != nullptr && row < prM) {
+          c2_hi = pr.C2 + (size_t)row * ld_out;
+          c2_lo = pr.C2_lo + (size_t)row * ld_out;
+        }
+        const float c2_coef = pr.c2_coef;
         const uint32_t acc = tcount & 1u;
         const uint32_t acc_round = tcount >> 1;
         ok = mbar_wait(smem_u32(&tmem_full_bar[acc]), acc_round & 1u, abort_flag, args.status, args.wait_limit_ns);
@@ -693,6 +704,24 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
             if (lane == 0) {
               if (CTAS == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty_bar[acc]), 0));
               else mbar_arrive(smem_u32(&tmem_empty_bar[acc]));
+            }
+          }
+          if (KIND == 1 && c2_hi != nullptr) {
+            // second linear term of a chain product: this thread's NC columns of its row, hi + lo
+#pragma unroll
+            for (int u = 0; u < UNITS; ++u) {
+              if (col0 + u * 8 >= prN) break;
+              const uint4 uh = __ldg(reinterpret_cast<const uint4*>(c2_hi + col0 + u * 8));
+              const uint4 ul = __ldg(reinterpret_cast<const uint4*>(c2_lo + col0 + u * 8));
+              const uint32_t wh[4] = {uh.x, uh.y, uh.z, uh.w};
+              const uint32_t wl[4] = {ul.x, ul.y, ul.z, ul.w};
+              float* o = v + u * 8;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                o[2 * e] = fmaf(c2_coef, __uint_as_float(wh[e] << 16) + __uint_as_float(wl[e] << 16), o[2 * e]);
+                o[2 * e + 1] = fmaf(c2_coef, __uint_as_float(wh[e] & 0xffff0000u) + __uint_as_float(wl[e] & 0xffff0000u),
+                                    o[2 * e + 1]);
+              }
             }
           }
           if (KIND == 0) {
@@ -744,6 +773,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
             apply_c_direct<NC>(pr, scale, row, col0, v);
           }
           // ---- outputs
+          if (mirror_hi) {
+            // lanes hold consecutive rows: one column of the tile is 64 contiguous bytes of the transposed tile
+#pragma unroll
+            for (int j = 0; j < NC; ++j)
+              if (col0 + j < prN) out_t[(size_t)(col0 + j) * ld_out] = __float2bfloat16_rn(v[j]);
+          }
           if (store_hi) {
             if (tma_out) {
 #pragma unroll

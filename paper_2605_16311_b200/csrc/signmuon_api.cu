@@ -36,7 +36,13 @@ struct ParamPlan {
   int32_t ldy, ldq;
   uint32_t n_words, word_off;
   uint32_t chunks_per_worker;
-  bool gs;               // the workers' Newton-Schulz iteration runs in Gram space (on-chip chain; short side <= 256)
+  bool gs;               // the Newton-Schulz iteration runs in Gram space: on chip (ns_chain_kernel) for a short side up
+                         // to 256, or ...
+  bool gs_mem;           // ... as a chain of symmetric s x s products through memory (grouped GEMM launches) for larger
+                         // matrices that are long enough for it to need fewer tensor-core operations
+  // Gram-space chain through memory: Q_1 (second buffer of the Q_k ping-pong; the first is q_off / qlo_off), R_k (hi
+  // only) and H_k (ping-pong); bytes into the workspace
+  size_t gc_q1_off, gc_q1lo_off, gc_r_off, gc_h_off[2], gc_hlo_off[2];
   bool fused_pack;       // sign+pack happens in the last apply epilogue
   size_t mom_off;        // bytes into the state buffer
   size_t y_off[2], lo_off[2], q_off, qlo_off, scales_off, partials_off;   // bytes into the workspace (matrix params)
@@ -52,7 +58,9 @@ struct ParamPlan {
 
 // indices of a parameter's tensor maps relative to tmap_base
 enum { TM_Y0_K128 = 0, TM_Y0_KBN, TM_Y0_MN, TM_Y1_K128, TM_Y1_KBN, TM_Y1_MN, TM_Q_K128, TM_Q_KBN, TM_LO0_K128, TM_MOM_F32,
-       TM_Q_BOX64, TM_LO1_K128, TM_LO0_MN, TM_LO1_MN, TM_QLO_K128, TM_QLO_KBN, TM_S8, TM_PER_PARAM };
+       TM_Q_BOX64, TM_LO1_K128, TM_LO0_MN, TM_LO1_MN, TM_QLO_K128, TM_QLO_KBN, TM_S8,
+       // Gram-space chain through memory (s x s matrices, {64 x 128} boxes: operand, C and output maps alike)
+       TM_GC_Q1, TM_GC_Q1LO, TM_GC_R, TM_GC_H0, TM_GC_H0LO, TM_GC_H1, TM_GC_H1LO, TM_PER_PARAM };
 
 struct LaunchPlan {        // one grouped GEMM launch
   size_t problem_base;     // index of its first problem in the problem array
@@ -63,7 +71,10 @@ struct LaunchPlan {        // one grouped GEMM launch
 
 // Tile tables.  The workers' first Gram launch and last apply launch also carry the parameters whose iteration runs in
 // Gram space (they take part in no other launch), so those two launches have tables of their own.
-enum { TT_GRAM_FIRST = 0, TT_APPLY_LAST, TT_GRAM, TT_APPLY, TT_LP_GRAM_FIRST, TT_LP_APPLY_LAST, TT_LP_GRAM, TT_LP_APPLY, TT_COUNT };
+enum { TT_GRAM_FIRST = 0, TT_APPLY_LAST, TT_GRAM, TT_APPLY, TT_LP_GRAM_FIRST, TT_LP_APPLY_LAST, TT_LP_GRAM, TT_LP_APPLY,
+       TT_GC_R, TT_GC_Q, TT_GC_HR, TT_GC_F,      // launches of the Gram-space chain through memory: workers ...
+       TT_LP_GC_R, TT_LP_GC_Q, TT_LP_GC_HR, TT_LP_GC_F,   // ... and local polar step (same order)
+       TT_COUNT };
 
 struct TileTable {
   std::vector<TileEntry> tiles;         // ordered by CTA
@@ -267,7 +278,14 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         pr.sym = (c->cfg.flags & SIGNMUON_FLAG_SIMT_GEMM) ? 0 : 1;   // square tiles only (bm == bn in every shape)
         pr.tmapOT = pl.tmap_base + TM_Q_BOX64;
         pr.diag_share = 1;                          // A and B are the same rows of the same matrix on diagonal tiles
-        if (local_polar_phase && gs) {              // -A/2 as a hi/lo pair for the chain; the +-1 operands are exact
+        if (gs && pl.gs_mem) {
+          // -A/2 as a hi/lo pair for the chain through memory: one segment (the contraction is long enough for the
+          // operands' rounding to average out), upper tiles only, hi part mirrored for the chain's operand loads
+          pr.gram_lo = 1;
+          pr.mirror_hi = 1;
+          pr.out_lo = reinterpret_cast<bf16*>(pl.qlo_off + m * qbytes);
+          pr.tmapO1 = pl.tmap_base + TM_QLO_K128;
+        } else if (local_polar_phase && gs) {       // -A/2 as a hi/lo pair for the chain; the +-1 operands are exact
           pr.gram_lo = 1;
           pr.sym = 0;
           pr.out_lo = reinterpret_cast<bf16*>(pl.qlo_off + m * qbytes);
@@ -306,21 +324,32 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
         }
       } else {
         pr.M = (int32_t)pl.rows; pr.N = (int32_t)pl.cols; pr.K = (int32_t)pl.s;
+        // the s x s factor: -A_k/2 of this iteration, or F_K when the iteration ran in Gram space (left in the Gram
+        // buffers by the on-chip chain, in the H buffer of parity K by the chain through memory)
+        size_t qf = q;
+        int tq = TM_Q_K128, tq_b = TM_Q_KBN;
+        if (gs && pl.gs_mem) {
+          qf = pl.gc_h_off[K & 1] + m * qbytes;
+          tq = tq_b = (K & 1) ? TM_GC_H1 : TM_GC_H0;
+        }
         if (pl.wide) {                      // Y' = (3/2 I - A/2) Y : A operand Q, B operand Y (contiguous along N)
-          pr.A = reinterpret_cast<const bf16*>(q); pr.a_sm = pl.ldq; pr.a_sk = 1;
+          pr.A = reinterpret_cast<const bf16*>(qf); pr.a_sm = pl.ldq; pr.a_sk = 1;
           pr.B = reinterpret_cast<const bf16*>(ysrc); pr.b_sn = 1; pr.b_sk = pl.ldy; pr.b_mn = 1;
-          pr.tmapA = pl.tmap_base + TM_Q_K128; pr.tmapB = pl.tmap_base + ty + 2;
+          pr.tmapA = pl.tmap_base + tq; pr.tmapB = pl.tmap_base + ty + 2;
         } else {                            // Y' = Y (3/2 I - A/2) : A operand Y, B operand Q (symmetric)
           pr.A = reinterpret_cast<const bf16*>(ysrc); pr.a_sm = pl.ldy; pr.a_sk = 1;
-          pr.B = reinterpret_cast<const bf16*>(q); pr.b_sn = pl.ldq; pr.b_sk = 1;
-          pr.tmapA = pl.tmap_base + ty; pr.tmapB = pl.tmap_base + TM_Q_KBN;
+          pr.B = reinterpret_cast<const bf16*>(qf); pr.b_sn = pl.ldq; pr.b_sk = 1;
+          pr.tmapA = pl.tmap_base + ty; pr.tmapB = pl.tmap_base + tq_b;
         }
         const bool split = c->split && !local_polar_phase;
         const size_t lo = pl.lo_off[split ? src : 0] + m * ybytes;       // lo part of Y_k
         const size_t lo_dst = pl.lo_off[split ? dst : 0] + m * ybytes;   // lo part of Y_{k+1}
         const int tlo = split && src ? TM_LO1_K128 : TM_LO0_K128, tlo_dst = split && dst ? TM_LO1_K128 : TM_LO0_K128;
         pr.own_coef = gs ? (float)std::pow(1.5, (double)K) : 1.5f;
-        if (split || gs) {      // Q Y ~ Qhi Yhi + Qlo Yhi + Qhi Ylo (three operand segments along K)
+        if (gs && pl.gs_mem) {
+          // F_K Y_0 in one segment (hi parts): over a contraction this long the operands' rounding averages out as it
+          // does in every product of the iteration on the full matrix
+        } else if (split || gs) {      // Q Y ~ Qhi Yhi + Qlo Yhi + Qhi Ylo (three operand segments along K)
           pr.nseg = local_polar_phase ? 2 : 3;        // (the +-1 vote matrix has no lo part)
           const int tlo_mn = src ? TM_LO1_MN : TM_LO0_MN;
           if (pl.wide) {
@@ -383,6 +412,91 @@ void append_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, bool gram, 
   }
 }
 
+// Problems of the Gram-space chain through memory (parameters with gs_mem), one launch stage at a time.  With
+// Q_k = -A_k / 2 (Q_0 is what the first Gram launch stores) and T_k = (3/2)^k (I + H_k) the printed iteration reads
+//     R_k     = Q_k Q_k + 3 Q_k
+//     Q_{k+1} = Q_k R_k + 9/4 Q_k                          (= -A_{k+1} / 2 with A_{k+1} = P_k A_k P_k)
+//     H_{k+1} = 2/3 (Q_k H_k + Q_k + 3/2 H_k),  H_1 = 2/3 Q_0,  F_K = (3/2)^K H_K     (T_{k+1} = P_k T_k)
+// Every line is one product with the apply epilogue y = scale (acc + own C + c2 C2): the tensor-core operands are the
+// hi parts, the linear terms enter as hi + lo.  All matrices are polynomials in A_0: symmetric and commuting, so only
+// the tiles on or above the diagonal are computed; the hi part (the next products' operand) is also stored mirrored,
+// the lo part is only ever read as a linear term of the same tile.  H_1 is never stored:
+// H_2 = 4/9 (Q_1 Q_0 + 3/2 Q_0 + 3/2 Q_1) uses Q_0 directly.  The last H launch scales its result to F_K.
+enum { GC_R = 0, GC_Q, GC_H };
+void append_gc_problems(signmuon_ctx* c, std::vector<GemmProblem>& out, int what, int k, int K, bool local_polar_phase) {
+  for (int32_t p : c->matrix_list) {
+    const ParamPlan& pl = c->plan[p];
+    if (!pl.gs_mem) continue;
+    const size_t qbytes = (size_t)pl.s * pl.ldq * 2;
+    // (the local polar step works in its own batch slot, index Wm)
+    for (int m = local_polar_phase ? c->Wm : 0; m < (local_polar_phase ? c->Wm + 1 : c->Wm); ++m) {
+      // Q_k lives in buffer k & 1 (buffer 0 = the Gram launch's output), H_k in H buffer k & 1
+      auto q_hi = [&](int kk) { return ((kk & 1) ? pl.gc_q1_off : pl.q_off) + m * qbytes; };
+      auto q_lo = [&](int kk) { return ((kk & 1) ? pl.gc_q1lo_off : pl.qlo_off) + m * qbytes; };
+      auto q_map = [&](int kk, bool lo) { return pl.tmap_base + ((kk & 1) ? (lo ? TM_GC_Q1LO : TM_GC_Q1) : (lo ? TM_QLO_K128 : TM_Q_K128)); };
+      auto h_map = [&](int kk, bool lo) { return pl.tmap_base + ((kk & 1) ? TM_GC_H1 : TM_GC_H0) + (lo ? 1 : 0); };
+      GemmProblem pr;
+      std::memset(&pr, 0, sizeof(pr));
+      pr.M = pr.N = pr.K = (int32_t)pl.s;
+      pr.a_sm = pr.b_sn = pl.ldq; pr.a_sk = pr.b_sk = 1;
+      pr.batch = pr.batch_c = pr.batch_o = m;
+      pr.param = p;
+      pr.epi = EPI_APPLY;
+      pr.c_mode = C_HILO;
+      pr.ldc = pr.ld_out = pl.ldq;
+      pr.tma_c = pr.tma_out = 1;
+      pr.scale_imm = 1.f;
+      pr.sym = 1;
+      pr.mirror_hi = 1;
+      pr.A = reinterpret_cast<const bf16*>(q_hi(k));
+      pr.tmapA = q_map(k, false);
+      pr.C = reinterpret_cast<const void*>(q_hi(k));
+      pr.C_lo = reinterpret_cast<const bf16*>(q_lo(k));
+      pr.tmapC0 = q_map(k, false); pr.tmapC1 = q_map(k, true);
+      if (what == GC_R) {
+        pr.B = pr.A; pr.tmapB = pr.tmapA;
+        pr.own_coef = 3.f;
+        pr.out = reinterpret_cast<void*>(pl.gc_r_off + m * qbytes);
+        pr.out_lo = reinterpret_cast<bf16*>(pl.gc_r_off + m * qbytes);     // (never written: hi only)
+        pr.hi_only = 1;
+        pr.tmapO0 = pr.tmapO1 = pl.tmap_base + TM_GC_R;
+      } else if (what == GC_Q) {
+        pr.B = reinterpret_cast<const bf16*>(pl.gc_r_off + m * qbytes); pr.tmapB = pl.tmap_base + TM_GC_R;
+        pr.own_coef = 2.25f;
+        pr.out = reinterpret_cast<void*>(q_hi(k + 1));
+        pr.out_lo = reinterpret_cast<bf16*>(q_lo(k + 1));
+        pr.tmapO0 = q_map(k + 1, false); pr.tmapO1 = q_map(k + 1, true);
+      } else {
+        const bool from_q0 = (k == 1);       // H_1 = 2/3 Q_0 is not stored
+        pr.C2 = reinterpret_cast<const bf16*>(q_hi(k));
+        pr.C2_lo = reinterpret_cast<const bf16*>(q_lo(k));
+        if (from_q0) {
+          pr.B = reinterpret_cast<const bf16*>(q_hi(0)); pr.tmapB = q_map(0, false);
+          pr.C = reinterpret_cast<const void*>(q_hi(0)); pr.C_lo = reinterpret_cast<const bf16*>(q_lo(0));
+          pr.tmapC0 = q_map(0, false); pr.tmapC1 = q_map(0, true);
+          pr.c2_coef = 1.5f;
+        } else {
+          pr.B = reinterpret_cast<const bf16*>(pl.gc_h_off[k & 1] + m * qbytes); pr.tmapB = h_map(k, false);
+          pr.C = reinterpret_cast<const void*>(pl.gc_h_off[k & 1] + m * qbytes);
+          pr.C_lo = reinterpret_cast<const bf16*>(pl.gc_hlo_off[k & 1] + m * qbytes);
+          pr.tmapC0 = h_map(k, false); pr.tmapC1 = h_map(k, true);
+          pr.c2_coef = 1.f;
+        }
+        pr.own_coef = 1.5f;
+        double scale = from_q0 ? 4.0 / 9.0 : 2.0 / 3.0;
+        const bool final_h = (k == K - 1);
+        if (final_h) scale *= std::pow(1.5, (double)K);
+        pr.scale_imm = (float)scale;
+        pr.hi_only = final_h ? 1 : 0;        // F_K is an operand only
+        pr.out = reinterpret_cast<void*>(pl.gc_h_off[(k + 1) & 1] + m * qbytes);
+        pr.out_lo = reinterpret_cast<bf16*>(pl.gc_hlo_off[(k + 1) & 1] + m * qbytes);
+        pr.tmapO0 = h_map(k + 1, false); pr.tmapO1 = h_map(k + 1, true);
+      }
+      out.push_back(pr);
+    }
+  }
+}
+
 int plan_layout(signmuon_ctx* c) {
   const int M = c->Wm;                    // batch slots of a matrix parameter: this context's own workers (1: Muon rule)
   const int K = c->cfg.ns_steps;
@@ -405,9 +519,17 @@ int plan_layout(signmuon_ctx* c) {
     pl.fused_pack = (sp.kind == SIGNMUON_PARAM_MATRIX) && K > 0 && (sp.cols % 32 == 0) && !c->muon;
     // Gram-space iteration for short sides up to 256: needs at least two iterations to pay, the tensor-core kernels,
     // and the Frobenius scale (with the spectral scale the products already run in split precision the regular way)
-    pl.gs = sp.kind == SIGNMUON_PARAM_MATRIX && K >= 2 && pl.s <= 256 &&
-            !(c->cfg.flags & (SIGNMUON_FLAG_SIMT_GEMM | SIGNMUON_FLAG_NO_GRAM_SPACE)) &&
-            c->cfg.ns_scale == SIGNMUON_SCALE_FRO;
+    const bool gs_ok = sp.kind == SIGNMUON_PARAM_MATRIX && K >= 2 &&
+                       !(c->cfg.flags & (SIGNMUON_FLAG_SIMT_GEMM | SIGNMUON_FLAG_NO_GRAM_SPACE)) &&
+                       c->cfg.ns_scale == SIGNMUON_SCALE_FRO;
+    // Larger short sides: the same chain as symmetric products through memory, where it takes fewer tensor-core
+    // operations.  On the tiles actually computed an iteration on the full matrix costs about 3.06 s^2 l multiply-adds
+    // (Gram, upper tiles only, plus apply); the chain costs one Gram and one apply product (3.06 s^2 l) plus 3 (K - 1)
+    // symmetric s^3 products (about 0.53 s^3 each on the upper tiles).
+    // Measured: long sides from twice the short one gain (ResNet-50's 512 x 1024 ... 1000 x 2048, GPT-2's 768 x 2304
+    // and 768 x 3072, Llama's 4096 x 11008), square matrices lose a little (768^2, 4096^2).
+    pl.gs_mem = gs_ok && pl.s > 256 && 2 * pl.l >= 3 * pl.s;
+    pl.gs = gs_ok && (pl.s <= 256 || pl.gs_mem);
     pl.ld8 = (int32_t)round_up((size_t)sp.cols, 16);
     pl.lp_fp8 = sp.kind == SIGNMUON_PARAM_MATRIX && c->lp && K > 0 &&
                 !(c->cfg.flags & (SIGNMUON_FLAG_SIMT_GEMM | SIGNMUON_FLAG_LP_GRAM_BF16));
@@ -550,6 +672,13 @@ int plan_layout(signmuon_ctx* c) {
     pl.q_off = off; off += round_up(slots * pl.s * pl.ldq * 2, 1024);
     if (c->split) { pl.lo_off[1] = off; off += ybytes; }
     if (c->split || pl.gs) { pl.qlo_off = off; off += round_up(slots * pl.s * pl.ldq * 2, 1024); }
+    if (pl.gs_mem) {
+      const size_t qb = round_up(slots * pl.s * pl.ldq * 2, 1024);
+      pl.gc_q1_off = off; off += qb;
+      pl.gc_q1lo_off = off; off += qb;
+      pl.gc_r_off = off; off += qb;
+      for (int i = 0; i < 2; ++i) { pl.gc_h_off[i] = off; off += qb; pl.gc_hlo_off[i] = off; off += qb; }
+    }
     if (pl.lp_fp8) { pl.s8_off = off; off += round_up((size_t)pl.rows * pl.ld8, 1024); }
   }
   // GEMM problems: K x (gram, apply) for the workers, and again for the local polar step
@@ -569,14 +698,40 @@ int plan_layout(signmuon_ctx* c) {
     if (!tt.used) { tt.used = true; tt.problem_base = lp.problem_base; tt.problem_count = lp.problem_count; }
     ls.push_back(lp);
   };
+  // one launch of the Gram-space chain through memory: the problems of `stages` (GC_*) of iteration k
+  auto add_gc_launch = [&](std::vector<LaunchPlan>& ls, std::initializer_list<int> stages, int k, bool lp_phase, int table) {
+    LaunchPlan lp;
+    lp.problem_base = c->problems.size();
+    for (int what : stages) append_gc_problems(c, c->problems, what, k, K, lp_phase);
+    lp.problem_count = c->problems.size() - lp.problem_base;
+    lp.tile_table = table;
+    lp.gram = false;
+    if (lp.problem_count == 0) return;
+    TileTable& tt = c->tables[table];
+    if (!tt.used) { tt.used = true; tt.problem_base = lp.problem_base; tt.problem_count = lp.problem_count; }
+    ls.push_back(lp);
+  };
+  // the chain through memory follows the first Gram launch (tables: R, Q, HR, F in this order from `t0`)
+  auto add_gc_chain = [&](std::vector<LaunchPlan>& ls, bool lp_phase, int t0) {
+    if (K < 2) return;
+    add_gc_launch(ls, {GC_R}, 0, lp_phase, t0);
+    add_gc_launch(ls, {GC_Q}, 0, lp_phase, t0 + 1);
+    for (int kk = 1; kk <= K - 2; ++kk) {
+      add_gc_launch(ls, {GC_H, GC_R}, kk, lp_phase, t0 + 2);
+      add_gc_launch(ls, {GC_Q}, kk, lp_phase, t0 + 1);
+    }
+    add_gc_launch(ls, {GC_H}, K - 1, lp_phase, t0 + 3);
+  };
   if (!c->matrix_list.empty()) {
     for (int k = 0; k < K; ++k) {
       add_launch(c->ns_launches, true, k, M, false, k == 0 ? TT_GRAM_FIRST : TT_GRAM);
+      if (k == 0) add_gc_chain(c->ns_launches, false, TT_GC_R);
       add_launch(c->ns_launches, false, k, M, false, k == K - 1 ? TT_APPLY_LAST : TT_APPLY);
     }
     if (c->lp) {
       for (int k = 0; k < K; ++k) {
         add_launch(c->lp_launches, true, k, 1, true, k == 0 ? TT_LP_GRAM_FIRST : TT_LP_GRAM);
+        if (k == 0) add_gc_chain(c->lp_launches, true, TT_LP_GC_R);
         add_launch(c->lp_launches, false, k, 1, true, k == K - 1 ? TT_LP_APPLY_LAST : TT_LP_APPLY);
       }
     }
@@ -601,7 +756,7 @@ int plan_layout(signmuon_ctx* c) {
     cs.problems.clear();
     for (int32_t p : c->matrix_list) {
       const ParamPlan& pl = c->plan[p];
-      if (!pl.gs || (set == 1 && !c->lp)) continue;
+      if (!pl.gs || pl.gs_mem || (set == 1 && !c->lp)) continue;
       const size_t qbytes = (size_t)pl.s * pl.ldq * 2;
       for (int m = (set ? M : 0); m < (set ? M + 1 : M); ++m) {
         ChainProblem cp;
@@ -1129,7 +1284,7 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
     if (pl.kind == SIGNMUON_PARAM_MATRIX) {
       d.y0 = reinterpret_cast<bf16*>(c->d_ws + pl.y_off[0]);
       d.y1 = reinterpret_cast<bf16*>(c->d_ws + pl.y_off[1]);
-      d.ylo = (c->split || pl.gs) ? reinterpret_cast<bf16*>(c->d_ws + pl.lo_off[0]) : nullptr;
+      d.ylo = (c->split || (pl.gs && !pl.gs_mem)) ? reinterpret_cast<bf16*>(c->d_ws + pl.lo_off[0]) : nullptr;
       d.yk_buf = pl.gs ? 1 : (c->cfg.ns_steps & 1);
       d.scales = reinterpret_cast<float*>(c->d_ws + pl.scales_off);
       d.partials = reinterpret_cast<float*>(c->d_ws + pl.partials_off);
@@ -1258,6 +1413,12 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
         ok = ok && encode_map(mp + TM_QLO_K128, c->d_ws + pl.qlo_off, pl.s, pl.s, slots, pl.ldq, qb, 128);
         ok = ok && encode_map(mp + TM_QLO_KBN, c->d_ws + pl.qlo_off, pl.s, pl.s, slots, pl.ldq, qb, bn);
       }
+      if (pl.gs_mem) {
+        const size_t offs[7] = {pl.gc_q1_off, pl.gc_q1lo_off, pl.gc_r_off, pl.gc_h_off[0], pl.gc_hlo_off[0], pl.gc_h_off[1],
+                                pl.gc_hlo_off[1]};
+        for (int i = 0; i < 7; ++i)
+          ok = ok && encode_map(mp + TM_GC_Q1 + i, c->d_ws + offs[i], pl.s, pl.s, slots, pl.ldq, qb, 128);
+      }
       if (pl.lp_fp8)          // FP8 copy of the vote matrix: {128 bytes x 128 rows} boxes serve K-major and MN-major tiles
         ok = ok && encode_map_u8(mp + TM_S8, c->d_ws + pl.s8_off, pl.cols, pl.rows, pl.ld8);
       if (pl.cols % 4 == 0)   // float32 momentum as the first iteration's C operand
@@ -1277,6 +1438,10 @@ int signmuon_bind(signmuon_ctx* c, void* dev_state, size_t state_bytes, void* de
       uint8_t* cbase = (pr.c_mode == C_F32) ? c->d_state : c->d_ws;
       pr.C = cbase + reinterpret_cast<size_t>(pr.C);
       if (pr.C_lo) pr.C_lo = reinterpret_cast<const bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.C_lo));
+      if (pr.c2_coef != 0.f) {
+        pr.C2 = reinterpret_cast<const bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.C2));
+        pr.C2_lo = reinterpret_cast<const bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.C2_lo));
+      }
       pr.out_lo = reinterpret_cast<bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.out_lo));
     } else if (pr.gram_lo) {
       pr.out_lo = reinterpret_cast<bf16*>(c->d_ws + reinterpret_cast<size_t>(pr.out_lo));

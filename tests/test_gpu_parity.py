@@ -235,13 +235,36 @@ def test_gram_space_iteration_against_oracle_and_full_matrix_iteration(K):
     run_and_check(wl, steps=1, flags=0)
 
 
+@pytest.mark.parametrize("K", [2, 5])
+def test_gram_space_chain_through_memory_against_oracle_and_full_matrix_iteration(K):
+    """Longer short sides iterate in Gram space as a chain of symmetric s x s products through memory (upper tiles
+    computed, hi part mirrored).  Held to the oracle's Alg. 4 like the per-iteration path, on shapes with ragged
+    tiles, wide and tall, and with the default flags as well."""
+    import numpy as np
+    from parity_utils import run_and_check
+    shapes = [(512, 2048), (2048, 512), (320, 512), (300, 1000), (1000, 300), (768, 2304), (264, 4096), (520, 520)]
+    wl = _wl(shapes, 3, K=K)
+    rep_gs, rep_full, cap_gs, cap_full = {}, {}, {}, {}
+    run_and_check(wl, steps=2, report=rep_gs, capture=cap_gs)
+    run_and_check(wl, steps=2, flags=B.FLAG_KEEP_POLAR | B.FLAG_NO_GRAM_SPACE, report=rep_full, capture=cap_full)
+    print("gram space:", rep_gs, "\nper iteration:", rep_full)
+    assert rep_gs["polar_relfro"] <= 2e-2 and rep_full["polar_relfro"] <= 2e-2
+    for m in range(wl.num_workers):
+        a = cap_gs["payloads"][0][m].cpu().numpy().view(np.uint8)
+        b = cap_full["payloads"][0][m].cpu().numpy().view(np.uint8)
+        assert int(np.unpackbits(a ^ b).sum()) <= 2e-3 * wl.numel
+    run_and_check(wl, steps=1, flags=0)
+    run_and_check(wl, steps=1, flags=B.FLAG_KEEP_POLAR | B.FLAG_GEMM_1CTA)
+
+
 def test_local_polar_step_in_gram_space_against_oracle_and_full_matrix_iteration():
-    """The local polar step of matrices with a short side up to 256 also iterates in Gram space (FP8 Gram of the
-    vote matrix, the on-chip chain, one apply launch that updates the weights).  Both that path and the per-iteration
+    """The local polar step also iterates in Gram space where the workers' iterations do (FP8 Gram of the vote matrix,
+    the on-chip chain or the chain through memory, one apply launch that updates the weights).  Both that path and the per-iteration
     one are held to the oracle's Alg. 4 on the vote matrix; the Gram-space path, whose product with the exact +-1 matrix
     carries only the rounding of F_K, is the more accurate of the two."""
     from parity_utils import run_and_check
-    shapes = [(64, 576), (576, 64), (100, 328), (200, 200), (256, 1024), (1024, 256), (64, 147), (16, 2048), (320, 512)]
+    shapes = [(64, 576), (576, 64), (100, 328), (200, 200), (256, 1024), (1024, 256), (64, 147), (16, 2048), (320, 512),
+              (512, 2048), (1000, 300), (520, 520)]
     wl = _wl(shapes, 4, local_polar=True, lr=0.01)
     rep_gs = run_and_check(wl, steps=2)
     rep_full = run_and_check(wl, steps=2, flags=B.FLAG_KEEP_POLAR | B.FLAG_NO_GRAM_SPACE)
