@@ -197,14 +197,48 @@ def time_oracle(wl, steps, warmup, budget_flops, min_seconds=0.0):
             "sample_seconds_per_step": per_sample_step, "extrapolated": True}
 
 
-# ncu DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the Newton-Schulz launches per unit of work, from
-# the captures summarised in profiles/ (small cases; the traffic of these launches grows in proportion to the entries
-# they process): bytes per (entry, worker) of one Gram launch and of one apply launch.
-NCU_NS_TRAFFIC_PER_ENTRY = {
-    # workload family -> (gram bytes per entry and worker, apply bytes per entry and worker, capture it comes from)
-    "large": (3.62, 12.04, "c5:4096x4096:4 (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
-    "c2_resnet50": (2.19, 7.87, "c2, matrices with a short side of 512 and more (profiles/ns_gemm_tc_kernel_c2_and_c5_4096.md)"),
+# ncu DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the grouped Newton-Schulz product launches per unit
+# of work, from the captures summarised in profiles/ns_gemm_tc_kernel_launch_metrics.md (small cases; the traffic of
+# these launches grows in proportion to the units they process).  Per path of a matrix (ns_path) and size class:
+#   full:   bytes per (entry, batch slot) of one Gram launch and of one apply launch (mean over the K apply launches);
+#   memory: bytes per (entry, batch slot) of the one Gram and of the one apply launch, and bytes per (entry of the
+#           s x s Gram matrix, batch slot) of the whole chain of 3 (K - 1) products at K = 5.
+NCU_NS_TRAFFIC = {
+    "large": {"full": (3.56, 11.6), "memory": (4.88, 22.6, 98.0),
+              "src": "c5:4096x4096:4 (full matrix) and c5:4096x11008:2 (Gram space through memory)"},
+    "small": {"full": (2.1, 7.1), "memory": (2.0, 6.6, 53.0),
+              "src": "c5:768x3072:16, per-iteration path (earlier capture) and Gram space through memory"},
 }
+# c2 (all of its 54 matrices iterate in Gram space) is small enough to capture whole: DRAM bytes of the 13 grouped
+# product launches of one step (the on-chip chain launch, 23.8 MB, not included)
+NCU_NS_TRAFFIC_C2_STEP = 3494.7e6
+
+
+def ns_traffic_per_launch(wl, launches):
+    """Mean DRAM traffic of a grouped Newton-Schulz product launch of this workload, scaled from the small captures
+    (None where no capture covers the workload's shapes and paths)."""
+    if wl.name.startswith("c2_resnet50") and not wl.local_polar and wl.ns_steps == 5:
+        return NCU_NS_TRAFFIC_C2_STEP / launches, "ncu capture of every product launch of one c2 step"
+    K = wl.ns_steps
+    total = 0.0
+    classes = set()
+    for p in wl.params:
+        if p.kind != "matrix":
+            continue
+        s_ = min(p.rows, p.cols)
+        path = ns_path(p, K)
+        if path == "chip" or (path == "memory" and K != 5):
+            return None, "no capture for this mix of shapes"
+        cls = "large" if s_ >= 2048 else "small"
+        classes.add(cls)
+        slots = wl.num_workers + (1 if wl.local_polar else 0)
+        c = NCU_NS_TRAFFIC[cls][path]
+        if path == "full":
+            total += slots * p.numel * K * (c[0] + c[1])
+        else:
+            total += slots * (p.numel * (c[0] + c[1]) + s_ * s_ * c[2])
+    src = "; ".join(NCU_NS_TRAFFIC[c]["src"] for c in sorted(classes))
+    return total / launches, "ncu captures of " + src + ", scaled by the units each launch kind processes"
 
 
 def max_over_ranks(values, dist=None, device="cpu"):
@@ -279,21 +313,31 @@ def kernel_report(wl, opt, stage_ms, peaks, clocks, timed_region_s, ns_scale="fr
                                      "frac_of_nominal_8000": a / NOMINAL_HBM_GBS}
     ns_ms = stage_ms["newton_schulz"] + stage_ms["local_polar"]
     if ns_ms > 0 and ns_flops > 0:
-        launches = 2 * K * (2 if wl.local_polar else 1)
+        launches = opt.ns_launches_per_step[0]     # grouped tensor-core product launches (workers + local polar step)
         tf = ns_flops / ns_ms / 1e9
         # The method's own memory traffic of the Newton-Schulz stage: the momentum is read once and one bit per entry
         # and worker is written (plus, for the local polar step, the +-1 matrix in and the weights in and out).
         method_bytes = sum(M * p.numel * (4 + 1 / 8) for p in mat) + \
             (sum(p.numel * (2 + 2 * gb[p.dtype]) for p in mat) if wl.local_polar else 0)
-        # What this implementation moves: per entry, batch slot and iteration the Gram product reads the bf16 iterate
-        # (2 B), the apply product reads it again as an operand (2 B) and moves the hi + lo pair in and out (8 B).  A
-        # matrix whose workers iterate in Gram space (short side <= 256, K >= 2, Frobenius scale) crosses HBM twice per
-        # step instead: hi + lo operands of the one Gram product (4 B), hi + lo operands of the one apply product (4 B)
-        # and the float32 momentum as its own term (4 B); the local polar step always iterates on the full matrix.
-        def gram_space(p):
-            return min(p.rows, p.cols) <= 256 and K >= 2 and ns_scale == "fro"
-        impl_bytes = sum(12.0 * p.numel * (M if gram_space(p) else K * M) + (12.0 * p.numel * K if wl.local_polar else 0.0)
-                         for p in mat)
+        # What this implementation moves through HBM, by the path a matrix takes (ns_path):
+        #  full   per entry, batch slot and iteration the Gram product reads the bf16 iterate (2 B), the apply product reads
+        #         it again as an operand (2 B) and moves the hi + lo pair in and out (8 B);
+        #  chip   (Gram space, chain on chip) the matrix crosses HBM twice per step: hi + lo operands of the one Gram
+        #         product (4 B), hi + lo operands of the one apply product (4 B), the float32 momentum as its own term (4 B);
+        #  memory (Gram space, chain of s x s products through memory) the one Gram and the one apply product read the hi
+        #         part (2 B each), the apply product the float32 momentum (4 B); each of the 3 (K - 1) chain products moves
+        #         about 16 B per entry of an s x s matrix (two hi operands 4 B, a hi + lo linear term 4 B or two of them
+        #         8 B, hi + lo results on the upper tiles and the mirrored hi part about 5 B).
+        # The local polar step's slot reads the +-1 matrix instead (1 B as FP8 for the Gram product, 2 B + 2 B as bf16
+        # for the apply product) and moves the weights in and out.
+        def slot_bytes(p, lp_slot):
+            path = ns_path(p, K, ns_scale)
+            s_, wb = min(p.rows, p.cols), gb[p.dtype]
+            if path == "full":
+                return 12.0 * p.numel * K
+            ends = (5.0 + 2 * wb) * p.numel if lp_slot else (12.0 if path == "chip" else 8.0) * p.numel
+            return ends + (16.0 * s_ * s_ * 3 * (K - 1) if path == "memory" else 0.0)
+        impl_bytes = sum(M * slot_bytes(p, False) + (slot_bytes(p, True) if wl.local_polar else 0.0) for p in mat)
         kernels["ns_gemm_tc"] = {
             "ms": ns_ms, "bound": "tensor", "launches": launches, "algorithmic_flops": ns_flops,
             "executed_flops": ns_exec, "achieved_tflops": tf, "executed_tflops": ns_exec / ns_ms / 1e9,
@@ -310,6 +354,19 @@ def kernel_report(wl, opt, stage_ms, peaks, clocks, timed_region_s, ns_scale="fr
     return kernels
 
 
+def ns_path(p, K, ns_scale="fro"):
+    """Which evaluation of Alg. 4's loop the library picks for a matrix parameter (its rule, restated): "chip" = Gram
+    space with the chain on chip (short side up to 256), "memory" = Gram space as a chain of symmetric s x s products
+    through memory (longer short sides when the long side is at least 1.5 times the short one), else "full" = every
+    iteration on the full matrix.  Gram space needs K >= 2 and the Frobenius scale."""
+    s_, l_ = min(p.rows, p.cols), max(p.rows, p.cols)
+    if K < 2 or ns_scale != "fro":
+        return "full"
+    if s_ <= 256:
+        return "chip"
+    return "memory" if 2 * l_ >= 3 * s_ else "full"
+
+
 def roofline_of(wl, kernels, peaks, clocks, timed_ns_seconds):
     """`roofline` object of the dominant kernel family."""
     dom = max(kernels, key=lambda k: kernels[k]["ms"])
@@ -324,14 +381,7 @@ def roofline_of(wl, kernels, peaks, clocks, timed_ns_seconds):
         near_max = bool(sm and mx and sm >= 0.9 * mx)
         use_sustained = timed_ns_seconds >= 1.0 and not near_max
         peak = peaks["bf16_tflops_sustained"] if use_sustained else peaks["bf16_tflops"]
-        fam = "c2_resnet50" if wl.name.startswith("c2") else "large"
-        g_b, a_b, src = NCU_NS_TRAFFIC_PER_ENTRY[fam]
-        # entries of the matrices that take part in every launch (those with a short side up to 256 iterate in Gram
-        # space and appear in the first Gram and the last apply launch only)
-        units = sum(p.numel for p in wl.params if p.kind == "matrix" and (min(p.rows, p.cols) > 256 or wl.ns_steps < 2)) * \
-            (wl.num_workers + (1 if wl.local_polar else 0)) / (2.0 if wl.local_polar else 1.0)
-        # mean over a step's Gram and apply launches (a local polar launch processes 1 / M of a workers' launch)
-        traffic = 0.5 * (g_b + a_b) * units
+        traffic, src = ns_traffic_per_launch(wl, launches)
         return {"kernel": "ns_gemm_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
                 "unit": "TFLOP/s", "frac": achieved / peak,
                 "frac_is": ("of measured sustained cuBLAS bf16 (timed Newton-Schulz work %.1f s, median SM clock %s MHz)"
@@ -345,7 +395,10 @@ def roofline_of(wl, kernels, peaks, clocks, timed_ns_seconds):
                 "executed_tflops": kd["executed_tflops"], "frac_executed": kd["executed_tflops"] / peak,
                 "frac_executed_of_nominal_2250": kd["executed_tflops"] / NOMINAL_BF16_TFLOPS,
                 "ms_per_launch": kd["ms"] / launches,
-                "traffic": traffic, "traffic_source": "ncu capture of " + src + ", scaled by (entries x batch slots)",
+                "note": "achieved counts Alg. 4's own 4 s^2 l K flops per matrix and batch slot; the library executes fewer "
+                        "(upper tiles of symmetric products, iterations carried out on the s x s Gram matrix), so frac can "
+                        "exceed 1: frac_executed is the rate of the tensor-core operations actually issued",
+                "traffic": traffic, "traffic_source": src,
                 "peak_source": peaks["source"]}
     achieved = kd["achieved_gbs"]
     return {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",

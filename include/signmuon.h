@@ -308,6 +308,12 @@ int signmuon_sign_agreement(signmuon_ctx* ctx, uint64_t* host_agree, uint64_t* h
 /* Number of kernels signmuon_step launches per call with the current configuration. */
 int signmuon_launches_per_step(const signmuon_ctx* ctx, int32_t* launches);
 
+/* Of those, the launches of the Newton-Schulz products (workers' iterations and local polar step together):
+ * `gemm_launches` grouped tensor-core product launches (Alg. 4's Gram and apply products, and the s x s products of
+ * iterations that run in Gram space through memory) and `chain_launches` launches of the on-chip Gram-space chain.
+ * Either pointer may be null.  Errors: INVALID_ARG (null context). */
+int signmuon_ns_launches_per_step(const signmuon_ctx* ctx, int32_t* gemm_launches, int32_t* chain_launches);
+
 /* Newton-Schulz floating-point operations of one step: 4 s^2 l K per matrix and worker (plus one
  * more "worker" for the local polar step), s = min(rows, cols), l = max(rows, cols). */
 int signmuon_ns_flops_per_step(const signmuon_ctx* ctx, double* flops);

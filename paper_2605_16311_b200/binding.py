@@ -29,7 +29,7 @@ EXPORTS = [
     "signmuon_step_host", "signmuon_packed_payload", "signmuon_payload_buffer", "signmuon_vote_update",
     "signmuon_local_sign_sum", "signmuon_vote_update_from_sums", "signmuon_exchange_flags",
     "signmuon_set_payload_peers", "signmuon_payload_segment", "signmuon_debug_tap",
-    "signmuon_status", "signmuon_launches_per_step", "signmuon_ns_flops_per_step", "signmuon_ns_executed_flops_per_step",
+    "signmuon_status", "signmuon_launches_per_step", "signmuon_ns_launches_per_step", "signmuon_ns_flops_per_step", "signmuon_ns_executed_flops_per_step",
     "signmuon_power_start_size", "signmuon_power_start_segment", "signmuon_set_power_start",
     "signmuon_sign_agreement", "signmuon_set_wait_limit", "signmuon_selftest_wait_timeout",
     "signmuon_momentum_norm_noalloc", "signmuon_destroy", "signmuon_error_string",
@@ -84,6 +84,7 @@ def load_library() -> C.CDLL:
     lib.signmuon_debug_tap.argtypes = [vp, i32, i32, i32, C.POINTER(vp), C.POINTER(sz), C.POINTER(C.c_int64)]
     lib.signmuon_status.argtypes = [vp, vp]
     lib.signmuon_launches_per_step.argtypes = [vp, C.POINTER(i32)]
+    lib.signmuon_ns_launches_per_step.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
     lib.signmuon_ns_flops_per_step.argtypes = [vp, C.POINTER(C.c_double)]
     lib.signmuon_ns_executed_flops_per_step.argtypes = [vp, C.POINTER(C.c_double)]
     lib.signmuon_power_start_size.argtypes = [vp, C.POINTER(sz)]
@@ -240,6 +241,12 @@ def signmuon_launches_per_step(ctx: int) -> int:
     n = C.c_int32()
     _check(load_library().signmuon_launches_per_step(ctx, C.byref(n)), "signmuon_launches_per_step")
     return n.value
+
+
+def signmuon_ns_launches_per_step(ctx: int):
+    g, ch = C.c_int32(), C.c_int32()
+    _check(load_library().signmuon_ns_launches_per_step(ctx, C.byref(g), C.byref(ch)), "signmuon_ns_launches_per_step")
+    return g.value, ch.value
 
 
 def signmuon_ns_flops_per_step(ctx: int) -> float:
@@ -507,6 +514,11 @@ class SignMuon:
     @property
     def launches_per_step(self) -> int:
         return signmuon_launches_per_step(self.ctx)
+
+    @property
+    def ns_launches_per_step(self):
+        """(grouped tensor-core product launches, on-chip chain launches) of the Newton-Schulz work of one step."""
+        return signmuon_ns_launches_per_step(self.ctx)
 
     @property
     def ns_flops_per_step(self) -> float:

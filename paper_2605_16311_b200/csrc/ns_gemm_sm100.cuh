@@ -693,6 +693,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
           const uint32_t b = g % EPI_BUFS;
           const uint32_t buf = epi_base + b * BUF_BYTES;
           const int col0 = n0 + ch * 64 + sub * NC;    // first of this thread's columns
+          // second linear term of a chain product: this thread's NC columns of its row, hi and lo parts (one cache line
+          // each), requested before the waits so that their latency is hidden
+          if (KIND == 1 && c2_hi != nullptr && col0 < prN) {
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(c2_hi + col0));
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(c2_lo + col0));
+          }
           ok = mbar_wait(smem_u32(&c_full_bar[b]), (g / EPI_BUFS) & 1u, abort_flag, args.status, args.wait_limit_ns);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
@@ -707,7 +713,6 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) ns_gemm_tc_kernel(const __gri
             }
           }
           if (KIND == 1 && c2_hi != nullptr) {
-            // second linear term of a chain product: this thread's NC columns of its row, hi + lo
 #pragma unroll
             for (int u = 0; u < UNITS; ++u) {
               if (col0 + u * 8 >= prN) break;

@@ -1792,6 +1792,15 @@ int signmuon_ns_flops_per_step(const signmuon_ctx* c, double* flops) {
   return SIGNMUON_OK;
 }
 
+int signmuon_ns_launches_per_step(const signmuon_ctx* c, int32_t* gemm_launches, int32_t* chain_launches) {
+  if (!c) return SIGNMUON_ERR_INVALID_ARG;
+  const bool lp = !c->matrix_list.empty() && c->lp && c->cfg.ns_steps > 0;
+  if (gemm_launches) *gemm_launches = (int32_t)(c->ns_launches.size() + (lp ? c->lp_launches.size() : 0));
+  if (chain_launches)
+    *chain_launches = (c->chain[0].problems.empty() ? 0 : 1) + ((lp && !c->chain[1].problems.empty()) ? 1 : 0);
+  return SIGNMUON_OK;
+}
+
 int signmuon_ns_executed_flops_per_step(const signmuon_ctx* c, double* flops) {
   if (!c || !flops) return SIGNMUON_ERR_INVALID_ARG;
   if (!c->bound) return SIGNMUON_ERR_NOT_BOUND;
