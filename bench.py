@@ -217,7 +217,7 @@ NCU_NS_TRAFFIC_C2_STEP = 3494.7e6
 def ns_traffic_per_launch(wl, launches):
     """Mean DRAM traffic of a grouped Newton-Schulz product launch of this workload, scaled from the small captures
     (None where no capture covers the workload's shapes and paths)."""
-    if wl.name.startswith("c2_resnet50") and not wl.local_polar and wl.ns_steps == 5:
+    if wl.name.startswith("c2_resnet50") and not wl.local_polar and wl.ns_steps == 5 and not NO_GRAM_SPACE:
         return NCU_NS_TRAFFIC_C2_STEP / launches, "ncu capture of every product launch of one c2 step"
     K = wl.ns_steps
     total = 0.0
@@ -354,13 +354,16 @@ def kernel_report(wl, opt, stage_ms, peaks, clocks, timed_region_s, ns_scale="fr
     return kernels
 
 
+NO_GRAM_SPACE = False      # set from --no-gram-space
+
+
 def ns_path(p, K, ns_scale="fro"):
     """Which evaluation of Alg. 4's loop the library picks for a matrix parameter (its rule, restated): "chip" = Gram
     space with the chain on chip (short side up to 256), "memory" = Gram space as a chain of symmetric s x s products
     through memory (longer short sides when the long side is at least 1.5 times the short one), else "full" = every
     iteration on the full matrix.  Gram space needs K >= 2 and the Frobenius scale."""
     s_, l_ = min(p.rows, p.cols), max(p.rows, p.cols)
-    if K < 2 or ns_scale != "fro":
+    if K < 2 or ns_scale != "fro" or NO_GRAM_SPACE:
         return "full"
     if s_ <= 256:
         return "chip"
@@ -422,7 +425,7 @@ def measure(wl, args, dev, dist, rank, world, local_rank, steps, warmup, with_e2
         kw = {"worker_offset": shard[0], "local_workers": shard[1]}
     opt = B.SignMuon(wl.params, wl.num_workers, momentum=wl.momentum, lr=wl.lr, ns_steps=wl.ns_steps,
                      local_polar=wl.local_polar, device=dev, host_staging=with_e2e, ns_scale=args.ns_scale,
-                     power_iters=args.power_iters, **kw)
+                     power_iters=args.power_iters, flags=(B.FLAG_NO_GRAM_SPACE if args.no_gram_space else 0), **kw)
     if args.ns_scale == "spectral":     # seeded start vectors of the power iteration, reused by every step
         flat = torch.zeros(opt.power_start_size, dtype=torch.float32, device=dev)
         for p, v in enumerate(wlmod.make_power_start(wl, 0, dev)):
@@ -752,10 +755,14 @@ def main():
     ap.add_argument("--ns-scale", default="fro", choices=["fro", "spectral"],
                     help="Alg. 4 scale: Frobenius norm (default, the benchmark configuration) or power iteration")
     ap.add_argument("--power-iters", type=int, default=2)
+    ap.add_argument("--no-gram-space", action="store_true",
+                    help="every Newton-Schulz iteration on the full matrix (the library's NO_GRAM_SPACE flag): for comparisons")
     ap.add_argument("--sweep", action="store_true", help="run the kernel sweep (config 5) and print one line per point")
     ap.add_argument("--sweep-workers", default="1,2,4,8,16,32")
     ap.add_argument("--sweep-shapes", default="", help="comma-separated ROWSxCOLS list (default: the whole sweep)")
     args = ap.parse_args()
+    global NO_GRAM_SPACE
+    NO_GRAM_SPACE = args.no_gram_space
     if args.sweep:
         run_sweep(args)
         return
