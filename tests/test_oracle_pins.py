@@ -91,6 +91,33 @@ def test_gram_space_evaluation_is_the_same_map_as_alg4(shape, K):
     assert np.max(np.abs(a_chain - a_lit)) <= 1e-12
 
 
+@pytest.mark.parametrize("shape,K", [((6, 40), 5), ((40, 6), 3), ((9, 14), 2), ((5, 17), 7)])
+def test_gram_space_chain_of_symmetric_products_is_the_same_map_as_alg4(shape, K):
+    """The form of the same reading that the CUDA path runs through memory for longer short sides: with Q_k = -A_k / 2
+    and T_k = (3/2)^k (I + H_k):  R_k = Q_k Q_k + 3 Q_k,  Q_{k+1} = Q_k R_k + 9/4 Q_k,
+    H_{k+1} = 2/3 (Q_k H_k + Q_k + 3/2 H_k) with H_1 = 2/3 Q_0,  Y_K = (3/2)^K (Y_0 + H_K Y_0);  every matrix of the
+    chain is symmetric (only its upper tiles are computed there).  Written out in numpy and compared with the oracle's
+    literal iteration."""
+    x = RNG.normal(size=shape)
+    wide = shape[0] <= shape[1]
+    y0 = x / np.linalg.norm(x)
+    q = -0.5 * (y0 @ y0.T if wide else y0.T @ y0)
+    h = (2.0 / 3.0) * q
+    for k in range(K - 1):                 # Q_{k+1} from Q_k; H_{k+2} from Q_{k+1}, H_{k+1}
+        r = q @ q + 3.0 * q
+        q = q @ r + 2.25 * q
+        h = (2.0 / 3.0) * (q @ h + q + 1.5 * h)
+        for m in (r, q, h):
+            assert np.max(np.abs(m - m.T)) <= 1e-14
+    f = 1.5 ** K * h
+    y_chain = 1.5 ** K * y0 + (f @ y0 if wide else y0 @ f)
+    y_literal = O.polar_ns(x, K)
+    assert np.max(np.abs(y_chain - y_literal)) <= 1e-12 * np.max(np.abs(y_literal))
+    # Q_{K-1} is -1/2 times the Gram matrix of the literal iterate Y_{K-1}
+    yk = O.polar_ns(x, K - 1)
+    assert np.max(np.abs(-2.0 * q - (yk @ yk.T if wide else yk.T @ yk))) <= 1e-12
+
+
 @pytest.mark.parametrize("K", [1, 2, 3, 4, 5])
 def test_newton_schulz_polar_error_bound(K):
     # tall 9 x 2 with singular values 0.8, 0.6: ||X||_F = 1, rho = ||I - X^T X||_op = 0.64
