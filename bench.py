@@ -226,7 +226,7 @@ def ns_traffic_per_launch(wl, launches):
         if p.kind != "matrix":
             continue
         s_ = min(p.rows, p.cols)
-        path = ns_path(p, K)
+        path = ns_path(p, K, wl=wl)
         if path == "chip" or (path == "memory" and K != 5):
             return None, "no capture for this mix of shapes"
         cls = "large" if s_ >= 2048 else "small"
@@ -331,7 +331,7 @@ def kernel_report(wl, opt, stage_ms, peaks, clocks, timed_region_s, ns_scale="fr
         # The local polar step's slot reads the +-1 matrix instead (1 B as FP8 for the Gram product, 2 B + 2 B as bf16
         # for the apply product) and moves the weights in and out.
         def slot_bytes(p, lp_slot):
-            path = ns_path(p, K, ns_scale)
+            path = ns_path(p, K, ns_scale, wl)
             s_, wb = min(p.rows, p.cols), gb[p.dtype]
             if path == "full":
                 return 12.0 * p.numel * K
@@ -357,17 +357,24 @@ def kernel_report(wl, opt, stage_ms, peaks, clocks, timed_region_s, ns_scale="fr
 NO_GRAM_SPACE = False      # set from --no-gram-space
 
 
-def ns_path(p, K, ns_scale="fro"):
+def ns_path(p, K, ns_scale="fro", wl=None):
     """Which evaluation of Alg. 4's loop the library picks for a matrix parameter (its rule, restated): "chip" = Gram
     space with the chain on chip (short side up to 256), "memory" = Gram space as a chain of symmetric s x s products
-    through memory (longer short sides when the long side is at least 1.5 times the short one), else "full" = every
-    iteration on the full matrix.  Gram space needs K >= 2 and the Frobenius scale."""
-    s_, l_ = min(p.rows, p.cols), max(p.rows, p.cols)
+    through memory (longer short sides when the long side is at least 1.5 times the short one, and when the matrices of
+    workload `wl` that qualify hold at least 8 M (entry, worker) pairs together), else "full" = every iteration on the
+    full matrix.  Gram space needs K >= 2 and the Frobenius scale."""
+    def qualifies(q):
+        s_, l_ = min(q.rows, q.cols), max(q.rows, q.cols)
+        return q.kind == "matrix" and s_ > 256 and 2 * l_ >= 3 * s_
     if K < 2 or ns_scale != "fro" or NO_GRAM_SPACE:
         return "full"
-    if s_ <= 256:
+    if min(p.rows, p.cols) <= 256:
         return "chip"
-    return "memory" if 2 * l_ >= 3 * s_ else "full"
+    if not qualifies(p):
+        return "full"
+    if wl is not None and sum(q.numel for q in wl.params if qualifies(q)) * wl.num_workers < 8.0e6:
+        return "full"
+    return "memory"
 
 
 def roofline_of(wl, kernels, peaks, clocks, timed_ns_seconds):

@@ -540,6 +540,15 @@ int plan_layout(signmuon_ctx* c) {
     else c->plain_list.push_back((int32_t)p);
     c->entries += pl.d;
   }
+  // The chain through memory adds 2K - 1 launches to a step (to the workers' iterations, and again to the local polar
+  // step): measured, that pays once the matrices that would take it hold about 8 M (entry, worker) pairs together
+  // (512 x 2048 from 8 workers on, 1024 x 4096 from 2); below that they iterate on the full matrix.
+  {
+    double pairs = 0;
+    for (const ParamPlan& pl : c->plan) if (pl.gs_mem) pairs += (double)pl.d * c->Wm;
+    if (pairs < 8.0e6)
+      for (ParamPlan& pl : c->plan) if (pl.gs_mem) pl.gs_mem = pl.gs = false;
+  }
   if (words >= (1ull << 32)) return SIGNMUON_ERR_BAD_SHAPE;
   c->words_per_worker = words;
   c->bits_pitch = round_up((size_t)words, 32);

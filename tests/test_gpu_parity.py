@@ -244,6 +244,14 @@ def test_gram_space_chain_through_memory_against_oracle_and_full_matrix_iteratio
     from parity_utils import run_and_check
     shapes = [(512, 2048), (2048, 512), (320, 512), (300, 1000), (1000, 300), (768, 2304), (264, 4096), (520, 520)]
     wl = _wl(shapes, 3, K=K)
+    # the path under test is the one taken: 2K launches for the square matrix, 2K - 1 more for the chain
+    from parity_utils import make_optimizer
+    opt = make_optimizer(wl, flags=0)
+    assert opt.ns_launches_per_step == (4 * K - 1, 0)
+    opt.close()
+    opt = make_optimizer(wl, flags=B.FLAG_NO_GRAM_SPACE)
+    assert opt.ns_launches_per_step == (2 * K, 0)
+    opt.close()
     rep_gs, rep_full, cap_gs, cap_full = {}, {}, {}, {}
     run_and_check(wl, steps=2, report=rep_gs, capture=cap_gs)
     run_and_check(wl, steps=2, flags=B.FLAG_KEEP_POLAR | B.FLAG_NO_GRAM_SPACE, report=rep_full, capture=cap_full)
@@ -264,7 +272,7 @@ def test_local_polar_step_in_gram_space_against_oracle_and_full_matrix_iteration
     carries only the rounding of F_K, is the more accurate of the two."""
     from parity_utils import run_and_check
     shapes = [(64, 576), (576, 64), (100, 328), (200, 200), (256, 1024), (1024, 256), (64, 147), (16, 2048), (320, 512),
-              (512, 2048), (1000, 300), (520, 520)]
+              (512, 2048), (1000, 300), (520, 520), (768, 2304)]
     wl = _wl(shapes, 4, local_polar=True, lr=0.01)
     rep_gs = run_and_check(wl, steps=2)
     rep_full = run_and_check(wl, steps=2, flags=B.FLAG_KEEP_POLAR | B.FLAG_NO_GRAM_SPACE)
