@@ -123,9 +123,12 @@ enum {
                                      CTA pairs on 256 x 256 tiles (same results; for comparison) */
   SIGNMUON_FLAG_LP_GRAM_BF16 = 32, /* run the first Gram product of the local polar step on the bf16 copy of the vote
                                      matrix instead of its FP8 (E4M3) copy (same result bit for bit; for comparison) */
-  SIGNMUON_FLAG_NO_GRAM_SPACE = 64, /* run every Newton-Schulz iteration on the full matrix, also for parameters with a
-                                     short side of at most 256 (whose iteration otherwise runs in Gram space on chip;
-                                     same map, two passes over the matrix instead of 2 K; for comparison) */
+  SIGNMUON_FLAG_NO_GRAM_SPACE = 64, /* run every Newton-Schulz iteration on the full matrix, also for the parameters
+                                     whose iteration otherwise runs on their s x s Gram matrix (Alg. 4's loop evaluated
+                                     as A_{k+1} = P_k A_k P_k, Y_K = (P_{K-1} ... P_0) Y_0: short sides up to 256 on
+                                     chip; longer short sides of matrices at least 1.5 times as long as a chain of
+                                     symmetric products through memory, when they hold 8 M (entry, worker) pairs
+                                     together; same map, two passes over the matrix instead of 2 K; for comparison) */
   SIGNMUON_FLAG_SIGN_AGREEMENT = 16 /* count, every step, how many of each worker's sign bits equal the vote
                                      (one more small kernel; read with signmuon_sign_agreement) */
 };
