@@ -496,6 +496,32 @@ def test_muon_rule_against_oracle(dtype, M, K):
     opt.close()
 
 
+def test_muon_rule_with_the_chain_through_memory():
+    """The Muon rule on a matrix large enough (one batch slot, 9.4 M entries) for its iteration to run in Gram space as
+    a chain through memory, whose last apply launch then updates the weights: direction against the oracle's PolarNS of
+    the GPU's own momentum."""
+    import oracle as O
+    from parity_utils import _np64
+    K, M = 5, 2
+    wl = _wl([(2048, 4608)], M, dtype="f32", K=K, lr=0.01)
+    opt = B.SignMuon(wl.params, M, momentum=0.9, lr=0.01, ns_steps=K, update_rule="muon")
+    assert opt.ns_launches_per_step == (2 + 2 * K - 1, 0)     # Gram, 2K - 1 chain launches, apply
+    w = wlmod.make_weights(wl, "cuda:0")
+    sig = wlmod.make_signal(wl, "cuda:0")
+    g = wlmod.make_grads(wl, sig, 0, "cuda:0")
+    w0 = _np64(w[0])
+    opt.step(w, g)
+    torch.cuda.synchronize()
+    assert opt.status() == B.OK
+    u_or = O.polar_ns_short_side(_np64(opt.tap(B.TAP_MOMENTUM, 0, 0)), K, 1e-12)
+    d_gpu = (w0 - _np64(w[0])) / 0.01
+    noise = np.linalg.norm(np.abs(w0) * 1.2e-7 / 0.01)
+    rel = max(np.linalg.norm(d_gpu - u_or) - noise, 0.0) / np.linalg.norm(u_or)
+    print("muon, chain through memory: direction off by", rel)
+    assert rel <= 2e-3
+    opt.close()
+
+
 @pytest.mark.parametrize("flags", [0, B.FLAG_GEMM_1CTA])
 def test_local_polar_first_gram_in_fp8_equals_bf16_bit_for_bit(flags):
     """The local polar step's first Gram product reads the vote matrix as E4M3 bytes (+-1 are exact, the fp32
